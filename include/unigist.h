@@ -1,0 +1,181 @@
+/*
+ * unigist.h -- C ABI of the UniGist gist-masked attention library for NVIDIA B200 (sm_100a).
+ *
+ * The library implements the attention operator of "UniGist: Towards General and
+ * Hardware-aligned Sequence-level Long Context Compression" (arXiv 2509.15763):
+ * one gist token is inserted after every r raw tokens (Eq. 2), every token attends to all
+ * sinks, all earlier gists and the raw tokens of its own gist unit plus the k units before
+ * it (Eq. 3), gists are moved to the right end of the sequence so the mask becomes
+ * tile-aligned (Section 4.2, "gist shift trick"), and at inference raw tokens outside the
+ * window are physically dropped from the KV cache (Section 4.3).
+ *
+ * Conventions that hold for every call
+ *  - Indices are 0-based.  s = sinks, T = raw tokens, r = ratio, n = T / r gists,
+ *    N = s + T + n.  The window is given as W raw tokens and means k = ceil(W / r)
+ *    previous gist units.
+ *  - "Interleaved" order is Eq. 2's Z.  "Shifted" order is [sinks | raw | gists], each kind
+ *    in its original order.  Attention calls take SHIFTED tensors.
+ *  - Dense tensors are [batch, N, heads, head_dim], head_dim contiguous, bf16 unless stated,
+ *    base pointers 16-byte aligned.  Query head h uses KV head h / (Hq / Hkv).
+ *  - Every pointer named "device" is memory of the current CUDA device; the CALLER owns every
+ *    buffer, the library never allocates or frees device memory.  Scratch comes in through
+ *    `workspace` (size from unigist_workspace_bytes / unigist_decode_workspace_bytes).
+ *  - `stream` is a cudaStream_t passed as void* (NULL = default stream).  Calls only enqueue
+ *    work; they do not synchronise.
+ *  - Return value: UNIGIST_OK or an error code; nothing is launched when arguments are
+ *    rejected.  unigist_last_error_string() describes the last failure of the calling thread.
+ *  - There is no CPU fallback: without a CUDA device the compute entry points return
+ *    UNIGIST_ERR_CUDA.
+ */
+#ifndef UNIGIST_H_
+#define UNIGIST_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  UNIGIST_OK = 0,
+  UNIGIST_ERR_INVALID_ARG = 1, /* null pointer, negative size, bad enum */
+  UNIGIST_ERR_SHAPE = 2,       /* T % r != 0, Hq % Hkv != 0, unsupported head_dim ... */
+  UNIGIST_ERR_ALIGNMENT = 3,   /* pointer or row size not 16-byte aligned */
+  UNIGIST_ERR_WORKSPACE = 4,   /* workspace missing or too small */
+  UNIGIST_ERR_UNSUPPORTED = 5,
+  UNIGIST_ERR_CUDA = 6,        /* a CUDA runtime / driver call failed */
+  UNIGIST_ERR_TIMEOUT = 7      /* a bounded device-side wait gave up */
+} unigist_status;
+
+/* dO passed to unigist_attn_bwd is fp32 (rounded to bf16 when it is read). */
+#define UNIGIST_FLAG_DOUT_FP32 1u
+
+enum { UNIGIST_PAGE_TOKENS = 64 }; /* tokens per KV-cache block */
+
+typedef enum {
+  UNIGIST_OP_FWD = 0,
+  UNIGIST_OP_BWD = 1,
+  UNIGIST_OP_COMPACT = 2
+} unigist_op;
+
+/* Problem statement of Section 4.1: (s, T, r, window) plus the attention shape. */
+typedef struct {
+  int32_t batch;        /* B >= 1 */
+  int32_t raw_len;      /* T, multiple of ratio */
+  int32_t num_sinks;    /* s >= 0 */
+  int32_t ratio;        /* r >= 1 */
+  int32_t window;       /* W >= 0 raw tokens; k = ceil(W / r) */
+  int32_t num_q_heads;  /* Hq */
+  int32_t num_kv_heads; /* Hkv, divides Hq */
+  int32_t head_dim;     /* D: 64 or 128 */
+  float softmax_scale;  /* 0 => 1 / sqrt(D) */
+  uint32_t flags;       /* UNIGIST_FLAG_* */
+} unigist_problem;
+
+/* Eq. 2: N = s + T + T / r.  Negative on a malformed problem. */
+int32_t unigist_total_len(const unigist_problem* p);
+/* Text after Eq. 3: number k of previous gist units in the local window, ceil(W / r). */
+int32_t unigist_window_units(const unigist_problem* p);
+/* Tokens left in the cache after compaction: s + n + min(k, n) * r (Section 4.3). */
+int32_t unigist_compact_len(const unigist_problem* p);
+/* Number of visible (query, key) pairs per head under Eq. 3; what "unmasked FLOPs" counts. */
+int64_t unigist_visible_pairs(const unigist_problem* p);
+/* Bytes of device scratch the given op needs for this problem (0 on a malformed problem). */
+size_t unigist_workspace_bytes(const unigist_problem* p, int32_t op);
+
+/*
+ * Gist shift index arrays (Section 4.2; the "original token indexes" the kernel design
+ * passes along).  shift_perm[sigma] = interleaved index of the token at shifted position
+ * sigma; unshift_perm = inverse; pos_ids[t] (interleaved order) = position id with each gist
+ * taking the id of the raw token right after it (Section 4.1, step 3).
+ * Each array has N int32 entries and may be NULL.  on_device = 0: host pointers, computed on
+ * the host, stream ignored.  on_device = 1: device pointers, filled by a kernel on `stream`.
+ */
+int32_t unigist_layout(const unigist_problem* p, int32_t* shift_perm, int32_t* unshift_perm,
+                       int32_t* pos_ids, int32_t on_device, void* stream);
+
+/*
+ * Gist shift / unshift of a [B, N, heads, D] device tensor with elements of elem_bytes
+ * (2 or 4) bytes (Section 4.2): dst[b, sigma] = src[b, shift_perm[sigma]] (shift) and
+ * dst[b, t] = src[b, unshift_perm[t]] (unshift).  src and dst must not overlap;
+ * heads * D * elem_bytes must be a multiple of 16.
+ */
+int32_t unigist_gist_shift(const unigist_problem* p, const void* src, void* dst, int32_t heads,
+                           int32_t elem_bytes, void* stream);
+int32_t unigist_gist_unshift(const unigist_problem* p, const void* src, void* dst, int32_t heads,
+                             int32_t elem_bytes, void* stream);
+
+/*
+ * Forward (Section 4.2 kernel; Eq. 3 mask): for each (b, head, row t)
+ *   S_tj = scale * q_t . k_j over visible j,  LSE_t = log sum_j exp(S_tj),  O_t = softmax(S_t) V.
+ * q [B,N,Hq,D], k, v [B,N,Hkv,D], o [B,N,Hq,D]: device bf16, SHIFTED order.
+ * lse [B,Hq,N]: device fp32, natural log, shifted order.  Masked-out tiles are never read.
+ */
+int32_t unigist_attn_fwd(const unigist_problem* p, const void* q, const void* k, const void* v,
+                         void* o, float* lse, void* workspace, size_t ws_bytes, void* stream);
+
+/*
+ * Backward of the forward above (the paper's backward kernel, Appendix speed-up table):
+ *   Delta = rowsum(dO o O), P = exp(S - LSE), dV = P^T dO, dP = dO V^T, dS = P o (dP - Delta),
+ *   dQ = scale dS K, dK = scale dS^T Q;  dK, dV summed over the query heads of a KV head.
+ * q, k, v, o, lse as in the forward; d_o [B,N,Hq,D] device bf16 (fp32 with
+ * UNIGIST_FLAG_DOUT_FP32); dq [B,N,Hq,D], dk, dv [B,N,Hkv,D] device bf16, all shifted.
+ * dK/dV are accumulated without atomics: each key tile is owned by one thread block.
+ */
+int32_t unigist_attn_bwd(const unigist_problem* p, const void* q, const void* k, const void* v,
+                         const void* o, const float* lse, const void* d_o, void* dq, void* dk,
+                         void* dv, void* workspace, size_t ws_bytes, void* stream);
+
+/*
+ * KV compaction (Section 4.3): after the last gist of a T-token prefix, keep the sinks, all n
+ * gists and the raw tokens of the last min(k, n) units; every other raw token is dropped.
+ * Cache order is [sinks | gists | window raw]; L = unigist_compact_len().
+ * The cache is paged: k_cache, v_cache [num_blocks, Hkv, 64, D] device bf16;
+ * block_table [B, max_blocks_per_seq] device int32 maps logical block -> physical block.
+ *
+ *  k, v != NULL: gather from the shifted tensors k, v [B,N,Hkv,D] into the pages named by the
+ *      first ceil(L / 64) entries of each block_table row (read only).
+ *  k == v == NULL: compact IN PLACE a paged cache that holds the whole shifted sequence
+ *      (logical position = shifted position; the first ceil(N / 64) entries of each row are
+ *      valid and distinct).  The row is rewritten: entries [0, ceil(L/64)) are the compacted
+ *      cache, entries [ceil(L/64), ceil(N/64)) list the freed physical blocks.  When
+ *      s, T, n and T - min(k,n)*r are multiples of 64 this is a block-table edit and no token
+ *      moves; otherwise kept tokens are staged through `workspace`
+ *      (unigist_workspace_bytes(p, UNIGIST_OP_COMPACT)).
+ * seq_lens [B] device int32 receives L.  kept_idx (nullable) [B, L] device int32 receives the
+ * SHIFTED position each cache entry came from.
+ */
+int32_t unigist_kv_compact(const unigist_problem* p, const void* k, const void* v, void* k_cache,
+                           void* v_cache, int32_t num_blocks, int32_t* block_table,
+                           int32_t max_blocks_per_seq, int32_t* seq_lens, int32_t* kept_idx,
+                           void* workspace, size_t ws_bytes, void* stream);
+
+/* Scratch for unigist_decode (split-KV partial results). */
+size_t unigist_decode_workspace_bytes(int32_t num_seqs, int32_t num_q_heads, int32_t num_kv_heads,
+                                      int32_t head_dim, int32_t max_blocks_per_seq);
+
+/*
+ * Decode over the compressed cache (Section 4.3; FlashDecoding-style split over keys): one
+ * query per sequence attends to ALL seq_lens[i] cache entries (what is left in a compacted
+ * cache is visible by construction; the caller appends the new token's K/V first).
+ * q, o [num_seqs, Hq, D] device bf16; k_cache, v_cache [num_blocks, Hkv, 64, D] device bf16;
+ * block_table [num_seqs, max_blocks_per_seq], seq_lens [num_seqs] device int32 (>= 1);
+ * lse [num_seqs, Hq] device fp32, nullable.  head_dim must be 128.
+ */
+int32_t unigist_decode(int32_t num_seqs, int32_t num_q_heads, int32_t num_kv_heads,
+                       int32_t head_dim, float softmax_scale, const void* q, const void* k_cache,
+                       const void* v_cache, int32_t num_blocks, const int32_t* block_table,
+                       int32_t max_blocks_per_seq, const int32_t* seq_lens, void* o, float* lse,
+                       void* workspace, size_t ws_bytes, void* stream);
+
+/* Number of kernels the library has launched in this process (all threads). */
+int64_t unigist_launch_count(void);
+
+/* Message for the last non-OK status returned to the calling thread ("" if none). */
+const char* unigist_last_error_string(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* UNIGIST_H_ */

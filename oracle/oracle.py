@@ -53,6 +53,8 @@ def lib() -> ctypes.CDLL:
         L.ug_oracle_attn_fwd.restype = i32
         L.ug_oracle_attn_bwd.argtypes = [i64] * 4 + [i32, i32, f64] + [p] * 7
         L.ug_oracle_attn_bwd.restype = i32
+        L.ug_oracle_attn_bwd_sample.argtypes = [i64] * 4 + [i32, i32, f64] + [p] * 4 + [i64, p, i64, p, p, p, p]
+        L.ug_oracle_attn_bwd_sample.restype = i32
         L.ug_oracle_kept_set.argtypes = [i64] * 4 + [p]
         L.ug_oracle_kept_set.restype = i64
         L.ug_oracle_decode.argtypes = [i64, i32, i32, f64] + [p] * 5
@@ -135,6 +137,22 @@ def attn_bwd_slice(s, T, r, k, scale, q, kk, v, dout):
     dv = np.empty_like(v)
     rc = lib().ug_oracle_attn_bwd(s, T, r, k, G, D, float(scale), _ptr(q), _ptr(kk),
                                   _ptr(v), _ptr(dout), _ptr(dq), _ptr(dk), _ptr(dv))
+    assert rc == 0, rc
+    return dq, dk, dv
+
+
+def attn_bwd_sample(s, T, r, k, scale, q, kk, v, dout, rows, keys):
+    """One (batch, KV head), sampled outputs: dq of `rows` [R,G,D]; dk, dv of `keys` [K,D]."""
+    q, kk, v, dout = _c64(q), _c64(kk), _c64(v), _c64(dout)
+    N, G, D = q.shape
+    rows = np.ascontiguousarray(rows, dtype=np.int64)
+    keys = np.ascontiguousarray(keys, dtype=np.int64)
+    dq = np.empty((len(rows), G, D))
+    dk = np.empty((len(keys), D))
+    dv = np.empty((len(keys), D))
+    rc = lib().ug_oracle_attn_bwd_sample(s, T, r, k, G, D, float(scale), _ptr(q), _ptr(kk), _ptr(v),
+                                         _ptr(dout), len(rows), _ptr(rows), len(keys), _ptr(keys),
+                                         _ptr(dq), _ptr(dk), _ptr(dv))
     assert rc == 0, rc
     return dq, dk, dv
 

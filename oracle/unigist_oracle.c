@@ -202,25 +202,42 @@ int32_t ug_oracle_attn_fwd(int64_t s, int64_t T, int64_t r, int64_t k,
 }
 
 /*
- * Backward for one (batch, KV head) slice.
- *   q, dout [N][G][D]; kk, v [N][D];  dq [N][G][D]; dk, dv [N][D].
+ * Backward for one (batch, KV head) slice, restricted to a sample of outputs.
+ *   q, dout [N][G][D]; kk, v [N][D].
+ *   dq_out [n_rows][G][D] = dQ of the listed query rows,
+ *   dk_out, dv_out [n_keys][D] = dK, dV of the listed key positions.
  * With P as in the forward:
  *   dV = P^T dO,  dP = dO V^T,  Delta_t = sum_j P_tj dP_tj,
  *   dS = P o (dP - Delta),  dQ = scale dS K,  dK = scale dS^T Q,
  * dK and dV summed over the G query heads of the slice.
- * Pass 1 walks rows (LSE, Delta, dQ); pass 2 walks key columns and evaluates
- * the column sums dV_j = sum_t P_tj dO_t and dK_j = scale sum_t dS_tj q_t.
+ * Pass 1 walks the query rows that are listed or that see a listed key (LSE, Delta, dQ);
+ * pass 2 walks the listed key columns and evaluates the column sums
+ * dV_j = sum_t P_tj dO_t and dK_j = scale sum_t dS_tj q_t.
  */
-int32_t ug_oracle_attn_bwd(int64_t s, int64_t T, int64_t r, int64_t k,
-                           int32_t G, int32_t D, double scale, const double *q,
-                           const double *kk, const double *v,
-                           const double *dout, double *dq, double *dk,
-                           double *dv) {
+int32_t ug_oracle_attn_bwd_sample(int64_t s, int64_t T, int64_t r, int64_t k,
+                                  int32_t G, int32_t D, double scale,
+                                  const double *q, const double *kk,
+                                  const double *v, const double *dout,
+                                  int64_t n_rows, const int64_t *rows,
+                                  int64_t n_keys, const int64_t *keys,
+                                  double *dq_out, double *dk_out,
+                                  double *dv_out) {
   if (r <= 0 || T % r != 0 || s < 0 || k < 0) return 1;
   const int64_t N = s + T + T / r;
   double *lse = (double *)malloc((size_t)N * G * sizeof(double));
   double *delta = (double *)malloc((size_t)N * G * sizeof(double));
-  if (!lse || !delta) return 2;
+  int64_t *slot = (int64_t *)malloc((size_t)N * sizeof(int64_t)); /* -1, -2 or dq slot */
+  if (!lse || !delta || !slot) return 2;
+  for (int64_t t = 0; t < N; ++t) slot[t] = -1; /* not needed */
+  for (int64_t a = 0; a < n_keys; ++a) {
+    if (keys[a] < 0 || keys[a] >= N) return 1;
+    for (int64_t t = keys[a]; t < N; ++t)
+      if (ug_oracle_visible(t, keys[a], s, r, k)) slot[t] = -2; /* needed, no dq */
+  }
+  for (int64_t a = 0; a < n_rows; ++a) {
+    if (rows[a] < 0 || rows[a] >= N) return 1;
+    slot[rows[a]] = a;
+  }
   int32_t err = 0;
 #pragma omp parallel
   {
@@ -233,6 +250,7 @@ int32_t ug_oracle_attn_bwd(int64_t s, int64_t T, int64_t r, int64_t k,
     } else {
 #pragma omp for schedule(dynamic, 4)
       for (int64_t t = 0; t < N; ++t) {
+        if (slot[t] == -1) continue;
         for (int64_t j = 0; j < N; ++j)
           mrow[j] = (uint8_t)ug_oracle_visible(t, j, s, r, k);
         for (int32_t g = 0; g < G; ++g) {
@@ -255,7 +273,10 @@ int32_t ug_oracle_attn_bwd(int64_t s, int64_t T, int64_t r, int64_t k,
             dp[j] = dot(dot_, v + (size_t)j * D, D);
             dl += sc[j] * dp[j];
           }
-          double *dqt = dq + ((size_t)t * G + g) * D;
+          lse[(size_t)t * G + g] = L;
+          delta[(size_t)t * G + g] = dl;
+          if (slot[t] < 0) continue;
+          double *dqt = dq_out + ((size_t)slot[t] * G + g) * D;
           for (int d = 0; d < D; ++d) dqt[d] = 0.0;
           for (int64_t j = 0; j < N; ++j) {
             if (!mrow[j]) continue;
@@ -263,8 +284,6 @@ int32_t ug_oracle_attn_bwd(int64_t s, int64_t T, int64_t r, int64_t k,
             const double *kj = kk + (size_t)j * D;
             for (int d = 0; d < D; ++d) dqt[d] += scale * ds * kj[d];
           }
-          lse[(size_t)t * G + g] = L;
-          delta[(size_t)t * G + g] = dl;
         }
       }
     }
@@ -273,10 +292,11 @@ int32_t ug_oracle_attn_bwd(int64_t s, int64_t T, int64_t r, int64_t k,
     free(dp);
   }
   if (!err) {
-#pragma omp parallel for schedule(dynamic, 4)
-    for (int64_t j = 0; j < N; ++j) {
-      double *dkj = dk + (size_t)j * D;
-      double *dvj = dv + (size_t)j * D;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int64_t a = 0; a < n_keys; ++a) {
+      const int64_t j = keys[a];
+      double *dkj = dk_out + (size_t)a * D;
+      double *dvj = dv_out + (size_t)a * D;
       const double *kj = kk + (size_t)j * D;
       const double *vj = v + (size_t)j * D;
       for (int d = 0; d < D; ++d) dkj[d] = dvj[d] = 0.0;
@@ -299,7 +319,26 @@ int32_t ug_oracle_attn_bwd(int64_t s, int64_t T, int64_t r, int64_t k,
   }
   free(lse);
   free(delta);
+  free(slot);
   return err;
+}
+
+/* The whole backward of one slice: every row and every key.
+ *   dq [N][G][D]; dk, dv [N][D]. */
+int32_t ug_oracle_attn_bwd(int64_t s, int64_t T, int64_t r, int64_t k,
+                           int32_t G, int32_t D, double scale, const double *q,
+                           const double *kk, const double *v,
+                           const double *dout, double *dq, double *dk,
+                           double *dv) {
+  if (r <= 0 || T % r != 0 || s < 0 || k < 0) return 1;
+  const int64_t N = s + T + T / r;
+  int64_t *all = (int64_t *)malloc((size_t)N * sizeof(int64_t));
+  if (!all) return 2;
+  for (int64_t t = 0; t < N; ++t) all[t] = t;
+  int32_t rc = ug_oracle_attn_bwd_sample(s, T, r, k, G, D, scale, q, kk, v, dout,
+                                         N, all, N, all, dq, dk, dv);
+  free(all);
+  return rc;
 }
 
 /*

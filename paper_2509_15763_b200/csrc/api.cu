@@ -1,0 +1,264 @@
+// C-ABI entry points: argument validation, error reporting, dispatch to the kernel launchers.
+#include <atomic>
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+
+#include "ug_common.cuh"
+
+namespace ug {
+
+static thread_local char g_err[512] = "";
+static std::atomic<int64_t> g_launches{0};
+
+int32_t fail(int32_t code, const char* fmt, ...) {
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(g_err, sizeof(g_err), fmt, ap);
+  va_end(ap);
+  return code;
+}
+
+void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+
+int32_t check_launch(const char* what) {
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return fail(UNIGIST_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
+  return UNIGIST_OK;
+}
+
+int32_t check_problem(const unigist_problem* p, Geom* g, float* scale) {
+  if (!p) return fail(UNIGIST_ERR_INVALID_ARG, "problem is NULL");
+  if (p->batch < 1 || p->raw_len < 1 || p->num_sinks < 0 || p->ratio < 1 || p->window < 0 ||
+      p->num_q_heads < 1 || p->num_kv_heads < 1)
+    return fail(UNIGIST_ERR_INVALID_ARG, "problem has a non-positive size");
+  if (p->raw_len % p->ratio != 0)
+    return fail(UNIGIST_ERR_SHAPE, "raw_len %d is not a multiple of ratio %d", p->raw_len,
+                p->ratio);
+  if (p->num_q_heads % p->num_kv_heads != 0)
+    return fail(UNIGIST_ERR_SHAPE, "num_q_heads %d is not a multiple of num_kv_heads %d",
+                p->num_q_heads, p->num_kv_heads);
+  if (p->head_dim != 64 && p->head_dim != 128)
+    return fail(UNIGIST_ERR_SHAPE, "head_dim %d is not 64 or 128", p->head_dim);
+  const int64_t n = p->raw_len / p->ratio;
+  const int64_t N = (int64_t)p->num_sinks + p->raw_len + n;
+  if (N > (int64_t)1 << 30) return fail(UNIGIST_ERR_SHAPE, "sequence too long");
+  if (!(p->softmax_scale >= 0.f) || std::isinf(p->softmax_scale))
+    return fail(UNIGIST_ERR_INVALID_ARG, "softmax_scale must be finite and >= 0");
+  if (g) {
+    g->s = p->num_sinks;
+    g->T = p->raw_len;
+    g->r = p->ratio;
+    g->n = (int)n;
+    g->N = (int)N;
+    const int64_t k = ((int64_t)p->window + p->ratio - 1) / p->ratio;
+    g->k = (int)(k < n ? k : n);
+  }
+  if (scale) *scale = p->softmax_scale > 0.f ? p->softmax_scale : 1.0f / sqrtf((float)p->head_dim);
+  return UNIGIST_OK;
+}
+
+static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+}  // namespace ug
+
+using namespace ug;
+
+extern "C" {
+
+int32_t unigist_total_len(const unigist_problem* p) {
+  Geom g;
+  if (check_problem(p, &g, nullptr) != UNIGIST_OK) return -1;
+  return g.N;
+}
+
+int32_t unigist_window_units(const unigist_problem* p) {
+  if (check_problem(p, nullptr, nullptr) != UNIGIST_OK) return -1;
+  return (int32_t)(((int64_t)p->window + p->ratio - 1) / p->ratio);
+}
+
+int32_t unigist_compact_len(const unigist_problem* p) {
+  Geom g;
+  if (check_problem(p, &g, nullptr) != UNIGIST_OK) return -1;
+  return g.s + g.n + g.k * g.r;
+}
+
+int64_t unigist_visible_pairs(const unigist_problem* p) {
+  Geom g;
+  if (check_problem(p, &g, nullptr) != UNIGIST_OK) return -1;
+  // Row counts of Eq. 3 summed over sink, raw and gist queries.
+  int64_t tot = (int64_t)g.s * (g.s + 1) / 2 + (int64_t)g.s * ((int64_t)g.T + g.n);
+  const int64_t r = g.r;
+  for (int64_t u = 0; u < g.n; ++u) {
+    const int64_t w = u < g.k ? u : g.k;
+    tot += r * r * w + r * (r + 1) / 2 + r * u;  // raw queries of unit u
+    tot += (w + 1) * r + u + 1;                  // gist query u
+  }
+  return tot;
+}
+
+size_t unigist_workspace_bytes(const unigist_problem* p, int32_t op) {
+  Geom g;
+  if (check_problem(p, &g, nullptr) != UNIGIST_OK) return 0;
+  switch (op) {
+    case UNIGIST_OP_FWD:
+      return 0;
+    case UNIGIST_OP_BWD: {
+      // Delta [B,Hq,N] fp32, plus a bf16 copy of dO when it arrives as fp32.
+      size_t b = align_up((size_t)p->batch * p->num_q_heads * g.N * sizeof(float), 256);
+      if (p->flags & UNIGIST_FLAG_DOUT_FP32)
+        b += align_up((size_t)p->batch * g.N * p->num_q_heads * p->head_dim * 2, 256);
+      return b;
+    }
+    case UNIGIST_OP_COMPACT: {
+      const size_t L = (size_t)g.s + g.n + (size_t)g.k * g.r;
+      return align_up(2 * (size_t)p->batch * L * p->num_kv_heads * p->head_dim * 2, 256);
+    }
+    default:
+      return 0;
+  }
+}
+
+int32_t unigist_layout(const unigist_problem* p, int32_t* sp, int32_t* up, int32_t* pos,
+                       int32_t on_device, void* stream) {
+  Geom g;
+  if (int32_t rc = check_problem(p, &g, nullptr)) return rc;
+  if (!on_device) {
+    for (int i = 0; i < g.N; ++i) {
+      if (sp) sp[i] = shift_perm(g, i);
+      if (up) up[i] = unshift_perm(g, i);
+      if (pos) {  // i is an interleaved index here
+        const int sig = unshift_perm(g, i);
+        pos[i] = sig < g.s + g.T ? sig : g.s + (sig - g.s - g.T + 1) * g.r;
+      }
+    }
+    return UNIGIST_OK;
+  }
+  return launch_layout(g, sp, up, pos, (cudaStream_t)stream);
+}
+
+static int32_t shift_common(const unigist_problem* p, const void* src, void* dst, int32_t heads,
+                            int32_t elem_bytes, void* stream, bool inverse) {
+  Geom g;
+  if (int32_t rc = check_problem(p, &g, nullptr)) return rc;
+  if (!src || !dst) return fail(UNIGIST_ERR_INVALID_ARG, "src/dst is NULL");
+  if (heads < 1 || (elem_bytes != 2 && elem_bytes != 4))
+    return fail(UNIGIST_ERR_INVALID_ARG, "heads must be >= 1 and elem_bytes 2 or 4");
+  const size_t row = (size_t)heads * p->head_dim * elem_bytes;
+  if (row % 16 || !aligned16(src) || !aligned16(dst))
+    return fail(UNIGIST_ERR_ALIGNMENT, "rows and pointers must be 16-byte aligned");
+  const char* a = (const char*)src;
+  const char* b = (const char*)dst;
+  const size_t tot = row * g.N * p->batch;
+  if (a < b + tot && b < a + tot) return fail(UNIGIST_ERR_INVALID_ARG, "src and dst overlap");
+  return launch_shift(g, p->batch, src, dst, row, inverse, (cudaStream_t)stream);
+}
+
+int32_t unigist_gist_shift(const unigist_problem* p, const void* src, void* dst, int32_t heads,
+                           int32_t elem_bytes, void* stream) {
+  return shift_common(p, src, dst, heads, elem_bytes, stream, false);
+}
+int32_t unigist_gist_unshift(const unigist_problem* p, const void* src, void* dst, int32_t heads,
+                             int32_t elem_bytes, void* stream) {
+  return shift_common(p, src, dst, heads, elem_bytes, stream, true);
+}
+
+int32_t unigist_attn_fwd(const unigist_problem* p, const void* q, const void* k, const void* v,
+                         void* o, float* lse, void* workspace, size_t ws_bytes, void* stream) {
+  Geom g;
+  float scale;
+  if (int32_t rc = check_problem(p, &g, &scale)) return rc;
+  (void)workspace;
+  (void)ws_bytes;
+  if (!q || !k || !v || !o || !lse) return fail(UNIGIST_ERR_INVALID_ARG, "a tensor is NULL");
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || !aligned16(lse))
+    return fail(UNIGIST_ERR_ALIGNMENT, "tensor pointers must be 16-byte aligned");
+  return launch_fwd_simt(g, *p, scale, q, k, v, o, lse, (cudaStream_t)stream);
+}
+
+int32_t unigist_attn_bwd(const unigist_problem* p, const void* q, const void* k, const void* v,
+                         const void* o, const float* lse, const void* d_o, void* dq, void* dk,
+                         void* dv, void* workspace, size_t ws_bytes, void* stream) {
+  Geom g;
+  float scale;
+  if (int32_t rc = check_problem(p, &g, &scale)) return rc;
+  if (!q || !k || !v || !o || !lse || !d_o || !dq || !dk || !dv)
+    return fail(UNIGIST_ERR_INVALID_ARG, "a tensor is NULL");
+  const void* ptrs[] = {q, k, v, o, lse, d_o, dq, dk, dv, workspace};
+  for (const void* x : ptrs)
+    if (!aligned16(x)) return fail(UNIGIST_ERR_ALIGNMENT, "tensor pointers must be 16-byte aligned");
+  const size_t need = unigist_workspace_bytes(p, UNIGIST_OP_BWD);
+  if (!workspace || ws_bytes < need)
+    return fail(UNIGIST_ERR_WORKSPACE, "backward needs %zu bytes of workspace, got %zu", need,
+                ws_bytes);
+  return launch_bwd_simt(g, *p, scale, q, k, v, o, lse, d_o, dq, dk, dv, (float*)workspace,
+                         (cudaStream_t)stream);
+}
+
+int32_t unigist_kv_compact(const unigist_problem* p, const void* k, const void* v, void* kc,
+                           void* vc, int32_t num_blocks, int32_t* table, int32_t max_blocks,
+                           int32_t* seq_lens, int32_t* kept_idx, void* workspace, size_t ws_bytes,
+                           void* stream) {
+  Geom g;
+  if (int32_t rc = check_problem(p, &g, nullptr)) return rc;
+  if (!kc || !vc || !table || !seq_lens) return fail(UNIGIST_ERR_INVALID_ARG, "a pointer is NULL");
+  if ((k == nullptr) != (v == nullptr))
+    return fail(UNIGIST_ERR_INVALID_ARG, "k and v must both be given or both be NULL");
+  if (!aligned16(k) || !aligned16(v) || !aligned16(kc) || !aligned16(vc) || !aligned16(workspace))
+    return fail(UNIGIST_ERR_ALIGNMENT, "tensor pointers must be 16-byte aligned");
+  const int L = g.s + g.n + g.k * g.r;
+  const int need_blocks = ((k ? L : g.N) + UNIGIST_PAGE_TOKENS - 1) / UNIGIST_PAGE_TOKENS;
+  if (num_blocks < 1 || max_blocks < need_blocks)
+    return fail(UNIGIST_ERR_SHAPE, "block table has %d entries per sequence, %d needed", max_blocks,
+                need_blocks);
+  if (k) {
+    return launch_compact_gather(g, *p, k, v, kc, vc, num_blocks, table, max_blocks, seq_lens,
+                                 kept_idx, (cudaStream_t)stream);
+  }
+  const bool edit_only = g.s % 64 == 0 && g.T % 64 == 0 && g.n % 64 == 0 && (g.k * g.r) % 64 == 0;
+  if (!edit_only) {
+    const size_t need = unigist_workspace_bytes(p, UNIGIST_OP_COMPACT);
+    if (!workspace || ws_bytes < need)
+      return fail(UNIGIST_ERR_WORKSPACE, "in-place compaction needs %zu bytes of workspace, got %zu",
+                  need, ws_bytes);
+  }
+  return launch_compact_inplace(g, *p, kc, vc, num_blocks, table, max_blocks, seq_lens, kept_idx,
+                                edit_only ? nullptr : workspace, (cudaStream_t)stream);
+}
+
+size_t unigist_decode_workspace_bytes(int32_t S, int32_t Hq, int32_t Hkv, int32_t D,
+                                      int32_t max_blocks) {
+  if (S < 1 || Hq < 1 || Hkv < 1 || D < 1 || max_blocks < 1) return 0;
+  const int splits = decode_num_splits(S, Hkv, max_blocks);
+  // per (seq, q head, split): D fp32 partial outputs + running max + running sum
+  return align_up((size_t)S * Hq * splits * (D + 2) * sizeof(float), 256);
+}
+
+int32_t unigist_decode(int32_t S, int32_t Hq, int32_t Hkv, int32_t D, float softmax_scale,
+                       const void* q, const void* kc, const void* vc, int32_t num_blocks,
+                       const int32_t* table, int32_t max_blocks, const int32_t* seq_lens, void* o,
+                       float* lse, void* workspace, size_t ws_bytes, void* stream) {
+  if (S < 1 || Hq < 1 || Hkv < 1 || max_blocks < 1 || num_blocks < 1)
+    return fail(UNIGIST_ERR_INVALID_ARG, "decode has a non-positive size");
+  if (Hq % Hkv) return fail(UNIGIST_ERR_SHAPE, "num_q_heads %d is not a multiple of num_kv_heads %d", Hq, Hkv);
+  if (D != 128) return fail(UNIGIST_ERR_SHAPE, "decode supports head_dim 128, got %d", D);
+  if (Hq / Hkv > 8) return fail(UNIGIST_ERR_UNSUPPORTED, "decode supports at most 8 query heads per KV head");
+  if (!q || !kc || !vc || !table || !seq_lens || !o) return fail(UNIGIST_ERR_INVALID_ARG, "a pointer is NULL");
+  if (!aligned16(q) || !aligned16(kc) || !aligned16(vc) || !aligned16(o) || !aligned16(workspace))
+    return fail(UNIGIST_ERR_ALIGNMENT, "tensor pointers must be 16-byte aligned");
+  if (!(softmax_scale >= 0.f) || std::isinf(softmax_scale))
+    return fail(UNIGIST_ERR_INVALID_ARG, "softmax_scale must be finite and >= 0");
+  const float scale = softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf((float)D);
+  const size_t need = unigist_decode_workspace_bytes(S, Hq, Hkv, D, max_blocks);
+  if (!workspace || ws_bytes < need)
+    return fail(UNIGIST_ERR_WORKSPACE, "decode needs %zu bytes of workspace, got %zu", need, ws_bytes);
+  return launch_decode(S, Hq, Hkv, D, scale, q, kc, vc, num_blocks, table, max_blocks, seq_lens, o,
+                       lse, workspace, (cudaStream_t)stream);
+}
+
+int64_t unigist_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+const char* unigist_last_error_string(void) { return g_err; }
+
+}  // extern "C"

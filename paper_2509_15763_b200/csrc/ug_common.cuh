@@ -1,0 +1,107 @@
+// Shared declarations of the UniGist CUDA library: problem geometry in shifted coordinates,
+// error reporting and launch bookkeeping.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "unigist.h"
+
+namespace ug {
+
+// Geometry of one sequence.  Shifted order = [sinks | raw | gists] (Section 4.2).
+struct Geom {
+  int s, T, r, k, n, N;  // k is clamped to n
+};
+
+// Columns a query row may see, per segment, numbered inside the segment and inclusive
+// (Eq. 3 rewritten for the shifted order).  hi < lo means "none".
+struct RowIv {
+  int hi_sink;  // sink columns [0, hi_sink]
+  int lo_raw;   // raw columns [lo_raw, hi_raw]
+  int hi_raw;
+  int hi_gist;  // gist columns [0, hi_gist]
+};
+
+__host__ __device__ inline RowIv row_intervals(const Geom& g, int sigma) {
+  RowIv v;
+  if (sigma < g.s) {  // sink query: earlier sinks only
+    v.hi_sink = sigma;
+    v.lo_raw = 0;
+    v.hi_raw = -1;
+    v.hi_gist = -1;
+  } else if (sigma < g.s + g.T) {  // raw query i of unit u
+    const int i = sigma - g.s;
+    const int u = i / g.r;
+    const int u0 = u > g.k ? u - g.k : 0;
+    v.hi_sink = g.s - 1;
+    v.lo_raw = u0 * g.r;
+    v.hi_raw = i;
+    v.hi_gist = u - 1;
+  } else {  // gist query u: its own unit's raw tokens and itself
+    const int u = sigma - g.s - g.T;
+    const int u0 = u > g.k ? u - g.k : 0;
+    v.hi_sink = g.s - 1;
+    v.lo_raw = u0 * g.r;
+    v.hi_raw = (u + 1) * g.r - 1;
+    v.hi_gist = u;
+  }
+  return v;
+}
+
+__host__ __device__ inline bool visible(const Geom& g, const RowIv& v, int col_sigma) {
+  if (col_sigma < g.s) return col_sigma <= v.hi_sink;
+  if (col_sigma < g.s + g.T) {
+    const int j = col_sigma - g.s;
+    return j >= v.lo_raw && j <= v.hi_raw;
+  }
+  return col_sigma - g.s - g.T <= v.hi_gist;
+}
+
+// Interleaved index of the token at shifted position sigma, and the inverse.
+__host__ __device__ inline int shift_perm(const Geom& g, int sigma) {
+  if (sigma < g.s) return sigma;
+  if (sigma < g.s + g.T) {
+    const int i = sigma - g.s;
+    return g.s + i + i / g.r;
+  }
+  const int u = sigma - g.s - g.T;
+  return g.s + u * (g.r + 1) + g.r;
+}
+__host__ __device__ inline int unshift_perm(const Geom& g, int t) {
+  if (t < g.s) return t;
+  const int q = t - g.s;
+  const int u = q / (g.r + 1), p = q % (g.r + 1);
+  return p == g.r ? g.s + g.T + u : g.s + u * g.r + p;
+}
+
+// Host side helpers (api.cu).
+int32_t fail(int32_t code, const char* fmt, ...);
+int32_t check_problem(const unigist_problem* p, Geom* g, float* scale);
+int32_t check_launch(const char* what);
+void count_launch(int n = 1);
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Kernel launchers (one per .cu file).
+int32_t launch_layout(const Geom& g, int32_t* sp, int32_t* up, int32_t* pos, cudaStream_t st);
+int32_t launch_shift(const Geom& g, int B, const void* src, void* dst, size_t row_bytes,
+                     bool inverse, cudaStream_t st);
+int32_t launch_fwd_simt(const Geom& g, const unigist_problem& p, float scale, const void* q,
+                        const void* k, const void* v, void* o, float* lse, cudaStream_t st);
+int32_t launch_bwd_simt(const Geom& g, const unigist_problem& p, float scale, const void* q,
+                        const void* k, const void* v, const void* o, const float* lse,
+                        const void* d_o, void* dq, void* dk, void* dv, float* delta,
+                        cudaStream_t st);
+int32_t launch_compact_gather(const Geom& g, const unigist_problem& p, const void* k,
+                              const void* v, void* kc, void* vc, int num_blocks,
+                              const int32_t* table, int max_blocks, int32_t* seq_lens,
+                              int32_t* kept_idx, cudaStream_t st);
+int32_t launch_compact_inplace(const Geom& g, const unigist_problem& p, void* kc, void* vc,
+                               int num_blocks, int32_t* table, int max_blocks, int32_t* seq_lens,
+                               int32_t* kept_idx, void* ws, cudaStream_t st);
+int32_t launch_decode(int S, int Hq, int Hkv, int D, float scale, const void* q, const void* kc,
+                      const void* vc, int num_blocks, const int32_t* table, int max_blocks,
+                      const int32_t* seq_lens, void* o, float* lse, void* ws, cudaStream_t st);
+int decode_num_splits(int S, int Hkv, int max_blocks);
+
+}  // namespace ug

@@ -1,0 +1,68 @@
+"""Host-side checks of the C ABI: the library loads, exports every declared symbol, and rejects
+malformed arguments without launching anything (no GPU needed)."""
+import ctypes
+import re
+from pathlib import Path
+
+import pytest
+
+import paper_2509_15763_b200 as ug
+from paper_2509_15763_b200 import binding, build
+from oracle import oracle
+
+ROOT = Path(__file__).resolve().parent.parent
+
+
+@pytest.fixture(scope="module", autouse=True)
+def built():
+    build.build()
+
+
+def test_every_declared_symbol_is_exported():
+    header = (ROOT / "include" / "unigist.h").read_text()
+    declared = set(re.findall(r"\b(unigist_[a-z_0-9]+)\s*\(", header))
+    assert declared, "no declarations found"
+    lib = ctypes.CDLL(str(binding.LIB_PATH))
+    for name in declared:
+        assert hasattr(lib, name), name
+    assert declared == set(binding.SYMBOLS)
+
+
+@pytest.mark.parametrize("s,T,r,W", [(0, 448, 7, 64), (5, 64, 4, 12), (3, 48, 8, 80), (0, 56, 7, 14)])
+def test_host_geometry_matches_oracle(s, T, r, W):
+    p = ug.Problem(1, T, r, W, 1, 1, 64, num_sinks=s)
+    k = oracle.window_units(W, r)
+    assert ug.unigist_total_len(p) == oracle.total_len(s, T, r)
+    assert ug.unigist_window_units(p) == k
+    assert ug.unigist_visible_pairs(p) == oracle.count_pairs(s, T, r, k)
+    assert ug.unigist_compact_len(p) == len(oracle.kept_set(s, T, r, k))
+
+
+def test_malformed_problems_are_rejected():
+    bad = [ug.Problem(1, 10, 3, 4, 1, 1, 64), ug.Problem(1, 16, 4, 4, 3, 2, 64),
+           ug.Problem(1, 16, 4, 4, 1, 1, 96), ug.Problem(0, 16, 4, 4, 1, 1, 64),
+           ug.Problem(1, 16, 4, -1, 1, 1, 64)]
+    for p in bad:
+        assert ug.unigist_total_len(p) < 0
+        assert ug.unigist_last_error_string()
+        assert ug.unigist_workspace_bytes(p, ug.OP_BWD) == 0
+
+
+def test_null_and_misaligned_pointers_are_rejected_before_any_launch():
+    lib = binding.lib()
+    p = ug.Problem(1, 16, 4, 4, 1, 1, 64).c()
+    before = ug.unigist_launch_count()
+    rc = lib.unigist_attn_fwd(ctypes.byref(p), None, None, None, None, None, None, 0, None)
+    assert rc == 1
+    buf = ctypes.create_string_buffer(4096)
+    a = ctypes.addressof(buf)
+    a += (-a) % 16
+    rc = lib.unigist_gist_shift(ctypes.byref(p), a + 2, a + 1024, 1, 2, None)
+    assert rc == 3
+    rc = lib.unigist_gist_shift(ctypes.byref(p), a, a + 16, 1, 2, None)  # overlap
+    assert rc == 1
+    rc = lib.unigist_attn_bwd(ctypes.byref(p), *([a] * 9), a, 0, None)  # workspace too small
+    assert rc == 4
+    rc = lib.unigist_decode(1, 6, 4, 128, 0.0, a, a, a, 1, a, 1, a, a, None, a, 1 << 20, None)
+    assert rc == 2
+    assert ug.unigist_launch_count() == before

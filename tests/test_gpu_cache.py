@@ -1,0 +1,161 @@
+"""GPU parity for KV compaction (bit-exact) and decode over the paged compressed cache."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2509_15763_b200 as ug
+from paper_2509_15763_b200 import synth
+from oracle import oracle
+
+from gpu_util import TOL_LSE, TOL_O_MAX, TOL_O_MEAN, check_close, f64
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+PG = ug.PAGE_TOKENS
+
+
+def read_cache(cache, table_row, length):
+    """Logical view [length, Hkv, D] of a paged cache."""
+    blocks = cache[table_row[: -(-length // PG)].long()]           # [nb, Hkv, PG, D]
+    return blocks.permute(0, 2, 1, 3).reshape(-1, cache.shape[1], cache.shape[3])[:length]
+
+
+COMPACT_CASES = [
+    # B, s, T, r, W, Hkv, D
+    (2, 0, 448, 7, 64, 1, 64),
+    (1, 5, 330, 5, 48, 2, 128),
+    (1, 64, 1024, 8, 512, 2, 128),     # page aligned: in place is a table edit
+    (2, 0, 2048, 16, 4096, 2, 128),    # window covers everything
+    (1, 3, 640, 4, 0, 1, 64),          # no window
+]
+
+
+@pytest.mark.parametrize("B,s,T,r,W,Hkv,D", COMPACT_CASES)
+@pytest.mark.parametrize("mode", ["gather", "inplace"])
+def test_compaction_matches_oracle(B, s, T, r, W, Hkv, D, mode):
+    p = ug.Problem(B, T, r, W, Hkv, Hkv, D, num_sinks=s)
+    N, L = ug.unigist_total_len(p), ug.unigist_compact_len(p)
+    k_units = oracle.window_units(W, r)
+    kept = oracle.kept_set(s, T, r, k_units)              # interleaved indices, cache order
+    sp, up, _ = oracle.layout(s, T, r)
+    assert len(kept) == L
+    g = torch.Generator().manual_seed(11)
+    k_sh = torch.randn(B, N, Hkv, D, generator=g).to(torch.bfloat16)  # shifted order
+    v_sh = torch.randn(B, N, Hkv, D, generator=g).to(torch.bfloat16)
+    nbN, nbL = -(-N // PG), -(-L // PG)
+    per_seq = nbN if mode == "inplace" else nbL
+    nblocks = B * per_seq + 3
+    table = torch.randperm(nblocks, generator=g)[: B * per_seq].to(torch.int32).reshape(B, per_seq)
+    kc = torch.randn(nblocks, Hkv, PG, D, generator=g).to(torch.bfloat16)
+    vc = torch.randn(nblocks, Hkv, PG, D, generator=g).to(torch.bfloat16)
+    if mode == "inplace":  # the cache holds the whole shifted sequence
+        for b in range(B):
+            pad = torch.zeros(nbN * PG - N, Hkv, D, dtype=torch.bfloat16)
+            for src, dst in ((k_sh, kc), (v_sh, vc)):
+                full = torch.cat([src[b], pad]).reshape(nbN, PG, Hkv, D).permute(0, 2, 1, 3)
+                dst[table[b].long()] = full
+    kc_d, vc_d, table_d = kc.to(DEV), vc.to(DEV), table.to(DEV)
+    lens = torch.zeros(B, dtype=torch.int32, device=DEV)
+    kept_idx = torch.full((B, L), -1, dtype=torch.int32, device=DEV)
+    ws = torch.empty(max(ug.unigist_workspace_bytes(p, ug.OP_COMPACT), 16), dtype=torch.uint8, device=DEV)
+    if mode == "gather":
+        ug.unigist_kv_compact(p, k_sh.to(DEV), v_sh.to(DEV), kc_d, vc_d, table_d, lens, kept_idx, ws)
+    else:
+        ug.unigist_kv_compact(p, None, None, kc_d, vc_d, table_d, lens, kept_idx, ws)
+    torch.cuda.synchronize()
+    assert lens.cpu().tolist() == [L] * B
+    # indices: bit-exact against the oracle's kept set (mapped into shifted positions)
+    want_idx = up[kept]
+    assert np.array_equal(kept_idx.cpu().numpy(), np.tile(want_idx, (B, 1)))
+    new_table = table_d.cpu()
+    for b in range(B):
+        assert sorted(new_table[b].tolist()) == sorted(table[b].tolist())  # a permutation of the row
+        for cache, src in ((kc_d, k_sh), (vc_d, v_sh)):
+            got = read_cache(cache.cpu(), new_table[b], L)
+            assert torch.equal(got, src[b, torch.from_numpy(want_idx).long()])
+    if mode == "gather":  # blocks outside the tables are untouched
+        spare = sorted(set(range(nblocks)) - set(table.flatten().tolist()))
+        assert torch.equal(kc_d.cpu()[spare], kc[spare])
+
+
+def run_decode(inp, lens=None):
+    d = {k: v.to(DEV) for k, v in inp.items()}
+    if lens is not None:
+        d["seq_lens"] = torch.tensor(lens, dtype=torch.int32, device=DEV)
+    S, Hq, D = d["q"].shape
+    Hkv = d["k_cache"].shape[1]
+    ws = torch.empty(ug.unigist_decode_workspace_bytes(S, Hq, Hkv, D, d["block_table"].shape[1]),
+                     dtype=torch.uint8, device=DEV)
+    o = torch.full_like(d["q"], float("nan"))
+    lse = torch.full((S, Hq), float("nan"), dtype=torch.float32, device=DEV)
+    ug.unigist_decode(d["q"], d["k_cache"], d["v_cache"], d["block_table"], d["seq_lens"], o, lse, ws)
+    torch.cuda.synchronize()
+    return o, lse, d["seq_lens"].cpu().tolist()
+
+
+def check_decode(inp, o, lse, lens, seqs):
+    Hq, D = inp["q"].shape[1:]
+    for i in seqs:
+        kl = read_cache(inp["k_cache"], inp["block_table"][i], lens[i])
+        vl = read_cache(inp["v_cache"], inp["block_table"][i], lens[i])
+        oo, ll = oracle.decode(D ** -0.5, f64(inp["q"][i:i + 1]), [f64(kl)], [f64(vl)])
+        check_close(f"decode O seq {i}", f64(o[i:i + 1]), oo, TOL_O_MAX, TOL_O_MEAN)
+        check_close(f"decode LSE seq {i}", f64(lse[i:i + 1]), ll, TOL_LSE)
+
+
+@pytest.mark.parametrize("S,Hq,Hkv,gists,window", [(3, 8, 2, 100, 37), (2, 4, 4, 1, 0), (5, 32, 8, 600, 128),
+                                                   (1, 8, 1, 64, 64), (2, 2, 1, 700, 1)])
+def test_decode_matches_oracle(S, Hq, Hkv, gists, window):
+    w = synth.DecodeWorkload("t", S, gists, window, Hq, Hkv, 128, seed=300 + S)
+    inp = synth.decode_inputs(w, spare_blocks=2)
+    inp["k_cache"][inp["block_table"][0, -1].long(), :, (w.seq_len - 1) % PG + 1:] = float("nan")  # unused slots
+    lens = [max(1, w.seq_len - 13 * i) for i in range(S)]  # ragged lengths
+    o, lse, lens = run_decode(inp, lens)
+    check_decode(inp, o, lse, lens, range(S))
+
+
+def test_decode_full_size_sampled():
+    w = synth.DECODE_WORKLOADS["decode_cache"]
+    inp = synth.decode_inputs(w)
+    o, lse, lens = run_decode(inp)
+    assert torch.isfinite(o.float()).all() and torch.isfinite(lse).all()
+    check_decode(inp, o, lse, lens, [0, 21, 42, 63])
+
+
+def test_compact_then_decode_equals_forward_row():
+    """Sections 4.1 and 4.3 jointly, on the GPU path: the query of the next token over the
+    compacted cache (plus its own K/V) reproduces its row of the uncompacted forward."""
+    s, T, r, W, Hq, Hkv, D = 0, 512, 8, 128, 8, 2, 128
+    w = synth.Workload("ext", 1, T + r, r, W, Hq, Hkv, D, seed=400)
+    inp = synth.attention_inputs(w, with_grad=False)
+    k_units = oracle.window_units(W, r)
+    N = oracle.total_len(s, T, r)
+    # prefix of T raw tokens, in shifted order
+    sp, _, _ = oracle.layout(s, T, r)
+    p = ug.Problem(1, T, r, W, Hq, Hkv, D)
+    L = ug.unigist_compact_len(p)
+    k_sh = inp["k"][:, torch.from_numpy(sp).long()].contiguous().to(DEV)
+    v_sh = inp["v"][:, torch.from_numpy(sp).long()].contiguous().to(DEV)
+    nb = -(-(L + 1) // PG)
+    kc = torch.zeros(nb + 1, Hkv, PG, D, dtype=torch.bfloat16, device=DEV)
+    vc = torch.zeros_like(kc)
+    table = torch.arange(nb, dtype=torch.int32, device=DEV).flip(0).reshape(1, nb).contiguous()
+    lens = torch.zeros(1, dtype=torch.int32, device=DEV)
+    ug.unigist_kv_compact(p, k_sh, v_sh, kc, vc, table, lens)
+    # append the next token (interleaved index N of the extended sequence)
+    blk, slot = table[0, L // PG].item(), L % PG
+    kc[blk, :, slot] = inp["k"][0, N].to(DEV)
+    vc[blk, :, slot] = inp["v"][0, N].to(DEV)
+    lens += 1
+    q = inp["q"][:, N].contiguous().to(DEV)
+    ws = torch.empty(ug.unigist_decode_workspace_bytes(1, Hq, Hkv, D, nb), dtype=torch.uint8, device=DEV)
+    o = torch.empty_like(q)
+    lse = torch.empty(1, Hq, dtype=torch.float32, device=DEV)
+    ug.unigist_decode(q, kc, vc, table, lens, o, lse, ws)
+    torch.cuda.synchronize()
+    G = Hq // Hkv
+    for hk in range(Hkv):
+        oo, ll = oracle.attn_fwd_slice(s, T + r, r, k_units, D ** -0.5, f64(inp["q"][0, :, hk * G:(hk + 1) * G]),
+                                       f64(inp["k"][0, :, hk]), f64(inp["v"][0, :, hk]), N, N + 1)
+        check_close("O", f64(o[0, hk * G:(hk + 1) * G]), oo[0], TOL_O_MAX, TOL_O_MEAN)
+        check_close("LSE", f64(lse[0, hk * G:(hk + 1) * G]), ll[0], TOL_LSE)

@@ -1,0 +1,133 @@
+"""GPU parity: the CUDA path (through the C ABI) against the fp64 oracle on the same seeded inputs."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2509_15763_b200 as ug
+from paper_2509_15763_b200 import synth
+from oracle import oracle
+
+from gpu_util import (TOL_GRAD, TOL_LSE, TOL_O_MAX, TOL_O_MEAN, check_close, f64, problem_of,
+                      run_attention)
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+# ------------------------------------------------------------------ layout and shift (bit-exact)
+@pytest.mark.parametrize("s,T,r", [(0, 448, 7), (5, 64, 4), (128, 4096, 8), (0, 16, 16), (3, 9, 1),
+                                   (0, 131072, 16)])
+def test_layout_device_matches_oracle(s, T, r):
+    p = ug.Problem(1, T, r, 64, 1, 1, 64, num_sinks=s)
+    N = ug.unigist_total_len(p)
+    sp, up, pos = (torch.full((N,), -1, dtype=torch.int32, device=DEV) for _ in range(3))
+    ug.unigist_layout(p, sp, up, pos)
+    a, b, c = oracle.layout(s, T, r)
+    assert np.array_equal(sp.cpu().numpy(), a)
+    assert np.array_equal(up.cpu().numpy(), b)
+    assert np.array_equal(pos.cpu().numpy(), c)
+    hs, hu, hp = (torch.empty(N, dtype=torch.int32) for _ in range(3))
+    ug.unigist_layout(p, hs, hu, hp)  # host variant
+    assert np.array_equal(hs.numpy(), a) and np.array_equal(hu.numpy(), b) and np.array_equal(hp.numpy(), c)
+
+
+@pytest.mark.parametrize("B,s,T,r,H,D,dtype", [(2, 0, 448, 7, 1, 64, torch.bfloat16),
+                                               (1, 5, 640, 4, 8, 128, torch.bfloat16),
+                                               (3, 2, 90, 9, 3, 64, torch.float32),
+                                               (1, 0, 16384, 8, 32, 128, torch.bfloat16)])
+def test_shift_unshift_bit_exact(B, s, T, r, H, D, dtype):
+    p = ug.Problem(B, T, r, 64, H, H, D, num_sinks=s)
+    N = ug.unigist_total_len(p)
+    g = torch.Generator().manual_seed(7)
+    x = torch.randn(B, N, H, D, generator=g).to(dtype)
+    sp, up, _ = oracle.layout(s, T, r)
+    xd = x.to(DEV)
+    y = torch.full_like(xd, float("nan"))
+    ug.unigist_gist_shift(p, xd, y)
+    assert torch.equal(y.cpu(), x[:, torch.from_numpy(sp).long()])
+    z = torch.full_like(xd, float("nan"))
+    ug.unigist_gist_unshift(p, y, z)
+    assert torch.equal(z.cpu(), x)
+
+
+# ------------------------------------------------------------------ forward + backward, whole problem
+SMALL = [
+    synth.WORKLOADS["tiny"],
+    synth.Workload("sinks_ragged", 2, 330, 5, 48, 4, 2, 64, num_sinks=7, seed=101),
+    synth.Workload("gqa_128", 1, 1536, 4, 256, 8, 2, 128, seed=102),
+    synth.Workload("full_window", 1, 384, 8, 4096, 2, 2, 128, seed=103),
+    synth.Workload("ratio_one", 1, 200, 1, 16, 2, 1, 64, seed=104),
+    synth.Workload("no_window", 1, 512, 16, 0, 2, 1, 128, num_sinks=3, seed=105),
+    synth.Workload("one_unit", 1, 12, 12, 12, 1, 1, 64, seed=106),
+    synth.Workload("odd_tiles", 1, 1000, 8, 200, 4, 4, 128, num_sinks=1, k_scale=0.5, seed=107),
+]
+
+
+@pytest.mark.parametrize("w", SMALL, ids=lambda w: w.name)
+def test_attention_matches_oracle(w):
+    fp32_dout = w.name == "tiny"  # the tiny workload states an fp32 dO
+    out = run_attention(w, backward=True, dout_fp32=fp32_dout)
+    inp = out["inputs"]
+    k = oracle.window_units(w.window, w.ratio)
+    scale = w.head_dim ** -0.5
+    q, kk, v, do = (f64(inp[n]) for n in ("q", "k", "v", "dout"))
+    o, lse = oracle.attn_fwd(w.num_sinks, w.raw_len, w.ratio, k, scale, q, kk, v)
+    check_close("O", f64(out["o"]), o, TOL_O_MAX, TOL_O_MEAN)
+    check_close("LSE", f64(out["lse"]), lse, TOL_LSE)
+    dq, dk, dv = oracle.attn_bwd(w.num_sinks, w.raw_len, w.ratio, k, scale, q, kk, v, do)
+    check_close("dQ", f64(out["dq"]), dq, TOL_GRAD)
+    check_close("dK", f64(out["dk"]), dk, TOL_GRAD)
+    check_close("dV", f64(out["dv"]), dv, TOL_GRAD)
+
+
+def test_forward_is_deterministic():
+    w = SMALL[2]
+    a = run_attention(w, backward=True)
+    b = run_attention(w, backward=True)
+    for n in ("o", "lse", "dq", "dk", "dv"):
+        assert torch.equal(a[n], b[n]), n
+
+
+# ------------------------------------------------------------------ full-size workloads, sampled outputs
+def _sample_rows(N, rng, blocks=6, width=16):
+    starts = [0, N - width] + list(rng.integers(0, N - width, size=blocks))
+    rows = sorted({int(s0) + i for s0 in starts for i in range(width)})
+    return np.array(rows, dtype=np.int64)
+
+
+@pytest.mark.parametrize("name,backward", [("llama8b_layer", True), ("train_batch", True),
+                                           ("long_prefill", False)])
+def test_full_size_sampled(name, backward):
+    w = synth.WORKLOADS[name]
+    out = run_attention(w, backward=backward)
+    inp = out["inputs"]
+    s, T, r = w.num_sinks, w.raw_len, w.ratio
+    k = oracle.window_units(w.window, r)
+    N, G = w.total_len, w.num_q_heads // w.num_kv_heads
+    scale = w.head_dim ** -0.5
+    rng = np.random.default_rng(w.seed)
+    b, hk = w.batch - 1, int(rng.integers(0, w.num_kv_heads))
+    hs = slice(hk * G, (hk + 1) * G)
+    q, kk, v = f64(inp["q"][b, :, hs]), f64(inp["k"][b, :, hk]), f64(inp["v"][b, :, hk])
+    # forward: blocks of rows, among them the first units, the window edge and the tail
+    o_gpu, lse_gpu = f64(out["o"][b, :, hs]), f64(out["lse"][b, hs])
+    for r0 in [0, (k + 1) * (r + 1) - 8, N // 2 + 3, N - 16]:
+        o, lse = oracle.attn_fwd_slice(s, T, r, k, scale, q, kk, v, r0, r0 + 16)
+        check_close(f"O rows {r0}", o_gpu[r0:r0 + 16], o, TOL_O_MAX, TOL_O_MEAN)
+        check_close(f"LSE rows {r0}", lse_gpu[:, r0:r0 + 16].T, lse, TOL_LSE)
+    # no row anywhere was left unwritten
+    assert torch.isfinite(out["lse_shifted"]).all()
+    assert torch.isfinite(out["o_shifted"].float()).all()
+    if not backward:
+        return
+    do = f64(inp["dout"][b, :, hs])
+    rows = np.concatenate([np.arange(0, 8), np.arange(N // 3, N // 3 + 8), np.arange(N - 8, N)])
+    last_gist = N - 1
+    keys = np.array([0, 1, r, (r + 1) * 5 + 2, N // 2, N // 2 + 1, N - 2 - (r + 1) * 3,
+                     last_gist - 40 * (r + 1), last_gist, N - 2], dtype=np.int64)
+    dq, dk, dv = oracle.attn_bwd_sample(s, T, r, k, scale, q, kk, v, do, rows, keys)
+    check_close("dQ rows", f64(out["dq"][b, rows][:, hs]), dq, TOL_GRAD)
+    check_close("dK keys", f64(out["dk"][b, keys, hk]), dk, TOL_GRAD)
+    check_close("dV keys", f64(out["dv"][b, keys, hk]), dv, TOL_GRAD)
+    for n in ("dq_shifted", "dk_shifted", "dv_shifted"):
+        assert torch.isfinite(out[n].float()).all(), n

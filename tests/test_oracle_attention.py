@@ -185,3 +185,13 @@ def test_decode_matches_library_softmax():
     sc = 0.2 * torch.from_numpy(qd) @ torch.from_numpy(kc).T
     assert np.allclose(o, (torch.softmax(sc, -1) @ torch.from_numpy(vc)).numpy(), atol=1e-13, rtol=0)
     assert np.allclose(lse, torch.logsumexp(sc, -1).numpy(), atol=1e-13, rtol=0)
+
+
+def test_sampled_backward_equals_full_backward():
+    s, T, r, k = 1, 32, 4, 2
+    N, G, D, scale = oracle.total_len(s, T, r), 2, 8, 0.45
+    q, kk, v, dout = rnd((N, G, D), 40), rnd((N, D), 41), rnd((N, D), 42), rnd((N, G, D), 43)
+    dq, dk, dv = oracle.attn_bwd_slice(s, T, r, k, scale, q, kk, v, dout)
+    rows, keys = [0, 7, 19, N - 1], [2, 9, 10, N - 2]
+    dq_s, dk_s, dv_s = oracle.attn_bwd_sample(s, T, r, k, scale, q, kk, v, dout, rows, keys)
+    assert np.array_equal(dq_s, dq[rows]) and np.array_equal(dk_s, dk[keys]) and np.array_equal(dv_s, dv[keys])
