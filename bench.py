@@ -1,0 +1,397 @@
+#!/usr/bin/env python
+"""Benchmark of the UniGist attention hot path on B200.
+
+One step = one pass of the whole path over one synthetic batch, in the order a training /
+prefill step runs it: gist shift of Q, K, V, dO -> forward (O, LSE) -> backward (dQ, dK, dV) ->
+unshift of O, dQ, dK, dV -> KV compaction into the paged cache -> one decode query per sequence
+over the compacted cache.  The headline value is the effective TFLOP/s of forward + backward
+counting only unmasked (visible) pairs: 14 * D * pairs * Hq * B FLOP per step / step time.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+
+With N > 1 (launched by torchrun) every rank runs an independent replica of the workload (the
+path has no exchange step); the value is the work of all ranks over the slowest rank's time.
+`--impl reference` times the fp64 CPU oracle on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+from pathlib import Path
+
+ROOT = Path(__file__).resolve().parent
+if str(ROOT) not in sys.path:
+    sys.path.insert(0, str(ROOT))
+
+METRIC = "effective_tflops_fwd_bwd_unmasked"
+UNIT = "TFLOP/s"
+
+# DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures
+# summarised under profiles/, keyed by (kernel, workload); None until a capture exists.
+NCU_TRAFFIC_BYTES = {}
+
+# FLOP per visible pair per query head that each attention kernel performs algorithmically,
+# in units of head_dim (a QK^T- or PV-shaped product is 2 * D FLOP per pair).
+KERNEL_FLOP_PER_PAIR_D = {
+    "fwd_simt_kernel": 4, "bwd_dq_simt_kernel": 6, "bwd_dkdv_simt_kernel": 8,
+    "attn_fwd_sm100_kernel": 4, "attn_bwd_dq_sm100_kernel": 6, "attn_bwd_dkdv_sm100_kernel": 8,
+}
+CUDA_CORE_KERNELS = {"fwd_simt_kernel", "bwd_dq_simt_kernel", "bwd_dkdv_simt_kernel"}
+
+
+def measured_peaks():
+    f = ROOT / "MEASURED_PEAKS.json"
+    if f.exists():
+        d = json.loads(f.read_text())
+        return {"hbm_gbs": d["hbm_gbs"], "bf16_tflops": d["bf16_tflops"],
+                "bf16_tflops_sustained": d.get("bf16_tflops_sustained", d["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.samples, self.proc = index, [], None
+
+    def __enter__(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+        return self
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.samples.append([x.strip() for x in line.split(",")])
+
+    def __exit__(self, *a):
+        if self.proc:
+            time.sleep(0.15)
+            self.proc.terminate()
+            self.thread.join(timeout=2)
+
+    def summary(self):
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for s in self.samples:
+            try:
+                sm.append(float(s[0]))
+                mx.append(float(s[1]))
+            except (ValueError, IndexError):
+                continue
+            for n, v in zip(names, s[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+def oracle_sample(w, seconds_hint: float = 20.0):
+    """Time the oracle (as it stands) on a bounded sample of workload `w`: forward + backward of
+    one KV group (G query heads) over the first T_s raw tokens.  -> (tflops, cores, description, s)."""
+    import numpy as np
+
+    from oracle import oracle
+    from paper_2509_15763_b200 import synth
+
+    T_s = min(w.raw_len, 8192 // w.ratio * w.ratio)
+    G = w.num_q_heads // w.num_kv_heads
+    ws = synth.Workload(w.name + "_sample", 1, T_s, w.ratio, w.window, G, 1, w.head_dim,
+                        num_sinks=w.num_sinks, k_scale=w.k_scale, seed=w.seed)
+    inp = synth.attention_inputs(ws)
+    f = lambda t: t.to(dtype=__import__("torch").float64).numpy()
+    q, k, v, do = f(inp["q"][0]), f(inp["k"][0, :, 0]), f(inp["v"][0, :, 0]), f(inp["dout"][0])
+    ku = oracle.window_units(w.window, w.ratio)
+    scale = w.head_dim ** -0.5
+    t0 = time.perf_counter()
+    oracle.attn_fwd_slice(ws.num_sinks, T_s, w.ratio, ku, scale, q, k, v)
+    oracle.attn_bwd_slice(ws.num_sinks, T_s, w.ratio, ku, scale, q, k, v, do)
+    dt = time.perf_counter() - t0
+    pairs = oracle.count_pairs(ws.num_sinks, T_s, w.ratio, ku)
+    flops = 14.0 * w.head_dim * pairs * G
+    desc = (f"oracle fwd+bwd of one KV group ({G} query heads) over the first {T_s} raw tokens "
+            f"(N={ws.total_len}) of {w.name}, {pairs} visible pairs per head")
+    return flops / dt / 1e12, oracle.num_threads(), desc, dt
+
+
+def run_reference(args, w):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    vals = []
+    for _ in range(args.warmup):
+        oracle_sample(w)
+    t_tot = 0.0
+    for _ in range(args.steps):
+        tf, cores, desc, dt = oracle_sample(w)
+        vals.append(tf)
+        t_tot += dt
+    value = statistics.mean(vals)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * t_tot / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic", "config": {"workload": w.name, "note": "each step is a bounded sample: " + desc},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+class Path_:
+    """Device buffers of one workload and the step that runs the whole path on them."""
+
+    def __init__(self, w, dev):
+        import torch
+
+        import paper_2509_15763_b200 as ug
+        from paper_2509_15763_b200 import synth
+
+        self.ug, self.torch, self.w, self.dev = ug, torch, w, dev
+        self.p = ug.Problem(w.batch, w.raw_len, w.ratio, w.window, w.num_q_heads, w.num_kv_heads, w.head_dim,
+                            num_sinks=w.num_sinks)
+        p = self.p
+        self.N = ug.unigist_total_len(p)
+        self.pairs = ug.unigist_visible_pairs(p)
+        host = synth.attention_inputs(w)
+        self.host_in = {k: v.pin_memory() for k, v in host.items()}
+        self.inter = {k: v.to(dev) for k, v in host.items()}                      # interleaved inputs
+        self.sh = {k: torch.empty_like(v) for k, v in self.inter.items()}         # shifted inputs
+        self.o_s = torch.empty_like(self.sh["q"])
+        self.lse = torch.empty(w.batch, w.num_q_heads, self.N, dtype=torch.float32, device=dev)
+        self.dq_s, self.dk_s, self.dv_s = (torch.empty_like(self.sh[n]) for n in ("q", "k", "v"))
+        self.out = {"o": torch.empty_like(self.o_s), "dq": torch.empty_like(self.dq_s),
+                    "dk": torch.empty_like(self.dk_s), "dv": torch.empty_like(self.dv_s)}
+        self.host_out = {k: torch.empty(v.shape, dtype=v.dtype).pin_memory() for k, v in self.out.items()}
+        self.ws = torch.empty(max(16, ug.unigist_workspace_bytes(p, ug.OP_BWD)), dtype=torch.uint8, device=dev)
+        L = ug.unigist_compact_len(p)
+        self.nb = -(-(L + 1) // ug.PAGE_TOKENS)
+        nblocks = w.batch * self.nb
+        self.kc = torch.zeros(nblocks, w.num_kv_heads, ug.PAGE_TOKENS, w.head_dim, dtype=torch.bfloat16, device=dev)
+        self.vc = torch.zeros_like(self.kc)
+        g = torch.Generator().manual_seed(w.seed)
+        self.table = torch.randperm(nblocks, generator=g).to(torch.int32).reshape(w.batch, self.nb).to(dev)
+        self.lens = torch.zeros(w.batch, dtype=torch.int32, device=dev)
+        self.qd = torch.empty(w.batch, w.num_q_heads, w.head_dim, dtype=torch.bfloat16, device=dev)
+        self.od = torch.empty_like(self.qd)
+        self.host_od = torch.empty(self.od.shape, dtype=self.od.dtype).pin_memory()
+        self.wsd = torch.empty(ug.unigist_decode_workspace_bytes(w.batch, w.num_q_heads, w.num_kv_heads,
+                                                                 w.head_dim, self.nb), dtype=torch.uint8, device=dev)
+        self.flops = 14.0 * w.head_dim * self.pairs * w.num_q_heads * w.batch
+
+    def step(self):
+        ug, p = self.ug, self.p
+        for n in ("q", "k", "v", "dout"):
+            ug.unigist_gist_shift(p, self.inter[n], self.sh[n])
+        ug.unigist_attn_fwd(p, self.sh["q"], self.sh["k"], self.sh["v"], self.o_s, self.lse)
+        ug.unigist_attn_bwd(p, self.sh["q"], self.sh["k"], self.sh["v"], self.o_s, self.lse, self.sh["dout"],
+                            self.dq_s, self.dk_s, self.dv_s, self.ws)
+        for n, t in (("o", self.o_s), ("dq", self.dq_s), ("dk", self.dk_s), ("dv", self.dv_s)):
+            ug.unigist_gist_unshift(p, t, self.out[n])
+        ug.unigist_kv_compact(p, self.sh["k"], self.sh["v"], self.kc, self.vc, self.table, self.lens)
+        self.qd.copy_(self.sh["q"][:, -1])
+        ug.unigist_decode(self.qd, self.kc, self.vc, self.table, self.lens, self.od, None, self.wsd)
+
+    def e2e_step(self):
+        for n in ("q", "k", "v", "dout"):
+            self.inter[n].copy_(self.host_in[n], non_blocking=True)
+        self.step()
+        for n in self.out:
+            self.host_out[n].copy_(self.out[n], non_blocking=True)
+        self.host_od.copy_(self.od, non_blocking=True)
+
+    def h2d_bytes(self):
+        return sum(t.numel() * t.element_size() for t in self.host_in.values())
+
+    def d2h_bytes(self):
+        return sum(t.numel() * t.element_size() for t in self.host_out.values()) + \
+            self.host_od.numel() * self.host_od.element_size()
+
+
+def bench_decode(dev, iters=20):
+    """Decode over the compressed-cache workload (64 sequences x 9216 cached tokens): GB/s of K+V."""
+    import torch
+
+    import paper_2509_15763_b200 as ug
+    from paper_2509_15763_b200 import synth
+
+    w = synth.DECODE_WORKLOADS["decode_cache"]
+    d = {k: v.to(dev) for k, v in synth.decode_inputs(w).items()}
+    ws = torch.empty(ug.unigist_decode_workspace_bytes(w.num_seqs, w.num_q_heads, w.num_kv_heads, w.head_dim,
+                                                       d["block_table"].shape[1]), dtype=torch.uint8, device=dev)
+    o = torch.empty_like(d["q"])
+    run = lambda: ug.unigist_decode(d["q"], d["k_cache"], d["v_cache"], d["block_table"], d["seq_lens"], o, None, ws)
+    for _ in range(3):
+        run()
+    torch.cuda.synchronize()
+    ug.unigist_kernel_timing(True)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(iters):
+        run()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / iters
+    split_ms = [ug.unigist_kernel_timing_get(i)[1] for i in range(ug.unigist_kernel_timing_count())
+                if ug.unigist_kernel_timing_get(i)[0] == "decode_split_kernel"]
+    ug.unigist_kernel_timing(False)
+    nbytes = w.num_seqs * w.seq_len * w.num_kv_heads * w.head_dim * 2 * 2
+    return {"workload": w.name, "kv_bytes": nbytes, "us_per_call": 1e3 * ms, "gbs": nbytes / (ms * 1e-3) / 1e9,
+            "split_kernel_us": 1e3 * statistics.mean(split_ms), "split_kernel_gbs": nbytes / (statistics.mean(split_ms) * 1e-3) / 1e9,
+            "l2_policy": "K+V (2.4 GB) exceed L2, every call streams from HBM"}
+
+
+def run_ours(args, w):
+    import torch
+
+    import paper_2509_15763_b200 as ug
+
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the path has no CPU fallback")
+    ug.binding.lib()
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_
+
+        dist = dist_
+        dist.init_process_group("nccl", device_id=dev)
+
+    def barrier():
+        if dist:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    path = Path_(w, dev)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)  # > 126 MB L2
+    for _ in range(max(args.warmup, 3)):
+        path.step()
+    barrier()
+
+    # ---- device-resident timing
+    ug.unigist_kernel_timing(True)
+    launches0 = ug.unigist_launch_count()
+    evs = []
+    barrier()
+    with ClockSampler(local) as clocks:
+        for _ in range(args.steps):
+            flush.fill_(1)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            path.step()
+            e1.record()
+            evs.append((e0, e1))
+        barrier()
+    launches = ug.unigist_launch_count() - launches0
+    step_ms = [a.elapsed_time(b) for a, b in evs]
+    total_ms = sum(step_ms)
+    per_kernel = {}
+    for i in range(ug.unigist_kernel_timing_count()):
+        name, ms = ug.unigist_kernel_timing_get(i)
+        cnt, tot = per_kernel.get(name, (0, 0.0))
+        per_kernel[name] = (cnt + 1, tot + ms)
+    ug.unigist_kernel_timing(False)
+
+    # ---- end to end: host buffers in, host buffers out
+    for _ in range(2):
+        path.e2e_step()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        path.e2e_step()
+    e1.record()
+    barrier()
+    e2e_ms = e0.elapsed_time(e1)
+
+    t = torch.tensor([total_ms, e2e_ms], dtype=torch.float64, device=dev)
+    if dist:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    total_ms, e2e_ms = t.tolist()
+    if rank != 0:
+        if dist:
+            dist.destroy_process_group()
+        return
+
+    peaks = measured_peaks()
+    value = world * path.flops * args.steps / (total_ms * 1e-3) / 1e12
+    e2e_value = world * path.flops * args.steps / (e2e_ms * 1e-3) / 1e12
+    attn = {k: v for k, v in per_kernel.items() if k in KERNEL_FLOP_PER_PAIR_D}
+    top = max(attn, key=lambda k: attn[k][1])
+    cnt, tot = attn[top]
+    top_flops = KERNEL_FLOP_PER_PAIR_D[top] * w.head_dim * path.pairs * w.num_q_heads * w.batch
+    achieved = top_flops / (tot / cnt * 1e-3) / 1e12
+    if top in CUDA_CORE_KERNELS:
+        # fp32 FMA pipe: 148 SMs x 128 lanes x 2 FLOP x 1.965 GHz
+        bound, peak, peak_src = "alu", 148 * 128 * 2 * 1.965e9 / 1e12, "derived from unit counts and max clock"
+    else:
+        bound, peak, peak_src = "tensor", peaks["bf16_tflops_sustained"], peaks["source"] + " sustained bf16"
+    kernel_share = {k: {"launches": c, "ms": round(m, 4), "share": round(m / sum(x[1] for x in per_kernel.values()), 4)}
+                    for k, (c, m) in sorted(per_kernel.items(), key=lambda kv: -kv[1][1])}
+    decode = bench_decode(dev)
+    cpu_tf, cores, desc, _ = oracle_sample(w)
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+        "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": w.name, "batch": w.batch, "raw_len": w.raw_len, "ratio": w.ratio, "window": w.window,
+                   "q_heads": w.num_q_heads, "kv_heads": w.num_kv_heads, "head_dim": w.head_dim,
+                   "total_len": path.N, "visible_pairs_per_head": path.pairs, "flop_per_step": path.flops,
+                   "l2": "256 MB buffer written between timed steps", "parallelism": f"replicas x{world}"},
+        "roofline": {"kernel": top, "bound": bound, "achieved": achieved, "peak": peak, "unit": UNIT,
+                     "frac": achieved / peak, "peak_source": peak_src,
+                     "traffic": NCU_TRAFFIC_BYTES.get((top, w.name))},
+        "pct_of_nominal_bf16_peak": 100.0 * value / world / 2250.0,
+        "kernels": kernel_share,
+        "decode": dict(decode, frac_of_measured_hbm=decode["split_kernel_gbs"] / peaks["hbm_gbs"],
+                       frac_of_nominal_8tbs=decode["split_kernel_gbs"] / 8000.0),
+        "cpu_baseline": {"value": cpu_tf, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc},
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": path.h2d_bytes(),
+                "d2h_bytes_per_step": path.d2h_bytes()},
+        "gpu_launches": launches,
+        "clocks": clocks.summary(),
+    }
+    print(json.dumps(line))
+    if dist:
+        dist.destroy_process_group()
+
+
+def main():
+    from paper_2509_15763_b200 import synth
+
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="llama8b_layer", choices=sorted(synth.WORKLOADS))
+    args = ap.parse_args()
+    w = synth.WORKLOADS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, w)
+    else:
+        run_ours(args, w)
+
+
+if __name__ == "__main__":
+    main()

@@ -169,6 +169,19 @@ int32_t unigist_decode(int32_t num_seqs, int32_t num_q_heads, int32_t num_kv_hea
                        int32_t max_blocks_per_seq, const int32_t* seq_lens, void* o, float* lse,
                        void* workspace, size_t ws_bytes, void* stream);
 
+/*
+ * Measurement aid (no counterpart in the paper): per-kernel device times.
+ * unigist_kernel_timing(1) clears the record list and makes every later kernel launch of the
+ * library record a CUDA event before and after itself on its stream (at most 4096 launches are
+ * kept); unigist_kernel_timing(0) stops recording.  unigist_kernel_timing_count() returns the
+ * number of recorded launches; unigist_kernel_timing_get(i, name, cap, &ms) waits for launch i
+ * to finish and returns its kernel name (copied into name[cap]) and duration in milliseconds.
+ * Not thread safe; meant for benchmarks.
+ */
+int32_t unigist_kernel_timing(int32_t enable);
+int32_t unigist_kernel_timing_count(void);
+int32_t unigist_kernel_timing_get(int32_t index, char* name, int32_t cap, float* ms);
+
 /* Number of kernels the library has launched in this process (all threads). */
 int64_t unigist_launch_count(void);
 

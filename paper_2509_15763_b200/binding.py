@@ -24,6 +24,7 @@ SYMBOLS = [
     "unigist_workspace_bytes", "unigist_layout", "unigist_gist_shift", "unigist_gist_unshift",
     "unigist_attn_fwd", "unigist_attn_bwd", "unigist_kv_compact", "unigist_decode_workspace_bytes",
     "unigist_decode", "unigist_launch_count", "unigist_last_error_string",
+    "unigist_kernel_timing", "unigist_kernel_timing_count", "unigist_kernel_timing_get",
 ]
 
 
@@ -86,6 +87,9 @@ def lib() -> ctypes.CDLL:
             "unigist_kv_compact": (i32, [P, vp, vp, vp, vp, i32, vp, i32, vp, vp, vp, sz, vp]),
             "unigist_decode_workspace_bytes": (sz, [i32] * 5),
             "unigist_decode": (i32, [i32, i32, i32, i32, f32, vp, vp, vp, i32, vp, i32, vp, vp, vp, vp, sz, vp]),
+            "unigist_kernel_timing": (i32, [i32]),
+            "unigist_kernel_timing_count": (i32, []),
+            "unigist_kernel_timing_get": (i32, [i32, ctypes.c_char_p, i32, ctypes.POINTER(ctypes.c_float)]),
             "unigist_launch_count": (i64, []),
             "unigist_last_error_string": (ctypes.c_char_p, []),
         }
@@ -139,6 +143,22 @@ def unigist_workspace_bytes(p: Problem, op: int) -> int:
 
 def unigist_launch_count() -> int:
     return lib().unigist_launch_count()
+
+
+def unigist_kernel_timing(enable: bool) -> None:
+    _check(lib().unigist_kernel_timing(int(enable)))
+
+
+def unigist_kernel_timing_count() -> int:
+    return lib().unigist_kernel_timing_count()
+
+
+def unigist_kernel_timing_get(index: int):
+    """-> (kernel name, milliseconds) of recorded launch `index` (waits for it to finish)."""
+    name = ctypes.create_string_buffer(128)
+    ms = ctypes.c_float()
+    _check(lib().unigist_kernel_timing_get(index, name, 128, ctypes.byref(ms)))
+    return name.value.decode(), ms.value
 
 
 def unigist_last_error_string() -> str:

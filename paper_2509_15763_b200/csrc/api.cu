@@ -22,6 +22,35 @@ int32_t fail(int32_t code, const char* fmt, ...) {
 
 void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
 
+namespace {
+struct TimingRecord {
+  const char* name;
+  cudaEvent_t e0, e1;
+};
+constexpr int kMaxRecords = 4096;
+bool g_timing = false;
+int g_num_records = 0;
+TimingRecord g_records[kMaxRecords];
+}  // namespace
+
+KernelScope::KernelScope(const char* name, cudaStream_t stream) : slot(-1), st(stream) {
+  count_launch();
+  if (!g_timing || g_num_records >= kMaxRecords) return;
+  TimingRecord& r = g_records[g_num_records];
+  if (cudaEventCreate(&r.e0) != cudaSuccess) return;
+  if (cudaEventCreate(&r.e1) != cudaSuccess) {
+    cudaEventDestroy(r.e0);
+    return;
+  }
+  r.name = name;
+  slot = g_num_records++;
+  cudaEventRecord(r.e0, st);
+}
+
+KernelScope::~KernelScope() {
+  if (slot >= 0) cudaEventRecord(g_records[slot].e1, st);
+}
+
 int32_t check_launch(const char* what) {
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return fail(UNIGIST_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
@@ -255,6 +284,31 @@ int32_t unigist_decode(int32_t S, int32_t Hq, int32_t Hkv, int32_t D, float soft
     return fail(UNIGIST_ERR_WORKSPACE, "decode needs %zu bytes of workspace, got %zu", need, ws_bytes);
   return launch_decode(S, Hq, Hkv, D, scale, q, kc, vc, num_blocks, table, max_blocks, seq_lens, o,
                        lse, workspace, (cudaStream_t)stream);
+}
+
+int32_t unigist_kernel_timing(int32_t enable) {
+  for (int i = 0; i < g_num_records; ++i) {
+    cudaEventDestroy(g_records[i].e0);
+    cudaEventDestroy(g_records[i].e1);
+  }
+  g_num_records = 0;
+  g_timing = enable != 0;
+  return UNIGIST_OK;
+}
+
+int32_t unigist_kernel_timing_count(void) { return g_num_records; }
+
+int32_t unigist_kernel_timing_get(int32_t index, char* name, int32_t cap, float* ms) {
+  if (index < 0 || index >= g_num_records || !ms) return fail(UNIGIST_ERR_INVALID_ARG, "no such timing record");
+  TimingRecord& r = g_records[index];
+  cudaError_t e = cudaEventSynchronize(r.e1);
+  if (e == cudaSuccess) e = cudaEventElapsedTime(ms, r.e0, r.e1);
+  if (e != cudaSuccess) return fail(UNIGIST_ERR_CUDA, "kernel timing: %s", cudaGetErrorString(e));
+  if (name && cap > 0) {
+    strncpy(name, r.name, (size_t)cap - 1);
+    name[cap - 1] = 0;
+  }
+  return UNIGIST_OK;
 }
 
 int64_t unigist_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }

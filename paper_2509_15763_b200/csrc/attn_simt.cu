@@ -448,10 +448,12 @@ int32_t launch_fwd_simt(const Geom& g, const unigist_problem& p, float scale, co
   auto go = [&](auto kern, int D) -> int32_t {
     const size_t smem = (size_t)(3 * TS * (D + 4) + TS * LDS_) * sizeof(float);
     if (int32_t rc = set_smem(kern, smem)) return rc;
-    kern<<<grid, 256, smem, st>>>(g, p.num_q_heads, p.num_kv_heads, scale, (const __nv_bfloat16*)q,
-                                  (const __nv_bfloat16*)k, (const __nv_bfloat16*)v,
-                                  (__nv_bfloat16*)o, lse);
-    count_launch();
+    {
+      KernelScope ks("fwd_simt_kernel", st);
+      kern<<<grid, 256, smem, st>>>(g, p.num_q_heads, p.num_kv_heads, scale, (const __nv_bfloat16*)q,
+                                    (const __nv_bfloat16*)k, (const __nv_bfloat16*)v,
+                                    (__nv_bfloat16*)o, lse);
+    }
     return check_launch("forward kernel");
   };
   return p.head_dim == 64 ? go(fwd_simt_kernel<64>, 64) : go(fwd_simt_kernel<128>, 128);
@@ -466,30 +468,34 @@ int32_t launch_bwd_simt(const Geom& g, const unigist_problem& p, float scale, co
   const long long rows = (long long)p.batch * g.N * p.num_q_heads;
   {
     const int blocks = (int)((rows + 7) / 8 < 148 * 16 ? (rows + 7) / 8 : 148 * 16);
+    KernelScope ks("bwd_delta_kernel", st);
     if (f32)
       bwd_delta_kernel<true><<<blocks, 256, 0, st>>>(g.N, p.num_q_heads, p.head_dim, rows, d_o,
                                                      (const __nv_bfloat16*)o, delta);
     else
       bwd_delta_kernel<false><<<blocks, 256, 0, st>>>(g.N, p.num_q_heads, p.head_dim, rows, d_o,
                                                       (const __nv_bfloat16*)o, delta);
-    count_launch();
-    if (int32_t rc = check_launch("delta kernel")) return rc;
   }
+  if (int32_t rc = check_launch("delta kernel")) return rc;
   auto go = [&](auto kq, auto kkv, int D) -> int32_t {
     const size_t smem_q = (size_t)(4 * TS * (D + 4) + TS * LDS_) * sizeof(float);
     const size_t smem_kv = (size_t)(4 * TS * (D + 4) + 2 * TS * LDS_ + 2 * TS) * sizeof(float);
     if (int32_t rc = set_smem(kq, smem_q)) return rc;
     if (int32_t rc = set_smem(kkv, smem_kv)) return rc;
-    kq<<<dim3(ntiles, p.num_q_heads, p.batch), 256, smem_q, st>>>(
-        g, p.num_q_heads, p.num_kv_heads, scale, f32, (const __nv_bfloat16*)q,
-        (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, d_o, lse, delta, (__nv_bfloat16*)dq);
-    count_launch();
+    {
+      KernelScope ks("bwd_dq_simt_kernel", st);
+      kq<<<dim3(ntiles, p.num_q_heads, p.batch), 256, smem_q, st>>>(
+          g, p.num_q_heads, p.num_kv_heads, scale, f32, (const __nv_bfloat16*)q,
+          (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, d_o, lse, delta, (__nv_bfloat16*)dq);
+    }
     if (int32_t rc = check_launch("dQ kernel")) return rc;
-    kkv<<<dim3(ntiles, p.num_kv_heads, p.batch), 256, smem_kv, st>>>(
-        g, p.num_q_heads, p.num_kv_heads, scale, f32, (const __nv_bfloat16*)q,
-        (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, d_o, lse, delta, (__nv_bfloat16*)dk,
-        (__nv_bfloat16*)dv);
-    count_launch();
+    {
+      KernelScope ks("bwd_dkdv_simt_kernel", st);
+      kkv<<<dim3(ntiles, p.num_kv_heads, p.batch), 256, smem_kv, st>>>(
+          g, p.num_q_heads, p.num_kv_heads, scale, f32, (const __nv_bfloat16*)q,
+          (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, d_o, lse, delta, (__nv_bfloat16*)dk,
+          (__nv_bfloat16*)dv);
+    }
     return check_launch("dK/dV kernel");
   };
   return p.head_dim == 64 ? go(bwd_dq_simt_kernel<64>, bwd_dkdv_simt_kernel<64>, 64)

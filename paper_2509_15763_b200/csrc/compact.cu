@@ -113,10 +113,12 @@ int32_t launch_compact_gather(const Geom& g, const unigist_problem& p, const voi
                               cudaStream_t st) {
   const int L = g.s + g.n + g.k * g.r, vecs = p.head_dim / 8;
   const long long total = (long long)p.batch * L * p.num_kv_heads * vecs;
-  compact_gather_kernel<<<grid_for(total), 256, 0, st>>>(
-      g, p.batch, p.num_kv_heads, vecs, L, (const uint4*)k, (const uint4*)v, (uint4*)kc, (uint4*)vc,
-      num_blocks, table, max_blocks, seq_lens, kept_idx);
-  count_launch();
+  {
+    KernelScope ks("compact_gather_kernel", st);
+    compact_gather_kernel<<<grid_for(total), 256, 0, st>>>(
+        g, p.batch, p.num_kv_heads, vecs, L, (const uint4*)k, (const uint4*)v, (uint4*)kc, (uint4*)vc,
+        num_blocks, table, max_blocks, seq_lens, kept_idx);
+  }
   return check_launch("compaction gather kernel");
 }
 
@@ -132,20 +134,26 @@ int32_t launch_compact_inplace(const Geom& g, const unigist_problem& p, void* kc
                                            cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
       if (e != cudaSuccess) return fail(UNIGIST_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
     }
-    compact_edit_table_kernel<<<p.batch, 256, smem, st>>>(g, L, table, max_blocks, seq_lens, kept_idx);
-    count_launch();
+    {
+      KernelScope ks("compact_edit_table_kernel", st);
+      compact_edit_table_kernel<<<p.batch, 256, smem, st>>>(g, L, table, max_blocks, seq_lens, kept_idx);
+    }
     return check_launch("compaction table edit kernel");
   }
   const long long total = (long long)p.batch * L * p.num_kv_heads * vecs;
-  compact_stage_kernel<false><<<grid_for(total), 256, 0, st>>>(
-      g, p.batch, p.num_kv_heads, vecs, L, (uint4*)kc, (uint4*)vc, num_blocks, table, max_blocks,
-      (uint4*)ws, seq_lens, kept_idx);
-  count_launch();
+  {
+    KernelScope ks("compact_stage_kernel", st);
+    compact_stage_kernel<false><<<grid_for(total), 256, 0, st>>>(
+        g, p.batch, p.num_kv_heads, vecs, L, (uint4*)kc, (uint4*)vc, num_blocks, table, max_blocks,
+        (uint4*)ws, seq_lens, kept_idx);
+  }
   if (int32_t rc = check_launch("compaction staging kernel")) return rc;
-  compact_stage_kernel<true><<<grid_for(total), 256, 0, st>>>(
-      g, p.batch, p.num_kv_heads, vecs, L, (uint4*)kc, (uint4*)vc, num_blocks, table, max_blocks,
-      (uint4*)ws, seq_lens, kept_idx);
-  count_launch();
+  {
+    KernelScope ks("compact_writeback_kernel", st);
+    compact_stage_kernel<true><<<grid_for(total), 256, 0, st>>>(
+        g, p.batch, p.num_kv_heads, vecs, L, (uint4*)kc, (uint4*)vc, num_blocks, table, max_blocks,
+        (uint4*)ws, seq_lens, kept_idx);
+  }
   return check_launch("compaction write-back kernel");
 }
 

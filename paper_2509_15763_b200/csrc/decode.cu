@@ -260,10 +260,12 @@ int32_t launch_decode(int S, int Hq, int Hkv, int D, float scale, const void* q,
     const size_t smem = split_smem(g);
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return fail(UNIGIST_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
-    kern<<<grid, THREADS, smem, st>>>(Hq, Hkv, scale * LOG2E, (const __nv_bfloat16*)q,
-                                      (const __nv_bfloat16*)kc, (const __nv_bfloat16*)vc, num_blocks,
-                                      table, max_blocks, seq_lens, splits, bps, (float*)ws);
-    count_launch();
+    {
+      KernelScope ks("decode_split_kernel", st);
+      kern<<<grid, THREADS, smem, st>>>(Hq, Hkv, scale * LOG2E, (const __nv_bfloat16*)q,
+                                        (const __nv_bfloat16*)kc, (const __nv_bfloat16*)vc, num_blocks,
+                                        table, max_blocks, seq_lens, splits, bps, (float*)ws);
+    }
     return check_launch("decode split kernel");
   };
   int32_t rc;
@@ -275,8 +277,10 @@ int32_t launch_decode(int S, int Hq, int Hkv, int D, float scale, const void* q,
     default: return fail(UNIGIST_ERR_UNSUPPORTED, "decode supports 1, 2, 4 or 8 query heads per KV head, got %d", G);
   }
   if (rc) return rc;
-  decode_combine_kernel<<<S * Hq, DD, 0, st>>>(splits, (const float*)ws, (__nv_bfloat16*)o, lse);
-  count_launch();
+  {
+    KernelScope ks("decode_combine_kernel", st);
+    decode_combine_kernel<<<S * Hq, DD, 0, st>>>(splits, (const float*)ws, (__nv_bfloat16*)o, lse);
+  }
   return check_launch("decode combine kernel");
 }
 

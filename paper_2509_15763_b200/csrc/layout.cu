@@ -18,8 +18,10 @@ int32_t launch_layout(const Geom& g, int32_t* sp, int32_t* up, int32_t* pos, cud
   const int threads = 256;
   int blocks = (g.N + threads - 1) / threads;
   if (blocks > 148 * 8) blocks = 148 * 8;
-  layout_kernel<<<blocks, threads, 0, st>>>(g, sp, up, pos);
-  count_launch();
+  {
+    KernelScope ks("layout_kernel", st);
+    layout_kernel<<<blocks, threads, 0, st>>>(g, sp, up, pos);
+  }
   return check_launch("layout kernel");
 }
 
@@ -65,11 +67,13 @@ int32_t launch_shift(const Geom& g, int B, const void* src, void* dst, size_t ro
   const long long total = (long long)B * g.N * vecs;
   long long want = (total + 255) / 256;
   const int blocks = (int)(want < 148 * 16 ? want : 148 * 16);
-  if (inverse)
-    shift_rows_kernel<true><<<blocks, 256, 0, st>>>(g, (const uint4*)src, (uint4*)dst, vecs, total);
-  else
-    shift_rows_kernel<false><<<blocks, 256, 0, st>>>(g, (const uint4*)src, (uint4*)dst, vecs, total);
-  count_launch();
+  {
+    KernelScope ks(inverse ? "unshift_rows_kernel" : "shift_rows_kernel", st);
+    if (inverse)
+      shift_rows_kernel<true><<<blocks, 256, 0, st>>>(g, (const uint4*)src, (uint4*)dst, vecs, total);
+    else
+      shift_rows_kernel<false><<<blocks, 256, 0, st>>>(g, (const uint4*)src, (uint4*)dst, vecs, total);
+  }
   return check_launch("gist shift kernel");
 }
 

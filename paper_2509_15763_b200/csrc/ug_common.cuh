@@ -80,6 +80,14 @@ int32_t fail(int32_t code, const char* fmt, ...);
 int32_t check_problem(const unigist_problem* p, Geom* g, float* scale);
 int32_t check_launch(const char* what);
 void count_launch(int n = 1);
+// Records a CUDA event before and after the kernels launched in its scope when per-kernel
+// timing is switched on; also counts the launch.
+struct KernelScope {
+  KernelScope(const char* name, cudaStream_t st);
+  ~KernelScope();
+  int slot;
+  cudaStream_t st;
+};
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 // Kernel launchers (one per .cu file).
