@@ -182,6 +182,15 @@ int32_t unigist_kernel_timing(int32_t enable);
 int32_t unigist_kernel_timing_count(void);
 int32_t unigist_kernel_timing_get(int32_t index, char* name, int32_t cap, float* ms);
 
+/*
+ * Device-side waits in the tensor-core kernels (on TMA and MMA completion barriers) are bounded:
+ * a wait that does not end within about a second of SM clock makes its thread block leave early
+ * and raises a flag instead of hanging the GPU.  This call synchronises the current device, then
+ * returns UNIGIST_ERR_TIMEOUT (and clears the flag) if any kernel gave up since the last call,
+ * UNIGIST_OK otherwise.  No counterpart in the paper.
+ */
+int32_t unigist_device_status(void);
+
 /* Number of kernels the library has launched in this process (all threads). */
 int64_t unigist_launch_count(void);
 

@@ -25,6 +25,7 @@ SYMBOLS = [
     "unigist_attn_fwd", "unigist_attn_bwd", "unigist_kv_compact", "unigist_decode_workspace_bytes",
     "unigist_decode", "unigist_launch_count", "unigist_last_error_string",
     "unigist_kernel_timing", "unigist_kernel_timing_count", "unigist_kernel_timing_get",
+    "unigist_device_status",
 ]
 
 
@@ -90,6 +91,7 @@ def lib() -> ctypes.CDLL:
             "unigist_kernel_timing": (i32, [i32]),
             "unigist_kernel_timing_count": (i32, []),
             "unigist_kernel_timing_get": (i32, [i32, ctypes.c_char_p, i32, ctypes.POINTER(ctypes.c_float)]),
+            "unigist_device_status": (i32, []),
             "unigist_launch_count": (i64, []),
             "unigist_last_error_string": (ctypes.c_char_p, []),
         }
@@ -159,6 +161,11 @@ def unigist_kernel_timing_get(index: int):
     ms = ctypes.c_float()
     _check(lib().unigist_kernel_timing_get(index, name, 128, ctypes.byref(ms)))
     return name.value.decode(), ms.value
+
+
+def unigist_device_status() -> None:
+    """Synchronise the device; raise UnigistError if a kernel gave up on a bounded wait."""
+    _check(lib().unigist_device_status())
 
 
 def unigist_last_error_string() -> str:

@@ -203,7 +203,18 @@ int32_t unigist_attn_fwd(const unigist_problem* p, const void* q, const void* k,
   if (!q || !k || !v || !o || !lse) return fail(UNIGIST_ERR_INVALID_ARG, "a tensor is NULL");
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || !aligned16(lse))
     return fail(UNIGIST_ERR_ALIGNMENT, "tensor pointers must be 16-byte aligned");
+  // Tensor-core path for sequences without sinks; the CUDA-core kernels cover sink prefixes.
+  if (g.s == 0) return launch_fwd_sm100(g, *p, scale, q, k, v, o, lse, (cudaStream_t)stream);
   return launch_fwd_simt(g, *p, scale, q, k, v, o, lse, (cudaStream_t)stream);
+}
+
+int32_t unigist_device_status(void) {
+  cudaError_t e = cudaDeviceSynchronize();
+  if (e != cudaSuccess) return fail(UNIGIST_ERR_CUDA, "cudaDeviceSynchronize: %s", cudaGetErrorString(e));
+  bool timed_out = false;
+  if (int32_t rc = fwd_sm100_take_timeout(&timed_out)) return rc;
+  if (timed_out) return fail(UNIGIST_ERR_TIMEOUT, "a kernel gave up on a bounded wait; its outputs are invalid");
+  return UNIGIST_OK;
 }
 
 int32_t unigist_attn_bwd(const unigist_problem* p, const void* q, const void* k, const void* v,

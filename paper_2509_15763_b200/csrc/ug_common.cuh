@@ -96,6 +96,9 @@ int32_t launch_shift(const Geom& g, int B, const void* src, void* dst, size_t ro
                      bool inverse, cudaStream_t st);
 int32_t launch_fwd_simt(const Geom& g, const unigist_problem& p, float scale, const void* q,
                         const void* k, const void* v, void* o, float* lse, cudaStream_t st);
+int32_t launch_fwd_sm100(const Geom& g, const unigist_problem& p, float scale, const void* q,
+                         const void* k, const void* v, void* o, float* lse, cudaStream_t st);
+int32_t fwd_sm100_take_timeout(bool* timed_out);
 int32_t launch_bwd_simt(const Geom& g, const unigist_problem& p, float scale, const void* q,
                         const void* k, const void* v, const void* o, const float* lse,
                         const void* d_o, void* dq, void* dk, void* dv, float* delta,

@@ -50,7 +50,7 @@ def run_attention(w: synth.Workload, backward: bool = True, dout_fp32: bool = Fa
             out[name] = torch.empty_like(t)
             ug.unigist_gist_unshift(p, t, out[name])
             out[name + "_shifted"] = t
-    torch.cuda.synchronize()
+    ug.unigist_device_status()  # synchronises; raises if a bounded device wait gave up
     return out
 
 
