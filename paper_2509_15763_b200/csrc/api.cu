@@ -212,8 +212,10 @@ int32_t unigist_device_status(void) {
   cudaError_t e = cudaDeviceSynchronize();
   if (e != cudaSuccess) return fail(UNIGIST_ERR_CUDA, "cudaDeviceSynchronize: %s", cudaGetErrorString(e));
   bool timed_out = false;
+  bool bwd_timed_out = false;
   if (int32_t rc = fwd_sm100_take_timeout(&timed_out)) return rc;
-  if (timed_out) return fail(UNIGIST_ERR_TIMEOUT, "a kernel gave up on a bounded wait; its outputs are invalid");
+  if (int32_t rc = bwd_sm100_take_timeout(&bwd_timed_out)) return rc;
+  if (timed_out || bwd_timed_out) return fail(UNIGIST_ERR_TIMEOUT, "a kernel gave up on a bounded wait; its outputs are invalid");
   return UNIGIST_OK;
 }
 
@@ -232,6 +234,8 @@ int32_t unigist_attn_bwd(const unigist_problem* p, const void* q, const void* k,
   if (!workspace || ws_bytes < need)
     return fail(UNIGIST_ERR_WORKSPACE, "backward needs %zu bytes of workspace, got %zu", need,
                 ws_bytes);
+  if (g.s == 0)
+    return launch_bwd_sm100(g, *p, scale, q, k, v, o, lse, d_o, dq, dk, dv, workspace, (cudaStream_t)stream);
   return launch_bwd_simt(g, *p, scale, q, k, v, o, lse, d_o, dq, dk, dv, (float*)workspace,
                          (cudaStream_t)stream);
 }

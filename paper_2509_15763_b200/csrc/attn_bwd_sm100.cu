@@ -1,0 +1,694 @@
+// Backward gist-masked attention on Blackwell tensor cores (tcgen05 + TMEM + TMA), no sinks.
+//
+// Three kernels on the SHIFTED sequence [raw (T) | gists (n)]:
+//   bwd_prep_kernel            Delta = rowsum(dO o O) (fp32) and, for an fp32 dO, its bf16 copy.
+//   attn_bwd_dkdv_sm100_kernel one thread block owns a 128-key tile of one KV head and walks every
+//                              128-query tile of every query head of the group that can see it:
+//                              S^T = K Q^T and dP^T = V dO^T (TMEM), P^T = exp2(S^T c - LSE),
+//                              dS^T = P^T o (dP^T - Delta), dV += P^T dO, dK += dS^T Q.  dK and dV
+//                              live in TMEM for the whole block: no atomics, deterministic.
+//   attn_bwd_dq_sm100_kernel   one thread block owns a 128-query tile of one query head and walks
+//                              the visible 64-key tiles: S, dP, dS as above, dQ += dS K in TMEM.
+// Tiles without a visible pair are never loaded; only "partial" tiles evaluate the mask.
+#include "sm100_ptx.cuh"
+#include "ug_common.cuh"
+
+namespace ug {
+namespace {
+
+using namespace sm100;
+
+constexpr float kLog2e = 1.4426950408889634f;
+__device__ unsigned int g_bwd_timeout = 0;
+
+// ------------------------------------------------------------------------------------------------
+// Delta and dO conversion: one warp per (batch, token, head) row.
+template <bool kF32>
+__global__ void __launch_bounds__(256)
+bwd_prep_kernel(int N, int Hq, int D, long long rows, const void* __restrict__ d_o,
+                const __nv_bfloat16* __restrict__ o, float* __restrict__ delta,
+                __nv_bfloat16* __restrict__ d_o_bf16) {
+  const int lane = threadIdx.x & 31;
+  const long long warp = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const long long nwarps = ((long long)gridDim.x * blockDim.x) >> 5;
+  for (long long rw = warp; rw < rows; rw += nwarps) {  // rw = (b*N + t)*Hq + h
+    float acc = 0.f;
+    for (int d = lane * 2; d < D; d += 64) {
+      float x0, x1;
+      if (kF32) {
+        const float2 t = *reinterpret_cast<const float2*>(reinterpret_cast<const float*>(d_o) + rw * D + d);
+        const __nv_bfloat162 r2 = __floats2bfloat162_rn(t.x, t.y);
+        *reinterpret_cast<__nv_bfloat162*>(d_o_bf16 + rw * D + d) = r2;
+        const float2 rr = __bfloat1622float2(r2);
+        x0 = rr.x;
+        x1 = rr.y;
+      } else {
+        const float2 rr = __bfloat1622float2(
+            *reinterpret_cast<const __nv_bfloat162*>(reinterpret_cast<const __nv_bfloat16*>(d_o) + rw * D + d));
+        x0 = rr.x;
+        x1 = rr.y;
+      }
+      const float2 oo = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(o + rw * D + d));
+      acc += x0 * oo.x + x1 * oo.y;
+    }
+#pragma unroll
+    for (int off = 16; off >= 1; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
+    if (lane == 0) {
+      const int h = (int)(rw % Hq);
+      const long long bt = rw / Hq;
+      const int t = (int)(bt % N);
+      const long long b = bt / N;
+      delta[(b * Hq + h) * N + t] = acc;
+    }
+  }
+}
+
+// Query rows (numbered inside the raw or the gist segment, inclusive) that see a given key:
+// Eq. 3 read column-wise.  An empty interval has lo > hi.
+__device__ __forceinline__ void key_q_interval(const Geom& g, bool key_is_raw, int key, bool key_valid,
+                                               bool q_is_raw, int& lo, int& hi) {
+  if (!key_valid) {
+    lo = 1;
+    hi = 0;
+    return;
+  }
+  if (key_is_raw) {
+    const int u = key / g.r;
+    if (q_is_raw) {
+      lo = key;
+      hi = min(g.T - 1, (u + g.k + 1) * g.r - 1);
+    } else {
+      lo = u;
+      hi = min(g.n - 1, u + g.k);
+    }
+  } else {
+    if (q_is_raw) {
+      lo = (key + 1) * g.r;
+      hi = g.T - 1;
+    } else {
+      lo = key;
+      hi = g.n - 1;
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// dK / dV kernel
+constexpr int KV_BM = 128;       // keys per block (TMEM lanes)
+constexpr int KV_BN = 128;       // queries per step
+constexpr int kKvThreads = 320;  // 8 compute warps, 1 TMA warp, 1 MMA warp
+
+template <int D>
+struct KvSmem {
+  static constexpr int kSlab = 128 * 128;
+  static constexpr int kTile = kSlab * (D / 64);
+  static constexpr int kStats = 2 * 2 * KV_BN * 4;  // [stage][lse2 | delta][128] fp32
+  static constexpr int kBytes = 6 * kTile + kStats + 1024 + 256;
+};
+
+template <int D>
+__global__ void __launch_bounds__(kKvThreads, 1)
+attn_bwd_dkdv_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const __grid_constant__ CUtensorMap tm_q_gist,
+                           const __grid_constant__ CUtensorMap tm_do_raw, const __grid_constant__ CUtensorMap tm_do_gist,
+                           const __grid_constant__ CUtensorMap tm_k_raw, const __grid_constant__ CUtensorMap tm_k_gist,
+                           const __grid_constant__ CUtensorMap tm_v_raw, const __grid_constant__ CUtensorMap tm_v_gist,
+                           Geom g, int Hq, int Hkv, float scale, const float* __restrict__ lse,
+                           const float* __restrict__ delta, __nv_bfloat16* __restrict__ dk,
+                           __nv_bfloat16* __restrict__ dv, int n_gist_kt) {
+  using SM = KvSmem<D>;
+  extern __shared__ unsigned char smem_dyn[];
+  const uint32_t base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
+  unsigned char* gen = smem_dyn + (base - smem_u32(smem_dyn));
+  const uint32_t sK = base, sV = base + SM::kTile;
+  const uint32_t sQ[2] = {base + 2 * SM::kTile, base + 4 * SM::kTile};
+  const uint32_t sDO[2] = {base + 3 * SM::kTile, base + 5 * SM::kTile};
+  float* stats = reinterpret_cast<float*>(gen + 6 * SM::kTile);  // [stage][2][128]
+  const uint32_t bars = base + 6 * SM::kTile + SM::kStats;
+  const uint32_t bar_kv = bars, bar_full[2] = {bars + 8, bars + 16}, bar_empty[2] = {bars + 24, bars + 32},
+                 bar_S = bars + 40, bar_dP = bars + 48, bar_P = bars + 56, bar_dS = bars + 64, bar_final = bars + 72,
+                 tmem_slot = bars + 80;
+  volatile uint32_t* tmem_slot_ptr = reinterpret_cast<volatile uint32_t*>(gen + 6 * SM::kTile + SM::kStats + 80);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int hk = blockIdx.y, b = blockIdx.z, G = Hq / Hkv;
+  // gist key tiles are seen by every later query: heaviest, scheduled first
+  const bool key_is_raw = (int)blockIdx.x >= n_gist_kt;
+  const int kt = key_is_raw ? blockIdx.x - n_gist_kt : blockIdx.x;
+  const int key_seg_len = key_is_raw ? g.T : g.n;
+  const int key_seg_base = key_is_raw ? g.s : g.s + g.T;
+  const int key_a = kt * KV_BM, key_b = min(key_a + KV_BM - 1, key_seg_len - 1);
+  const bool key_tile_whole = key_a + KV_BM - 1 <= key_seg_len - 1;
+
+  // query tiles that see this key tile: raw-segment tiles [rq_lo, rq_hi], gist-segment tiles [gq_lo, gq_hi]
+  int a_lo, a_hi, b_lo, b_hi, c_lo, c_hi, d_lo, d_hi;
+  key_q_interval(g, key_is_raw, key_a, true, true, a_lo, a_hi);   // first key vs raw queries
+  key_q_interval(g, key_is_raw, key_b, true, true, b_lo, b_hi);   // last key vs raw queries
+  key_q_interval(g, key_is_raw, key_a, true, false, c_lo, c_hi);  // first key vs gist queries
+  key_q_interval(g, key_is_raw, key_b, true, false, d_lo, d_hi);  // last key vs gist queries
+  const int n_raw_q = b_hi >= a_lo ? b_hi / KV_BN - a_lo / KV_BN + 1 : 0;
+  const int rq_lo = a_lo / KV_BN;
+  const int n_gist_q = d_hi >= c_lo ? d_hi / KV_BN - c_lo / KV_BN + 1 : 0;
+  const int gq_lo = c_lo / KV_BN;
+  const int n_iter = (n_raw_q + n_gist_q) * G;
+
+  if (threadIdx.x == 0) {
+    mbar_init(bar_kv, 1);
+    mbar_init(bar_full[0], 1);
+    mbar_init(bar_full[1], 1);
+    mbar_init(bar_empty[0], 1);
+    mbar_init(bar_empty[1], 1);
+    mbar_init(bar_S, 1);
+    mbar_init(bar_dP, 1);
+    mbar_init(bar_P, 256);
+    mbar_init(bar_dS, 256);
+    mbar_init(bar_final, 1);
+    mbar_fence_init();
+  }
+  if (warp == 9) tmem_alloc(tmem_slot, 512);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot_ptr;
+  const uint32_t t_dK = tmem, t_dV = tmem + 128, t_A = tmem + 256, t_B = tmem + 384;
+  bool ok = true;
+
+  auto tile_of = [&](int it, bool& q_is_raw, int& qt, int& head) {
+    const int t = it / G;
+    head = hk * G + (it - t * G);
+    q_is_raw = t < n_raw_q;
+    qt = q_is_raw ? rq_lo + t : gq_lo + (t - n_raw_q);
+  };
+
+  if (warp == 8) {
+    // ------------------------------------------------------------ producer: K, V once; Q, dO, LSE, Delta per step
+    if (lane == 0) {
+      mbar_arrive_expect_tx(bar_kv, 2 * SM::kTile);
+      const CUtensorMap* mk = key_is_raw ? &tm_k_raw : &tm_k_gist;
+      const CUtensorMap* mv = key_is_raw ? &tm_v_raw : &tm_v_gist;
+#pragma unroll
+      for (int sl = 0; sl < D / 64; ++sl) {
+        tma_load_4d(sK + sl * SM::kSlab, mk, bar_kv, sl * 64, hk, key_a, b);
+        tma_load_4d(sV + sl * SM::kSlab, mv, bar_kv, sl * 64, hk, key_a, b);
+      }
+    }
+    for (int it = 0; it < n_iter; ++it) {
+      const int st = it & 1;
+      bool q_is_raw;
+      int qt, head;
+      tile_of(it, q_is_raw, qt, head);
+      if (it >= 2) ok = mbar_wait(bar_empty[st], ((it >> 1) - 1) & 1);
+      if (!ok) break;
+      const int q_seg_len = q_is_raw ? g.T : g.n, q_seg_base = q_is_raw ? g.s : g.s + g.T;
+      float* ls = stats + st * 2 * KV_BN;
+      const long long row_base = ((long long)b * Hq + head) * g.N + q_seg_base;
+#pragma unroll
+      for (int i = 0; i < KV_BN / 32; ++i) {
+        const int c = lane + 32 * i, row = qt * KV_BN + c;
+        const bool valid = row < q_seg_len;
+        // rows past the segment get LSE = +inf, so their P is exactly zero
+        ls[c] = valid ? lse[row_base + row] * kLog2e : INFINITY;
+        ls[KV_BN + c] = valid ? delta[row_base + row] : 0.f;
+      }
+      __syncwarp();
+      if (lane == 0) {
+        mbar_arrive_expect_tx(bar_full[st], 2 * SM::kTile);
+        const CUtensorMap* mq = q_is_raw ? &tm_q_raw : &tm_q_gist;
+        const CUtensorMap* md = q_is_raw ? &tm_do_raw : &tm_do_gist;
+#pragma unroll
+        for (int sl = 0; sl < D / 64; ++sl) {
+          tma_load_4d(sQ[st] + sl * SM::kSlab, mq, bar_full[st], sl * 64, head, qt * KV_BN, b);
+          tma_load_4d(sDO[st] + sl * SM::kSlab, md, bar_full[st], sl * 64, head, qt * KV_BN, b);
+        }
+      }
+      __syncwarp();
+    }
+    if (!ok) atomicExch(&g_bwd_timeout, 1u);
+  } else if (warp == 9) {
+    // ------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc_s = make_idesc_bf16(KV_BM, KV_BN, false, false);
+      constexpr uint32_t idesc_acc = make_idesc_bf16(KV_BM, D, false, true);
+      // A operand of the accumulating MMAs: bf16 pairs in TMEM; query columns [0,64) are packed at
+      // columns [0,32) of the buffer, query columns [64,128) at columns [64,96)
+      auto a_col = [](int kk) { return (kk / 4) * 64 + (kk % 4) * 8; };
+      ok = mbar_wait(bar_kv, 0);
+      for (int it = 0; it < n_iter && ok; ++it) {
+        const int st = it & 1;
+        ok = mbar_wait(bar_full[st], (it >> 1) & 1);
+        if (!ok) break;
+        tc_fence_after();
+#pragma unroll
+        for (int kk = 0; kk < D / 16; ++kk) {
+          const uint32_t off = (kk / 4) * SM::kSlab + (kk % 4) * 32;
+          umma_ss(t_A, make_smem_desc(sK + off, 16, 1024), make_smem_desc(sQ[st] + off, 16, 1024), idesc_s, kk > 0);
+        }
+        umma_commit(bar_S);
+        if (it > 0) {
+          const int ps = (it - 1) & 1;
+          ok = mbar_wait(bar_dS, (it - 1) & 1);
+          if (!ok) break;
+          tc_fence_after();
+#pragma unroll
+          for (int kk = 0; kk < KV_BN / 16; ++kk)
+            umma_ts(t_dK, t_B + a_col(kk), make_smem_desc(sQ[ps] + kk * 2048, SM::kSlab, 1024), idesc_acc,
+                    (it > 1 || kk > 0) ? 1u : 0u);
+          umma_commit(bar_empty[ps]);
+        }
+#pragma unroll
+        for (int kk = 0; kk < D / 16; ++kk) {
+          const uint32_t off = (kk / 4) * SM::kSlab + (kk % 4) * 32;
+          umma_ss(t_B, make_smem_desc(sV + off, 16, 1024), make_smem_desc(sDO[st] + off, 16, 1024), idesc_s, kk > 0);
+        }
+        umma_commit(bar_dP);
+        ok = mbar_wait(bar_P, it & 1);
+        if (!ok) break;
+        tc_fence_after();
+#pragma unroll
+        for (int kk = 0; kk < KV_BN / 16; ++kk)
+          umma_ts(t_dV, t_A + a_col(kk), make_smem_desc(sDO[st] + kk * 2048, SM::kSlab, 1024), idesc_acc,
+                  (it > 0 || kk > 0) ? 1u : 0u);
+      }
+      if (ok && n_iter > 0) {
+        const int ps = (n_iter - 1) & 1;
+        ok = mbar_wait(bar_dS, (n_iter - 1) & 1);
+        if (ok) {
+          tc_fence_after();
+#pragma unroll
+          for (int kk = 0; kk < KV_BN / 16; ++kk)
+            umma_ts(t_dK, t_B + a_col(kk), make_smem_desc(sQ[ps] + kk * 2048, SM::kSlab, 1024), idesc_acc,
+                    (n_iter > 1 || kk > 0) ? 1u : 0u);
+          umma_commit(bar_final);
+        }
+      }
+      if (!ok) atomicExch(&g_bwd_timeout, 1u);
+    }
+  } else {
+    // ------------------------------------------------------------ compute: thread = key (TMEM lane), 64 query columns
+    const int qd = warp & 3, hf = warp >> 2;
+    const int key = key_a + qd * 32 + lane;
+    const bool key_valid = key <= key_b;
+    const uint32_t lane_base = static_cast<uint32_t>(qd * 32) << 16;
+    const float scale_log2 = scale * kLog2e;
+    int my_lo[2], my_hi[2];  // [0]: vs raw queries, [1]: vs gist queries
+    key_q_interval(g, key_is_raw, key, key_valid, true, my_lo[0], my_hi[0]);
+    key_q_interval(g, key_is_raw, key, key_valid, false, my_lo[1], my_hi[1]);
+
+    for (int it = 0; it < n_iter && ok; ++it) {
+      const int st = it & 1;
+      bool q_is_raw;
+      int qt, head;
+      tile_of(it, q_is_raw, qt, head);
+      const int q0 = qt * KV_BN, q_seg_len = q_is_raw ? g.T : g.n;
+      const int qb = min(q0 + KV_BN - 1, q_seg_len - 1);
+      // full: every (query, key) pair of the tile is visible -> no mask arithmetic
+      const int t_lo = q_is_raw ? b_lo : d_lo, t_hi = q_is_raw ? a_hi : c_hi;
+      const bool full = key_tile_whole && q0 >= t_lo && qb <= t_hi;
+      const int lo = my_lo[q_is_raw ? 0 : 1] - q0 - 64 * hf, hi = my_hi[q_is_raw ? 0 : 1] - q0 - 64 * hf;
+      const float* ls = stats + st * 2 * KV_BN + 64 * hf;
+      const float* dl = ls + KV_BN;
+      ok = mbar_wait(bar_full[st], (it >> 1) & 1) && mbar_wait(bar_S, it & 1);
+      if (!ok) break;
+      tc_fence_after();
+      float p[64];
+#pragma unroll
+      for (int c = 0; c < 2; ++c) {
+        uint32_t v[32];
+        tmem_ld(t_A + lane_base + 64 * hf + 32 * c, v);
+        tmem_wait_ld();
+        uint32_t pk[16];
+#pragma unroll
+        for (int i = 0; i < 32; i += 4) {
+          const float4 l4 = *reinterpret_cast<const float4*>(ls + 32 * c + i);
+          const float lv[4] = {l4.x, l4.y, l4.z, l4.w};
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            float x = fmaf(__uint_as_float(v[i + e]), scale_log2, -lv[e]);
+            if (!full) {
+              const int col = 32 * c + i + e;
+              x = (col >= lo && col <= hi) ? x : -INFINITY;
+            }
+            p[32 * c + i + e] = ex2(x);
+          }
+          pk[i / 2] = pack_bf16(p[32 * c + i], p[32 * c + i + 1]);
+          pk[i / 2 + 1] = pack_bf16(p[32 * c + i + 2], p[32 * c + i + 3]);
+        }
+        tmem_st(t_A + lane_base + 64 * hf + 16 * c, pk);
+      }
+      tmem_wait_st();
+      tc_fence_before();
+      mbar_arrive(bar_P);
+      ok = mbar_wait(bar_dP, it & 1);
+      if (!ok) break;
+      tc_fence_after();
+#pragma unroll
+      for (int c = 0; c < 2; ++c) {
+        uint32_t v[32];
+        tmem_ld(t_B + lane_base + 64 * hf + 32 * c, v);
+        tmem_wait_ld();
+        uint32_t pk[16];
+#pragma unroll
+        for (int i = 0; i < 32; i += 4) {
+          const float4 d4 = *reinterpret_cast<const float4*>(dl + 32 * c + i);
+          const float dv4[4] = {d4.x, d4.y, d4.z, d4.w};
+          float ds[4];
+#pragma unroll
+          for (int e = 0; e < 4; ++e) ds[e] = p[32 * c + i + e] * (__uint_as_float(v[i + e]) - dv4[e]);
+          pk[i / 2] = pack_bf16(ds[0], ds[1]);
+          pk[i / 2 + 1] = pack_bf16(ds[2], ds[3]);
+        }
+        tmem_st(t_B + lane_base + 64 * hf + 16 * c, pk);
+      }
+      tmem_wait_st();
+      tc_fence_before();
+      mbar_arrive(bar_dS);
+    }
+    if (ok && n_iter > 0) ok = mbar_wait(bar_final, 0);
+    if (ok) {
+      tc_fence_after();
+      const long long tok = (long long)b * g.N + key_seg_base + key;
+      // D = 128: this warp stores columns [64 hf, 64 hf + 64) of dK and of dV; D = 64: hf picks dK or dV
+      constexpr int kChunks = 2;
+#pragma unroll
+      for (int which = 0; which < (D == 128 ? 2 : 1); ++which) {
+        const bool is_dk = D == 128 ? which == 0 : hf == 0;
+        const int col0 = D == 128 ? 64 * hf : 0;
+        const uint32_t tsrc = (is_dk ? t_dK : t_dV) + lane_base + col0;
+        __nv_bfloat16* dst = (is_dk ? dk : dv) + (tok * Hkv + hk) * D + col0;
+        const float mul = is_dk ? scale : 1.f;
+#pragma unroll
+        for (int c = 0; c < kChunks; ++c) {
+          uint32_t v[32];
+          if (n_iter > 0) {
+            tmem_ld(tsrc + 32 * c, v);
+            tmem_wait_ld();
+          } else {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) v[i] = 0u;
+          }
+          if (key_valid) {
+#pragma unroll
+            for (int i = 0; i < 32; i += 8) {
+              uint4 pk;
+              pk.x = pack_bf16(__uint_as_float(v[i]) * mul, __uint_as_float(v[i + 1]) * mul);
+              pk.y = pack_bf16(__uint_as_float(v[i + 2]) * mul, __uint_as_float(v[i + 3]) * mul);
+              pk.z = pack_bf16(__uint_as_float(v[i + 4]) * mul, __uint_as_float(v[i + 5]) * mul);
+              pk.w = pack_bf16(__uint_as_float(v[i + 6]) * mul, __uint_as_float(v[i + 7]) * mul);
+              *reinterpret_cast<uint4*>(dst + 32 * c + i) = pk;
+            }
+          }
+        }
+      }
+    } else {
+      atomicExch(&g_bwd_timeout, 1u);
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 9) {
+    __syncwarp();
+    tmem_dealloc(tmem, 512);
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// dQ kernel
+constexpr int DQ_BM = 128;  // query rows per block
+constexpr int DQ_BN = 64;   // keys per step
+constexpr int kDqThreads = 192;
+
+template <int D>
+struct DqSmem {
+  static constexpr int kQSlab = DQ_BM * 128, kQTile = kQSlab * (D / 64);
+  static constexpr int kKSlab = DQ_BN * 128, kKTile = kKSlab * (D / 64);
+  static constexpr int kBytes = 2 * kQTile + 2 * kKTile + 1024 + 128;
+};
+
+template <int D>
+__global__ void __launch_bounds__(kDqThreads, 2)
+attn_bwd_dq_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const __grid_constant__ CUtensorMap tm_q_gist,
+                         const __grid_constant__ CUtensorMap tm_do_raw, const __grid_constant__ CUtensorMap tm_do_gist,
+                         const __grid_constant__ CUtensorMap tm_k_raw, const __grid_constant__ CUtensorMap tm_k_gist,
+                         const __grid_constant__ CUtensorMap tm_v_raw, const __grid_constant__ CUtensorMap tm_v_gist,
+                         Geom g, int Hq, int Hkv, float scale, const float* __restrict__ lse,
+                         const float* __restrict__ delta, __nv_bfloat16* __restrict__ dq, int n_raw_qt) {
+  using SM = DqSmem<D>;
+  extern __shared__ unsigned char smem_dyn[];
+  const uint32_t base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
+  unsigned char* gen = smem_dyn + (base - smem_u32(smem_dyn));
+  const uint32_t sQ = base, sDO = base + SM::kQTile, sK = base + 2 * SM::kQTile, sV = sK + SM::kKTile;
+  const uint32_t bars = sV + SM::kKTile;
+  const uint32_t bar_q = bars, bar_k = bars + 8, bar_v = bars + 16, bar_s = bars + 24, bar_p = bars + 32,
+                 bar_pv = bars + 40, tmem_slot = bars + 48;
+  volatile uint32_t* tmem_slot_ptr =
+      reinterpret_cast<volatile uint32_t*>(gen + 2 * SM::kQTile + 2 * SM::kKTile + 48);
+
+  const int warp = threadIdx.x >> 5;
+  const int h = blockIdx.y, b = blockIdx.z, hk = h / (Hq / Hkv);
+  const int qt_lin = gridDim.x - 1 - blockIdx.x;  // heaviest tiles first
+  const bool q_is_raw = qt_lin < n_raw_qt;
+  const int qt = q_is_raw ? qt_lin : qt_lin - n_raw_qt;
+  const int seg_len = q_is_raw ? g.T : g.n;
+  const int seg_base = q_is_raw ? g.s : g.s + g.T;
+  const int row_a = qt * DQ_BM, row_b = min(row_a + DQ_BM - 1, seg_len - 1);
+  const RowIv iv_a = row_intervals(g, seg_base + row_a), iv_b = row_intervals(g, seg_base + row_b);
+  // visible 64-key tiles: raw tiles [raw_lo, raw_hi] then gist tiles [0, n_gist)
+  const int raw_lo = iv_a.lo_raw / DQ_BN, n_raw = iv_b.hi_raw / DQ_BN - raw_lo + 1;
+  const int n_gist = iv_b.hi_gist >= 0 ? iv_b.hi_gist / DQ_BN + 1 : 0;
+  const int nt = n_raw + n_gist;
+
+  if (threadIdx.x == 0) {
+    mbar_init(bar_q, 1);
+    mbar_init(bar_k, 1);
+    mbar_init(bar_v, 1);
+    mbar_init(bar_s, 1);
+    mbar_init(bar_p, 128);
+    mbar_init(bar_pv, 1);
+    mbar_fence_init();
+  }
+  if (warp == 5) tmem_alloc(tmem_slot, 256);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot_ptr;
+  const uint32_t t_S = tmem, t_dP = tmem + 64, t_dQ = tmem + 128;
+  bool ok = true;
+
+  if (warp == 4) {
+    if (elect_one()) {
+      mbar_arrive_expect_tx(bar_q, 2 * SM::kQTile);
+      const CUtensorMap* mq = q_is_raw ? &tm_q_raw : &tm_q_gist;
+      const CUtensorMap* md = q_is_raw ? &tm_do_raw : &tm_do_gist;
+#pragma unroll
+      for (int sl = 0; sl < D / 64; ++sl) {
+        tma_load_4d(sQ + sl * SM::kQSlab, mq, bar_q, sl * 64, h, row_a, b);
+        tma_load_4d(sDO + sl * SM::kQSlab, md, bar_q, sl * 64, h, row_a, b);
+      }
+      for (int j = 0; j < nt && ok; ++j) {
+        const bool is_raw = j < n_raw;
+        const int idx = is_raw ? raw_lo + j : j - n_raw;
+        const CUtensorMap* mk = is_raw ? &tm_k_raw : &tm_k_gist;
+        const CUtensorMap* mv = is_raw ? &tm_v_raw : &tm_v_gist;
+        if (j > 0) ok = mbar_wait(bar_s, (j - 1) & 1);  // dP(j-1) done: V buffer free
+        if (!ok) break;
+        mbar_arrive_expect_tx(bar_v, SM::kKTile);
+#pragma unroll
+        for (int sl = 0; sl < D / 64; ++sl) tma_load_4d(sV + sl * SM::kKSlab, mv, bar_v, sl * 64, hk, idx * DQ_BN, b);
+        if (j > 0) ok = mbar_wait(bar_pv, (j - 1) & 1);  // dQ MMA (j-1) done: K buffer free
+        if (!ok) break;
+        mbar_arrive_expect_tx(bar_k, SM::kKTile);
+#pragma unroll
+        for (int sl = 0; sl < D / 64; ++sl) tma_load_4d(sK + sl * SM::kKSlab, mk, bar_k, sl * 64, hk, idx * DQ_BN, b);
+      }
+      if (!ok) atomicExch(&g_bwd_timeout, 1u);
+    }
+  } else if (warp == 5) {
+    if (elect_one()) {
+      constexpr uint32_t idesc_s = make_idesc_bf16(DQ_BM, DQ_BN, false, false);
+      constexpr uint32_t idesc_dq = make_idesc_bf16(DQ_BM, D, false, true);
+      ok = mbar_wait(bar_q, 0);
+      for (int j = 0; j < nt && ok; ++j) {
+        ok = mbar_wait(bar_k, j & 1) && mbar_wait(bar_v, j & 1);
+        if (!ok) break;
+        tc_fence_after();
+#pragma unroll
+        for (int kk = 0; kk < D / 16; ++kk) {
+          const uint32_t qoff = (kk / 4) * SM::kQSlab + (kk % 4) * 32, koff = (kk / 4) * SM::kKSlab + (kk % 4) * 32;
+          umma_ss(t_S, make_smem_desc(sQ + qoff, 16, 1024), make_smem_desc(sK + koff, 16, 1024), idesc_s, kk > 0);
+        }
+#pragma unroll
+        for (int kk = 0; kk < D / 16; ++kk) {
+          const uint32_t qoff = (kk / 4) * SM::kQSlab + (kk % 4) * 32, koff = (kk / 4) * SM::kKSlab + (kk % 4) * 32;
+          umma_ss(t_dP, make_smem_desc(sDO + qoff, 16, 1024), make_smem_desc(sV + koff, 16, 1024), idesc_s, kk > 0);
+        }
+        umma_commit(bar_s);
+        ok = mbar_wait(bar_p, j & 1);
+        if (!ok) break;
+        tc_fence_after();
+#pragma unroll
+        for (int kk = 0; kk < DQ_BN / 16; ++kk)
+          umma_ts(t_dQ, t_S + kk * 8, make_smem_desc(sK + kk * 2048, SM::kKSlab, 1024), idesc_dq,
+                  (j > 0 || kk > 0) ? 1u : 0u);
+        umma_commit(bar_pv);
+      }
+      if (!ok) atomicExch(&g_bwd_timeout, 1u);
+    }
+  } else {
+    const int r_in_tile = threadIdx.x;
+    const int row = min(row_a + r_in_tile, row_b);
+    const bool valid = row_a + r_in_tile <= row_b;
+    const RowIv my = row_intervals(g, seg_base + row);
+    const uint32_t lane_base = static_cast<uint32_t>(warp * 32) << 16;
+    const float scale_log2 = scale * kLog2e;
+    const long long stat_idx = ((long long)b * Hq + h) * g.N + seg_base + row;
+    const float lse2 = lse[stat_idx] * kLog2e, dl = delta[stat_idx];
+    for (int j = 0; j < nt && ok; ++j) {
+      const bool is_raw = j < n_raw;
+      const int col0 = (is_raw ? raw_lo + j : j - n_raw) * DQ_BN;
+      bool full;
+      int lo, hi;
+      if (is_raw) {
+        full = col0 >= iv_b.lo_raw && col0 + DQ_BN - 1 <= iv_a.hi_raw;
+        lo = my.lo_raw - col0;
+        hi = my.hi_raw - col0;
+      } else {
+        full = col0 + DQ_BN - 1 <= iv_a.hi_gist;
+        lo = 0;
+        hi = my.hi_gist - col0;
+      }
+      ok = mbar_wait(bar_s, j & 1);
+      if (!ok) break;
+      tc_fence_after();
+#pragma unroll
+      for (int c = 0; c < DQ_BN / 32; ++c) {
+        uint32_t sv[32], dv_[32];
+        tmem_ld(t_S + lane_base + 32 * c, sv);
+        tmem_ld(t_dP + lane_base + 32 * c, dv_);
+        tmem_wait_ld();
+        uint32_t pk[16];
+#pragma unroll
+        for (int i = 0; i < 32; i += 2) {
+          float x0 = fmaf(__uint_as_float(sv[i]), scale_log2, -lse2);
+          float x1 = fmaf(__uint_as_float(sv[i + 1]), scale_log2, -lse2);
+          if (!full) {
+            const int col = 32 * c + i;
+            x0 = (col >= lo && col <= hi) ? x0 : -INFINITY;
+            x1 = (col + 1 >= lo && col + 1 <= hi) ? x1 : -INFINITY;
+          }
+          const float ds0 = ex2(x0) * (__uint_as_float(dv_[i]) - dl);
+          const float ds1 = ex2(x1) * (__uint_as_float(dv_[i + 1]) - dl);
+          pk[i / 2] = pack_bf16(ds0, ds1);
+        }
+        tmem_st(t_S + lane_base + 16 * c, pk);
+      }
+      tmem_wait_st();
+      tc_fence_before();
+      mbar_arrive(bar_p);
+    }
+    if (ok) ok = mbar_wait(bar_pv, (nt - 1) & 1);
+    if (ok) {
+      tc_fence_after();
+      const long long tok = (long long)b * g.N + seg_base + row_a + r_in_tile;
+      __nv_bfloat16* drow = dq + (tok * Hq + h) * D;
+#pragma unroll
+      for (int c = 0; c < D / 32; ++c) {
+        uint32_t v[32];
+        tmem_ld(t_dQ + lane_base + 32 * c, v);
+        tmem_wait_ld();
+        if (valid) {
+#pragma unroll
+          for (int i = 0; i < 32; i += 8) {
+            uint4 pk;
+            pk.x = pack_bf16(__uint_as_float(v[i]) * scale, __uint_as_float(v[i + 1]) * scale);
+            pk.y = pack_bf16(__uint_as_float(v[i + 2]) * scale, __uint_as_float(v[i + 3]) * scale);
+            pk.z = pack_bf16(__uint_as_float(v[i + 4]) * scale, __uint_as_float(v[i + 5]) * scale);
+            pk.w = pack_bf16(__uint_as_float(v[i + 6]) * scale, __uint_as_float(v[i + 7]) * scale);
+            *reinterpret_cast<uint4*>(drow + 32 * c + i) = pk;
+          }
+        }
+      }
+    } else {
+      atomicExch(&g_bwd_timeout, 1u);
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 5) {
+    __syncwarp();
+    tmem_dealloc(tmem, 256);
+  }
+}
+
+}  // namespace
+
+int32_t launch_bwd_sm100(const Geom& g, const unigist_problem& p, float scale, const void* q, const void* k,
+                         const void* v, const void* o, const float* lse, const void* d_o, void* dq, void* dk,
+                         void* dv, void* workspace, cudaStream_t st) {
+  const int D = p.head_dim, Hq = p.num_q_heads, Hkv = p.num_kv_heads, B = p.batch;
+  const bool f32 = (p.flags & UNIGIST_FLAG_DOUT_FP32) != 0;
+  float* delta = static_cast<float*>(workspace);
+  const size_t delta_bytes = ((size_t)B * Hq * g.N * sizeof(float) + 255) / 256 * 256;
+  __nv_bfloat16* do_bf16 = reinterpret_cast<__nv_bfloat16*>(static_cast<char*>(workspace) + delta_bytes);
+  const void* do_src = f32 ? static_cast<const void*>(do_bf16) : d_o;
+  {
+    const long long rows = (long long)B * g.N * Hq;
+    const int blocks = (int)((rows + 7) / 8 < 148 * 16 ? (rows + 7) / 8 : 148 * 16);
+    KernelScope ks("bwd_prep_kernel", st);
+    if (f32)
+      bwd_prep_kernel<true><<<blocks, 256, 0, st>>>(g.N, Hq, D, rows, d_o, (const __nv_bfloat16*)o, delta, do_bf16);
+    else
+      bwd_prep_kernel<false><<<blocks, 256, 0, st>>>(g.N, Hq, D, rows, d_o, (const __nv_bfloat16*)o, delta, nullptr);
+  }
+  if (int32_t rc = check_launch("backward prep kernel")) return rc;
+
+  CUtensorMap mq[2], md[2], mk[2], mv[2], mk64[2], mv64[2];
+  const long long first[2] = {g.s, (long long)g.s + g.T}, len[2] = {g.T, g.n};
+  for (int sgm = 0; sgm < 2; ++sgm) {
+    if (int32_t rc = encode_segment_map(&mq[sgm], q, D, Hq, g.N, B, first[sgm], len[sgm], 128)) return rc;
+    if (int32_t rc = encode_segment_map(&md[sgm], do_src, D, Hq, g.N, B, first[sgm], len[sgm], 128)) return rc;
+    if (int32_t rc = encode_segment_map(&mk[sgm], k, D, Hkv, g.N, B, first[sgm], len[sgm], 128)) return rc;
+    if (int32_t rc = encode_segment_map(&mv[sgm], v, D, Hkv, g.N, B, first[sgm], len[sgm], 128)) return rc;
+    if (int32_t rc = encode_segment_map(&mk64[sgm], k, D, Hkv, g.N, B, first[sgm], len[sgm], DQ_BN)) return rc;
+    if (int32_t rc = encode_segment_map(&mv64[sgm], v, D, Hkv, g.N, B, first[sgm], len[sgm], DQ_BN)) return rc;
+  }
+  const int n_raw_t = (g.T + 127) / 128, n_gist_t = (g.n + 127) / 128;
+
+  auto go_kv = [&](auto kern, size_t smem) -> int32_t {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return fail(UNIGIST_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
+    {
+      KernelScope ks("attn_bwd_dkdv_sm100_kernel", st);
+      kern<<<dim3(n_raw_t + n_gist_t, Hkv, B), kKvThreads, smem, st>>>(
+          mq[0], mq[1], md[0], md[1], mk[0], mk[1], mv[0], mv[1], g, Hq, Hkv, scale, lse, delta,
+          (__nv_bfloat16*)dk, (__nv_bfloat16*)dv, n_gist_t);
+    }
+    return check_launch("tcgen05 dK/dV kernel");
+  };
+  auto go_q = [&](auto kern, size_t smem) -> int32_t {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return fail(UNIGIST_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
+    {
+      KernelScope ks("attn_bwd_dq_sm100_kernel", st);
+      kern<<<dim3(n_raw_t + n_gist_t, Hq, B), kDqThreads, smem, st>>>(
+          mq[0], mq[1], md[0], md[1], mk64[0], mk64[1], mv64[0], mv64[1], g, Hq, Hkv, scale, lse, delta,
+          (__nv_bfloat16*)dq, n_raw_t);
+    }
+    return check_launch("tcgen05 dQ kernel");
+  };
+  if (D == 64) {
+    if (int32_t rc = go_kv(attn_bwd_dkdv_sm100_kernel<64>, KvSmem<64>::kBytes)) return rc;
+    return go_q(attn_bwd_dq_sm100_kernel<64>, DqSmem<64>::kBytes);
+  }
+  if (int32_t rc = go_kv(attn_bwd_dkdv_sm100_kernel<128>, KvSmem<128>::kBytes)) return rc;
+  return go_q(attn_bwd_dq_sm100_kernel<128>, DqSmem<128>::kBytes);
+}
+
+int32_t bwd_sm100_take_timeout(bool* timed_out) {
+  unsigned int flag = 0, zero = 0;
+  cudaError_t e = cudaMemcpyFromSymbol(&flag, g_bwd_timeout, sizeof(flag));
+  if (e == cudaSuccess && flag) e = cudaMemcpyToSymbol(g_bwd_timeout, &zero, sizeof(zero));
+  if (e != cudaSuccess) return fail(UNIGIST_ERR_CUDA, "reading the device status: %s", cudaGetErrorString(e));
+  *timed_out = flag != 0;
+  return UNIGIST_OK;
+}
+
+}  // namespace ug

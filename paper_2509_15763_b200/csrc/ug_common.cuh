@@ -99,6 +99,11 @@ int32_t launch_fwd_simt(const Geom& g, const unigist_problem& p, float scale, co
 int32_t launch_fwd_sm100(const Geom& g, const unigist_problem& p, float scale, const void* q,
                          const void* k, const void* v, void* o, float* lse, cudaStream_t st);
 int32_t fwd_sm100_take_timeout(bool* timed_out);
+int32_t launch_bwd_sm100(const Geom& g, const unigist_problem& p, float scale, const void* q,
+                         const void* k, const void* v, const void* o, const float* lse,
+                         const void* d_o, void* dq, void* dk, void* dv, void* workspace,
+                         cudaStream_t st);
+int32_t bwd_sm100_take_timeout(bool* timed_out);
 int32_t launch_bwd_simt(const Geom& g, const unigist_problem& p, float scale, const void* q,
                         const void* k, const void* v, const void* o, const float* lse,
                         const void* d_o, void* dq, void* dk, void* dv, float* delta,
