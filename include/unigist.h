@@ -183,6 +183,34 @@ int32_t unigist_kernel_timing_count(void);
 int32_t unigist_kernel_timing_get(int32_t index, char* name, int32_t cap, float* ms);
 
 /*
+ * unigist_decode for callers that have no device memory to hand over as scratch and may not
+ * allocate any.  (The paper has no counterpart; this exists for deployment.)  Typical cases: a
+ * plugin called from inside an inference server that has already claimed the whole GPU for its
+ * own memory pool, so a cudaMalloc from the plugin would fail or stall the device; or a decode
+ * loop with a hard latency budget, where an allocation's implicit device-wide synchronisation is
+ * not acceptable.
+ *
+ * Same arguments and results as unigist_decode, minus workspace / ws_bytes.  The split-KV
+ * partial results are kept in a fixed array of UNIGIST_DECODE_STATIC_SCRATCH_BYTES bytes that is
+ * part of the library image: every GPU that loads the library holds that much global memory
+ * until the process exits.  The call allocates and frees nothing.
+ *  - A problem whose unigist_decode_workspace_bytes() exceeds the array is rejected with
+ *    UNIGIST_ERR_WORKSPACE before anything is launched (use unigist_decode, or fewer sequences).
+ *  - The first call on each device looks up the array's device address (with that device
+ *    current); make that first call outside any stream capture.
+ *  - All calls on a device share the one array.  Nothing in it has to start at zero (each call
+ *    overwrites every slot it later reads), so back-to-back calls on one stream are fine, but two
+ *    calls that may overlap on the GPU (different streams, different host threads) race on it
+ *    and must be serialised by the caller.
+ */
+#define UNIGIST_DECODE_STATIC_SCRATCH_BYTES (8u << 20)
+int32_t unigist_decode_static(int32_t num_seqs, int32_t num_q_heads, int32_t num_kv_heads,
+                              int32_t head_dim, float softmax_scale, const void* q,
+                              const void* k_cache, const void* v_cache, int32_t num_blocks,
+                              const int32_t* block_table, int32_t max_blocks_per_seq,
+                              const int32_t* seq_lens, void* o, float* lse, void* stream);
+
+/*
  * Device-side waits in the tensor-core kernels (on TMA and MMA completion barriers) are bounded:
  * a wait that does not end within about a second of SM clock makes its thread block leave early
  * and raises a flag instead of hanging the GPU.  This call synchronises the current device, then

@@ -25,7 +25,7 @@ SYMBOLS = [
     "unigist_attn_fwd", "unigist_attn_bwd", "unigist_kv_compact", "unigist_decode_workspace_bytes",
     "unigist_decode", "unigist_launch_count", "unigist_last_error_string",
     "unigist_kernel_timing", "unigist_kernel_timing_count", "unigist_kernel_timing_get",
-    "unigist_device_status",
+    "unigist_device_status", "unigist_decode_static",
 ]
 
 
@@ -92,6 +92,7 @@ def lib() -> ctypes.CDLL:
             "unigist_kernel_timing_count": (i32, []),
             "unigist_kernel_timing_get": (i32, [i32, ctypes.c_char_p, i32, ctypes.POINTER(ctypes.c_float)]),
             "unigist_device_status": (i32, []),
+            "unigist_decode_static": (i32, [i32, i32, i32, i32, f32, vp, vp, vp, i32, vp, i32, vp, vp, vp, vp]),
             "unigist_launch_count": (i64, []),
             "unigist_last_error_string": (ctypes.c_char_p, []),
         }
@@ -161,6 +162,21 @@ def unigist_kernel_timing_get(index: int):
     ms = ctypes.c_float()
     _check(lib().unigist_kernel_timing_get(index, name, 128, ctypes.byref(ms)))
     return name.value.decode(), ms.value
+
+
+DECODE_STATIC_SCRATCH_BYTES = 8 << 20
+
+
+def unigist_decode_static(q, k_cache, v_cache, block_table, seq_lens, o, lse=None,
+                          softmax_scale: float = 0.0, stream=None):
+    """unigist_decode without a workspace argument: scratch is the library's built-in array, so
+    nothing is allocated.  Calls on one device must not overlap; see include/unigist.h."""
+    _dev(q, k_cache, v_cache, block_table, seq_lens, o, lse)
+    S, Hq, D = q.shape
+    _check(lib().unigist_decode_static(S, Hq, k_cache.shape[1], D, softmax_scale, _ptr(q), _ptr(k_cache),
+                                       _ptr(v_cache), k_cache.shape[0], _ptr(block_table),
+                                       block_table.shape[1], _ptr(seq_lens), _ptr(o), _ptr(lse),
+                                       _stream(stream)))
 
 
 def unigist_device_status() -> None:

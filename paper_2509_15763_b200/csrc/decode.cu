@@ -285,3 +285,69 @@ int32_t launch_decode(int S, int Hq, int Hkv, int D, float scale, const void* q,
 }
 
 }  // namespace ug
+
+// ------------------------------------------------------------------------------------------------
+// Decode without caller-provided scratch.  The split-KV partial results go to a fixed array that
+// is part of the library image, so this entry point needs no allocation from anyone.
+#include <cmath>
+#include <mutex>
+
+namespace {
+
+// Lives in the global memory of every GPU that loads the library, from load until process exit.
+static __device__ __align__(256) unsigned char g_decode_static_scratch[UNIGIST_DECODE_STATIC_SCRATCH_BYTES];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mutex;
+void* g_static_scratch_ptr[kMaxDevices] = {};
+
+// In host code the array's name is only a handle; the device address has to be asked for, once
+// per device, with that device current.
+int32_t static_scratch_address(void** out) {
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return ug::fail(UNIGIST_ERR_CUDA, "cudaGetDevice: %s", cudaGetErrorString(e));
+  if (dev < 0 || dev >= kMaxDevices) return ug::fail(UNIGIST_ERR_UNSUPPORTED, "device ordinal %d out of range", dev);
+  std::lock_guard<std::mutex> lock(g_static_mutex);
+  if (!g_static_scratch_ptr[dev]) {
+    void* ptr = nullptr;
+    e = cudaGetSymbolAddress(&ptr, g_decode_static_scratch);
+    if (e != cudaSuccess || !ptr)
+      return ug::fail(UNIGIST_ERR_CUDA, "cudaGetSymbolAddress(static decode scratch): %s", cudaGetErrorString(e));
+    g_static_scratch_ptr[dev] = ptr;
+  }
+  *out = g_static_scratch_ptr[dev];
+  return UNIGIST_OK;
+}
+
+}  // namespace
+
+extern "C" int32_t unigist_decode_static(int32_t S, int32_t Hq, int32_t Hkv, int32_t D, float softmax_scale,
+                                         const void* q, const void* kc, const void* vc, int32_t num_blocks,
+                                         const int32_t* table, int32_t max_blocks, const int32_t* seq_lens,
+                                         void* o, float* lse, void* stream) {
+  using namespace ug;
+  if (S < 1 || Hq < 1 || Hkv < 1 || max_blocks < 1 || num_blocks < 1)
+    return fail(UNIGIST_ERR_INVALID_ARG, "decode has a non-positive size");
+  if (Hq % Hkv) return fail(UNIGIST_ERR_SHAPE, "num_q_heads %d is not a multiple of num_kv_heads %d", Hq, Hkv);
+  if (D != 128) return fail(UNIGIST_ERR_SHAPE, "decode supports head_dim 128, got %d", D);
+  const int G = Hq / Hkv;
+  if (G != 1 && G != 2 && G != 4 && G != 8)
+    return fail(UNIGIST_ERR_UNSUPPORTED, "decode supports 1, 2, 4 or 8 query heads per KV head, got %d", G);
+  if (!q || !kc || !vc || !table || !seq_lens || !o) return fail(UNIGIST_ERR_INVALID_ARG, "a pointer is NULL");
+  if (!aligned16(q) || !aligned16(kc) || !aligned16(vc) || !aligned16(o))
+    return fail(UNIGIST_ERR_ALIGNMENT, "tensor pointers must be 16-byte aligned");
+  if (!(softmax_scale >= 0.f) || std::isinf(softmax_scale))
+    return fail(UNIGIST_ERR_INVALID_ARG, "softmax_scale must be finite and >= 0");
+  const size_t need = unigist_decode_workspace_bytes(S, Hq, Hkv, D, max_blocks);
+  if (need > (size_t)UNIGIST_DECODE_STATIC_SCRATCH_BYTES)
+    return fail(UNIGIST_ERR_WORKSPACE,
+                "this decode needs %zu bytes of scratch but the built-in array holds %zu: use unigist_decode "
+                "with a caller-provided workspace, or decode fewer sequences per call",
+                need, (size_t)UNIGIST_DECODE_STATIC_SCRATCH_BYTES);
+  void* scratch = nullptr;
+  if (int32_t rc = static_scratch_address(&scratch)) return rc;
+  const float scale = softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf((float)D);
+  return launch_decode(S, Hq, Hkv, D, scale, q, kc, vc, num_blocks, table, max_blocks, seq_lens, o, lse, scratch,
+                       (cudaStream_t)stream);
+}
