@@ -196,7 +196,7 @@ attn_bwd_dkdv_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const _
       bool q_is_raw;
       int qt, head;
       tile_of(it, q_is_raw, qt, head);
-      if (it >= 2) ok = mbar_wait(bar_empty[st], ((it >> 1) - 1) & 1);
+      if (it >= 2) ok = mbar_wait_warp(bar_empty[st], ((it >> 1) - 1) & 1);
       if (!ok) break;
       const int q_seg_len = q_is_raw ? g.T : g.n, q_seg_base = q_is_raw ? g.s : g.s + g.T;
       float* ls = stats + st * 2 * KV_BN;
@@ -306,7 +306,7 @@ attn_bwd_dkdv_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const _
       const int lo = my_lo[q_is_raw ? 0 : 1] - q0 - 64 * hf, hi = my_hi[q_is_raw ? 0 : 1] - q0 - 64 * hf;
       const float* ls = stats + st * 2 * KV_BN + 64 * hf;
       const float* dl = ls + KV_BN;
-      ok = mbar_wait(bar_full[st], (it >> 1) & 1) && mbar_wait(bar_S, it & 1);
+      ok = mbar_wait_warp(bar_full[st], (it >> 1) & 1) && mbar_wait_warp(bar_S, it & 1);
       if (!ok) break;
       tc_fence_after();
       float p[64];
@@ -337,7 +337,7 @@ attn_bwd_dkdv_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const _
       tmem_wait_st();
       tc_fence_before();
       mbar_arrive(bar_P);
-      ok = mbar_wait(bar_dP, it & 1);
+      ok = mbar_wait_warp(bar_dP, it & 1);
       if (!ok) break;
       tc_fence_after();
 #pragma unroll
@@ -362,7 +362,7 @@ attn_bwd_dkdv_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const _
       tc_fence_before();
       mbar_arrive(bar_dS);
     }
-    if (ok && n_iter > 0) ok = mbar_wait(bar_final, 0);
+    if (ok && n_iter > 0) ok = mbar_wait_warp(bar_final, 0);
     if (ok) {
       tc_fence_after();
       const long long tok = (long long)b * g.N + key_seg_base + key;
@@ -555,7 +555,7 @@ attn_bwd_dq_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const __g
         lo = 0;
         hi = my.hi_gist - col0;
       }
-      ok = mbar_wait(bar_s, j & 1);
+      ok = mbar_wait_warp(bar_s, j & 1);
       if (!ok) break;
       tc_fence_after();
 #pragma unroll
@@ -584,7 +584,7 @@ attn_bwd_dq_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const __g
       tc_fence_before();
       mbar_arrive(bar_p);
     }
-    if (ok) ok = mbar_wait(bar_pv, (nt - 1) & 1);
+    if (ok) ok = mbar_wait_warp(bar_pv, (nt - 1) & 1);
     if (ok) {
       tc_fence_after();
       const long long tok = (long long)b * g.N + seg_base + row_a + r_in_tile;

@@ -199,7 +199,7 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const __grid
         lo = 0;
         hi = my.hi_gist - col0;
       }
-      ok = mbar_wait(bar_s, j & 1);
+      ok = mbar_wait_warp(bar_s, j & 1);
       if (!ok) break;
       tc_fence_after();
 
@@ -267,7 +267,7 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const __grid
       tc_fence_before();
       mbar_arrive(bar_p);
     }
-    if (ok) ok = mbar_wait(bar_pv, (nt - 1) & 1);
+    if (ok) ok = mbar_wait_warp(bar_pv, (nt - 1) & 1);
     if (ok) {
       tc_fence_after();
       const float inv_l = 1.f / l_run;
@@ -300,7 +300,10 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const __grid
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 5) tmem_dealloc(tmem, kTmemCols);
+  if (warp == 5) {
+    __syncwarp();
+    tmem_dealloc(tmem, kTmemCols);
+  }
 }
 
 }  // namespace
