@@ -1,17 +1,23 @@
 // Forward gist-masked attention on Blackwell tensor cores (tcgen05 + TMEM + TMA), no sinks.
 //
-// The SHIFTED sequence is [raw (T) | gists (n)].  A thread block owns one 128-row query tile of one
-// segment and one query head.  From the closed-form row intervals it derives the list of 128-key
-// tiles that hold a visible pair: the tile of the query rows' own segment that contains the
-// diagonal comes first (every row sees itself there, so the running maximum is finite from the
-// first tile on), then the rest; masked-out tiles are never loaded.  Per key tile:
+// The SHIFTED sequence is [raw (T) | gists (n)].  A thread block runs TWO query streams at once,
+// each a 128-row query tile of one query head: either the same tile of two neighbouring heads of
+// one KV group (when the group size is even: both streams then walk the same key tiles under the
+// same mask), or two neighbouring tiles of one head.  Both streams read the same K / V tiles, which
+// are loaded once into a ring in shared memory.  From the closed-form row intervals each stream
+// derives the interval of 128-key tiles that hold a visible pair; the block walks the union (own
+// segment first, downwards from the diagonal, then the other segment) and a stream skips the tiles
+// outside its own interval.  Masked-out tiles are never loaded.  Per key tile and stream:
 //   TMA:      K, V tiles -> shared memory (128-byte swizzle), one tensor map per segment so a tile
 //             never straddles segments and rows past a segment's end read as zero.
 //   tcgen05:  S = Q K^T into TMEM (fp32);   O += P V with P (bf16) read from TMEM.
-//   softmax:  128 threads, one query row each: row max, lazy rescale of O, exp2, row sum, P -> TMEM.
-//             Only tiles classified "partial" evaluate the mask; "full" tiles skip it.
-// Roles: warps 0-3 softmax / epilogue, warp 4 TMA producer, warp 5 MMA issuer and TMEM owner.
-// Two thread blocks share an SM (256 TMEM columns each) so one block's MMAs overlap the other's softmax.
+//   softmax:  one warpgroup per stream, one query row per thread: row max, lazy rescale of O,
+//             exp2, row sum, P -> TMEM.  Only tiles classified "partial" evaluate the mask.
+// The MMA issue order PV0(j), S0(j+1), PV1(j), S1(j+1) lets one stream's softmax run under the
+// other stream's matrix products.
+// Roles: warps 0-3 softmax of stream 0, warps 4-7 softmax of stream 1, warp 8 TMA producer,
+// warp 9 MMA issuer and TMEM owner; the third warpgroup hands most of its registers to the two
+// softmax warpgroups, which keep a whole score row (128 values) per thread.  TMEM: S0 | S1 | O0 | O1, 128 columns each.
 #include "sm100_ptx.cuh"
 #include "ug_common.cuh"
 
@@ -22,8 +28,14 @@ using namespace sm100;
 
 constexpr int BM = 128;  // query rows per tile
 constexpr int BN = 128;  // keys per tile
-constexpr int kThreads = 192;
-constexpr uint32_t kTmemCols = 256;
+constexpr int kStages = 4;  // ring slots; K and V tiles alternate through them
+constexpr int kThreads = 384;  // 3 warpgroups: softmax 0, softmax 1, {TMA, MMA, 2 idle warps}
+constexpr uint32_t kTmemCols = 512;
+// Register split after launch (168 per thread for 384 threads): the two softmax warpgroups grow, the
+// third shrinks.  The total must not exceed what the block was launched with, or the growing
+// warpgroups would wait forever.
+constexpr int kRegsLaunch = 168, kRegsSoftmax = 216, kRegsOther = 72;
+static_assert(2 * kRegsSoftmax + kRegsOther <= 3 * kRegsLaunch, "register split exceeds the block's allocation");
 constexpr float kRescaleThreshold = 8.0f;  // log2 units: O is rescaled only when the max grows by > 2^8
 
 __device__ unsigned int g_fwd_timeout = 0;
@@ -32,11 +44,43 @@ template <int D>
 struct FwdSmem {
   static constexpr int kSlab = BM * 128;          // bytes of one [128 rows x 64 bf16] slab
   static constexpr int kTile = kSlab * (D / 64);  // bytes of one [128 x D] tile
-  static constexpr int kBytes = 3 * kTile + 1024 /*align*/ + 128 /*barriers*/;
+  static constexpr int kBarOff = (2 + kStages) * kTile;
+  static constexpr int kBytes = kBarOff + 1024 /*align*/ + 256 /*barriers*/;
 };
 
-// Key tiles a query tile visits: `n_first` tiles of its own segment in descending order starting
-// at `first_hi`, then `n_second` tiles of the other segment ascending from `second_lo`.
+// One query stream: a 128-row tile of one head, with the key-tile interval it can see.
+struct Stream {
+  bool valid;
+  int h, row_a, row_b;      // head; first / last row inside the segment
+  RowIv iv_a, iv_b;         // visible intervals of the first / last row
+  int raw_lo, raw_hi, n_gist;  // raw key tiles [raw_lo, raw_hi], gist key tiles [0, n_gist)
+  __device__ bool sees(bool is_raw, int idx) const {
+    return valid && (is_raw ? (idx >= raw_lo && idx <= raw_hi) : idx < n_gist);
+  }
+};
+
+__device__ Stream make_stream(const Geom& g, bool valid, int h, int qt, bool q_is_raw) {
+  Stream s;
+  s.valid = valid;
+  s.h = h;
+  const int seg_len = q_is_raw ? g.T : g.n;
+  const int seg_base = q_is_raw ? g.s : g.s + g.T;
+  s.row_a = qt * BM;
+  s.row_b = min(s.row_a + BM - 1, seg_len - 1);
+  if (!valid) {
+    s.row_a = s.row_b = 0;
+  }
+  s.iv_a = row_intervals(g, seg_base + s.row_a);
+  s.iv_b = row_intervals(g, seg_base + s.row_b);
+  s.raw_lo = s.iv_a.lo_raw / BN;
+  s.raw_hi = s.iv_b.hi_raw / BN;
+  s.n_gist = s.iv_b.hi_gist >= 0 ? s.iv_b.hi_gist / BN + 1 : 0;
+  return s;
+}
+
+// Key tiles the block visits: the union of its streams' intervals; `n_first` tiles of the query
+// rows' own segment in descending order from `first_hi`, then `n_second` tiles of the other
+// segment ascending from `second_lo`.
 struct TileSeq {
   int n_first, first_hi, n_second, second_lo;
   bool first_is_raw;
@@ -52,10 +96,19 @@ struct TileSeq {
   }
 };
 
-__device__ TileSeq make_tile_seq(const RowIv& iv_a, const RowIv& iv_b, bool q_is_raw) {
-  const int raw_lo = iv_a.lo_raw / BN, raw_hi = iv_b.hi_raw / BN;  // hi_raw >= lo_raw always
+__device__ TileSeq make_tile_seq(const Stream& a, const Stream& b, bool q_is_raw) {
+  int raw_lo, raw_hi, n_gist;
+  if (a.valid && b.valid) {
+    raw_lo = min(a.raw_lo, b.raw_lo);
+    raw_hi = max(a.raw_hi, b.raw_hi);
+    n_gist = max(a.n_gist, b.n_gist);
+  } else {
+    const Stream& s = a.valid ? a : b;
+    raw_lo = s.raw_lo;
+    raw_hi = s.raw_hi;
+    n_gist = s.n_gist;
+  }
   const int n_raw = raw_hi - raw_lo + 1;
-  const int n_gist = iv_b.hi_gist >= 0 ? iv_b.hi_gist / BN + 1 : 0;
   TileSeq s;
   s.first_is_raw = q_is_raw;
   if (q_is_raw) {
@@ -72,235 +125,347 @@ __device__ TileSeq make_tile_seq(const RowIv& iv_a, const RowIv& iv_b, bool q_is
   return s;
 }
 
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+
+// Bit e of the result: column 32 * c + e lies inside [lo, hi].
+__device__ __forceinline__ uint32_t chunk_mask(int lo, int hi, int c) {
+  const int a = max(lo - 32 * c, 0), b = min(hi - 32 * c, 31);
+  return a > b ? 0u : ((0xffffffffu >> (31 - b)) & (0xffffffffu << a));
+}
+
+// Row maximum of the raw scores of one tile; kMasked: only columns [lo, hi] count.
+template <bool kMasked>
+__device__ __forceinline__ float row_max(const uint32_t (&sc)[BN], int lo, int hi) {
+  float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
+#pragma unroll
+  for (int c = 0; c < BN / 32; ++c) {
+    if (kMasked) {
+      const uint32_t bits = chunk_mask(lo, hi, c);
+#pragma unroll
+      for (int e = 0; e < 32; e += 2) {
+        const float x0 = (bits >> e) & 1u ? __uint_as_float(sc[c * 32 + e]) : -INFINITY;
+        const float x1 = (bits >> (e + 1)) & 1u ? __uint_as_float(sc[c * 32 + e + 1]) : -INFINITY;
+        if (e & 2) m1 = max3(m1, x0, x1); else m0 = max3(m0, x0, x1);
+      }
+    } else {
+#pragma unroll
+      for (int e = 0; e < 32; e += 8) {
+        m0 = max3(m0, __uint_as_float(sc[c * 32 + e]), __uint_as_float(sc[c * 32 + e + 1]));
+        m1 = max3(m1, __uint_as_float(sc[c * 32 + e + 2]), __uint_as_float(sc[c * 32 + e + 3]));
+        m2 = max3(m2, __uint_as_float(sc[c * 32 + e + 4]), __uint_as_float(sc[c * 32 + e + 5]));
+        m3 = max3(m3, __uint_as_float(sc[c * 32 + e + 6]), __uint_as_float(sc[c * 32 + e + 7]));
+      }
+    }
+  }
+  return fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
+}
+
+// p = 2^(s * scale_log2 - m) for one row of a tile, written to TMEM as bf16 pairs; returns the row sum.
+template <bool kMasked>
+__device__ __forceinline__ float row_exp(const uint32_t (&sc)[BN], uint32_t t_p, float scale_log2, float m, int lo,
+                                         int hi) {
+  float l0 = 0.f, l1 = 0.f, l2 = 0.f, l3 = 0.f;
+#pragma unroll
+  for (int c = 0; c < BN / 32; ++c) {
+    uint32_t bits = 0xffffffffu;
+    if (kMasked) bits = chunk_mask(lo, hi, c);
+    uint32_t pk[16];
+#pragma unroll
+    for (int e = 0; e < 32; e += 4) {
+      float x[4];
+#pragma unroll
+      for (int t = 0; t < 4; ++t) {
+        x[t] = fmaf(__uint_as_float(sc[c * 32 + e + t]), scale_log2, -m);
+        if (kMasked) x[t] = (bits >> (e + t)) & 1u ? x[t] : -INFINITY;
+        x[t] = ex2(x[t]);
+      }
+      l0 += x[0];
+      l1 += x[1];
+      l2 += x[2];
+      l3 += x[3];
+      pk[e / 2] = pack_bf16(x[0], x[1]);
+      pk[e / 2 + 1] = pack_bf16(x[2], x[3]);
+    }
+    tmem_st(t_p + c * 16, pk);
+  }
+  return (l0 + l1) + (l2 + l3);
+}
+
 template <int D>
-__global__ void __launch_bounds__(kThreads, 2)
+__global__ void __launch_bounds__(kThreads, 1)
 attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const __grid_constant__ CUtensorMap tm_q_gist,
                       const __grid_constant__ CUtensorMap tm_k_raw, const __grid_constant__ CUtensorMap tm_k_gist,
                       const __grid_constant__ CUtensorMap tm_v_raw, const __grid_constant__ CUtensorMap tm_v_gist,
                       Geom g, int Hq, int Hkv, float scale_log2, __nv_bfloat16* __restrict__ o,
-                      float* __restrict__ lse, int n_raw_qt) {
+                      float* __restrict__ lse, int n_raw_units, int n_raw_qt, int n_gist_qt, int pair_heads) {
   using SM = FwdSmem<D>;
   extern __shared__ unsigned char smem_dyn[];
   const uint32_t base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
-  const uint32_t sQ = base, sK = base + SM::kTile, sV = base + 2 * SM::kTile;
-  const uint32_t bars = base + 3 * SM::kTile;
-  const uint32_t bar_q = bars, bar_k = bars + 8, bar_v = bars + 16, bar_s = bars + 24, bar_p = bars + 32,
-                 bar_pv = bars + 40, tmem_slot = bars + 48;
+  const uint32_t sQ[2] = {base, base + SM::kTile};
+  const uint32_t ring = base + 2 * SM::kTile;
+  const uint32_t bars = base + SM::kBarOff;
+  const uint32_t bar_q = bars, bar_o = bars + 8;
+  const uint32_t bar_s[2] = {bars + 16, bars + 24}, bar_p[2] = {bars + 32, bars + 40};
+  const uint32_t bar_full = bars + 48, bar_empty = bars + 48 + 8 * kStages;  // arrays of kStages
+  const uint32_t tmem_slot = bars + 48 + 16 * kStages;
   unsigned char* gen_base = smem_dyn + (base - smem_u32(smem_dyn));
-  volatile uint32_t* tmem_slot_ptr = reinterpret_cast<volatile uint32_t*>(gen_base + 3 * SM::kTile + 48);
+  volatile uint32_t* tmem_slot_ptr =
+      reinterpret_cast<volatile uint32_t*>(gen_base + SM::kBarOff + 48 + 16 * kStages);
 
   const int warp = threadIdx.x >> 5;
-  const int h = blockIdx.y, b = blockIdx.z, hk = h / (Hq / Hkv);
-  // heaviest tiles first: gist tiles from the end, then raw tiles from the end
-  const int qt_lin = gridDim.x - 1 - blockIdx.x;
-  const bool q_is_raw = qt_lin < n_raw_qt;
-  const int qt = q_is_raw ? qt_lin : qt_lin - n_raw_qt;
-  const int seg_len = q_is_raw ? g.T : g.n;
+  const int b = blockIdx.z;
+  // heaviest units first: gist units from the end, then raw units from the end
+  const int u_lin = gridDim.x - 1 - blockIdx.x;
+  const bool q_is_raw = u_lin < n_raw_units;
+  const int u = q_is_raw ? u_lin : u_lin - n_raw_units;
+  const int n_qt = q_is_raw ? n_raw_qt : n_gist_qt;
   const int seg_base = q_is_raw ? g.s : g.s + g.T;  // shifted position of the segment's row 0
-  const int row_a = qt * BM, row_b = min(row_a + BM - 1, seg_len - 1);
-  const RowIv iv_a = row_intervals(g, seg_base + row_a), iv_b = row_intervals(g, seg_base + row_b);
-  const TileSeq seq = make_tile_seq(iv_a, iv_b, q_is_raw);
+  int qt[2], hh[2];
+  bool sv[2];
+  if (pair_heads) {
+    qt[0] = qt[1] = u;
+    hh[0] = 2 * blockIdx.y;
+    hh[1] = hh[0] + 1;
+    sv[0] = sv[1] = true;
+  } else {
+    qt[0] = 2 * u;
+    qt[1] = 2 * u + 1;
+    hh[0] = hh[1] = blockIdx.y;
+    sv[0] = true;
+    sv[1] = qt[1] < n_qt;
+  }
+  const int hk = hh[0] / (Hq / Hkv);  // both streams share the KV head
+  const Stream str0 = make_stream(g, sv[0], hh[0], qt[0], q_is_raw), str1 = make_stream(g, sv[1], hh[1], qt[1], q_is_raw);
+  const TileSeq seq = make_tile_seq(str0, str1, q_is_raw);
   const int nt = seq.count();
 
   if (threadIdx.x == 0) {
     mbar_init(bar_q, 1);
-    mbar_init(bar_k, 1);
-    mbar_init(bar_v, 1);
-    mbar_init(bar_s, 1);
-    mbar_init(bar_p, 128);
-    mbar_init(bar_pv, 1);
+    mbar_init(bar_o, 1);
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(bar_s[i], 1);
+      mbar_init(bar_p[i], 128);
+    }
+    for (int i = 0; i < kStages; ++i) {
+      mbar_init(bar_full + 8 * i, 1);
+      mbar_init(bar_empty + 8 * i, 1);
+    }
     mbar_fence_init();
   }
-  if (warp == 5) tmem_alloc(tmem_slot, kTmemCols);
+  if (warp == 9) tmem_alloc(tmem_slot, kTmemCols);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot_ptr;
-  const uint32_t tmem_S = tmem, tmem_P = tmem, tmem_O = tmem + 128;
   bool ok = true;
-
-  if (warp == 4) {
+  if (warp >= 8) {
+    reg_dealloc<kRegsOther>();
+  if (warp == 8) {
     // ------------------------------------------------------------ TMA producer
     if (elect_one()) {
       const CUtensorMap* mq = q_is_raw ? &tm_q_raw : &tm_q_gist;
-      mbar_arrive_expect_tx(bar_q, SM::kTile);
+      mbar_arrive_expect_tx(bar_q, (sv[1] ? 2 : 1) * SM::kTile);
+      for (int i = 0; i < 2; ++i) {
+        if (!sv[i]) continue;
 #pragma unroll
-      for (int sl = 0; sl < D / 64; ++sl) tma_load_4d(sQ + sl * SM::kSlab, mq, bar_q, sl * 64, h, row_a, b);
-      for (int j = 0; j < nt && ok; ++j) {
+        for (int sl = 0; sl < D / 64; ++sl)
+          tma_load_4d(sQ[i] + sl * SM::kSlab, mq, bar_q, sl * 64, hh[i], qt[i] * BM, b);
+      }
+      for (int t = 0; t < 2 * nt && ok; ++t) {  // item t: K tile of step t/2 (even t) or its V tile (odd t)
         bool is_raw;
         int idx;
-        seq.at(j, is_raw, idx);
-        const CUtensorMap* mk = is_raw ? &tm_k_raw : &tm_k_gist;
-        const CUtensorMap* mv = is_raw ? &tm_v_raw : &tm_v_gist;
-        if (j > 0) ok = mbar_wait(bar_s, (j - 1) & 1);  // S(j-1) done: K buffer free
+        seq.at(t >> 1, is_raw, idx);
+        const CUtensorMap* m = (t & 1) ? (is_raw ? &tm_v_raw : &tm_v_gist) : (is_raw ? &tm_k_raw : &tm_k_gist);
+        const int slot = t % kStages, use = t / kStages;
+        if (use > 0) ok = mbar_wait(bar_empty + 8 * slot, (use - 1) & 1);
         if (!ok) break;
-        mbar_arrive_expect_tx(bar_k, SM::kTile);
+        mbar_arrive_expect_tx(bar_full + 8 * slot, SM::kTile);
 #pragma unroll
-        for (int sl = 0; sl < D / 64; ++sl) tma_load_4d(sK + sl * SM::kSlab, mk, bar_k, sl * 64, hk, idx * BN, b);
-        if (j > 0) ok = mbar_wait(bar_pv, (j - 1) & 1);  // PV(j-1) done: V buffer free
-        if (!ok) break;
-        mbar_arrive_expect_tx(bar_v, SM::kTile);
-#pragma unroll
-        for (int sl = 0; sl < D / 64; ++sl) tma_load_4d(sV + sl * SM::kSlab, mv, bar_v, sl * 64, hk, idx * BN, b);
+        for (int sl = 0; sl < D / 64; ++sl)
+          tma_load_4d(ring + slot * SM::kTile + sl * SM::kSlab, m, bar_full + 8 * slot, sl * 64, hk, idx * BN, b);
       }
       if (!ok) atomicExch(&g_fwd_timeout, 1u);
     }
-  } else if (warp == 5) {
+  } else if (warp == 9) {
     // ------------------------------------------------------------ MMA issuer
     if (elect_one()) {
       constexpr uint32_t idesc_qk = make_idesc_bf16(BM, BN, false, false);
       constexpr uint32_t idesc_pv = make_idesc_bf16(BM, D, false, true);
-      ok = mbar_wait(bar_q, 0);
-      for (int j = 0; j < nt && ok; ++j) {
-        ok = mbar_wait(bar_k, j & 1);
-        if (!ok) break;
-        tc_fence_after();
+      int n_s[2] = {0, 0}, n_pv[2] = {0, 0};  // products issued so far per stream
+      auto issue_s = [&](int i, uint32_t sK) {
 #pragma unroll
         for (int kk = 0; kk < D / 16; ++kk) {
           const uint32_t off = (kk / 4) * SM::kSlab + (kk % 4) * 32;
-          umma_ss(tmem_S, make_smem_desc(sQ + off, 16, 1024), make_smem_desc(sK + off, 16, 1024), idesc_qk,
-                  kk > 0);
+          umma_ss(tmem + i * 128, make_smem_desc(sQ[i] + off, 16, 1024), make_smem_desc(sK + off, 16, 1024),
+                  idesc_qk, kk > 0);
         }
-        umma_commit(bar_s);
-        ok = mbar_wait(bar_p, j & 1) && mbar_wait(bar_v, j & 1);
-        if (!ok) break;
-        tc_fence_after();
+        umma_commit(bar_s[i]);
+        ++n_s[i];
+      };
+      auto issue_pv = [&](int i, uint32_t sV) {
 #pragma unroll
         for (int kk = 0; kk < BN / 16; ++kk) {
           // V tile is MN-major: 16 keys = 2048 B per k step, 64-column groups SM::kSlab apart
-          umma_ts(tmem_O, tmem_P + kk * 8, make_smem_desc(sV + kk * 2048, SM::kSlab, 1024), idesc_pv,
-                  (j > 0 || kk > 0) ? 1u : 0u);
+          umma_ts(tmem + 256 + i * 128, tmem + i * 128 + kk * 8, make_smem_desc(sV + kk * 2048, SM::kSlab, 1024),
+                  idesc_pv, (n_pv[i] > 0 || kk > 0) ? 1u : 0u);
         }
-        umma_commit(bar_pv);
+        ++n_pv[i];
+      };
+      auto slot_of = [&](int t) { return t % kStages; };
+      auto wait_full = [&](int t) { return mbar_wait(bar_full + 8 * slot_of(t), (t / kStages) & 1); };
+      bool is_raw, nx_raw = false;
+      int idx, nx_idx = 0;
+      ok = mbar_wait(bar_q, 0);
+      if (ok && nt > 0) {
+        seq.at(0, is_raw, idx);
+        ok = wait_full(0);
+        if (ok) {
+          tc_fence_after();
+          if (str0.sees(is_raw, idx)) issue_s(0, ring + slot_of(0) * SM::kTile);
+          if (str1.sees(is_raw, idx)) issue_s(1, ring + slot_of(0) * SM::kTile);
+          umma_commit(bar_empty + 8 * slot_of(0));
+        }
       }
+      for (int j = 0; j < nt && ok; ++j) {
+        seq.at(j, is_raw, idx);
+        const bool has_next = j + 1 < nt;
+        if (has_next) seq.at(j + 1, nx_raw, nx_idx);
+        const int tv = 2 * j + 1, tk = 2 * j + 2;
+        ok = wait_full(tv);
+        if (!ok) break;
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+          const Stream& si = i ? str1 : str0;
+          if (si.sees(is_raw, idx)) {
+            ok = mbar_wait(bar_p[i], n_pv[i] & 1);
+            if (!ok) break;
+            tc_fence_after();
+            issue_pv(i, ring + slot_of(tv) * SM::kTile);
+          }
+          if (i == 1) umma_commit(bar_empty + 8 * slot_of(tv));
+          if (has_next) {
+            if (i == 0) {
+              ok = wait_full(tk);
+              if (!ok) break;
+              tc_fence_after();
+            }
+            if (si.sees(nx_raw, nx_idx)) issue_s(i, ring + slot_of(tk) * SM::kTile);
+            if (i == 1) umma_commit(bar_empty + 8 * slot_of(tk));
+          }
+        }
+      }
+      if (ok) umma_commit(bar_o);
       if (!ok) atomicExch(&g_fwd_timeout, 1u);
     }
+  }
   } else {
+    reg_alloc<kRegsSoftmax>();
     // ------------------------------------------------------------ softmax + epilogue (one row per thread)
-    const int r_in_tile = threadIdx.x;  // 0..127
-    const int row = min(row_a + r_in_tile, row_b);
-    const RowIv my = row_intervals(g, seg_base + row);
-    const uint32_t lane_base = static_cast<uint32_t>(warp * 32) << 16;
-    float m_run = -INFINITY, l_run = 0.f;
+    const int i = warp >> 2;  // stream
+    const Stream me = i ? str1 : str0;
+    if (me.valid) {
+      const int r_in_tile = threadIdx.x & 127;
+      const int row = min(me.row_a + r_in_tile, me.row_b);
+      const RowIv my = row_intervals(g, seg_base + row);
+      const uint32_t lane_base = static_cast<uint32_t>((warp & 3) * 32) << 16;
+      const uint32_t tS = tmem + i * 128 + lane_base, tO = tmem + 256 + i * 128 + lane_base;
+      float m_run = -INFINITY, l_run = 0.f;
+      int cnt = 0;
 
-    for (int j = 0; j < nt && ok; ++j) {
-      bool is_raw;
-      int idx;
-      seq.at(j, is_raw, idx);
-      const int col0 = idx * BN;
-      bool full;
-      int lo, hi;  // visible columns of this row, relative to the tile
-      if (is_raw) {
-        full = col0 >= iv_b.lo_raw && col0 + BN - 1 <= iv_a.hi_raw;
-        lo = my.lo_raw - col0;
-        hi = my.hi_raw - col0;
-      } else {
-        full = col0 + BN - 1 <= iv_a.hi_gist;
-        lo = 0;
-        hi = my.hi_gist - col0;
-      }
-      ok = mbar_wait_warp(bar_s, j & 1);
-      if (!ok) break;
-      tc_fence_after();
-
-      // pass 1: row maximum of the raw scores
-      float mx = -INFINITY;
-#pragma unroll
-      for (int c = 0; c < BN / 32; ++c) {
-        uint32_t v[32];
-        tmem_ld(tmem_S + lane_base + c * 32, v);
-        tmem_wait_ld();
-        if (full) {
-#pragma unroll
-          for (int i = 0; i < 32; ++i) mx = fmaxf(mx, __uint_as_float(v[i]));
+      for (int j = 0; j < nt && ok; ++j) {
+        bool is_raw;
+        int idx;
+        seq.at(j, is_raw, idx);
+        if (!me.sees(is_raw, idx)) continue;
+        const int col0 = idx * BN;
+        bool full;
+        int lo, hi;  // visible columns of this row, relative to the tile
+        if (is_raw) {
+          full = col0 >= me.iv_b.lo_raw && col0 + BN - 1 <= me.iv_a.hi_raw;
+          lo = my.lo_raw - col0;
+          hi = my.hi_raw - col0;
         } else {
-#pragma unroll
-          for (int i = 0; i < 32; ++i) {
-            const int col = c * 32 + i;
-            const float x = (col >= lo && col <= hi) ? __uint_as_float(v[i]) : -INFINITY;
-            mx = fmaxf(mx, x);
-          }
+          full = col0 + BN - 1 <= me.iv_a.hi_gist;
+          lo = 0;
+          hi = my.hi_gist - col0;
         }
-      }
-      const float mx_s = mx * scale_log2;
-      const bool need = mx_s > m_run + kRescaleThreshold;  // also true for the first visible tile
-      if (__any_sync(0xffffffffu, need)) {
-        const float m_new = need ? mx_s : m_run;
-        const float f = need ? ex2(m_run - m_new) : 1.f;  // m_run = -inf gives 0
-        l_run *= f;
-        m_run = m_new;
-        if (j > 0) {  // S(j) complete implies PV(j-1) complete: O is stable here
+        ok = mbar_wait_warp(bar_s[i], cnt & 1);
+        if (!ok) break;
+        tc_fence_after();
+
+        // the whole score row of this tile sits in registers between the two passes
+        uint32_t sc[BN];
 #pragma unroll
-          for (int c = 0; c < D / 32; ++c) {
-            uint32_t v[32];
-            tmem_ld(tmem_O + lane_base + c * 32, v);
-            tmem_wait_ld();
-#pragma unroll
-            for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) * f);
-            tmem_st(tmem_O + lane_base + c * 32, v);
-          }
-        }
-      }
-      // pass 2: p = 2^(s * scale_log2 - m), row sum, bf16 P into TMEM (over the first 64 columns of S)
-#pragma unroll
-      for (int c = 0; c < BN / 32; ++c) {
-        uint32_t v[32];
-        tmem_ld(tmem_S + lane_base + c * 32, v);
+        for (int c = 0; c < BN / 32; ++c) tmem_ld32(tS + c * 32, sc + c * 32);
         tmem_wait_ld();
-        uint32_t pk[16];
+        const float mx = full ? row_max<false>(sc, lo, hi) : row_max<true>(sc, lo, hi);
+        const float mx_s = mx * scale_log2;
+        const bool need = mx_s > m_run + kRescaleThreshold;  // also true for the first visible tile
+        if (__any_sync(0xffffffffu, need)) {
+          const float m_new = need ? mx_s : m_run;
+          const float f = need ? ex2(m_run - m_new) : 1.f;  // m_run = -inf gives 0
+          l_run *= f;
+          m_run = m_new;
+          if (cnt > 0) {  // S of this step complete implies the previous PV complete: O is stable here
 #pragma unroll
-        for (int i = 0; i < 32; i += 2) {
-          float x0 = fmaf(__uint_as_float(v[i]), scale_log2, -m_run);
-          float x1 = fmaf(__uint_as_float(v[i + 1]), scale_log2, -m_run);
-          if (!full) {
-            const int col = c * 32 + i;
-            x0 = (col >= lo && col <= hi) ? x0 : -INFINITY;
-            x1 = (col + 1 >= lo && col + 1 <= hi) ? x1 : -INFINITY;
-          }
-          const float p0 = ex2(x0), p1 = ex2(x1);
-          l_run += p0 + p1;
-          pk[i / 2] = pack_bf16(p0, p1);
-        }
-        tmem_st(tmem_P + lane_base + c * 16, pk);
-      }
-      tmem_wait_st();
-      tc_fence_before();
-      mbar_arrive(bar_p);
-    }
-    if (ok) ok = mbar_wait_warp(bar_pv, (nt - 1) & 1);
-    if (ok) {
-      tc_fence_after();
-      const float inv_l = 1.f / l_run;
-      const bool valid = row_a + r_in_tile <= row_b;
-      const long long tok = (long long)b * g.N + seg_base + row_a + r_in_tile;
-      __nv_bfloat16* orow = o + (tok * Hq + h) * D;
+            for (int c = 0; c < D / 32; ++c) {
+              uint32_t v[32];
+              tmem_ld(tO + c * 32, v);
+              tmem_wait_ld();
 #pragma unroll
-      for (int c = 0; c < D / 32; ++c) {
-        uint32_t v[32];
-        tmem_ld(tmem_O + lane_base + c * 32, v);
-        tmem_wait_ld();
-        if (valid) {
-#pragma unroll
-          for (int i = 0; i < 32; i += 8) {
-            uint4 pk;
-            pk.x = pack_bf16(__uint_as_float(v[i]) * inv_l, __uint_as_float(v[i + 1]) * inv_l);
-            pk.y = pack_bf16(__uint_as_float(v[i + 2]) * inv_l, __uint_as_float(v[i + 3]) * inv_l);
-            pk.z = pack_bf16(__uint_as_float(v[i + 4]) * inv_l, __uint_as_float(v[i + 5]) * inv_l);
-            pk.w = pack_bf16(__uint_as_float(v[i + 6]) * inv_l, __uint_as_float(v[i + 7]) * inv_l);
-            *reinterpret_cast<uint4*>(orow + c * 32 + i) = pk;
+              for (int e = 0; e < 32; ++e) v[e] = __float_as_uint(__uint_as_float(v[e]) * f);
+              tmem_st(tO + c * 32, v);
+            }
           }
         }
+        // p = 2^(s * scale_log2 - m), row sum, bf16 P into TMEM (over the first 64 columns of S)
+        const float tile_sum = full ? row_exp<false>(sc, tS, scale_log2, m_run, lo, hi)
+                                    : row_exp<true>(sc, tS, scale_log2, m_run, lo, hi);
+        l_run += tile_sum;
+        tmem_wait_st();
+        tc_fence_before();
+        mbar_arrive(bar_p[i]);
+        ++cnt;
       }
-      if (valid)
-        lse[((long long)b * Hq + h) * g.N + seg_base + row_a + r_in_tile] =
-            (m_run + log2f(l_run)) * 0.6931471805599453f;
-    } else {
-      atomicExch(&g_fwd_timeout, 1u);
+      if (ok) ok = mbar_wait_warp(bar_o, 0);
+      if (ok) {
+        tc_fence_after();
+        const float inv_l = 1.f / l_run;
+        const bool valid = me.row_a + r_in_tile <= me.row_b;
+        const long long tok = (long long)b * g.N + seg_base + me.row_a + r_in_tile;
+        __nv_bfloat16* orow = o + (tok * Hq + me.h) * D;
+#pragma unroll
+        for (int c = 0; c < D / 32; ++c) {
+          uint32_t v[32];
+          tmem_ld(tO + c * 32, v);
+          tmem_wait_ld();
+          if (valid) {
+#pragma unroll
+            for (int e = 0; e < 32; e += 8) {
+              uint4 pk;
+              pk.x = pack_bf16(__uint_as_float(v[e]) * inv_l, __uint_as_float(v[e + 1]) * inv_l);
+              pk.y = pack_bf16(__uint_as_float(v[e + 2]) * inv_l, __uint_as_float(v[e + 3]) * inv_l);
+              pk.z = pack_bf16(__uint_as_float(v[e + 4]) * inv_l, __uint_as_float(v[e + 5]) * inv_l);
+              pk.w = pack_bf16(__uint_as_float(v[e + 6]) * inv_l, __uint_as_float(v[e + 7]) * inv_l);
+              *reinterpret_cast<uint4*>(orow + c * 32 + e) = pk;
+            }
+          }
+        }
+        if (valid)
+          lse[((long long)b * Hq + me.h) * g.N + seg_base + me.row_a + r_in_tile] =
+              (m_run + log2f(l_run)) * 0.6931471805599453f;
+      } else {
+        atomicExch(&g_fwd_timeout, 1u);
+      }
     }
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 5) {
+  if (warp == 9) {
     __syncwarp();
     tmem_dealloc(tmem, kTmemCols);
   }
@@ -345,7 +510,12 @@ int32_t launch_fwd_sm100(const Geom& g, const unigist_problem& p, float scale, c
   if (int32_t rc = encode_segment_map(&mv_raw, v, D, Hkv, g.N, B, g.s, g.T, BN)) return rc;
   if (int32_t rc = encode_segment_map(&mv_gist, v, D, Hkv, g.N, B, g.s + g.T, g.n, BN)) return rc;
   const int n_raw_qt = (g.T + BM - 1) / BM, n_gist_qt = (g.n + BM - 1) / BM;
-  dim3 grid(n_raw_qt + n_gist_qt, Hq, B);
+  // Two streams per block: neighbouring heads of a KV group when the group size is even,
+  // otherwise neighbouring query tiles of one head.
+  const int pair_heads = (Hq / Hkv) % 2 == 0 ? 1 : 0;
+  const int n_raw_units = pair_heads ? n_raw_qt : (n_raw_qt + 1) / 2;
+  const int n_gist_units = pair_heads ? n_gist_qt : (n_gist_qt + 1) / 2;
+  dim3 grid(n_raw_units + n_gist_units, pair_heads ? Hq / 2 : Hq, B);
   const float scale_log2 = scale * 1.4426950408889634f;
   auto go = [&](auto kern, size_t smem) -> int32_t {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
@@ -353,7 +523,7 @@ int32_t launch_fwd_sm100(const Geom& g, const unigist_problem& p, float scale, c
     {
       KernelScope ks("attn_fwd_sm100_kernel", st);
       kern<<<grid, kThreads, smem, st>>>(mq_raw, mq_gist, mk_raw, mk_gist, mv_raw, mv_gist, g, Hq, Hkv, scale_log2,
-                                         (__nv_bfloat16*)o, lse, n_raw_qt);
+                                         (__nv_bfloat16*)o, lse, n_raw_units, n_raw_qt, n_gist_qt, pair_heads);
     }
     return check_launch("tcgen05 forward kernel");
   };
