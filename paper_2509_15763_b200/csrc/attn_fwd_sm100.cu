@@ -15,9 +15,10 @@
 //             exp2, row sum, P -> TMEM.  Only tiles classified "partial" evaluate the mask.
 // The MMA issue order PV0(j), S0(j+1), PV1(j), S1(j+1) lets one stream's softmax run under the
 // other stream's matrix products.
-// Roles: warps 0-3 softmax of stream 0, warps 4-7 softmax of stream 1, warp 8 TMA producer,
-// warp 9 MMA issuer and TMEM owner; the third warpgroup hands most of its registers to the two
-// softmax warpgroups, which keep a whole score row (128 values) per thread.  TMEM: S0 | S1 | O0 | O1, 128 columns each.
+// Roles: one softmax warpgroup per stream (kSplit = 1: a thread owns a whole query row and keeps its
+// 128 scores of a tile in registers; kSplit = 2: two threads share a row), then one more warpgroup
+// with the TMA producer warp and the MMA issuer / TMEM owner warp, which hands most of its registers
+// to the softmax warpgroups.  TMEM: S0 | S1 | O0 | O1, 128 columns each.
 #include "sm100_ptx.cuh"
 #include "ug_common.cuh"
 
@@ -29,13 +30,19 @@ using namespace sm100;
 constexpr int BM = 128;  // query rows per tile
 constexpr int BN = 128;  // keys per tile
 constexpr int kStages = 4;  // ring slots; K and V tiles alternate through them
-constexpr int kThreads = 384;  // 3 warpgroups: softmax 0, softmax 1, {TMA, MMA, 2 idle warps}
+constexpr int kSplit = 1;              // threads per query row: each takes BN / kSplit score columns
+constexpr int kCols = BN / kSplit;     // score columns per thread and tile
+constexpr int kSmWarps = 8 * kSplit;   // softmax warps: 2 streams x kSplit column parts x 4 lane quarters
+constexpr int kTmaWarp = kSmWarps, kMmaWarp = kSmWarps + 1;
+constexpr int kThreads = (kSmWarps + 4) * 32;  // the last warpgroup: TMA warp, MMA warp, 2 idle warps
 constexpr uint32_t kTmemCols = 512;
-// Register split after launch (168 per thread for 384 threads): the two softmax warpgroups grow, the
-// third shrinks.  The total must not exceed what the block was launched with, or the growing
+// Register split after launch: the softmax warpgroups grow, the last warpgroup shrinks.  The total must not exceed what the block was launched with, or the growing
 // warpgroups would wait forever.
-constexpr int kRegsLaunch = 168, kRegsSoftmax = 216, kRegsOther = 72;
-static_assert(2 * kRegsSoftmax + kRegsOther <= 3 * kRegsLaunch, "register split exceeds the block's allocation");
+constexpr int kRegsLaunch = kSplit == 1 ? 168 : 96;  // 65536 / kThreads, rounded down to a multiple of 8
+constexpr int kRegsSoftmax = kSplit == 1 ? 216 : 104, kRegsOther = kSplit == 1 ? 72 : 64;
+static_assert(kThreads * (kRegsLaunch + 8) > 65536 && kThreads * kRegsLaunch <= 65536, "kRegsLaunch is stale");
+static_assert((kSmWarps / 4) * kRegsSoftmax + kRegsOther <= (kSmWarps / 4 + 1) * kRegsLaunch,
+              "register split exceeds the block's allocation");
 constexpr float kRescaleThreshold = 8.0f;  // log2 units: O is rescaled only when the max grows by > 2^8
 
 __device__ unsigned int g_fwd_timeout = 0;
@@ -45,7 +52,8 @@ struct FwdSmem {
   static constexpr int kSlab = BM * 128;          // bytes of one [128 rows x 64 bf16] slab
   static constexpr int kTile = kSlab * (D / 64);  // bytes of one [128 x D] tile
   static constexpr int kBarOff = (2 + kStages) * kTile;
-  static constexpr int kBytes = kBarOff + 1024 /*align*/ + 256 /*barriers*/;
+  static constexpr int kXchOff = kBarOff + 256;  // [2 streams][kSplit][128 rows] fp32 exchange slots
+  static constexpr int kBytes = kXchOff + 2 * kSplit * BM * 4 + 1024 /*align*/;
 };
 
 // One query stream: a 128-row tile of one head, with the key-tile interval it can see.
@@ -139,10 +147,10 @@ __device__ __forceinline__ uint32_t chunk_mask(int lo, int hi, int c) {
 
 // Row maximum of the raw scores of one tile; kMasked: only columns [lo, hi] count.
 template <bool kMasked>
-__device__ __forceinline__ float row_max(const uint32_t (&sc)[BN], int lo, int hi) {
+__device__ __forceinline__ float row_max(const uint32_t (&sc)[kCols], int lo, int hi) {
   float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
 #pragma unroll
-  for (int c = 0; c < BN / 32; ++c) {
+  for (int c = 0; c < kCols / 32; ++c) {
     if (kMasked) {
       const uint32_t bits = chunk_mask(lo, hi, c);
 #pragma unroll
@@ -166,11 +174,11 @@ __device__ __forceinline__ float row_max(const uint32_t (&sc)[BN], int lo, int h
 
 // p = 2^(s * scale_log2 - m) for one row of a tile, written to TMEM as bf16 pairs; returns the row sum.
 template <bool kMasked>
-__device__ __forceinline__ float row_exp(const uint32_t (&sc)[BN], uint32_t t_p, float scale_log2, float m, int lo,
+__device__ __forceinline__ float row_exp(const uint32_t (&sc)[kCols], uint32_t t_p, float scale_log2, float m, int lo,
                                          int hi) {
   float l0 = 0.f, l1 = 0.f, l2 = 0.f, l3 = 0.f;
 #pragma unroll
-  for (int c = 0; c < BN / 32; ++c) {
+  for (int c = 0; c < kCols / 32; ++c) {
     uint32_t bits = 0xffffffffu;
     if (kMasked) bits = chunk_mask(lo, hi, c);
     uint32_t pk[16];
@@ -248,7 +256,7 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const __grid
     mbar_init(bar_o, 1);
     for (int i = 0; i < 2; ++i) {
       mbar_init(bar_s[i], 1);
-      mbar_init(bar_p[i], 128);
+      mbar_init(bar_p[i], 128 * kSplit);
     }
     for (int i = 0; i < kStages; ++i) {
       mbar_init(bar_full + 8 * i, 1);
@@ -256,15 +264,15 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const __grid
     }
     mbar_fence_init();
   }
-  if (warp == 9) tmem_alloc(tmem_slot, kTmemCols);
+  if (warp == kMmaWarp) tmem_alloc(tmem_slot, kTmemCols);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot_ptr;
   bool ok = true;
-  if (warp >= 8) {
+  if (warp >= kSmWarps) {
     reg_dealloc<kRegsOther>();
-  if (warp == 8) {
+  if (warp == kTmaWarp) {
     // ------------------------------------------------------------ TMA producer
     if (elect_one()) {
       const CUtensorMap* mq = q_is_raw ? &tm_q_raw : &tm_q_gist;
@@ -290,27 +298,32 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const __grid
       }
       if (!ok) atomicExch(&g_fwd_timeout, 1u);
     }
-  } else if (warp == 9) {
+  } else if (warp == kMmaWarp) {
     // ------------------------------------------------------------ MMA issuer
     if (elect_one()) {
       constexpr uint32_t idesc_qk = make_idesc_bf16(BM, BN, false, false);
       constexpr uint32_t idesc_pv = make_idesc_bf16(BM, D, false, true);
       int n_s[2] = {0, 0}, n_pv[2] = {0, 0};  // products issued so far per stream
+      // descriptors: constant high word, low word = start address / 16 stepped per 16-element k step
+      constexpr uint32_t kHi = smem_desc_hi(1024);
+      const uint32_t q_lo[2] = {smem_desc_lo(sQ[0], 16), smem_desc_lo(sQ[1], 16)};
       auto issue_s = [&](int i, uint32_t sK) {
+        const uint32_t k_lo = smem_desc_lo(sK, 16);
 #pragma unroll
         for (int kk = 0; kk < D / 16; ++kk) {
-          const uint32_t off = (kk / 4) * SM::kSlab + (kk % 4) * 32;
-          umma_ss(tmem + i * 128, make_smem_desc(sQ[i] + off, 16, 1024), make_smem_desc(sK + off, 16, 1024),
-                  idesc_qk, kk > 0);
+          const uint32_t off = ((kk / 4) * SM::kSlab + (kk % 4) * 32) >> 4;
+          umma_ss(tmem + i * 128, smem_desc_join(q_lo[i] + off, kHi), smem_desc_join(k_lo + off, kHi), idesc_qk,
+                  kk > 0);
         }
         umma_commit(bar_s[i]);
         ++n_s[i];
       };
       auto issue_pv = [&](int i, uint32_t sV) {
+        // V tile is MN-major: 16 keys = 2048 B per k step, 64-column groups SM::kSlab apart
+        const uint32_t v_lo = smem_desc_lo(sV, SM::kSlab);
 #pragma unroll
         for (int kk = 0; kk < BN / 16; ++kk) {
-          // V tile is MN-major: 16 keys = 2048 B per k step, 64-column groups SM::kSlab apart
-          umma_ts(tmem + 256 + i * 128, tmem + i * 128 + kk * 8, make_smem_desc(sV + kk * 2048, SM::kSlab, 1024),
+          umma_ts(tmem + 256 + i * 128, tmem + i * 128 + kk * 8, smem_desc_join(v_lo + kk * (2048 >> 4), kHi),
                   idesc_pv, (n_pv[i] > 0 || kk > 0) ? 1u : 0u);
         }
         ++n_pv[i];
@@ -365,14 +378,16 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const __grid
   } else {
     reg_alloc<kRegsSoftmax>();
     // ------------------------------------------------------------ softmax + epilogue (one row per thread)
-    const int i = warp >> 2;  // stream
+    const int i = warp / (4 * kSplit);  // stream
+    const int part = (warp >> 2) % kSplit;  // which BN / kSplit columns of the row
+    float* xch = reinterpret_cast<float*>(gen_base + SM::kXchOff) + i * kSplit * BM;
     const Stream me = i ? str1 : str0;
     if (me.valid) {
-      const int r_in_tile = threadIdx.x & 127;
+      const int r_in_tile = (warp & 3) * 32 + (threadIdx.x & 31);
       const int row = min(me.row_a + r_in_tile, me.row_b);
       const RowIv my = row_intervals(g, seg_base + row);
       const uint32_t lane_base = static_cast<uint32_t>((warp & 3) * 32) << 16;
-      const uint32_t tS = tmem + i * 128 + lane_base, tO = tmem + 256 + i * 128 + lane_base;
+      const uint32_t tS = tmem + i * 128 + lane_base, tO = tmem + 256 + i * 128 + lane_base + part * (D / kSplit);
       float m_run = -INFINITY, l_run = 0.f;
       int cnt = 0;
 
@@ -386,23 +401,29 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const __grid
         int lo, hi;  // visible columns of this row, relative to the tile
         if (is_raw) {
           full = col0 >= me.iv_b.lo_raw && col0 + BN - 1 <= me.iv_a.hi_raw;
-          lo = my.lo_raw - col0;
-          hi = my.hi_raw - col0;
+          lo = my.lo_raw - col0 - part * kCols;
+          hi = my.hi_raw - col0 - part * kCols;
         } else {
           full = col0 + BN - 1 <= me.iv_a.hi_gist;
-          lo = 0;
-          hi = my.hi_gist - col0;
+          lo = -part * kCols;
+          hi = my.hi_gist - col0 - part * kCols;
         }
         ok = mbar_wait_warp(bar_s[i], cnt & 1);
         if (!ok) break;
         tc_fence_after();
 
         // the whole score row of this tile sits in registers between the two passes
-        uint32_t sc[BN];
+        uint32_t sc[kCols];
 #pragma unroll
-        for (int c = 0; c < BN / 32; ++c) tmem_ld32(tS + c * 32, sc + c * 32);
+        for (int c = 0; c < kCols / 32; ++c) tmem_ld32(tS + part * kCols + c * 32, sc + c * 32);
         tmem_wait_ld();
-        const float mx = full ? row_max<false>(sc, lo, hi) : row_max<true>(sc, lo, hi);
+        float mx = full ? row_max<false>(sc, lo, hi) : row_max<true>(sc, lo, hi);
+        if (kSplit > 1) {  // the threads that share a row agree on its maximum
+          xch[part * BM + r_in_tile] = mx;
+          named_barrier_sync(1 + i, 128 * kSplit);
+#pragma unroll
+          for (int q = 0; q < kSplit; ++q) mx = fmaxf(mx, xch[q * BM + r_in_tile]);
+        }
         const float mx_s = mx * scale_log2;
         const bool need = mx_s > m_run + kRescaleThreshold;  // also true for the first visible tile
         if (__any_sync(0xffffffffu, need)) {
@@ -412,7 +433,7 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const __grid
           m_run = m_new;
           if (cnt > 0) {  // S of this step complete implies the previous PV complete: O is stable here
 #pragma unroll
-            for (int c = 0; c < D / 32; ++c) {
+            for (int c = 0; c < D / kSplit / 32; ++c) {
               uint32_t v[32];
               tmem_ld(tO + c * 32, v);
               tmem_wait_ld();
@@ -423,8 +444,8 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const __grid
           }
         }
         // p = 2^(s * scale_log2 - m), row sum, bf16 P into TMEM (over the first 64 columns of S)
-        const float tile_sum = full ? row_exp<false>(sc, tS, scale_log2, m_run, lo, hi)
-                                    : row_exp<true>(sc, tS, scale_log2, m_run, lo, hi);
+        const float tile_sum = full ? row_exp<false>(sc, tS + part * (kCols / 2), scale_log2, m_run, lo, hi)
+                                    : row_exp<true>(sc, tS + part * (kCols / 2), scale_log2, m_run, lo, hi);
         l_run += tile_sum;
         tmem_wait_st();
         tc_fence_before();
@@ -434,12 +455,19 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const __grid
       if (ok) ok = mbar_wait_warp(bar_o, 0);
       if (ok) {
         tc_fence_after();
+        if (kSplit > 1) {  // row sum = sum of the parts (no thread reads a max slot any more: all P are consumed)
+          xch[part * BM + r_in_tile] = l_run;
+          named_barrier_sync(1 + i, 128 * kSplit);
+          l_run = 0.f;
+#pragma unroll
+          for (int q = 0; q < kSplit; ++q) l_run += xch[q * BM + r_in_tile];
+        }
         const float inv_l = 1.f / l_run;
         const bool valid = me.row_a + r_in_tile <= me.row_b;
         const long long tok = (long long)b * g.N + seg_base + me.row_a + r_in_tile;
-        __nv_bfloat16* orow = o + (tok * Hq + me.h) * D;
+        __nv_bfloat16* orow = o + (tok * Hq + me.h) * D + part * (D / kSplit);
 #pragma unroll
-        for (int c = 0; c < D / 32; ++c) {
+        for (int c = 0; c < D / kSplit / 32; ++c) {
           uint32_t v[32];
           tmem_ld(tO + c * 32, v);
           tmem_wait_ld();
@@ -455,7 +483,7 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const __grid
             }
           }
         }
-        if (valid)
+        if (valid && part == 0)
           lse[((long long)b * Hq + me.h) * g.N + seg_base + me.row_a + r_in_tile] =
               (m_run + log2f(l_run)) * 0.6931471805599453f;
       } else {
@@ -465,7 +493,7 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const __grid
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 9) {
+  if (warp == kMmaWarp) {
     __syncwarp();
     tmem_dealloc(tmem, kTmemCols);
   }
