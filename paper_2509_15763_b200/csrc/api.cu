@@ -138,6 +138,9 @@ size_t unigist_workspace_bytes(const unigist_problem* p, int32_t op) {
       size_t b = align_up((size_t)p->batch * p->num_q_heads * g.N * sizeof(float), 256);
       if (p->flags & UNIGIST_FLAG_DOUT_FP32)
         b += align_up((size_t)p->batch * g.N * p->num_q_heads * p->head_dim * 2, 256);
+      // fp32 dQ accumulator of the fused tensor-core backward (head_dim 128, no sinks)
+      if (p->head_dim == 128 && g.s == 0)
+        b += align_up((size_t)p->batch * g.N * p->num_q_heads * p->head_dim * sizeof(float), 256);
       return b;
     }
     case UNIGIST_OP_COMPACT: {

@@ -27,11 +27,14 @@ template <bool kF32>
 __global__ void __launch_bounds__(256)
 bwd_prep_kernel(int N, int Hq, int D, long long rows, const void* __restrict__ d_o,
                 const __nv_bfloat16* __restrict__ o, float* __restrict__ delta,
-                __nv_bfloat16* __restrict__ d_o_bf16) {
+                __nv_bfloat16* __restrict__ d_o_bf16, float* __restrict__ dq32) {
   const int lane = threadIdx.x & 31;
   const long long warp = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const long long nwarps = ((long long)gridDim.x * blockDim.x) >> 5;
   for (long long rw = warp; rw < rows; rw += nwarps) {  // rw = (b*N + t)*Hq + h
+    if (dq32) {  // the fused backward accumulates dQ into this fp32 buffer: start it at zero
+      for (int d = lane * 4; d < D; d += 128) *reinterpret_cast<float4*>(dq32 + rw * D + d) = make_float4(0.f, 0.f, 0.f, 0.f);
+    }
     float acc = 0.f;
     for (int d = lane * 2; d < D; d += 64) {
       float x0, x1;
@@ -618,6 +621,463 @@ attn_bwd_dq_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const __g
   }
 }
 
+// ------------------------------------------------------------------------------------------------
+// Fused backward for head_dim 128: one kernel, five matrix products per (key tile, query tile) pair.
+//
+// A thread block owns a 128-key tile of one KV head (dK, dV in TMEM for its lifetime: no atomics,
+// deterministic) and walks every 128-query tile of every query head of the group that sees it:
+//   S^T = K Q^T, dP^T = V dO^T        (both operands in shared memory)          -> TMEM
+//   P^T = exp2(S^T c - LSE)            bf16, written over S^T in TMEM
+//   dV += P^T dO                       (P^T read from TMEM)
+//   dS^T = P^T o (dP^T - Delta)        bf16, written to shared memory [key][query]
+//   dK += dS^T Q                       (dS^T from shared memory, query-contiguous = K-major A)
+//   dQ^T = K^T dS^T                    (K tile as MN-major A, dS^T as MN-major B) -> TMEM, over dP^T
+// dQ^T (head_dim x queries, fp32) is then added into an fp32 dQ buffer in global memory with
+// coalesced red.global.add (lane = head_dim index), since several key tiles contribute to one
+// query tile; a small kernel scales and rounds that buffer to bf16 afterwards.
+// MMA issue order per step i:  dV(i), S(i+1), dQ(i), dK(i), dP(i+1)  so that the exponentials of
+// step i+1 and the dQ read-out of step i run under matrix products.
+// Warps: 0-7 compute (thread = key, 64 query columns each), 8-11 dQ read-out, 12 TMA, 13 MMA.
+// Which backward head_dim 128 takes: the fused kernel below, or the two kernels above.
+constexpr bool kFusedBackward = true;
+constexpr int kFuThreads = 512;
+constexpr int kFuRegsLaunch = 128, kFuRegsCompute = 168, kFuRegsReadout = 96, kFuRegsOther = 80;
+static_assert(kFuThreads * kFuRegsLaunch == 65536, "launch register count is stale");
+static_assert(2 * kFuRegsCompute + kFuRegsReadout + kFuRegsOther <= 4 * kFuRegsLaunch,
+              "register split exceeds the block's allocation");
+
+// One 32-query chunk of P^T for one key: p = 2^(s * c - lse2[q]); kMasked: bit e of `bits` says query e sees the key.
+template <bool kMasked>
+__device__ __forceinline__ void fused_p_chunk(const uint32_t (&v)[32], const float* __restrict__ ls, float scale_log2,
+                                              uint32_t bits, float* __restrict__ p, uint32_t (&pk)[16]) {
+#pragma unroll
+  for (int i = 0; i < 32; i += 4) {
+    const float4 l4 = *reinterpret_cast<const float4*>(ls + i);
+    const float lv[4] = {l4.x, l4.y, l4.z, l4.w};
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      float x = fmaf(__uint_as_float(v[i + e]), scale_log2, -lv[e]);
+      if (kMasked) x = (bits >> (i + e)) & 1u ? x : -INFINITY;
+      p[i + e] = ex2(x);
+    }
+    pk[i / 2] = pack_bf16(p[i], p[i + 1]);
+    pk[i / 2 + 1] = pack_bf16(p[i + 2], p[i + 3]);
+  }
+}
+
+struct FuSmem {
+  static constexpr int kSlab = 128 * 128;    // [128 rows x 64 bf16]
+  static constexpr int kTile = 2 * kSlab;    // [128 x 128] bf16
+  static constexpr int kOffK = 0, kOffV = kTile, kOffQ = 2 * kTile, kOffDO = 4 * kTile, kOffDS = 6 * kTile;
+  static constexpr int kOffStats = 7 * kTile;             // [stage][lse2 | delta][128] fp32
+  static constexpr int kOffBars = kOffStats + 2 * 2 * 128 * 4;
+  static constexpr int kUsed = kOffBars + 192;
+  static constexpr int kBytes = 232448;  // all a block may have; the 1024-byte alignment slack comes out of it
+};
+
+__global__ void __launch_bounds__(kFuThreads, 1)
+attn_bwd_fused_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const __grid_constant__ CUtensorMap tm_q_gist,
+                            const __grid_constant__ CUtensorMap tm_do_raw, const __grid_constant__ CUtensorMap tm_do_gist,
+                            const __grid_constant__ CUtensorMap tm_k_raw, const __grid_constant__ CUtensorMap tm_k_gist,
+                            const __grid_constant__ CUtensorMap tm_v_raw, const __grid_constant__ CUtensorMap tm_v_gist,
+                            Geom g, int Hq, int Hkv, float scale, const float* __restrict__ lse,
+                            const float* __restrict__ delta, float* __restrict__ dq32,
+                            __nv_bfloat16* __restrict__ dk, __nv_bfloat16* __restrict__ dv, int n_gist_kt) {
+  using SM = FuSmem;
+  constexpr int D = 128;
+  extern __shared__ unsigned char smem_dyn[];
+  const uint32_t raw_base = smem_u32(smem_dyn);
+  const uint32_t base = (raw_base + 1023u) & ~1023u;
+  if (base - raw_base + SM::kUsed > SM::kBytes) {  // cannot happen with a 1024-aligned window; never run past it
+    if (threadIdx.x == 0) atomicExch(&g_bwd_timeout, 1u);
+    return;
+  }
+  unsigned char* gen = smem_dyn + (base - raw_base);
+  const uint32_t sK = base + SM::kOffK, sV = base + SM::kOffV, sDS = base + SM::kOffDS;
+  const uint32_t sQ0 = base + SM::kOffQ, sDO0 = base + SM::kOffDO;  // stage st at + st * kTile
+  float* stats = reinterpret_cast<float*>(gen + SM::kOffStats);
+  const uint32_t bars = base + SM::kOffBars;
+  const uint32_t bar_kv = bars, bar_S = bars + 8, bar_dP = bars + 16, bar_P = bars + 24, bar_dS = bars + 32,
+                 bar_dSfree = bars + 40, bar_dQ = bars + 48, bar_dQfree = bars + 56, bar_final = bars + 64;
+  const uint32_t full_q0 = bars + 72, empty_q0 = bars + 88, full_do0 = bars + 104, empty_do0 = bars + 120;  // + 8 * st
+  const uint32_t tmem_slot = bars + 136;
+  volatile uint32_t* tmem_slot_ptr = reinterpret_cast<volatile uint32_t*>(gen + SM::kOffBars + 136);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  // blockIdx.x = key tile rank * Hkv + KV head.  Gist key tiles are seen by every later query: they are
+  // the heaviest and come first, for all KV heads, before any raw key tile.
+  const int hk = blockIdx.x % Hkv, rank = blockIdx.x / Hkv, b = blockIdx.z, G = Hq / Hkv;
+  const bool key_is_raw = rank >= n_gist_kt;
+  const int kt = key_is_raw ? rank - n_gist_kt : rank;
+  const int key_seg_len = key_is_raw ? g.T : g.n;
+  const int key_seg_base = key_is_raw ? g.s : g.s + g.T;
+  const int key_a = kt * 128, key_b = min(key_a + 127, key_seg_len - 1);
+  const bool key_tile_whole = key_a + 127 <= key_seg_len - 1;
+
+  // query tiles that see this key tile, per query segment
+  int a_lo, a_hi, b_lo, b_hi, c_lo, c_hi, d_lo, d_hi;
+  key_q_interval(g, key_is_raw, key_a, true, true, a_lo, a_hi);   // first key vs raw queries
+  key_q_interval(g, key_is_raw, key_b, true, true, b_lo, b_hi);   // last key vs raw queries
+  key_q_interval(g, key_is_raw, key_a, true, false, c_lo, c_hi);  // first key vs gist queries
+  key_q_interval(g, key_is_raw, key_b, true, false, d_lo, d_hi);  // last key vs gist queries
+  const int n_raw_q = b_hi >= a_lo ? b_hi / 128 - a_lo / 128 + 1 : 0;
+  const int rq_lo = a_lo / 128;
+  const int n_gist_q = d_hi >= c_lo ? d_hi / 128 - c_lo / 128 + 1 : 0;
+  const int gq_lo = c_lo / 128;
+  const int n_iter = (n_raw_q + n_gist_q) * G;
+
+  if (threadIdx.x == 0) {
+    mbar_init(bar_kv, 1);
+    mbar_init(bar_S, 1);
+    mbar_init(bar_dP, 1);
+    mbar_init(bar_P, 256);
+    mbar_init(bar_dS, 256);
+    mbar_init(bar_dSfree, 1);
+    mbar_init(bar_dQ, 1);
+    mbar_init(bar_dQfree, 128);
+    mbar_init(bar_final, 1);
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(full_q0 + 8 * i, 1);
+      mbar_init(empty_q0 + 8 * i, 1);
+      mbar_init(full_do0 + 8 * i, 1);
+      mbar_init(empty_do0 + 8 * i, 1);
+    }
+    mbar_fence_init();
+  }
+  if (warp == 13) tmem_alloc(tmem_slot, 512);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot_ptr;
+  const uint32_t t_dK = tmem, t_dV = tmem + 128, t_S = tmem + 256, t_dP = tmem + 384;
+  bool ok = true;
+
+  // Step order: raw query tiles from the last one down, then gist query tiles from the last one down, the
+  // G heads of a tile back to back.  Every key tile's visible range ends at the last tile of a segment, so
+  // thread blocks that run side by side walk the same Q / dO / dQ tiles at the same time and share them in L2.
+  auto tile_of = [&](int it, bool& q_is_raw, int& qt, int& head) {
+    const int t = it / G;
+    head = hk * G + (it - t * G);
+    q_is_raw = t < n_raw_q;
+    qt = q_is_raw ? rq_lo + (n_raw_q - 1 - t) : gq_lo + (n_gist_q - 1 - (t - n_raw_q));
+  };
+
+  if (warp >= 12) {
+    reg_dealloc<kFuRegsOther>();
+    if (warp == 12) {
+      // ---------------------------------------------------------- producer: K, V once; Q, dO, LSE, Delta per step
+      if (lane == 0) {
+        mbar_arrive_expect_tx(bar_kv, 2 * SM::kTile);
+        const CUtensorMap* mk = key_is_raw ? &tm_k_raw : &tm_k_gist;
+        const CUtensorMap* mv = key_is_raw ? &tm_v_raw : &tm_v_gist;
+#pragma unroll
+        for (int sl = 0; sl < 2; ++sl) {
+          tma_load_4d(sK + sl * SM::kSlab, mk, bar_kv, sl * 64, hk, key_a, b);
+          tma_load_4d(sV + sl * SM::kSlab, mv, bar_kv, sl * 64, hk, key_a, b);
+        }
+      }
+      for (int it = 0; it < n_iter; ++it) {
+        const int st = it & 1;
+        bool q_is_raw;
+        int qt, head;
+        tile_of(it, q_is_raw, qt, head);
+        if (it >= 2) ok = mbar_wait_warp(empty_q0 + 8 * st, ((it >> 1) - 1) & 1);
+        if (!ok) break;
+        const int q_seg_len = q_is_raw ? g.T : g.n, q_seg_base = q_is_raw ? g.s : g.s + g.T;
+        float* ls = stats + st * 256;
+        const long long row_base = ((long long)b * Hq + head) * g.N + q_seg_base;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const int c = lane + 32 * i, row = qt * 128 + c;
+          const bool valid = row < q_seg_len;
+          // rows past the segment get LSE = +inf, so their P is exactly zero
+          ls[c] = valid ? lse[row_base + row] * kLog2e : INFINITY;
+          ls[128 + c] = valid ? delta[row_base + row] : 0.f;
+        }
+        __syncwarp();
+        if (lane == 0) {
+          mbar_arrive_expect_tx(full_q0 + 8 * st, SM::kTile);
+          const CUtensorMap* mq = q_is_raw ? &tm_q_raw : &tm_q_gist;
+#pragma unroll
+          for (int sl = 0; sl < 2; ++sl)
+            tma_load_4d(sQ0 + st * SM::kTile + sl * SM::kSlab, mq, full_q0 + 8 * st, sl * 64, head, qt * 128, b);
+        }
+        if (it >= 2) ok = mbar_wait_warp(empty_do0 + 8 * st, ((it >> 1) - 1) & 1);
+        if (!ok) break;
+        if (lane == 0) {
+          mbar_arrive_expect_tx(full_do0 + 8 * st, SM::kTile);
+          const CUtensorMap* md = q_is_raw ? &tm_do_raw : &tm_do_gist;
+#pragma unroll
+          for (int sl = 0; sl < 2; ++sl)
+            tma_load_4d(sDO0 + st * SM::kTile + sl * SM::kSlab, md, full_do0 + 8 * st, sl * 64, head, qt * 128, b);
+        }
+        __syncwarp();
+      }
+      if (!ok && lane == 0) atomicExch(&g_bwd_timeout, 1u);
+    } else if (warp == 13) {
+      // ---------------------------------------------------------- MMA issuer
+      if (lane == 0) {
+        constexpr uint32_t idesc_s = make_idesc_bf16(128, 128, false, false);   // K-major A and B
+        constexpr uint32_t idesc_acc = make_idesc_bf16(128, 128, false, true);  // K-major A, MN-major B
+        constexpr uint32_t idesc_dq = make_idesc_bf16(128, 128, true, true);    // MN-major A and B
+        constexpr uint32_t kHi = smem_desc_hi(1024);
+        constexpr uint32_t kStage = SM::kTile >> 4;  // stage st of Q / dO: + st * kStage on the low word
+        const uint32_t k_lo = smem_desc_lo(sK, 16), v_lo = smem_desc_lo(sV, 16);
+        const uint32_t kT_lo = smem_desc_lo(sK, SM::kSlab);    // K tile read as MN-major A (head_dim contiguous)
+        const uint32_t ds_lo = smem_desc_lo(sDS, 16);          // dS^T as K-major A (queries contiguous)
+        const uint32_t dsT_lo = smem_desc_lo(sDS, SM::kSlab);  // dS^T as MN-major B
+        const uint32_t q_lo = smem_desc_lo(sQ0, 16), qT_lo = smem_desc_lo(sQ0, SM::kSlab);
+        const uint32_t do_lo = smem_desc_lo(sDO0, 16), doT_lo = smem_desc_lo(sDO0, SM::kSlab);
+        // K-major operands step 32 B per 16 elements inside a 64-element slab; MN-major ones 2048 B
+        auto koff = [](int kk) { return (uint32_t)(((kk / 4) * SM::kSlab + (kk % 4) * 32) >> 4); };
+        auto moff = [](int kk) { return (uint32_t)((kk * 2048) >> 4); };
+        // bf16 pairs of P^T in TMEM: query columns [0,64) packed at [0,32), [64,128) at [64,96)
+        auto a_col = [](int kk) { return (uint32_t)((kk / 4) * 64 + (kk % 4) * 8); };
+        auto issue_S = [&](int st) {
+#pragma unroll
+          for (int kk = 0; kk < 8; ++kk)
+            umma_ss(t_S, smem_desc_join(k_lo + koff(kk), kHi), smem_desc_join(q_lo + st * kStage + koff(kk), kHi),
+                    idesc_s, kk > 0);
+          umma_commit(bar_S);
+        };
+        auto issue_dP = [&](int st) {
+#pragma unroll
+          for (int kk = 0; kk < 8; ++kk)
+            umma_ss(t_dP, smem_desc_join(v_lo + koff(kk), kHi), smem_desc_join(do_lo + st * kStage + koff(kk), kHi),
+                    idesc_s, kk > 0);
+          umma_commit(bar_dP);
+        };
+        ok = mbar_wait(bar_kv, 0);
+        if (ok && n_iter > 0) {
+          ok = mbar_wait(full_q0, 0);
+          if (ok) {
+            tc_fence_after();
+            issue_S(0);
+            ok = mbar_wait(full_do0, 0);
+          }
+          if (ok) {
+            tc_fence_after();
+            issue_dP(0);
+          }
+        }
+        for (int it = 0; it < n_iter && ok; ++it) {
+          const int st = it & 1, ph = it & 1;
+          const bool has_next = it + 1 < n_iter;
+          ok = mbar_wait(bar_P, ph);
+          if (!ok) break;
+          tc_fence_after();
+#pragma unroll
+          for (int kk = 0; kk < 8; ++kk)  // dV += P^T dO
+            umma_ts(t_dV, t_S + a_col(kk), smem_desc_join(doT_lo + st * kStage + moff(kk), kHi), idesc_acc,
+                    (it > 0 || kk > 0) ? 1u : 0u);
+          umma_commit(empty_do0 + 8 * st);
+          if (has_next) {
+            ok = mbar_wait(full_q0 + 8 * (st ^ 1), ((it + 1) >> 1) & 1);
+            if (!ok) break;
+            tc_fence_after();
+            issue_S(st ^ 1);
+          }
+          ok = mbar_wait(bar_dS, ph);
+          if (!ok) break;
+          tc_fence_after();
+#pragma unroll
+          for (int kk = 0; kk < 8; ++kk)  // dQ^T = K^T dS^T  (contraction over the 128 keys)
+            umma_ss(t_dP, smem_desc_join(kT_lo + moff(kk), kHi), smem_desc_join(dsT_lo + moff(kk), kHi), idesc_dq,
+                    kk > 0);
+          umma_commit(bar_dQ);
+#pragma unroll
+          for (int kk = 0; kk < 8; ++kk)  // dK += dS^T Q  (contraction over the 128 queries)
+            umma_ss(t_dK, smem_desc_join(ds_lo + koff(kk), kHi), smem_desc_join(qT_lo + st * kStage + moff(kk), kHi),
+                    idesc_acc, (it > 0 || kk > 0) ? 1u : 0u);
+          umma_commit(empty_q0 + 8 * st);
+          umma_commit(bar_dSfree);
+          if (has_next) {
+            ok = mbar_wait(bar_dQfree, ph) && mbar_wait(full_do0 + 8 * (st ^ 1), ((it + 1) >> 1) & 1);
+            if (!ok) break;
+            tc_fence_after();
+            issue_dP(st ^ 1);
+          }
+        }
+        if (ok) umma_commit(bar_final);
+        if (!ok) atomicExch(&g_bwd_timeout, 1u);
+      }
+    }
+  } else if (warp >= 8) {
+    // ------------------------------------------------------------ dQ read-out: lane = head_dim index
+    reg_dealloc<kFuRegsReadout>();
+    const int qd = warp & 3;
+    const int dcol = qd * 32 + lane;
+    const uint32_t lane_base = static_cast<uint32_t>(qd * 32) << 16;
+    for (int it = 0; it < n_iter && ok; ++it) {
+      bool q_is_raw;
+      int qt, head;
+      tile_of(it, q_is_raw, qt, head);
+      const int q_seg_len = q_is_raw ? g.T : g.n, q_seg_base = q_is_raw ? g.s : g.s + g.T;
+      const int q0 = qt * 128;
+      const int nq = min(128, q_seg_len - q0);
+      float* dst = dq32 + (((long long)b * g.N + q_seg_base + q0) * Hq + head) * D + dcol;
+      const long long row_stride = (long long)Hq * D;
+      ok = mbar_wait_warp(bar_dQ, it & 1);
+      if (!ok) break;
+      tc_fence_after();
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        uint32_t v[32];
+        tmem_ld32(t_dP + lane_base + 32 * c, v);
+        tmem_wait_ld();
+        if (c == 3) {
+          // everything is in registers: the columns may be overwritten.  A releasing arrival would
+          // first wait for the reductions below (and of the earlier chunks) to be performed.
+          tc_fence_before();
+          mbar_arrive_relaxed(bar_dQfree);
+        }
+        if (32 * c < nq) {
+#pragma unroll
+          for (int e = 0; e < 32; ++e) {
+            if (32 * c + e < nq) atomicAdd(dst + (32 * c + e) * row_stride, __uint_as_float(v[e]));
+          }
+        }
+      }
+    }
+    if (!ok && lane == 0) atomicExch(&g_bwd_timeout, 1u);
+  } else {
+    // ------------------------------------------------------------ compute: thread = key (TMEM lane), 64 query columns
+    reg_alloc<kFuRegsCompute>();
+    const int qd = warp & 3, hf = warp >> 2;
+    const int krow = qd * 32 + lane;
+    const int key = key_a + krow;
+    const bool key_valid = key <= key_b;
+    const uint32_t lane_base = static_cast<uint32_t>(qd * 32) << 16;
+    const float scale_log2 = scale * kLog2e;
+    int my_lo_r, my_hi_r, my_lo_g, my_hi_g;  // queries that see this key: raw segment, gist segment
+    key_q_interval(g, key_is_raw, key, key_valid, true, my_lo_r, my_hi_r);
+    key_q_interval(g, key_is_raw, key, key_valid, false, my_lo_g, my_hi_g);
+    // this thread's row of the dS^T tile in shared memory: slab hf, row krow, 16-byte chunks swizzled by row
+    unsigned char* ds_row = gen + SM::kOffDS + hf * SM::kSlab + krow * 128;
+    const int swz = krow & 7;
+
+    for (int it = 0; it < n_iter && ok; ++it) {
+      const int st = it & 1;
+      bool q_is_raw;
+      int qt, head;
+      tile_of(it, q_is_raw, qt, head);
+      const int q0 = qt * 128, q_seg_len = q_is_raw ? g.T : g.n;
+      const int qb = min(q0 + 127, q_seg_len - 1);
+      // full: every (query, key) pair of the tile is visible -> no mask arithmetic
+      const int t_lo = q_is_raw ? b_lo : d_lo, t_hi = q_is_raw ? a_hi : c_hi;
+      const bool full = key_tile_whole && q0 >= t_lo && qb <= t_hi;
+      const int lo = (q_is_raw ? my_lo_r : my_lo_g) - q0 - 64 * hf, hi = (q_is_raw ? my_hi_r : my_hi_g) - q0 - 64 * hf;
+      const float* ls = stats + st * 256 + 64 * hf;
+      const float* dl = ls + 128;
+      ok = mbar_wait_warp(full_q0 + 8 * st, (it >> 1) & 1) && mbar_wait_warp(bar_S, it & 1);
+      if (!ok) break;
+      tc_fence_after();
+      float p[64];
+#pragma unroll
+      for (int c = 0; c < 2; ++c) {
+        uint32_t v[32];
+        tmem_ld32(t_S + lane_base + 64 * hf + 32 * c, v);
+        tmem_wait_ld();
+        uint32_t pk[16];
+        if (full) {
+          fused_p_chunk<false>(v, ls + 32 * c, scale_log2, 0u, p + 32 * c, pk);
+        } else {
+          const int a = max(lo - 32 * c, 0), bb = min(hi - 32 * c, 31);
+          const uint32_t bits = a > bb ? 0u : ((0xffffffffu >> (31 - bb)) & (0xffffffffu << a));
+          fused_p_chunk<true>(v, ls + 32 * c, scale_log2, bits, p + 32 * c, pk);
+        }
+        tmem_st(t_S + lane_base + 64 * hf + 16 * c, pk);
+      }
+      tmem_wait_st();
+      tc_fence_before();
+      mbar_arrive(bar_P);
+      ok = mbar_wait_warp(bar_dP, it & 1);
+      if (ok && it > 0) ok = mbar_wait_warp(bar_dSfree, (it - 1) & 1);  // the previous dS^T has been consumed
+      if (!ok) break;
+      tc_fence_after();
+#pragma unroll
+      for (int c = 0; c < 2; ++c) {
+        uint32_t v[32];
+        tmem_ld32(t_dP + lane_base + 64 * hf + 32 * c, v);
+        tmem_wait_ld();
+#pragma unroll
+        for (int i = 0; i < 32; i += 8) {  // 8 queries = one 16-byte chunk of this key's dS^T row
+          const float4 d0 = *reinterpret_cast<const float4*>(dl + 32 * c + i);
+          const float4 d1 = *reinterpret_cast<const float4*>(dl + 32 * c + i + 4);
+          const float* pp = p + 32 * c + i;
+          uint4 w;
+          w.x = pack_bf16(pp[0] * (__uint_as_float(v[i]) - d0.x), pp[1] * (__uint_as_float(v[i + 1]) - d0.y));
+          w.y = pack_bf16(pp[2] * (__uint_as_float(v[i + 2]) - d0.z), pp[3] * (__uint_as_float(v[i + 3]) - d0.w));
+          w.z = pack_bf16(pp[4] * (__uint_as_float(v[i + 4]) - d1.x), pp[5] * (__uint_as_float(v[i + 5]) - d1.y));
+          w.w = pack_bf16(pp[6] * (__uint_as_float(v[i + 6]) - d1.z), pp[7] * (__uint_as_float(v[i + 7]) - d1.w));
+          const int chunk = 4 * c + i / 8;
+          *reinterpret_cast<uint4*>(ds_row + ((chunk ^ swz) << 4)) = w;
+        }
+      }
+      tc_fence_before();  // the dP^T columns may be overwritten (by dQ^T) once every thread has arrived
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // dS^T visible to the tensor core's reads
+      mbar_arrive(bar_dS);
+    }
+    if (ok && n_iter > 0) ok = mbar_wait_warp(bar_final, 0);
+    if (ok) {
+      tc_fence_after();
+      const long long tok = (long long)b * g.N + key_seg_base + key;
+      // this warp stores columns [64 hf, 64 hf + 64) of dK and of dV
+#pragma unroll
+      for (int which = 0; which < 2; ++which) {
+        const bool is_dk = which == 0;
+        const uint32_t tsrc = (is_dk ? t_dK : t_dV) + lane_base + 64 * hf;
+        __nv_bfloat16* dst = (is_dk ? dk : dv) + (tok * Hkv + hk) * D + 64 * hf;
+        const float mul = is_dk ? scale : 1.f;
+#pragma unroll
+        for (int c = 0; c < 2; ++c) {
+          uint32_t v[32];
+          if (n_iter > 0) {
+            tmem_ld32(tsrc + 32 * c, v);
+            tmem_wait_ld();
+          } else {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) v[i] = 0u;
+          }
+          if (key_valid) {
+#pragma unroll
+            for (int i = 0; i < 32; i += 8) {
+              uint4 pk;
+              pk.x = pack_bf16(__uint_as_float(v[i]) * mul, __uint_as_float(v[i + 1]) * mul);
+              pk.y = pack_bf16(__uint_as_float(v[i + 2]) * mul, __uint_as_float(v[i + 3]) * mul);
+              pk.z = pack_bf16(__uint_as_float(v[i + 4]) * mul, __uint_as_float(v[i + 5]) * mul);
+              pk.w = pack_bf16(__uint_as_float(v[i + 6]) * mul, __uint_as_float(v[i + 7]) * mul);
+              *reinterpret_cast<uint4*>(dst + 32 * c + i) = pk;
+            }
+          }
+        }
+      }
+    } else {
+      atomicExch(&g_bwd_timeout, 1u);
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 13) {
+    __syncwarp();
+    tmem_dealloc(tmem, 512);
+  }
+}
+
+// dQ (bf16) = scale * dQ accumulated in fp32; 8 elements per thread.
+__global__ void __launch_bounds__(256)
+dq_convert_kernel(const float4* __restrict__ src, uint4* __restrict__ dst, long long n8, float scale) {
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n8; i += (long long)gridDim.x * blockDim.x) {
+    const float4 a = __ldcs(src + 2 * i), c = __ldcs(src + 2 * i + 1);
+    uint4 o;
+    o.x = pack_bf16(a.x * scale, a.y * scale);
+    o.y = pack_bf16(a.z * scale, a.w * scale);
+    o.z = pack_bf16(c.x * scale, c.y * scale);
+    o.w = pack_bf16(c.z * scale, c.w * scale);
+    dst[i] = o;
+  }
+}
+
 }  // namespace
 
 int32_t launch_bwd_sm100(const Geom& g, const unigist_problem& p, float scale, const void* q, const void* k,
@@ -629,14 +1089,17 @@ int32_t launch_bwd_sm100(const Geom& g, const unigist_problem& p, float scale, c
   const size_t delta_bytes = ((size_t)B * Hq * g.N * sizeof(float) + 255) / 256 * 256;
   __nv_bfloat16* do_bf16 = reinterpret_cast<__nv_bfloat16*>(static_cast<char*>(workspace) + delta_bytes);
   const void* do_src = f32 ? static_cast<const void*>(do_bf16) : d_o;
+  const size_t do_bytes = f32 ? ((size_t)B * g.N * Hq * D * 2 + 255) / 256 * 256 : 0;
+  const bool fused = kFusedBackward && D == 128;  // head_dim 64 keeps the two-kernel path
+  float* dq32 = fused ? reinterpret_cast<float*>(static_cast<char*>(workspace) + delta_bytes + do_bytes) : nullptr;
   {
     const long long rows = (long long)B * g.N * Hq;
     const int blocks = (int)((rows + 7) / 8 < 148 * 16 ? (rows + 7) / 8 : 148 * 16);
     KernelScope ks("bwd_prep_kernel", st);
     if (f32)
-      bwd_prep_kernel<true><<<blocks, 256, 0, st>>>(g.N, Hq, D, rows, d_o, (const __nv_bfloat16*)o, delta, do_bf16);
+      bwd_prep_kernel<true><<<blocks, 256, 0, st>>>(g.N, Hq, D, rows, d_o, (const __nv_bfloat16*)o, delta, do_bf16, dq32);
     else
-      bwd_prep_kernel<false><<<blocks, 256, 0, st>>>(g.N, Hq, D, rows, d_o, (const __nv_bfloat16*)o, delta, nullptr);
+      bwd_prep_kernel<false><<<blocks, 256, 0, st>>>(g.N, Hq, D, rows, d_o, (const __nv_bfloat16*)o, delta, nullptr, dq32);
   }
   if (int32_t rc = check_launch("backward prep kernel")) return rc;
 
@@ -674,12 +1137,32 @@ int32_t launch_bwd_sm100(const Geom& g, const unigist_problem& p, float scale, c
     }
     return check_launch("tcgen05 dQ kernel");
   };
-  if (D == 64) {
+  if (!fused && D == 64) {
     if (int32_t rc = go_kv(attn_bwd_dkdv_sm100_kernel<64>, KvSmem<64>::kBytes)) return rc;
     return go_q(attn_bwd_dq_sm100_kernel<64>, DqSmem<64>::kBytes);
   }
-  if (int32_t rc = go_kv(attn_bwd_dkdv_sm100_kernel<128>, KvSmem<128>::kBytes)) return rc;
-  return go_q(attn_bwd_dq_sm100_kernel<128>, DqSmem<128>::kBytes);
+  if (!fused) {
+    if (int32_t rc = go_kv(attn_bwd_dkdv_sm100_kernel<128>, KvSmem<128>::kBytes)) return rc;
+    return go_q(attn_bwd_dq_sm100_kernel<128>, DqSmem<128>::kBytes);
+  }
+  cudaError_t e = cudaFuncSetAttribute(attn_bwd_fused_sm100_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       FuSmem::kBytes);
+  if (e != cudaSuccess) return fail(UNIGIST_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
+  {
+    KernelScope ks("attn_bwd_fused_sm100_kernel", st);
+    attn_bwd_fused_sm100_kernel<<<dim3((n_raw_t + n_gist_t) * Hkv, 1, B), kFuThreads, FuSmem::kBytes, st>>>(
+        mq[0], mq[1], md[0], md[1], mk[0], mk[1], mv[0], mv[1], g, Hq, Hkv, scale, lse, delta, dq32,
+        (__nv_bfloat16*)dk, (__nv_bfloat16*)dv, n_gist_t);
+  }
+  if (int32_t rc = check_launch("tcgen05 fused backward kernel")) return rc;
+  {
+    const long long n8 = (long long)B * g.N * Hq * D / 8;
+    const int blocks = (int)((n8 + 255) / 256 < 148 * 16 ? (n8 + 255) / 256 : 148 * 16);
+    KernelScope ks("dq_convert_kernel", st);
+    dq_convert_kernel<<<blocks, 256, 0, st>>>(reinterpret_cast<const float4*>(dq32), reinterpret_cast<uint4*>(dq), n8,
+                                              scale);
+  }
+  return check_launch("dQ convert kernel");
 }
 
 int32_t bwd_sm100_take_timeout(bool* timed_out) {
