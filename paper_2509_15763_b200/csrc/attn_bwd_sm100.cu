@@ -632,9 +632,9 @@ attn_bwd_dq_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const __g
 //   dS^T = P^T o (dP^T - Delta)        bf16, written to shared memory [key][query]
 //   dK += dS^T Q                       (dS^T from shared memory, query-contiguous = K-major A)
 //   dQ^T = K^T dS^T                    (K tile as MN-major A, dS^T as MN-major B) -> TMEM, over dP^T
-// dQ^T (head_dim x queries, fp32) is then added into an fp32 dQ buffer in global memory with
-// coalesced red.global.add (lane = head_dim index), since several key tiles contribute to one
-// query tile; a small kernel scales and rounds that buffer to bf16 afterwards.
+// dQ^T (head_dim x queries, fp32) is then added into an fp32 dQ buffer in global memory by TMA
+// reductions from small staging buffers, since several key tiles contribute to one query tile; a
+// small kernel scales and rounds that buffer to bf16 afterwards.
 // MMA issue order per step i:  dV(i), S(i+1), dQ(i), dK(i), dP(i+1)  so that the exponentials of
 // step i+1 and the dQ read-out of step i run under matrix products.
 // Warps: 0-7 compute (thread = key, 64 query columns each), 8-11 dQ read-out, 12 TMA, 13 MMA.
@@ -668,7 +668,8 @@ __device__ __forceinline__ void fused_p_chunk(const uint32_t (&v)[32], const flo
 struct FuSmem {
   static constexpr int kSlab = 128 * 128;    // [128 rows x 64 bf16]
   static constexpr int kTile = 2 * kSlab;    // [128 x 128] bf16
-  static constexpr int kOffK = 0, kOffV = kTile, kOffQ = 2 * kTile, kOffDO = 4 * kTile, kOffDS = 6 * kTile;
+  static constexpr int kOffK = 0, kOffV = kTile, kOffQ = 2 * kTile /* 2 stages */, kOffDO = 4 * kTile, kOffDS = 5 * kTile;
+  static constexpr int kOffStage = 6 * kTile;             // dQ staging: [4 warps][2 buffers][32 queries][32 floats]
   static constexpr int kOffStats = 7 * kTile;             // [stage][lse2 | delta][128] fp32
   static constexpr int kOffBars = kOffStats + 2 * 2 * 128 * 4;
   static constexpr int kUsed = kOffBars + 192;
@@ -680,8 +681,9 @@ attn_bwd_fused_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const 
                             const __grid_constant__ CUtensorMap tm_do_raw, const __grid_constant__ CUtensorMap tm_do_gist,
                             const __grid_constant__ CUtensorMap tm_k_raw, const __grid_constant__ CUtensorMap tm_k_gist,
                             const __grid_constant__ CUtensorMap tm_v_raw, const __grid_constant__ CUtensorMap tm_v_gist,
+                            const __grid_constant__ CUtensorMap tm_dq_raw, const __grid_constant__ CUtensorMap tm_dq_gist,
                             Geom g, int Hq, int Hkv, float scale, const float* __restrict__ lse,
-                            const float* __restrict__ delta, float* __restrict__ dq32,
+                            const float* __restrict__ delta,
                             __nv_bfloat16* __restrict__ dk, __nv_bfloat16* __restrict__ dv, int n_gist_kt) {
   using SM = FuSmem;
   constexpr int D = 128;
@@ -694,12 +696,12 @@ attn_bwd_fused_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const 
   }
   unsigned char* gen = smem_dyn + (base - raw_base);
   const uint32_t sK = base + SM::kOffK, sV = base + SM::kOffV, sDS = base + SM::kOffDS;
-  const uint32_t sQ0 = base + SM::kOffQ, sDO0 = base + SM::kOffDO;  // stage st at + st * kTile
+  const uint32_t sQ0 = base + SM::kOffQ /* stage st at + st * kTile */, sDO = base + SM::kOffDO;
   float* stats = reinterpret_cast<float*>(gen + SM::kOffStats);
   const uint32_t bars = base + SM::kOffBars;
   const uint32_t bar_kv = bars, bar_S = bars + 8, bar_dP = bars + 16, bar_P = bars + 24, bar_dS = bars + 32,
                  bar_dSfree = bars + 40, bar_dQ = bars + 48, bar_dQfree = bars + 56, bar_final = bars + 64;
-  const uint32_t full_q0 = bars + 72, empty_q0 = bars + 88, full_do0 = bars + 104, empty_do0 = bars + 120;  // + 8 * st
+  const uint32_t full_q0 = bars + 72, empty_q0 = bars + 88 /* + 8 * st */, full_do = bars + 104, empty_do = bars + 120;
   const uint32_t tmem_slot = bars + 136;
   volatile uint32_t* tmem_slot_ptr = reinterpret_cast<volatile uint32_t*>(gen + SM::kOffBars + 136);
 
@@ -739,9 +741,9 @@ attn_bwd_fused_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const 
     for (int i = 0; i < 2; ++i) {
       mbar_init(full_q0 + 8 * i, 1);
       mbar_init(empty_q0 + 8 * i, 1);
-      mbar_init(full_do0 + 8 * i, 1);
-      mbar_init(empty_do0 + 8 * i, 1);
     }
+    mbar_init(full_do, 1);
+    mbar_init(empty_do, 1);
     mbar_fence_init();
   }
   if (warp == 13) tmem_alloc(tmem_slot, 512);
@@ -802,14 +804,13 @@ attn_bwd_fused_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const 
           for (int sl = 0; sl < 2; ++sl)
             tma_load_4d(sQ0 + st * SM::kTile + sl * SM::kSlab, mq, full_q0 + 8 * st, sl * 64, head, qt * 128, b);
         }
-        if (it >= 2) ok = mbar_wait_warp(empty_do0 + 8 * st, ((it >> 1) - 1) & 1);
+        if (it >= 1) ok = mbar_wait_warp(empty_do, (it - 1) & 1);  // one dO buffer: free once dV of the step before is done
         if (!ok) break;
         if (lane == 0) {
-          mbar_arrive_expect_tx(full_do0 + 8 * st, SM::kTile);
+          mbar_arrive_expect_tx(full_do, SM::kTile);
           const CUtensorMap* md = q_is_raw ? &tm_do_raw : &tm_do_gist;
 #pragma unroll
-          for (int sl = 0; sl < 2; ++sl)
-            tma_load_4d(sDO0 + st * SM::kTile + sl * SM::kSlab, md, full_do0 + 8 * st, sl * 64, head, qt * 128, b);
+          for (int sl = 0; sl < 2; ++sl) tma_load_4d(sDO + sl * SM::kSlab, md, full_do, sl * 64, head, qt * 128, b);
         }
         __syncwarp();
       }
@@ -827,7 +828,7 @@ attn_bwd_fused_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const 
         const uint32_t ds_lo = smem_desc_lo(sDS, 16);          // dS^T as K-major A (queries contiguous)
         const uint32_t dsT_lo = smem_desc_lo(sDS, SM::kSlab);  // dS^T as MN-major B
         const uint32_t q_lo = smem_desc_lo(sQ0, 16), qT_lo = smem_desc_lo(sQ0, SM::kSlab);
-        const uint32_t do_lo = smem_desc_lo(sDO0, 16), doT_lo = smem_desc_lo(sDO0, SM::kSlab);
+        const uint32_t do_lo = smem_desc_lo(sDO, 16), doT_lo = smem_desc_lo(sDO, SM::kSlab);
         // K-major operands step 32 B per 16 elements inside a 64-element slab; MN-major ones 2048 B
         auto koff = [](int kk) { return (uint32_t)(((kk / 4) * SM::kSlab + (kk % 4) * 32) >> 4); };
         auto moff = [](int kk) { return (uint32_t)((kk * 2048) >> 4); };
@@ -840,11 +841,10 @@ attn_bwd_fused_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const 
                     idesc_s, kk > 0);
           umma_commit(bar_S);
         };
-        auto issue_dP = [&](int st) {
+        auto issue_dP = [&]() {
 #pragma unroll
           for (int kk = 0; kk < 8; ++kk)
-            umma_ss(t_dP, smem_desc_join(v_lo + koff(kk), kHi), smem_desc_join(do_lo + st * kStage + koff(kk), kHi),
-                    idesc_s, kk > 0);
+            umma_ss(t_dP, smem_desc_join(v_lo + koff(kk), kHi), smem_desc_join(do_lo + koff(kk), kHi), idesc_s, kk > 0);
           umma_commit(bar_dP);
         };
         ok = mbar_wait(bar_kv, 0);
@@ -853,11 +853,11 @@ attn_bwd_fused_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const 
           if (ok) {
             tc_fence_after();
             issue_S(0);
-            ok = mbar_wait(full_do0, 0);
+            ok = mbar_wait(full_do, 0);
           }
           if (ok) {
             tc_fence_after();
-            issue_dP(0);
+            issue_dP();
           }
         }
         for (int it = 0; it < n_iter && ok; ++it) {
@@ -868,9 +868,9 @@ attn_bwd_fused_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const 
           tc_fence_after();
 #pragma unroll
           for (int kk = 0; kk < 8; ++kk)  // dV += P^T dO
-            umma_ts(t_dV, t_S + a_col(kk), smem_desc_join(doT_lo + st * kStage + moff(kk), kHi), idesc_acc,
+            umma_ts(t_dV, t_S + a_col(kk), smem_desc_join(doT_lo + moff(kk), kHi), idesc_acc,
                     (it > 0 || kk > 0) ? 1u : 0u);
-          umma_commit(empty_do0 + 8 * st);
+          umma_commit(empty_do);
           if (has_next) {
             ok = mbar_wait(full_q0 + 8 * (st ^ 1), ((it + 1) >> 1) & 1);
             if (!ok) break;
@@ -892,10 +892,10 @@ attn_bwd_fused_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const 
           umma_commit(empty_q0 + 8 * st);
           umma_commit(bar_dSfree);
           if (has_next) {
-            ok = mbar_wait(bar_dQfree, ph) && mbar_wait(full_do0 + 8 * (st ^ 1), ((it + 1) >> 1) & 1);
+            ok = mbar_wait(bar_dQfree, ph) && mbar_wait(full_do, (it + 1) & 1);
             if (!ok) break;
             tc_fence_after();
-            issue_dP(st ^ 1);
+            issue_dP();
           }
         }
         if (ok) umma_commit(bar_final);
@@ -904,19 +904,19 @@ attn_bwd_fused_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const 
     }
   } else if (warp >= 8) {
     // ------------------------------------------------------------ dQ read-out: lane = head_dim index
+    // Each warp moves its 32 head_dim rows of dQ^T, 32 queries at a time, through its own staging buffers
+    // ([32 queries][32 floats], two of them) and has the TMA unit add them into the fp32 dQ tensor.
     reg_dealloc<kFuRegsReadout>();
     const int qd = warp & 3;
-    const int dcol = qd * 32 + lane;
     const uint32_t lane_base = static_cast<uint32_t>(qd * 32) << 16;
+    float* stage_gen = reinterpret_cast<float*>(gen + SM::kOffStage) + qd * 2 * 1024;
+    const uint32_t stage_sh = base + SM::kOffStage + qd * 2 * 4096;
     for (int it = 0; it < n_iter && ok; ++it) {
       bool q_is_raw;
       int qt, head;
       tile_of(it, q_is_raw, qt, head);
-      const int q_seg_len = q_is_raw ? g.T : g.n, q_seg_base = q_is_raw ? g.s : g.s + g.T;
-      const int q0 = qt * 128;
-      const int nq = min(128, q_seg_len - q0);
-      float* dst = dq32 + (((long long)b * g.N + q_seg_base + q0) * Hq + head) * D + dcol;
-      const long long row_stride = (long long)Hq * D;
+      const CUtensorMap* mdq = q_is_raw ? &tm_dq_raw : &tm_dq_gist;
+      const int nq = (q_is_raw ? g.T : g.n) - qt * 128;  // rows of this tile inside the segment (may exceed 128)
       ok = mbar_wait_warp(bar_dQ, it & 1);
       if (!ok) break;
       tc_fence_after();
@@ -925,20 +925,25 @@ attn_bwd_fused_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const 
         uint32_t v[32];
         tmem_ld32(t_dP + lane_base + 32 * c, v);
         tmem_wait_ld();
-        if (c == 3) {
-          // everything is in registers: the columns may be overwritten.  A releasing arrival would
-          // first wait for the reductions below (and of the earlier chunks) to be performed.
+        if (c == 3) {  // everything is in registers: the columns may be overwritten
           tc_fence_before();
           mbar_arrive_relaxed(bar_dQfree);
         }
-        if (32 * c < nq) {
+        // the reduction issued two chunks ago has finished reading this buffer
+        if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+        __syncwarp();
+        float* sb = stage_gen + (c & 1) * 1024 + lane;
 #pragma unroll
-          for (int e = 0; e < 32; ++e) {
-            if (32 * c + e < nq) atomicAdd(dst + (32 * c + e) * row_stride, __uint_as_float(v[e]));
-          }
+        for (int e = 0; e < 32; ++e) sb[e * 32] = __uint_as_float(v[e]);
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        __syncwarp();
+        if (lane == 0 && 32 * c < nq) {  // rows past the segment's end are clipped by the tensor map
+          tma_reduce_add_4d(mdq, stage_sh + (c & 1) * 4096, qd * 32, head, qt * 128 + 32 * c, b);
+          asm volatile("cp.async.bulk.commit_group;" ::: "memory");
         }
       }
     }
+    if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
     if (!ok && lane == 0) atomicExch(&g_bwd_timeout, 1u);
   } else {
     // ------------------------------------------------------------ compute: thread = key (TMEM lane), 64 query columns
@@ -1145,13 +1150,16 @@ int32_t launch_bwd_sm100(const Geom& g, const unigist_problem& p, float scale, c
     if (int32_t rc = go_kv(attn_bwd_dkdv_sm100_kernel<128>, KvSmem<128>::kBytes)) return rc;
     return go_q(attn_bwd_dq_sm100_kernel<128>, DqSmem<128>::kBytes);
   }
+  CUtensorMap mdq[2];
+  for (int sgm = 0; sgm < 2; ++sgm)
+    if (int32_t rc = encode_segment_map_f32(&mdq[sgm], dq32, D, Hq, g.N, B, first[sgm], len[sgm], 32, 32)) return rc;
   cudaError_t e = cudaFuncSetAttribute(attn_bwd_fused_sm100_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        FuSmem::kBytes);
   if (e != cudaSuccess) return fail(UNIGIST_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
   {
     KernelScope ks("attn_bwd_fused_sm100_kernel", st);
     attn_bwd_fused_sm100_kernel<<<dim3((n_raw_t + n_gist_t) * Hkv, 1, B), kFuThreads, FuSmem::kBytes, st>>>(
-        mq[0], mq[1], md[0], md[1], mk[0], mk[1], mv[0], mv[1], g, Hq, Hkv, scale, lse, delta, dq32,
+        mq[0], mq[1], md[0], md[1], mk[0], mk[1], mv[0], mv[1], mdq[0], mdq[1], g, Hq, Hkv, scale, lse, delta,
         (__nv_bfloat16*)dk, (__nv_bfloat16*)dv, n_gist_t);
   }
   if (int32_t rc = check_launch("tcgen05 fused backward kernel")) return rc;

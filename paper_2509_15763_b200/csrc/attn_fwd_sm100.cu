@@ -501,11 +501,11 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const __grid
 
 }  // namespace
 
-int32_t encode_segment_map(CUtensorMap* map, const void* base, int D, int H, long long N, int B,
-                           long long seg_first_row, long long seg_rows, int box_rows) {
-  typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                               const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                               CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+namespace {
+typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                             const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                             CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+int32_t get_encode_fn(EncodeFn* out) {
   static EncodeFn encode = nullptr;
   if (!encode) {
     void* fn = nullptr;
@@ -515,16 +515,37 @@ int32_t encode_segment_map(CUtensorMap* map, const void* base, int D, int H, lon
       return fail(UNIGIST_ERR_CUDA, "cuTensorMapEncodeTiled is not available: %s", cudaGetErrorString(e));
     encode = reinterpret_cast<EncodeFn>(fn);
   }
+  *out = encode;
+  return UNIGIST_OK;
+}
+int32_t encode_map(CUtensorMap* map, const void* base, int D, int H, long long N, int B, long long seg_first_row,
+                   long long seg_rows, int box_cols, int box_rows, int elem_bytes) {
+  EncodeFn encode;
+  if (int32_t rc = get_encode_fn(&encode)) return rc;
+  const cuuint64_t eb = (cuuint64_t)elem_bytes;
   const cuuint64_t dims[4] = {(cuuint64_t)D, (cuuint64_t)H, (cuuint64_t)seg_rows, (cuuint64_t)B};
-  const cuuint64_t strides[3] = {(cuuint64_t)D * 2, (cuuint64_t)H * D * 2, (cuuint64_t)N * H * D * 2};
-  const cuuint32_t box[4] = {64, 1, (cuuint32_t)box_rows, 1};
+  const cuuint64_t strides[3] = {(cuuint64_t)D * eb, (cuuint64_t)H * D * eb, (cuuint64_t)N * H * D * eb};
+  const cuuint32_t box[4] = {(cuuint32_t)box_cols, 1, (cuuint32_t)box_rows, 1};
   const cuuint32_t estr[4] = {1, 1, 1, 1};
-  void* addr = const_cast<char*>(static_cast<const char*>(base)) + seg_first_row * H * D * 2;
-  CUresult r = encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, addr, dims, strides, box, estr,
-                      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+  void* addr = const_cast<char*>(static_cast<const char*>(base)) + seg_first_row * H * D * elem_bytes;
+  const bool bf16 = elem_bytes == 2;
+  CUresult r = encode(map, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, addr, dims,
+                      strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                      bf16 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                       CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) return fail(UNIGIST_ERR_CUDA, "cuTensorMapEncodeTiled failed with code %d", (int)r);
   return UNIGIST_OK;
+}
+}  // namespace
+
+int32_t encode_segment_map(CUtensorMap* map, const void* base, int D, int H, long long N, int B,
+                           long long seg_first_row, long long seg_rows, int box_rows) {
+  return encode_map(map, base, D, H, N, B, seg_first_row, seg_rows, 64, box_rows, 2);
+}
+
+int32_t encode_segment_map_f32(CUtensorMap* map, const void* base, int D, int H, long long N, int B,
+                               long long seg_first_row, long long seg_rows, int box_cols, int box_rows) {
+  return encode_map(map, base, D, H, N, B, seg_first_row, seg_rows, box_cols, box_rows, 4);
 }
 
 int32_t launch_fwd_sm100(const Geom& g, const unigist_problem& p, float scale, const void* q, const void* k,

@@ -72,6 +72,16 @@ __device__ __forceinline__ void tma_load_4d(uint32_t smem_dst, const CUtensorMap
       : "memory");
 }
 
+// Adds a shared-memory tile into global memory through a tiled tensor map (fp32 add at the L2);
+// completion is tracked by the issuing thread's bulk async-group.
+__device__ __forceinline__ void tma_reduce_add_4d(const CUtensorMap* map, uint32_t smem_src, int c0, int c1, int c2,
+                                                  int c3) {
+  asm volatile(
+      "cp.reduce.async.bulk.tensor.4d.global.shared::cta.add.tile.bulk_group [%0, {%2, %3, %4, %5}], [%1];"
+      ::"l"(reinterpret_cast<uint64_t>(map)), "r"(smem_src), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+      : "memory");
+}
+
 // ------------------------------------------------------------------ tensor memory
 __device__ __forceinline__ void tmem_alloc(uint32_t smem_slot, uint32_t ncols) {  // whole warp
   asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_slot), "r"(ncols)
@@ -220,5 +230,10 @@ __device__ __forceinline__ bool elect_one() {
 // out-of-range rows read as zero).
 int32_t encode_segment_map(CUtensorMap* map, const void* base, int D, int H, long long N, int B,
                            long long seg_first_row, long long seg_rows, int box_rows);
+
+// The same for an fp32 tensor, box = box_cols x 1 x box_rows x 1, no swizzle (rows of the box are
+// box_cols * 4 contiguous bytes in shared memory).  Used for reductions into the tensor.
+int32_t encode_segment_map_f32(CUtensorMap* map, const void* base, int D, int H, long long N, int B,
+                               long long seg_first_row, long long seg_rows, int box_cols, int box_rows);
 
 }  // namespace ug
