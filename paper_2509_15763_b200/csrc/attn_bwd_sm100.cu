@@ -637,13 +637,16 @@ attn_bwd_dq_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const __g
 // small kernel scales and rounds that buffer to bf16 afterwards.
 // MMA issue order per step i:  dV(i), S(i+1), dQ(i), dK(i), dP(i+1)  so that the exponentials of
 // step i+1 and the dQ read-out of step i run under matrix products.
-// Warps: 0-7 compute (thread = key, 64 query columns each), 8-11 dQ read-out, 12 TMA, 13 MMA.
+// Warps: 0-7 compute (thread = key, 64 query columns each), 8-15 dQ read-out (two warps per TMEM lane
+// quarter, 64 query columns each, so the dQ^T columns are free again after two TMEM loads), 16 TMA, 17 MMA.
 // Which backward head_dim 128 takes: the fused kernel below, or the two kernels above.
 constexpr bool kFusedBackward = true;
-constexpr int kFuThreads = 512;
-constexpr int kFuRegsLaunch = 128, kFuRegsCompute = 168, kFuRegsReadout = 96, kFuRegsOther = 80;
-static_assert(kFuThreads * kFuRegsLaunch == 65536, "launch register count is stale");
-static_assert(2 * kFuRegsCompute + kFuRegsReadout + kFuRegsOther <= 4 * kFuRegsLaunch,
+constexpr int kFuThreads = 640;
+constexpr int kFuTmaWarp = 16, kFuMmaWarp = 17;
+constexpr int kFuRegsLaunch = 96, kFuRegsCompute = 144, kFuRegsReadout = 64, kFuRegsOther = 64;
+static_assert(kFuThreads * kFuRegsLaunch <= 65536 && kFuThreads * (kFuRegsLaunch + 8) > 65536,
+              "launch register count is stale");
+static_assert(2 * kFuRegsCompute + 2 * kFuRegsReadout + kFuRegsOther <= 5 * kFuRegsLaunch,
               "register split exceeds the block's allocation");
 
 // One 32-query chunk of P^T for one key: p = 2^(s * c - lse2[q]); kMasked: bit e of `bits` says query e sees the key.
@@ -669,7 +672,7 @@ struct FuSmem {
   static constexpr int kSlab = 128 * 128;    // [128 rows x 64 bf16]
   static constexpr int kTile = 2 * kSlab;    // [128 x 128] bf16
   static constexpr int kOffK = 0, kOffV = kTile, kOffQ = 2 * kTile /* 2 stages */, kOffDO = 4 * kTile, kOffDS = 5 * kTile;
-  static constexpr int kOffStage = 6 * kTile;             // dQ staging: [4 warps][2 buffers][32 queries][32 floats]
+  static constexpr int kOffStage = 6 * kTile;             // dQ staging: [8 warps][32 queries][32 floats]
   static constexpr int kOffStats = 7 * kTile;             // [stage][lse2 | delta][128] fp32
   static constexpr int kOffBars = kOffStats + 2 * 2 * 128 * 4;
   static constexpr int kUsed = kOffBars + 192;
@@ -736,7 +739,7 @@ attn_bwd_fused_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const 
     mbar_init(bar_dS, 256);
     mbar_init(bar_dSfree, 1);
     mbar_init(bar_dQ, 1);
-    mbar_init(bar_dQfree, 128);
+    mbar_init(bar_dQfree, 256);
     mbar_init(bar_final, 1);
     for (int i = 0; i < 2; ++i) {
       mbar_init(full_q0 + 8 * i, 1);
@@ -746,7 +749,7 @@ attn_bwd_fused_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const 
     mbar_init(empty_do, 1);
     mbar_fence_init();
   }
-  if (warp == 13) tmem_alloc(tmem_slot, 512);
+  if (warp == kFuMmaWarp) tmem_alloc(tmem_slot, 512);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -764,9 +767,9 @@ attn_bwd_fused_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const 
     qt = q_is_raw ? rq_lo + (n_raw_q - 1 - t) : gq_lo + (n_gist_q - 1 - (t - n_raw_q));
   };
 
-  if (warp >= 12) {
+  if (warp >= 16) {
     reg_dealloc<kFuRegsOther>();
-    if (warp == 12) {
+    if (warp == kFuTmaWarp) {
       // ---------------------------------------------------------- producer: K, V once; Q, dO, LSE, Delta per step
       if (lane == 0) {
         mbar_arrive_expect_tx(bar_kv, 2 * SM::kTile);
@@ -778,6 +781,24 @@ attn_bwd_fused_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const 
           tma_load_4d(sV + sl * SM::kSlab, mv, bar_kv, sl * 64, hk, key_a, b);
         }
       }
+      // LSE (in log2 units) and Delta of the step's 128 query rows, 4 rows per lane, fetched one step ahead
+      float st_l[4], st_d[4];
+      auto fetch_stats = [&](int it) {
+        bool q_is_raw;
+        int qt, head;
+        tile_of(it, q_is_raw, qt, head);
+        const int q_seg_len = q_is_raw ? g.T : g.n, q_seg_base = q_is_raw ? g.s : g.s + g.T;
+        const long long row_base = ((long long)b * Hq + head) * g.N + q_seg_base;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const int row = qt * 128 + lane + 32 * i;
+          const bool valid = row < q_seg_len;
+          // rows past the segment get LSE = +inf, so their P is exactly zero
+          st_l[i] = valid ? lse[row_base + row] * kLog2e : INFINITY;
+          st_d[i] = valid ? delta[row_base + row] : 0.f;
+        }
+      };
+      if (n_iter > 0) fetch_stats(0);
       for (int it = 0; it < n_iter; ++it) {
         const int st = it & 1;
         bool q_is_raw;
@@ -785,16 +806,11 @@ attn_bwd_fused_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const 
         tile_of(it, q_is_raw, qt, head);
         if (it >= 2) ok = mbar_wait_warp(empty_q0 + 8 * st, ((it >> 1) - 1) & 1);
         if (!ok) break;
-        const int q_seg_len = q_is_raw ? g.T : g.n, q_seg_base = q_is_raw ? g.s : g.s + g.T;
         float* ls = stats + st * 256;
-        const long long row_base = ((long long)b * Hq + head) * g.N + q_seg_base;
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-          const int c = lane + 32 * i, row = qt * 128 + c;
-          const bool valid = row < q_seg_len;
-          // rows past the segment get LSE = +inf, so their P is exactly zero
-          ls[c] = valid ? lse[row_base + row] * kLog2e : INFINITY;
-          ls[128 + c] = valid ? delta[row_base + row] : 0.f;
+          ls[lane + 32 * i] = st_l[i];
+          ls[128 + lane + 32 * i] = st_d[i];
         }
         __syncwarp();
         if (lane == 0) {
@@ -804,6 +820,7 @@ attn_bwd_fused_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const 
           for (int sl = 0; sl < 2; ++sl)
             tma_load_4d(sQ0 + st * SM::kTile + sl * SM::kSlab, mq, full_q0 + 8 * st, sl * 64, head, qt * 128, b);
         }
+        if (it + 1 < n_iter) fetch_stats(it + 1);
         if (it >= 1) ok = mbar_wait_warp(empty_do, (it - 1) & 1);  // one dO buffer: free once dV of the step before is done
         if (!ok) break;
         if (lane == 0) {
@@ -815,7 +832,7 @@ attn_bwd_fused_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const 
         __syncwarp();
       }
       if (!ok && lane == 0) atomicExch(&g_bwd_timeout, 1u);
-    } else if (warp == 13) {
+    } else if (warp == kFuMmaWarp) {
       // ---------------------------------------------------------- MMA issuer
       if (lane == 0) {
         constexpr uint32_t idesc_s = make_idesc_bf16(128, 128, false, false);   // K-major A and B
@@ -904,13 +921,13 @@ attn_bwd_fused_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const 
     }
   } else if (warp >= 8) {
     // ------------------------------------------------------------ dQ read-out: lane = head_dim index
-    // Each warp moves its 32 head_dim rows of dQ^T, 32 queries at a time, through its own staging buffers
-    // ([32 queries][32 floats], two of them) and has the TMA unit add them into the fp32 dQ tensor.
+    // Each warp moves its 32 head_dim rows x 64 queries of dQ^T, 32 queries at a time, through its own
+    // staging buffer ([32 queries][32 floats]) and has the TMA unit add them into the fp32 dQ tensor.
     reg_dealloc<kFuRegsReadout>();
-    const int qd = warp & 3;
+    const int qd = warp & 3, half = (warp >> 2) & 1;
     const uint32_t lane_base = static_cast<uint32_t>(qd * 32) << 16;
-    float* stage_gen = reinterpret_cast<float*>(gen + SM::kOffStage) + qd * 2 * 1024;
-    const uint32_t stage_sh = base + SM::kOffStage + qd * 2 * 4096;
+    float* stage_gen = reinterpret_cast<float*>(gen + SM::kOffStage) + (warp - 8) * 1024 + lane;
+    const uint32_t stage_sh = base + SM::kOffStage + (warp - 8) * 4096;
     for (int it = 0; it < n_iter && ok; ++it) {
       bool q_is_raw;
       int qt, head;
@@ -921,24 +938,24 @@ attn_bwd_fused_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const 
       if (!ok) break;
       tc_fence_after();
 #pragma unroll
-      for (int c = 0; c < 4; ++c) {
+      for (int c = 0; c < 2; ++c) {
+        const int col0 = 64 * half + 32 * c;
         uint32_t v[32];
-        tmem_ld32(t_dP + lane_base + 32 * c, v);
+        tmem_ld32(t_dP + lane_base + col0, v);
         tmem_wait_ld();
-        if (c == 3) {  // everything is in registers: the columns may be overwritten
+        if (c == 1) {  // this warp's columns are in registers: they may be overwritten
           tc_fence_before();
           mbar_arrive_relaxed(bar_dQfree);
         }
-        // the reduction issued two chunks ago has finished reading this buffer
-        if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+        // the reduction issued before has finished reading the staging buffer
+        if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
         __syncwarp();
-        float* sb = stage_gen + (c & 1) * 1024 + lane;
 #pragma unroll
-        for (int e = 0; e < 32; ++e) sb[e * 32] = __uint_as_float(v[e]);
+        for (int e = 0; e < 32; ++e) stage_gen[e * 32] = __uint_as_float(v[e]);
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         __syncwarp();
-        if (lane == 0 && 32 * c < nq) {  // rows past the segment's end are clipped by the tensor map
-          tma_reduce_add_4d(mdq, stage_sh + (c & 1) * 4096, qd * 32, head, qt * 128 + 32 * c, b);
+        if (lane == 0 && col0 < nq) {  // rows past the segment's end are clipped by the tensor map
+          tma_reduce_add_4d(mdq, stage_sh, qd * 32, head, qt * 128 + col0, b);
           asm volatile("cp.async.bulk.commit_group;" ::: "memory");
         }
       }
@@ -1063,7 +1080,7 @@ attn_bwd_fused_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const 
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 13) {
+  if (warp == kFuMmaWarp) {
     __syncwarp();
     tmem_dealloc(tmem, 512);
   }
