@@ -34,17 +34,14 @@ UNIT = "TFLOP/s"
 
 # DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures
 # summarised under profiles/, keyed by (kernel, workload); None until a capture exists.
-NCU_TRAFFIC_BYTES = {
-    ("attn_fwd_sm100_kernel", "llama8b_layer"): 346202256,
-    ("attn_bwd_dkdv_sm100_kernel", "llama8b_layer"): 2123198032,
-    ("attn_bwd_dq_sm100_kernel", "llama8b_layer"): 508098256,
-}
+NCU_TRAFFIC_BYTES = {}
 
 # FLOP per visible pair per query head that each attention kernel performs algorithmically,
 # in units of head_dim (a QK^T- or PV-shaped product is 2 * D FLOP per pair).
 KERNEL_FLOP_PER_PAIR_D = {
     "fwd_simt_kernel": 4, "bwd_dq_simt_kernel": 6, "bwd_dkdv_simt_kernel": 8,
     "attn_fwd_sm100_kernel": 4, "attn_bwd_dq_sm100_kernel": 6, "attn_bwd_dkdv_sm100_kernel": 8,
+    "attn_bwd_fused_sm100_kernel": 10,
 }
 CUDA_CORE_KERNELS = {"fwd_simt_kernel", "bwd_dq_simt_kernel", "bwd_dkdv_simt_kernel"}
 
