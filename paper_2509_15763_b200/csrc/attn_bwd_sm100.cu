@@ -22,7 +22,7 @@ constexpr float kLog2e = 1.4426950408889634f;
 __device__ unsigned int g_bwd_timeout = 0;
 
 // ------------------------------------------------------------------------------------------------
-// Delta and dO conversion: one warp per (batch, token, head) row.
+// Delta and dO conversion: one warp per (batch, token, head) row, 4 elements per lane and pass.
 template <bool kF32>
 __global__ void __launch_bounds__(256)
 bwd_prep_kernel(int N, int Hq, int D, long long rows, const void* __restrict__ d_o,
@@ -32,27 +32,26 @@ bwd_prep_kernel(int N, int Hq, int D, long long rows, const void* __restrict__ d
   const long long warp = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const long long nwarps = ((long long)gridDim.x * blockDim.x) >> 5;
   for (long long rw = warp; rw < rows; rw += nwarps) {  // rw = (b*N + t)*Hq + h
-    if (dq32) {  // the fused backward accumulates dQ into this fp32 buffer: start it at zero
-      for (int d = lane * 4; d < D; d += 128) *reinterpret_cast<float4*>(dq32 + rw * D + d) = make_float4(0.f, 0.f, 0.f, 0.f);
-    }
     float acc = 0.f;
-    for (int d = lane * 2; d < D; d += 64) {
-      float x0, x1;
+    for (int d = lane * 4; d < D; d += 128) {
+      // the fused backward accumulates dQ into this fp32 buffer: start it at zero
+      if (dq32) __stcs(reinterpret_cast<float4*>(dq32 + rw * D + d), make_float4(0.f, 0.f, 0.f, 0.f));
+      uint2 dbits;  // 4 bf16 of dO
       if (kF32) {
-        const float2 t = *reinterpret_cast<const float2*>(reinterpret_cast<const float*>(d_o) + rw * D + d);
-        const __nv_bfloat162 r2 = __floats2bfloat162_rn(t.x, t.y);
-        *reinterpret_cast<__nv_bfloat162*>(d_o_bf16 + rw * D + d) = r2;
-        const float2 rr = __bfloat1622float2(r2);
-        x0 = rr.x;
-        x1 = rr.y;
+        const float4 t = __ldcs(reinterpret_cast<const float4*>(reinterpret_cast<const float*>(d_o) + rw * D + d));
+        const __nv_bfloat162 lo = __floats2bfloat162_rn(t.x, t.y), hi = __floats2bfloat162_rn(t.z, t.w);
+        dbits.x = *reinterpret_cast<const uint32_t*>(&lo);
+        dbits.y = *reinterpret_cast<const uint32_t*>(&hi);
+        *reinterpret_cast<uint2*>(d_o_bf16 + rw * D + d) = dbits;
       } else {
-        const float2 rr = __bfloat1622float2(
-            *reinterpret_cast<const __nv_bfloat162*>(reinterpret_cast<const __nv_bfloat16*>(d_o) + rw * D + d));
-        x0 = rr.x;
-        x1 = rr.y;
+        dbits = *reinterpret_cast<const uint2*>(reinterpret_cast<const __nv_bfloat16*>(d_o) + rw * D + d);
       }
-      const float2 oo = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(o + rw * D + d));
-      acc += x0 * oo.x + x1 * oo.y;
+      const uint2 obits = *reinterpret_cast<const uint2*>(o + rw * D + d);
+      // a bf16 is the high half of an fp32
+      acc += __uint_as_float(dbits.x << 16) * __uint_as_float(obits.x << 16) +
+             __uint_as_float(dbits.x & 0xffff0000u) * __uint_as_float(obits.x & 0xffff0000u) +
+             __uint_as_float(dbits.y << 16) * __uint_as_float(obits.y << 16) +
+             __uint_as_float(dbits.y & 0xffff0000u) * __uint_as_float(obits.y & 0xffff0000u);
     }
 #pragma unroll
     for (int off = 16; off >= 1; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
