@@ -218,7 +218,9 @@ int32_t unigist_device_status(void) {
   bool bwd_timed_out = false;
   if (int32_t rc = fwd_sm100_take_timeout(&timed_out)) return rc;
   if (int32_t rc = bwd_sm100_take_timeout(&bwd_timed_out)) return rc;
-  if (timed_out || bwd_timed_out) return fail(UNIGIST_ERR_TIMEOUT, "a kernel gave up on a bounded wait; its outputs are invalid");
+  bool dec_timed_out = false;
+  if (int32_t rc = decode_take_timeout(&dec_timed_out)) return rc;
+  if (timed_out || bwd_timed_out || dec_timed_out) return fail(UNIGIST_ERR_TIMEOUT, "a kernel gave up on a bounded wait; its outputs are invalid");
   return UNIGIST_OK;
 }
 

@@ -548,6 +548,20 @@ int32_t encode_segment_map_f32(CUtensorMap* map, const void* base, int D, int H,
   return encode_map(map, base, D, H, N, B, seg_first_row, seg_rows, box_cols, box_rows, 4);
 }
 
+int32_t encode_map_2d_bf16(CUtensorMap* map, const void* base, long long rows, int cols, int box_rows, int box_cols) {
+  EncodeFn encode;
+  if (int32_t rc = get_encode_fn(&encode)) return rc;
+  const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  const cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+  const cuuint32_t box[2] = {(cuuint32_t)box_cols, (cuuint32_t)box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  CUresult r = encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return fail(UNIGIST_ERR_CUDA, "cuTensorMapEncodeTiled failed with code %d", (int)r);
+  return UNIGIST_OK;
+}
+
 int32_t launch_fwd_sm100(const Geom& g, const unigist_problem& p, float scale, const void* q, const void* k,
                          const void* v, void* o, float* lse, cudaStream_t st) {
   const int D = p.head_dim, Hq = p.num_q_heads, Hkv = p.num_kv_heads, B = p.batch;

@@ -1,206 +1,246 @@
 // Decode attention over the compacted, paged KV cache (Section 4.3): one query per sequence,
 // every cache entry visible.  Split over keys: each thread block streams a contiguous range of
-// 64-token pages of one (sequence, KV head) through shared memory with 16-byte asynchronous
-// copies (a page of one KV head is one contiguous 64 * D * 2 byte run), keeps a running
-// (max, sum, output) for the G query heads that share the KV head, and a second kernel merges
-// the splits.  HBM-bound: K and V are read exactly once.
+// 64-token pages of one (sequence, KV head) through a ring in shared memory and a second kernel
+// merges the splits.  HBM-bound: K and V are read exactly once.
+//   producer warp:  per page one K and one V tile (64 tokens x 128 dims, 16 KB each) by TMA, 128-byte
+//                   swizzle, into a 3-stage ring guarded by full / empty mbarriers; two thread blocks
+//                   per SM keep about 128 KB of loads in flight.
+//   consumer warps: three warps, one per ring stage, each takes every third page on its own and keeps a running
+//                   (max, sum, output) for the G query heads of the KV head: S = Q K^T and O += P V
+//                   with warp-level mma (m16n8k16, query heads padded to 16 rows), fragments
+//                   fetched with ldmatrix.  The warps merge once, at the end.
 #include <cmath>
 
+#include "sm100_ptx.cuh"
 #include "ug_common.cuh"
 
 namespace ug {
 namespace {
 
+using namespace sm100;
+
 constexpr int PG = UNIGIST_PAGE_TOKENS;
 constexpr int DD = 128;                     // head_dim
 constexpr int STAGES = 3;
 constexpr int PAGE_BYTES = PG * DD * 2;     // one K (or V) page of one KV head
-constexpr int THREADS = 256;
+constexpr int SLAB_BYTES = PAGE_BYTES / 2;  // [64 tokens x 64 dims], rows of 128 bytes
+constexpr int STAGE_BYTES = 2 * PAGE_BYTES;
+constexpr int kConsumers = STAGES;  // page i lives in stage i % STAGES and belongs to warp i % STAGES: every barrier
+                                    // has one waiter, which sees each of its phases in turn
+constexpr int THREADS = (kConsumers + 1) * 32;
 constexpr float LOG2E = 1.4426950408889634f;
 
-__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gsrc) {
-  const uint32_t d = (uint32_t)__cvta_generic_to_shared(smem_dst);
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(d), "l"(gsrc) : "memory");
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory"); }
+__device__ unsigned int g_decode_timeout = 0;
 
-__device__ __forceinline__ void unpack8(const uint4& raw, float (&f)[8]) {
-  const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    f[2 * i] = __uint_as_float(w[i] << 16);
-    f[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
-  }
+__device__ __forceinline__ void tma_load_2d(uint32_t smem_dst, const CUtensorMap* map, uint32_t bar, int c0, int c1) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(smem_dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1)
+      : "memory");
 }
+__device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+__device__ __forceinline__ void ldsm_x4_trans(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+// D (16x8 fp32) += A (16x16 bf16, row) * B (16x8 bf16, col)
+__device__ __forceinline__ void mma_bf16(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                         uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+               : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+               : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+struct DecSmem {
+  static constexpr int kOffBars = STAGES * STAGE_BYTES;
+  static constexpr int kOffMerge = kOffBars + 64;                      // [warps][8 heads][128 + 2] fp32
+  static constexpr int kBytes = kOffMerge + kConsumers * 8 * (DD + 2) * 4 + 1024 /*align*/;
+};
 
 // Partial results per (seq, q head, split): o[D] unnormalised, then m (log2 domain), l.
-template <int G>
 __global__ void __launch_bounds__(THREADS, 2)
-decode_split_kernel(int Hq, int Hkv, float scale_log2, const __nv_bfloat16* __restrict__ q,
-                    const __nv_bfloat16* __restrict__ kc, const __nv_bfloat16* __restrict__ vc,
-                    int num_blocks, const int32_t* __restrict__ table, int max_blocks,
-                    const int32_t* __restrict__ seq_lens, int splits, int blocks_per_split,
-                    float* __restrict__ part) {
-  extern __shared__ __align__(128) unsigned char smem_raw[];
-  unsigned char* stage = smem_raw;                                     // STAGES * 2 * PAGE_BYTES
-  float* sc = reinterpret_cast<float*>(smem_raw + STAGES * 2 * PAGE_BYTES);  // [G][PG]
-  float* run_m = sc + G * PG;                                         // [G]
-  float* run_l = run_m + G;
-  float* fac = run_l + G;
+decode_split_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v, int Hq,
+                    int Hkv, int G, float scale_log2, const __nv_bfloat16* __restrict__ q, int num_blocks,
+                    const int32_t* __restrict__ table, int max_blocks, const int32_t* __restrict__ seq_lens,
+                    int splits, int blocks_per_split, float* __restrict__ part) {
+  extern __shared__ unsigned char smem_dyn[];
+  const uint32_t base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
+  unsigned char* gen = smem_dyn + (base - smem_u32(smem_dyn));
+  const uint32_t bars = base + DecSmem::kOffBars;  // full[s] at + 8 s, empty[s] at + 8 (STAGES + s)
+  float* merge = reinterpret_cast<float*>(gen + DecSmem::kOffMerge);
   const int split = blockIdx.x, hk = blockIdx.y, seq = blockIdx.z;
-  const int tid = threadIdx.x;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int len = seq_lens[seq];
   const int nblk = (len + PG - 1) / PG;
   const int b0 = min(split * blocks_per_split, nblk);
   const int b1 = min(b0 + blocks_per_split, min(nblk, max_blocks));
-  const int32_t* row = table + (long long)seq * max_blocks;
+  const int npages = b1 - b0;
 
-  // query fragments: thread (c = tid % 8) owns elements [8c, 8c+8) and [64+8c, 64+8c+8)
-  const int c8 = tid & 7;
-  float qf[G][16];
-#pragma unroll
-  for (int g = 0; g < G; ++g) {
-    const __nv_bfloat16* qp = q + ((long long)seq * Hq + hk * G + g) * DD;
-    float a[8], b[8];
-    unpack8(*reinterpret_cast<const uint4*>(qp + c8 * 8), a);
-    unpack8(*reinterpret_cast<const uint4*>(qp + 64 + c8 * 8), b);
-#pragma unroll
-    for (int e = 0; e < 8; ++e) {
-      qf[g][e] = a[e] * scale_log2;
-      qf[g][8 + e] = b[e] * scale_log2;
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < STAGES; ++i) {
+      mbar_init(bars + 8 * i, 1);
+      mbar_init(bars + 8 * (STAGES + i), 1);
     }
+    mbar_fence_init();
   }
-  if (tid < G) {
-    run_m[tid] = -INFINITY;
-    run_l[tid] = 0.f;
-  }
-  float acc[G][8];
-#pragma unroll
-  for (int g = 0; g < G; ++g)
-#pragma unroll
-    for (int e = 0; e < 8; ++e) acc[g][e] = 0.f;
+  __syncthreads();
+  bool ok = true;
 
-  auto issue = [&](int blk_idx, int st) {
-    if (blk_idx < b1) {
-      int phys = row[blk_idx];
-      phys = min(max(phys, 0), num_blocks - 1);  // never read outside the cache
-      const char* ksrc = reinterpret_cast<const char*>(kc) + ((long long)phys * Hkv + hk) * PAGE_BYTES;
-      const char* vsrc = reinterpret_cast<const char*>(vc) + ((long long)phys * Hkv + hk) * PAGE_BYTES;
-      unsigned char* kd = stage + st * 2 * PAGE_BYTES;
-      unsigned char* vd = kd + PAGE_BYTES;
-#pragma unroll
-      for (int i = 0; i < PAGE_BYTES / 16 / THREADS; ++i) {
-        const int off = (i * THREADS + tid) * 16;
-        cp_async16(kd + off, ksrc + off);
-        cp_async16(vd + off, vsrc + off);
+  if (warp == kConsumers) {
+    // ------------------------------------------------------------ producer
+    const int32_t* row = table + (long long)seq * max_blocks;
+    int32_t phys_mine = 0;
+    for (int i = 0; i < npages && ok; ++i) {
+      if ((i & 31) == 0) {  // the next 32 block-table entries, one per lane
+        const int idx = b0 + i + lane;
+        phys_mine = idx < b1 ? row[idx] : 0;
+        phys_mine = min(max(phys_mine, 0), num_blocks - 1);  // never read outside the cache
       }
-    }
-    cp_async_commit();  // empty groups keep the wait arithmetic uniform
-  };
-
-#pragma unroll
-  for (int s = 0; s < STAGES - 1; ++s) issue(b0 + s, s);
-
-  for (int blk = b0; blk < b1; ++blk) {
-    const int st = (blk - b0) % STAGES;
-    cp_async_wait<STAGES - 2>();
-    __syncthreads();  // page `blk` has landed; everyone is done with the stage refilled next
-    issue(blk + STAGES - 1, (blk - b0 + STAGES - 1) % STAGES);
-    const unsigned char* ks = stage + st * 2 * PAGE_BYTES;
-    const unsigned char* vs = ks + PAGE_BYTES;
-    const int nvalid = min(PG, len - blk * PG);
-
-    // scores: 8 threads per token, 32 tokens per pass
-#pragma unroll
-    for (int pass = 0; pass < PG / 32; ++pass) {
-      const int tok = pass * 32 + (tid >> 3);
-      float ka[8], kb[8];
-      unpack8(*reinterpret_cast<const uint4*>(ks + tok * (DD * 2) + c8 * 16), ka);
-      unpack8(*reinterpret_cast<const uint4*>(ks + tok * (DD * 2) + 128 + c8 * 16), kb);
-#pragma unroll
-      for (int g = 0; g < G; ++g) {
-        float d = 0.f;
-#pragma unroll
-        for (int e = 0; e < 8; ++e) d += qf[g][e] * ka[e] + qf[g][8 + e] * kb[e];
-        d += __shfl_xor_sync(0xffffffffu, d, 1);
-        d += __shfl_xor_sync(0xffffffffu, d, 2);
-        d += __shfl_xor_sync(0xffffffffu, d, 4);
-        if (c8 == 0) sc[g * PG + tok] = tok < nvalid ? d : -INFINITY;
-      }
-    }
-    __syncthreads();
-    // running softmax: warp g owns query head g
-    if ((tid >> 5) < G) {
-      const int g = tid >> 5, lane = tid & 31;
-      const float s0 = sc[g * PG + lane], s1 = sc[g * PG + 32 + lane];
-      float mx = fmaxf(s0, s1);
-#pragma unroll
-      for (int o = 16; o >= 1; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-      const float mo = run_m[g];
-      const float mn = fmaxf(mo, mx);  // finite: token 0 of the page is always valid
-      const float p0 = exp2f(s0 - mn), p1 = exp2f(s1 - mn);
-      float ps = p0 + p1;
-#pragma unroll
-      for (int o = 16; o >= 1; o >>= 1) ps += __shfl_xor_sync(0xffffffffu, ps, o);
-      sc[g * PG + lane] = p0;
-      sc[g * PG + 32 + lane] = p1;
+      const int phys = __shfl_sync(0xffffffffu, phys_mine, i & 31);
+      const int st = i % STAGES, use = i / STAGES;
+      if (use > 0) ok = mbar_wait_warp(bars + 8 * (STAGES + st), (use - 1) & 1);
+      if (!ok) break;
       if (lane == 0) {
-        const float f = exp2f(mo - mn);
-        fac[g] = f;
-        run_l[g] = run_l[g] * f + ps;
-        run_m[g] = mn;
+        const uint32_t full = bars + 8 * st, dst = base + st * STAGE_BYTES;
+        const int row0 = (phys * Hkv + hk) * PG;
+        mbar_arrive_expect_tx(full, STAGE_BYTES);
+        tma_load_2d(dst, &tm_k, full, 0, row0);
+        tma_load_2d(dst + SLAB_BYTES, &tm_k, full, 64, row0);
+        tma_load_2d(dst + PAGE_BYTES, &tm_v, full, 0, row0);
+        tma_load_2d(dst + PAGE_BYTES + SLAB_BYTES, &tm_v, full, 64, row0);
+      }
+      __syncwarp();
+    }
+    if (!ok && lane == 0) atomicExch(&g_decode_timeout, 1u);
+  } else {
+    // ------------------------------------------------------------ consumer: pages warp, warp + 3, ...
+    const int g = lane >> 2, qc = lane & 3;  // query head (row of the padded 16 x 128 Q), column pair
+    // A fragments of Q for the 8 k-steps of 16 dims: rows 8..15 are padding (zero)
+    uint32_t qa0[8], qa2[8];
+    {
+      const __nv_bfloat16* qp = q + ((long long)seq * Hq + hk * G + min(g, G - 1)) * DD;
+#pragma unroll
+      for (int ks = 0; ks < 8; ++ks) {
+        const uint32_t lo = *reinterpret_cast<const uint32_t*>(qp + 16 * ks + 2 * qc);
+        const uint32_t hi = *reinterpret_cast<const uint32_t*>(qp + 16 * ks + 8 + 2 * qc);
+        qa0[ks] = g < G ? lo : 0u;
+        qa2[ks] = g < G ? hi : 0u;
       }
     }
-    __syncthreads();
-    // O += P V: thread owns 8 output columns (piece) for 4 tokens of the page
-    {
-      const int piece = tid & 15, tg = tid >> 4;
+    float o[16][4];
 #pragma unroll
-      for (int g = 0; g < G; ++g) {
-        const float f = fac[g];
+    for (int i = 0; i < 16; ++i)
 #pragma unroll
-        for (int e = 0; e < 8; ++e) acc[g][e] *= f;
-      }
+      for (int e = 0; e < 4; ++e) o[i][e] = 0.f;
+    float m_run = -INFINITY, l_run = 0.f;  // of row g (the 4 lanes of a quad hold the same values)
+    const int lr = lane & 7, lj = lane >> 3;  // ldmatrix: this lane supplies row lr of matrix lj
+
+    for (int i = warp; i < npages && ok; i += kConsumers) {
+      const int st = i % STAGES, use = i / STAGES;
+      ok = mbar_wait_warp(bars + 8 * st, use & 1);
+      if (!ok) break;
+      const uint32_t sK = base + st * STAGE_BYTES, sV = sK + PAGE_BYTES;
+      const int nvalid = min(PG, len - (b0 + i) * PG);
+      // S = Q K^T: 8 token tiles of 8, fp32
+      float s[8][4];
 #pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const int tok = tg * 4 + i;
-        if (tok < nvalid) {
-          float vf[8];
-          unpack8(*reinterpret_cast<const uint4*>(vs + tok * (DD * 2) + piece * 16), vf);
+      for (int nt = 0; nt < 8; ++nt) {
 #pragma unroll
-          for (int g = 0; g < G; ++g) {
-            const float p = sc[g * PG + tok];
+        for (int e = 0; e < 4; ++e) s[nt][e] = 0.f;
+        const int t = 8 * nt + lr;  // token whose row address this lane supplies
 #pragma unroll
-            for (int e = 0; e < 8; ++e) acc[g][e] += p * vf[e];
-          }
+        for (int kq = 0; kq < 4; ++kq) {  // 32 dims = 4 chunks of 16 bytes per ldmatrix.x4
+          const int chunk = (kq & 1) * 4 + lj;
+          uint32_t k0, k1, k2, k3;
+          ldsm_x4(sK + (kq >> 1) * SLAB_BYTES + t * 128 + ((chunk ^ (t & 7)) << 4), k0, k1, k2, k3);
+          mma_bf16(s[nt], qa0[2 * kq], 0u, qa2[2 * kq], 0u, k0, k1);
+          mma_bf16(s[nt], qa0[2 * kq + 1], 0u, qa2[2 * kq + 1], 0u, k2, k3);
         }
       }
+      // running softmax of row g over the page's 64 tokens (this lane: tokens 8 nt + 2 qc + {0, 1})
+      float mx = -INFINITY;
+#pragma unroll
+      for (int nt = 0; nt < 8; ++nt) {
+        const int tok = 8 * nt + 2 * qc;
+        s[nt][0] = tok < nvalid ? s[nt][0] * scale_log2 : -INFINITY;
+        s[nt][1] = tok + 1 < nvalid ? s[nt][1] * scale_log2 : -INFINITY;
+        mx = fmaxf(mx, fmaxf(s[nt][0], s[nt][1]));
+      }
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+      const float m_new = fmaxf(m_run, mx);  // finite: token 0 of a page is always valid
+      const float f = ex2(m_run - m_new);
+      m_run = m_new;
+      float ps = 0.f;
+      uint32_t pa[8];  // P as bf16 pairs: pa[nt] = tokens 8 nt + 2 qc + {0, 1} of row g
+#pragma unroll
+      for (int nt = 0; nt < 8; ++nt) {
+        const float p0 = ex2(s[nt][0] - m_new), p1 = ex2(s[nt][1] - m_new);
+        ps += p0 + p1;
+        pa[nt] = pack_bf16(p0, p1);
+      }
+      ps += __shfl_xor_sync(0xffffffffu, ps, 1);
+      ps += __shfl_xor_sync(0xffffffffu, ps, 2);
+      l_run = l_run * f + ps;
+#pragma unroll
+      for (int i2 = 0; i2 < 16; ++i2) {
+        o[i2][0] *= f;
+        o[i2][1] *= f;
+      }
+      // O += P V: 4 k-steps of 16 tokens, 16 dim tiles of 8
+#pragma unroll
+      for (int ks = 0; ks < 4; ++ks) {
+        const int t = 16 * ks + (lj & 1) * 8 + lr;
+#pragma unroll
+        for (int np = 0; np < 8; ++np) {  // dim tiles 2 np, 2 np + 1
+          const int chunk = 2 * np + (lj >> 1);  // 16-byte chunk of the 256-byte V row
+          uint32_t v0, v1, v2, v3;
+          ldsm_x4_trans(sV + (chunk >> 3) * SLAB_BYTES + t * 128 + (((chunk & 7) ^ (t & 7)) << 4), v0, v1, v2, v3);
+          mma_bf16(o[2 * np], pa[2 * ks], 0u, pa[2 * ks + 1], 0u, v0, v1);
+          mma_bf16(o[2 * np + 1], pa[2 * ks], 0u, pa[2 * ks + 1], 0u, v2, v3);
+        }
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bars + 8 * (STAGES + st));  // the stage may be refilled
+    }
+    if (!ok && lane == 0) atomicExch(&g_decode_timeout, 1u);
+    // this warp's partial result for row g -> shared memory
+    if (g < G) {
+      float* mrow = merge + (warp * 8 + g) * (DD + 2);
+#pragma unroll
+      for (int nt = 0; nt < 16; ++nt) {
+        mrow[8 * nt + 2 * qc] = o[nt][0];
+        mrow[8 * nt + 2 * qc + 1] = o[nt][1];
+      }
+      if (qc == 0) {
+        mrow[DD] = m_run;
+        mrow[DD + 1] = l_run;
+      }
     }
   }
-  cp_async_wait<0>();
   __syncthreads();
-  // reduce the 16 token groups through shared memory (the page stages are free now)
-  float* red = reinterpret_cast<float*>(stage);  // [16][G][DD]
-  {
-    const int piece = tid & 15, tg = tid >> 4;
-#pragma unroll
-    for (int g = 0; g < G; ++g)
-#pragma unroll
-      for (int e = 0; e < 8; ++e) red[(tg * G + g) * DD + piece * 8 + e] = acc[g][e];
-  }
-  __syncthreads();
-  for (int idx = tid; idx < G * DD; idx += THREADS) {
+  // merge the consumer warps
+  for (int idx = threadIdx.x; idx < G * DD; idx += THREADS) {
     const int g = idx / DD, d = idx % DD;
-    float s = 0.f;
+    float M = -INFINITY;
 #pragma unroll
-    for (int tg = 0; tg < 16; ++tg) s += red[(tg * G + g) * DD + d];
+    for (int w = 0; w < kConsumers; ++w) M = fmaxf(M, merge[(w * 8 + g) * (DD + 2) + DD]);
+    float acc = 0.f, L = 0.f;
+#pragma unroll
+    for (int w = 0; w < kConsumers; ++w) {
+      const float* mrow = merge + (w * 8 + g) * (DD + 2);
+      const float wgt = mrow[DD] == -INFINITY ? 0.f : ex2(mrow[DD] - M);
+      acc += wgt * mrow[d];
+      L += wgt * mrow[DD + 1];
+    }
     const long long slot = ((long long)seq * Hq + hk * G + g) * splits + split;
-    part[slot * (DD + 2) + d] = s;
+    part[slot * (DD + 2) + d] = acc;
     if (d == 0) {
-      part[slot * (DD + 2) + DD] = run_m[g];
-      part[slot * (DD + 2) + DD + 1] = run_l[g];
+      part[slot * (DD + 2) + DD] = M;
+      part[slot * (DD + 2) + DD + 1] = L;
     }
   }
 }
@@ -223,8 +263,6 @@ decode_combine_kernel(int splits, const float* __restrict__ part, __nv_bfloat16*
   o[sh * DD + threadIdx.x] = __float2bfloat16_rn(acc / L);
   if (lse && threadIdx.x == 0) lse[sh] = (M + log2f(L)) * 0.6931471805599453f;
 }
-
-size_t split_smem(int G) { return (size_t)STAGES * 2 * PAGE_BYTES + (size_t)(G * PG + 3 * G) * sizeof(float); }
 
 }  // namespace
 
@@ -253,35 +291,38 @@ int32_t launch_decode(int S, int Hq, int Hkv, int D, float scale, const void* q,
                       const int32_t* seq_lens, void* o, float* lse, void* ws, cudaStream_t st) {
   (void)D;
   const int G = Hq / Hkv;
+  if (G < 1 || G > 8) return fail(UNIGIST_ERR_UNSUPPORTED, "decode supports 1 to 8 query heads per KV head, got %d", G);
   const int splits = decode_num_splits(S, Hkv, max_blocks);
   const int bps = (max_blocks + splits - 1) / splits;
-  dim3 grid(splits, Hkv, S);
-  auto go = [&](auto kern, int g) -> int32_t {
-    const size_t smem = split_smem(g);
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return fail(UNIGIST_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
-    {
-      KernelScope ks("decode_split_kernel", st);
-      kern<<<grid, THREADS, smem, st>>>(Hq, Hkv, scale * LOG2E, (const __nv_bfloat16*)q,
-                                        (const __nv_bfloat16*)kc, (const __nv_bfloat16*)vc, num_blocks,
-                                        table, max_blocks, seq_lens, splits, bps, (float*)ws);
-    }
-    return check_launch("decode split kernel");
-  };
-  int32_t rc;
-  switch (G) {
-    case 1: rc = go(decode_split_kernel<1>, 1); break;
-    case 2: rc = go(decode_split_kernel<2>, 2); break;
-    case 4: rc = go(decode_split_kernel<4>, 4); break;
-    case 8: rc = go(decode_split_kernel<8>, 8); break;
-    default: return fail(UNIGIST_ERR_UNSUPPORTED, "decode supports 1, 2, 4 or 8 query heads per KV head, got %d", G);
+  // the caches as 2-D tensors [num_blocks * Hkv * 64 tokens, 128 dims], tiles of 64 tokens x 64 dims
+  CUtensorMap mk, mv;
+  const long long rows = (long long)num_blocks * Hkv * PG;
+  if (int32_t rc = encode_map_2d_bf16(&mk, kc, rows, DD, PG, 64)) return rc;
+  if (int32_t rc = encode_map_2d_bf16(&mv, vc, rows, DD, PG, 64)) return rc;
+  cudaError_t e = cudaFuncSetAttribute(decode_split_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       DecSmem::kBytes);
+  if (e != cudaSuccess) return fail(UNIGIST_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
+  {
+    KernelScope ks("decode_split_kernel", st);
+    decode_split_kernel<<<dim3(splits, Hkv, S), THREADS, DecSmem::kBytes, st>>>(
+        mk, mv, Hq, Hkv, G, scale * LOG2E, (const __nv_bfloat16*)q, num_blocks, table, max_blocks, seq_lens, splits, bps,
+        (float*)ws);
   }
-  if (rc) return rc;
+  if (int32_t rc = check_launch("decode split kernel")) return rc;
   {
     KernelScope ks("decode_combine_kernel", st);
     decode_combine_kernel<<<S * Hq, DD, 0, st>>>(splits, (const float*)ws, (__nv_bfloat16*)o, lse);
   }
   return check_launch("decode combine kernel");
+}
+
+int32_t decode_take_timeout(bool* timed_out) {
+  unsigned int flag = 0, zero = 0;
+  cudaError_t e = cudaMemcpyFromSymbol(&flag, g_decode_timeout, sizeof(flag));
+  if (e == cudaSuccess && flag) e = cudaMemcpyToSymbol(g_decode_timeout, &zero, sizeof(zero));
+  if (e != cudaSuccess) return fail(UNIGIST_ERR_CUDA, "reading the device status: %s", cudaGetErrorString(e));
+  *timed_out = flag != 0;
+  return UNIGIST_OK;
 }
 
 }  // namespace ug

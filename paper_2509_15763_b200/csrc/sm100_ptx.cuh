@@ -236,4 +236,7 @@ int32_t encode_segment_map(CUtensorMap* map, const void* base, int D, int H, lon
 int32_t encode_segment_map_f32(CUtensorMap* map, const void* base, int D, int H, long long N, int B,
                                long long seg_first_row, long long seg_rows, int box_cols, int box_rows);
 
+// A [rows, cols] bf16 matrix (cols contiguous) with boxes of box_rows x box_cols, 128-byte swizzle.
+int32_t encode_map_2d_bf16(CUtensorMap* map, const void* base, long long rows, int cols, int box_rows, int box_cols);
+
 }  // namespace ug

@@ -119,5 +119,6 @@ int32_t launch_decode(int S, int Hq, int Hkv, int D, float scale, const void* q,
                       const void* vc, int num_blocks, const int32_t* table, int max_blocks,
                       const int32_t* seq_lens, void* o, float* lse, void* ws, cudaStream_t st);
 int decode_num_splits(int S, int Hkv, int max_blocks);
+int32_t decode_take_timeout(bool* timed_out);
 
 }  // namespace ug
