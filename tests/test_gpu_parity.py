@@ -60,6 +60,12 @@ SMALL = [
     synth.Workload("no_window", 1, 512, 16, 0, 2, 1, 128, num_sinks=3, seed=105),
     synth.Workload("one_unit", 1, 12, 12, 12, 1, 1, 64, seed=106),
     synth.Workload("odd_tiles", 1, 1000, 8, 200, 4, 4, 128, num_sinks=1, k_scale=0.5, seed=107),
+    # tensor-core paths (no sinks) with ragged last tiles in both segments, batch > 1, odd and even group sizes
+    synth.Workload("ragged_128", 2, 1000, 8, 200, 4, 2, 128, k_scale=0.5, seed=108),
+    synth.Workload("ragged_mha_128", 1, 1096, 4, 300, 3, 3, 128, seed=109),
+    synth.Workload("ragged_group3_128", 1, 777, 7, 77, 6, 2, 128, seed=110),
+    synth.Workload("ragged_64", 2, 1000, 8, 200, 4, 2, 64, seed=111),
+    synth.Workload("tiny_window_128", 1, 2048, 16, 16, 2, 1, 128, seed=112),
 ]
 
 
