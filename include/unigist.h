@@ -51,6 +51,17 @@ typedef enum {
 /* dO passed to unigist_attn_bwd is fp32 (rounded to bf16 when it is read). */
 #define UNIGIST_FLAG_DOUT_FP32 1u
 
+/*
+ * q, k, v, o, d_o, dq, dk, dv of unigist_attn_fwd / unigist_attn_bwd are in INTERLEAVED order (Eq. 2)
+ * instead of shifted order: the gist shift of Section 4.2 then happens inside the tile addressing of
+ * the loads (a raw tile is r rows of each of 128 / r consecutive gist units, a gist tile is one row per
+ * unit) and outputs are stored at their interleaved row, so no separate shift / unshift pass is needed.
+ * lse stays in shifted order (it is the tensor the backward reads back).  Supported when ratio divides
+ * 128, head_dim is 128 and there are no sinks; otherwise the calls return UNIGIST_ERR_UNSUPPORTED and
+ * the caller uses unigist_gist_shift / unigist_gist_unshift.
+ */
+#define UNIGIST_FLAG_INTERLEAVED 2u
+
 enum { UNIGIST_PAGE_TOKENS = 64 }; /* tokens per KV-cache block */
 
 typedef enum {

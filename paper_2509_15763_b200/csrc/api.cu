@@ -90,6 +90,17 @@ int32_t check_problem(const unigist_problem* p, Geom* g, float* scale) {
 
 static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
+// UNIGIST_FLAG_INTERLEAVED needs the tile addressing of the tensor-core kernels for head_dim 128.
+int32_t check_interleaved(const unigist_problem* p, const Geom& g) {
+  if (!(p->flags & UNIGIST_FLAG_INTERLEAVED)) return UNIGIST_OK;
+  if (g.s != 0 || p->head_dim != 128 || 128 % g.r != 0)
+    return fail(UNIGIST_ERR_UNSUPPORTED,
+                "interleaved tensors need no sinks, head_dim 128 and a ratio that divides 128 "
+                "(got s = %d, D = %d, r = %d): shift the tensors with unigist_gist_shift instead",
+                g.s, p->head_dim, g.r);
+  return UNIGIST_OK;
+}
+
 }  // namespace ug
 
 using namespace ug;
@@ -206,6 +217,7 @@ int32_t unigist_attn_fwd(const unigist_problem* p, const void* q, const void* k,
   if (!q || !k || !v || !o || !lse) return fail(UNIGIST_ERR_INVALID_ARG, "a tensor is NULL");
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || !aligned16(lse))
     return fail(UNIGIST_ERR_ALIGNMENT, "tensor pointers must be 16-byte aligned");
+  if (int32_t rc = check_interleaved(p, g)) return rc;
   // Tensor-core path for sequences without sinks; the CUDA-core kernels cover sink prefixes.
   if (g.s == 0) return launch_fwd_sm100(g, *p, scale, q, k, v, o, lse, (cudaStream_t)stream);
   return launch_fwd_simt(g, *p, scale, q, k, v, o, lse, (cudaStream_t)stream);
@@ -235,6 +247,7 @@ int32_t unigist_attn_bwd(const unigist_problem* p, const void* q, const void* k,
   const void* ptrs[] = {q, k, v, o, lse, d_o, dq, dk, dv, workspace};
   for (const void* x : ptrs)
     if (!aligned16(x)) return fail(UNIGIST_ERR_ALIGNMENT, "tensor pointers must be 16-byte aligned");
+  if (int32_t rc = check_interleaved(p, g)) return rc;
   const size_t need = unigist_workspace_bytes(p, UNIGIST_OP_BWD);
   if (!workspace || ws_bytes < need)
     return fail(UNIGIST_ERR_WORKSPACE, "backward needs %zu bytes of workspace, got %zu", need,

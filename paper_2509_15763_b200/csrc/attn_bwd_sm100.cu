@@ -25,7 +25,7 @@ __device__ unsigned int g_bwd_timeout = 0;
 // Delta and dO conversion: one warp per (batch, token, head) row, 4 elements per lane and pass.
 template <bool kF32>
 __global__ void __launch_bounds__(256)
-bwd_prep_kernel(int N, int Hq, int D, long long rows, const void* __restrict__ d_o,
+bwd_prep_kernel(Geom g, int interleaved, int Hq, int D, long long rows, const void* __restrict__ d_o,
                 const __nv_bfloat16* __restrict__ o, float* __restrict__ delta,
                 __nv_bfloat16* __restrict__ d_o_bf16, float* __restrict__ dq32) {
   const int lane = threadIdx.x & 31;
@@ -58,9 +58,10 @@ bwd_prep_kernel(int N, int Hq, int D, long long rows, const void* __restrict__ d
     if (lane == 0) {
       const int h = (int)(rw % Hq);
       const long long bt = rw / Hq;
-      const int t = (int)(bt % N);
-      const long long b = bt / N;
-      delta[(b * Hq + h) * N + t] = acc;
+      const int t = (int)(bt % g.N);
+      const long long b = bt / g.N;
+      // Delta is kept in shifted order, whatever the order of dO and O
+      delta[(b * Hq + h) * g.N + (interleaved ? unshift_perm(g, t) : t)] = acc;
     }
   }
 }
@@ -686,7 +687,7 @@ attn_bwd_fused_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const 
                             const __grid_constant__ CUtensorMap tm_dq_raw, const __grid_constant__ CUtensorMap tm_dq_gist,
                             Geom g, int Hq, int Hkv, float scale, const float* __restrict__ lse,
                             const float* __restrict__ delta,
-                            __nv_bfloat16* __restrict__ dk, __nv_bfloat16* __restrict__ dv, int n_gist_kt) {
+                            __nv_bfloat16* __restrict__ dk, __nv_bfloat16* __restrict__ dv, int n_gist_kt, int interleaved) {
   using SM = FuSmem;
   constexpr int D = 128;
   extern __shared__ unsigned char smem_dyn[];
@@ -770,14 +771,16 @@ attn_bwd_fused_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const 
     reg_dealloc<kFuRegsOther>();
     if (warp == kFuTmaWarp) {
       // ---------------------------------------------------------- producer: K, V once; Q, dO, LSE, Delta per step
+      // tile coordinate: its first unit (a raw tile of an interleaved tensor spans 128 / r gist units)
+      auto first_unit = [&](bool is_raw, int row0) { return interleaved && is_raw ? row0 / g.r : row0; };
       if (lane == 0) {
         mbar_arrive_expect_tx(bar_kv, 2 * SM::kTile);
         const CUtensorMap* mk = key_is_raw ? &tm_k_raw : &tm_k_gist;
         const CUtensorMap* mv = key_is_raw ? &tm_v_raw : &tm_v_gist;
 #pragma unroll
         for (int sl = 0; sl < 2; ++sl) {
-          tma_load_4d(sK + sl * SM::kSlab, mk, bar_kv, sl * 64, hk, key_a, b);
-          tma_load_4d(sV + sl * SM::kSlab, mv, bar_kv, sl * 64, hk, key_a, b);
+          tma_load_5d(sK + sl * SM::kSlab, mk, bar_kv, sl * 64, hk, 0, first_unit(key_is_raw, key_a), b);
+          tma_load_5d(sV + sl * SM::kSlab, mv, bar_kv, sl * 64, hk, 0, first_unit(key_is_raw, key_a), b);
         }
       }
       // LSE (in log2 units) and Delta of the step's 128 query rows, 4 rows per lane, fetched one step ahead
@@ -817,7 +820,8 @@ attn_bwd_fused_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const 
           const CUtensorMap* mq = q_is_raw ? &tm_q_raw : &tm_q_gist;
 #pragma unroll
           for (int sl = 0; sl < 2; ++sl)
-            tma_load_4d(sQ0 + st * SM::kTile + sl * SM::kSlab, mq, full_q0 + 8 * st, sl * 64, head, qt * 128, b);
+            tma_load_5d(sQ0 + st * SM::kTile + sl * SM::kSlab, mq, full_q0 + 8 * st, sl * 64, head, 0,
+                        first_unit(q_is_raw, qt * 128), b);
         }
         if (it + 1 < n_iter) fetch_stats(it + 1);
         if (it >= 1) ok = mbar_wait_warp(empty_do, (it - 1) & 1);  // one dO buffer: free once dV of the step before is done
@@ -826,7 +830,8 @@ attn_bwd_fused_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const 
           mbar_arrive_expect_tx(full_do, SM::kTile);
           const CUtensorMap* md = q_is_raw ? &tm_do_raw : &tm_do_gist;
 #pragma unroll
-          for (int sl = 0; sl < 2; ++sl) tma_load_4d(sDO + sl * SM::kSlab, md, full_do, sl * 64, head, qt * 128, b);
+          for (int sl = 0; sl < 2; ++sl)
+            tma_load_5d(sDO + sl * SM::kSlab, md, full_do, sl * 64, head, 0, first_unit(q_is_raw, qt * 128), b);
         }
         __syncwarp();
       }
@@ -1042,7 +1047,7 @@ attn_bwd_fused_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const 
     if (ok && n_iter > 0) ok = mbar_wait_warp(bar_final, 0);
     if (ok) {
       tc_fence_after();
-      const long long tok = (long long)b * g.N + key_seg_base + key;
+      const long long tok = (long long)b * g.N + seg_row_to_token(g, interleaved != 0, key_is_raw, key_valid ? key : key_a);
       // this warp stores columns [64 hf, 64 hf + 64) of dK and of dV
 #pragma unroll
       for (int which = 0; which < 2; ++which) {
@@ -1085,17 +1090,30 @@ attn_bwd_fused_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const 
   }
 }
 
-// dQ (bf16) = scale * dQ accumulated in fp32; 8 elements per thread.
+// dQ (bf16) = scale * dQ accumulated in fp32 (shifted order, head_dim 128).  One warp per token: Hq rows of
+// 128 floats, 4 per lane; the bf16 row goes to the token's shifted or interleaved position.
 __global__ void __launch_bounds__(256)
-dq_convert_kernel(const float4* __restrict__ src, uint4* __restrict__ dst, long long n8, float scale) {
-  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n8; i += (long long)gridDim.x * blockDim.x) {
-    const float4 a = __ldcs(src + 2 * i), c = __ldcs(src + 2 * i + 1);
-    uint4 o;
-    o.x = pack_bf16(a.x * scale, a.y * scale);
-    o.y = pack_bf16(a.z * scale, a.w * scale);
-    o.z = pack_bf16(c.x * scale, c.y * scale);
-    o.w = pack_bf16(c.z * scale, c.w * scale);
-    dst[i] = o;
+dq_convert_kernel(Geom g, int interleaved, int Hq, long long tokens, const float* __restrict__ src,
+                  __nv_bfloat16* __restrict__ dst, float scale) {
+  const int lane = threadIdx.x & 31;
+  const long long warp = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const long long nwarps = ((long long)gridDim.x * blockDim.x) >> 5;
+  for (long long tk = warp; tk < tokens; tk += nwarps) {  // tk = b * N + sigma
+    const long long b = tk / g.N;
+    const int sigma = (int)(tk - b * g.N);
+    const long long out_tk = b * g.N + (interleaved ? shift_perm(g, sigma) : sigma);
+    const float4* s4 = reinterpret_cast<const float4*>(src + tk * Hq * 128) + lane;
+    uint2* d2 = reinterpret_cast<uint2*>(dst + out_tk * Hq * 128) + lane;
+    for (int h0 = 0; h0 < Hq; h0 += 4) {
+      float4 a[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u)
+        if (h0 + u < Hq) a[u] = __ldcs(s4 + (h0 + u) * 32);
+#pragma unroll
+      for (int u = 0; u < 4; ++u)
+        if (h0 + u < Hq)
+          d2[(h0 + u) * 32] = make_uint2(pack_bf16(a[u].x * scale, a[u].y * scale), pack_bf16(a[u].z * scale, a[u].w * scale));
+    }
   }
 }
 
@@ -1106,6 +1124,7 @@ int32_t launch_bwd_sm100(const Geom& g, const unigist_problem& p, float scale, c
                          void* dv, void* workspace, cudaStream_t st) {
   const int D = p.head_dim, Hq = p.num_q_heads, Hkv = p.num_kv_heads, B = p.batch;
   const bool f32 = (p.flags & UNIGIST_FLAG_DOUT_FP32) != 0;
+  const bool il = (p.flags & UNIGIST_FLAG_INTERLEAVED) != 0;
   float* delta = static_cast<float*>(workspace);
   const size_t delta_bytes = ((size_t)B * Hq * g.N * sizeof(float) + 255) / 256 * 256;
   __nv_bfloat16* do_bf16 = reinterpret_cast<__nv_bfloat16*>(static_cast<char*>(workspace) + delta_bytes);
@@ -1118,15 +1137,22 @@ int32_t launch_bwd_sm100(const Geom& g, const unigist_problem& p, float scale, c
     const int blocks = (int)((rows + 7) / 8 < 148 * 16 ? (rows + 7) / 8 : 148 * 16);
     KernelScope ks("bwd_prep_kernel", st);
     if (f32)
-      bwd_prep_kernel<true><<<blocks, 256, 0, st>>>(g.N, Hq, D, rows, d_o, (const __nv_bfloat16*)o, delta, do_bf16, dq32);
+      bwd_prep_kernel<true><<<blocks, 256, 0, st>>>(g, il ? 1 : 0, Hq, D, rows, d_o, (const __nv_bfloat16*)o, delta, do_bf16, dq32);
     else
-      bwd_prep_kernel<false><<<blocks, 256, 0, st>>>(g.N, Hq, D, rows, d_o, (const __nv_bfloat16*)o, delta, nullptr, dq32);
+      bwd_prep_kernel<false><<<blocks, 256, 0, st>>>(g, il ? 1 : 0, Hq, D, rows, d_o, (const __nv_bfloat16*)o, delta, nullptr, dq32);
   }
   if (int32_t rc = check_launch("backward prep kernel")) return rc;
 
   CUtensorMap mq[2], md[2], mk[2], mv[2], mk64[2], mv64[2];
   const long long first[2] = {g.s, (long long)g.s + g.T}, len[2] = {g.T, g.n};
   for (int sgm = 0; sgm < 2; ++sgm) {
+    if (fused) {  // 128-row tile maps that read shifted or interleaved tensors
+      if (int32_t rc = encode_tile_map(&mq[sgm], q, D, Hq, B, g.s, g.T, g.r, il, sgm == 0)) return rc;
+      if (int32_t rc = encode_tile_map(&md[sgm], do_src, D, Hq, B, g.s, g.T, g.r, il, sgm == 0)) return rc;
+      if (int32_t rc = encode_tile_map(&mk[sgm], k, D, Hkv, B, g.s, g.T, g.r, il, sgm == 0)) return rc;
+      if (int32_t rc = encode_tile_map(&mv[sgm], v, D, Hkv, B, g.s, g.T, g.r, il, sgm == 0)) return rc;
+      continue;
+    }
     if (int32_t rc = encode_segment_map(&mq[sgm], q, D, Hq, g.N, B, first[sgm], len[sgm], 128)) return rc;
     if (int32_t rc = encode_segment_map(&md[sgm], do_src, D, Hq, g.N, B, first[sgm], len[sgm], 128)) return rc;
     if (int32_t rc = encode_segment_map(&mk[sgm], k, D, Hkv, g.N, B, first[sgm], len[sgm], 128)) return rc;
@@ -1176,15 +1202,14 @@ int32_t launch_bwd_sm100(const Geom& g, const unigist_problem& p, float scale, c
     KernelScope ks("attn_bwd_fused_sm100_kernel", st);
     attn_bwd_fused_sm100_kernel<<<dim3((n_raw_t + n_gist_t) * Hkv, 1, B), kFuThreads, FuSmem::kBytes, st>>>(
         mq[0], mq[1], md[0], md[1], mk[0], mk[1], mv[0], mv[1], mdq[0], mdq[1], g, Hq, Hkv, scale, lse, delta,
-        (__nv_bfloat16*)dk, (__nv_bfloat16*)dv, n_gist_t);
+        (__nv_bfloat16*)dk, (__nv_bfloat16*)dv, n_gist_t, il ? 1 : 0);
   }
   if (int32_t rc = check_launch("tcgen05 fused backward kernel")) return rc;
   {
-    const long long n8 = (long long)B * g.N * Hq * D / 8;
-    const int blocks = (int)((n8 + 255) / 256 < 148 * 16 ? (n8 + 255) / 256 : 148 * 16);
+    const long long tokens = (long long)B * g.N;
+    const int blocks = (int)((tokens + 7) / 8 < 148 * 16 ? (tokens + 7) / 8 : 148 * 16);
     KernelScope ks("dq_convert_kernel", st);
-    dq_convert_kernel<<<blocks, 256, 0, st>>>(reinterpret_cast<const float4*>(dq32), reinterpret_cast<uint4*>(dq), n8,
-                                              scale);
+    dq_convert_kernel<<<blocks, 256, 0, st>>>(g, il ? 1 : 0, Hq, tokens, dq32, (__nv_bfloat16*)dq, scale);
   }
   return check_launch("dQ convert kernel");
 }

@@ -209,7 +209,8 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const __grid
                       const __grid_constant__ CUtensorMap tm_k_raw, const __grid_constant__ CUtensorMap tm_k_gist,
                       const __grid_constant__ CUtensorMap tm_v_raw, const __grid_constant__ CUtensorMap tm_v_gist,
                       Geom g, int Hq, int Hkv, float scale_log2, __nv_bfloat16* __restrict__ o,
-                      float* __restrict__ lse, int n_raw_units, int n_raw_qt, int n_gist_qt, int pair_heads) {
+                      float* __restrict__ lse, int n_raw_units, int n_raw_qt, int n_gist_qt, int pair_heads,
+                      int interleaved) {
   using SM = FwdSmem<D>;
   extern __shared__ unsigned char smem_dyn[];
   const uint32_t base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
@@ -275,13 +276,15 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const __grid
   if (warp == kTmaWarp) {
     // ------------------------------------------------------------ TMA producer
     if (elect_one()) {
+      // tile coordinate: its first unit (a raw tile of an interleaved tensor spans 128 / r gist units)
+      auto first_unit = [&](bool is_raw, int row0) { return interleaved && is_raw ? row0 / g.r : row0; };
       const CUtensorMap* mq = q_is_raw ? &tm_q_raw : &tm_q_gist;
       mbar_arrive_expect_tx(bar_q, (sv[1] ? 2 : 1) * SM::kTile);
       for (int i = 0; i < 2; ++i) {
         if (!sv[i]) continue;
 #pragma unroll
         for (int sl = 0; sl < D / 64; ++sl)
-          tma_load_4d(sQ[i] + sl * SM::kSlab, mq, bar_q, sl * 64, hh[i], qt[i] * BM, b);
+          tma_load_5d(sQ[i] + sl * SM::kSlab, mq, bar_q, sl * 64, hh[i], 0, first_unit(q_is_raw, qt[i] * BM), b);
       }
       for (int t = 0; t < 2 * nt && ok; ++t) {  // item t: K tile of step t/2 (even t) or its V tile (odd t)
         bool is_raw;
@@ -294,7 +297,8 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const __grid
         mbar_arrive_expect_tx(bar_full + 8 * slot, SM::kTile);
 #pragma unroll
         for (int sl = 0; sl < D / 64; ++sl)
-          tma_load_4d(ring + slot * SM::kTile + sl * SM::kSlab, m, bar_full + 8 * slot, sl * 64, hk, idx * BN, b);
+          tma_load_5d(ring + slot * SM::kTile + sl * SM::kSlab, m, bar_full + 8 * slot, sl * 64, hk, 0,
+                      first_unit(is_raw, idx * BN), b);
       }
       if (!ok) atomicExch(&g_fwd_timeout, 1u);
     }
@@ -464,7 +468,7 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const __grid
         }
         const float inv_l = 1.f / l_run;
         const bool valid = me.row_a + r_in_tile <= me.row_b;
-        const long long tok = (long long)b * g.N + seg_base + me.row_a + r_in_tile;
+        const long long tok = (long long)b * g.N + seg_row_to_token(g, interleaved != 0, q_is_raw, me.row_a + r_in_tile);
         __nv_bfloat16* orow = o + (tok * Hq + me.h) * D + part * (D / kSplit);
 #pragma unroll
         for (int c = 0; c < D / kSplit / 32; ++c) {
@@ -548,6 +552,42 @@ int32_t encode_segment_map_f32(CUtensorMap* map, const void* base, int D, int H,
   return encode_map(map, base, D, H, N, B, seg_first_row, seg_rows, box_cols, box_rows, 4);
 }
 
+int32_t encode_tile_map(CUtensorMap* map, const void* base, int D, int H, int B, int s, int T, int r,
+                        bool interleaved, bool raw_segment) {
+  EncodeFn encode;
+  if (int32_t rc = get_encode_fn(&encode)) return rc;
+  const long long n = T / r, N = (long long)s + T + n;
+  const cuuint64_t row_bytes = (cuuint64_t)H * D * 2;
+  long long first_row, units, unit_rows, unit_stride_rows;
+  if (!interleaved) {
+    first_row = raw_segment ? s : (long long)s + T;
+    units = raw_segment ? T : n;
+    unit_rows = 1;
+    unit_stride_rows = 1;
+  } else if (raw_segment) {
+    first_row = s;
+    units = n;
+    unit_rows = r;
+    unit_stride_rows = r + 1;
+  } else {
+    first_row = (long long)s + r;  // the first gist sits after the first r raw rows
+    units = n;
+    unit_rows = 1;
+    unit_stride_rows = r + 1;
+  }
+  const cuuint64_t dims[5] = {(cuuint64_t)D, (cuuint64_t)H, (cuuint64_t)unit_rows, (cuuint64_t)units, (cuuint64_t)B};
+  const cuuint64_t strides[4] = {(cuuint64_t)D * 2, row_bytes, row_bytes * (cuuint64_t)unit_stride_rows,
+                                 row_bytes * (cuuint64_t)N};
+  const cuuint32_t box[5] = {64, 1, (cuuint32_t)unit_rows, (cuuint32_t)(128 / unit_rows), 1};
+  const cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+  void* addr = const_cast<char*>(static_cast<const char*>(base)) + first_row * row_bytes;
+  CUresult rc = encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, addr, dims, strides, box, estr,
+                       CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                       CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (rc != CUDA_SUCCESS) return fail(UNIGIST_ERR_CUDA, "cuTensorMapEncodeTiled failed with code %d", (int)rc);
+  return UNIGIST_OK;
+}
+
 int32_t encode_map_2d_bf16(CUtensorMap* map, const void* base, long long rows, int cols, int box_rows, int box_cols) {
   EncodeFn encode;
   if (int32_t rc = get_encode_fn(&encode)) return rc;
@@ -566,12 +606,13 @@ int32_t launch_fwd_sm100(const Geom& g, const unigist_problem& p, float scale, c
                          const void* v, void* o, float* lse, cudaStream_t st) {
   const int D = p.head_dim, Hq = p.num_q_heads, Hkv = p.num_kv_heads, B = p.batch;
   CUtensorMap mq_raw, mq_gist, mk_raw, mk_gist, mv_raw, mv_gist;
-  if (int32_t rc = encode_segment_map(&mq_raw, q, D, Hq, g.N, B, g.s, g.T, BM)) return rc;
-  if (int32_t rc = encode_segment_map(&mq_gist, q, D, Hq, g.N, B, g.s + g.T, g.n, BM)) return rc;
-  if (int32_t rc = encode_segment_map(&mk_raw, k, D, Hkv, g.N, B, g.s, g.T, BN)) return rc;
-  if (int32_t rc = encode_segment_map(&mk_gist, k, D, Hkv, g.N, B, g.s + g.T, g.n, BN)) return rc;
-  if (int32_t rc = encode_segment_map(&mv_raw, v, D, Hkv, g.N, B, g.s, g.T, BN)) return rc;
-  if (int32_t rc = encode_segment_map(&mv_gist, v, D, Hkv, g.N, B, g.s + g.T, g.n, BN)) return rc;
+  const bool il = (p.flags & UNIGIST_FLAG_INTERLEAVED) != 0;
+  if (int32_t rc = encode_tile_map(&mq_raw, q, D, Hq, B, g.s, g.T, g.r, il, true)) return rc;
+  if (int32_t rc = encode_tile_map(&mq_gist, q, D, Hq, B, g.s, g.T, g.r, il, false)) return rc;
+  if (int32_t rc = encode_tile_map(&mk_raw, k, D, Hkv, B, g.s, g.T, g.r, il, true)) return rc;
+  if (int32_t rc = encode_tile_map(&mk_gist, k, D, Hkv, B, g.s, g.T, g.r, il, false)) return rc;
+  if (int32_t rc = encode_tile_map(&mv_raw, v, D, Hkv, B, g.s, g.T, g.r, il, true)) return rc;
+  if (int32_t rc = encode_tile_map(&mv_gist, v, D, Hkv, B, g.s, g.T, g.r, il, false)) return rc;
   const int n_raw_qt = (g.T + BM - 1) / BM, n_gist_qt = (g.n + BM - 1) / BM;
   // Two streams per block: neighbouring heads of a KV group when the group size is even,
   // otherwise neighbouring query tiles of one head.
@@ -586,7 +627,7 @@ int32_t launch_fwd_sm100(const Geom& g, const unigist_problem& p, float scale, c
     {
       KernelScope ks("attn_fwd_sm100_kernel", st);
       kern<<<grid, kThreads, smem, st>>>(mq_raw, mq_gist, mk_raw, mk_gist, mv_raw, mv_gist, g, Hq, Hkv, scale_log2,
-                                         (__nv_bfloat16*)o, lse, n_raw_units, n_raw_qt, n_gist_qt, pair_heads);
+                                         (__nv_bfloat16*)o, lse, n_raw_units, n_raw_qt, n_gist_qt, pair_heads, il ? 1 : 0);
     }
     return check_launch("tcgen05 forward kernel");
   };

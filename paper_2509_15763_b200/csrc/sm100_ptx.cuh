@@ -72,6 +72,14 @@ __device__ __forceinline__ void tma_load_4d(uint32_t smem_dst, const CUtensorMap
       : "memory");
 }
 
+__device__ __forceinline__ void tma_load_5d(uint32_t smem_dst, const CUtensorMap* map, uint32_t bar, int c0,
+                                            int c1, int c2, int c3, int c4) {
+  asm volatile(
+      "cp.async.bulk.tensor.5d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
+      ::"r"(smem_dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4)
+      : "memory");
+}
+
 // Adds a shared-memory tile into global memory through a tiled tensor map (fp32 add at the L2);
 // completion is tracked by the issuing thread's bulk async-group.
 __device__ __forceinline__ void tma_reduce_add_4d(const CUtensorMap* map, uint32_t smem_src, int c0, int c1, int c2,
@@ -230,6 +238,15 @@ __device__ __forceinline__ bool elect_one() {
 // out-of-range rows read as zero).
 int32_t encode_segment_map(CUtensorMap* map, const void* base, int D, int H, long long N, int B,
                            long long seg_first_row, long long seg_rows, int box_rows);
+
+// 128-row tile maps over one segment of a [B, N, H, D] bf16 tensor with five dimensions
+// (D, H, row in unit, unit, B), so that one kernel reads shifted and interleaved tensors alike:
+//   shifted:           unit = row of the segment, one row per unit;         tile = 128 units
+//   interleaved raw:   unit = gist unit (r raw rows, stride r + 1 rows);    tile = 128 / r units x r rows
+//   interleaved gist:  unit = gist unit, its one gist row;                  tile = 128 units
+// A tile starts at coordinates (d, h, 0, first unit, b); units past the segment read as zero.
+int32_t encode_tile_map(CUtensorMap* map, const void* base, int D, int H, int B, int s, int T, int r,
+                        bool interleaved, bool raw_segment);
 
 // The same for an fp32 tensor, box = box_cols x 1 x box_rows x 1, no swizzle (rows of the box are
 // box_cols * 4 contiguous bytes in shared memory).  Used for reductions into the tensor.

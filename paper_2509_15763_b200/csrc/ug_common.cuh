@@ -75,10 +75,18 @@ __host__ __device__ inline int unshift_perm(const Geom& g, int t) {
   return p == g.r ? g.s + g.T + u : g.s + u * g.r + p;
 }
 
+// Row of a [B, N, H, D] tensor that holds row `row` of the raw (is_raw) or gist segment: in shifted
+// order, or in interleaved order (Eq. 2) when the caller's tensors were never shifted.
+__host__ __device__ inline int seg_row_to_token(const Geom& g, bool interleaved, bool is_raw, int row) {
+  if (!interleaved) return (is_raw ? g.s : g.s + g.T) + row;
+  return is_raw ? g.s + row + row / g.r : g.s + row * (g.r + 1) + g.r;
+}
+
 // Host side helpers (api.cu).
 int32_t fail(int32_t code, const char* fmt, ...);
 int32_t check_problem(const unigist_problem* p, Geom* g, float* scale);
 int32_t check_launch(const char* what);
+int32_t check_interleaved(const unigist_problem* p, const Geom& g);
 void count_launch(int n = 1);
 // Records a CUDA event before and after the kernels launched in its scope when per-kernel
 // timing is switched on; also counts the launch.

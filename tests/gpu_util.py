@@ -17,6 +17,30 @@ def problem_of(w: synth.Workload, flags: int = 0) -> ug.Problem:
                       w.head_dim, num_sinks=w.num_sinks, flags=flags)
 
 
+def run_attention_interleaved(w: synth.Workload, backward: bool = True, inputs=None):
+    """The same results as run_attention, computed with UNIGIST_FLAG_INTERLEAVED: the library reads the
+    interleaved tensors as they are and writes o, dq, dk, dv interleaved; no shift / unshift call."""
+    dev = torch.device("cuda:0")
+    inp = inputs or synth.attention_inputs(w, with_grad=backward)
+    p = problem_of(w, ug.FLAG_INTERLEAVED)
+    N = ug.unigist_total_len(p)
+    d = {k: v.to(dev) for k, v in inp.items()}
+    o = torch.full_like(d["q"], float("nan"))
+    lse_s = torch.full((w.batch, w.num_q_heads, N), float("nan"), device=dev, dtype=torch.float32)
+    ug.unigist_attn_fwd(p, d["q"], d["k"], d["v"], o, lse_s)
+    up = torch.empty(N, dtype=torch.int32, device=dev)
+    ug.unigist_layout(p, None, up, None)
+    out = {"inputs": inp, "o": o, "lse": lse_s[:, :, up.long()], "lse_shifted": lse_s}
+    if backward:
+        ws = torch.empty(max(ug.unigist_workspace_bytes(p, ug.OP_BWD), 16), dtype=torch.uint8, device=dev)
+        out["dq"] = torch.full_like(d["q"], float("nan"))
+        out["dk"] = torch.full_like(d["k"], float("nan"))
+        out["dv"] = torch.full_like(d["v"], float("nan"))
+        ug.unigist_attn_bwd(p, d["q"], d["k"], d["v"], o, lse_s, d["dout"], out["dq"], out["dk"], out["dv"], ws)
+    ug.unigist_device_status()
+    return out
+
+
 def run_attention(w: synth.Workload, backward: bool = True, dout_fp32: bool = False, inputs=None):
     """-> dict of CUDA tensors in INTERLEAVED order: o, lse [B,Hq,N], dq, dk, dv, plus inputs."""
     dev = torch.device("cuda:0")

@@ -8,7 +8,7 @@ from paper_2509_15763_b200 import synth
 from oracle import oracle
 
 from gpu_util import (TOL_GRAD, TOL_LSE, TOL_O_MAX, TOL_O_MEAN, check_close, f64, problem_of,
-                      run_attention)
+                      run_attention, run_attention_interleaved)
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
@@ -84,6 +84,42 @@ def test_attention_matches_oracle(w):
     check_close("dQ", f64(out["dq"]), dq, TOL_GRAD)
     check_close("dK", f64(out["dk"]), dk, TOL_GRAD)
     check_close("dV", f64(out["dv"]), dv, TOL_GRAD)
+
+
+INTERLEAVED = [w for w in SMALL if w.num_sinks == 0 and w.head_dim == 128 and 128 % w.ratio == 0]
+
+
+@pytest.mark.parametrize("w", INTERLEAVED, ids=lambda w: w.name)
+def test_interleaved_tensors_match_oracle(w):
+    """UNIGIST_FLAG_INTERLEAVED: the shift happens inside the tile addressing, no shift / unshift pass."""
+    out = run_attention_interleaved(w)
+    inp = out["inputs"]
+    k = oracle.window_units(w.window, w.ratio)
+    scale = w.head_dim ** -0.5
+    q, kk, v, do = (f64(inp[n]) for n in ("q", "k", "v", "dout"))
+    o, lse = oracle.attn_fwd(0, w.raw_len, w.ratio, k, scale, q, kk, v)
+    check_close("O", f64(out["o"]), o, TOL_O_MAX, TOL_O_MEAN)
+    check_close("LSE", f64(out["lse"]), lse, TOL_LSE)
+    dq, dk, dv = oracle.attn_bwd(0, w.raw_len, w.ratio, k, scale, q, kk, v, do)
+    check_close("dQ", f64(out["dq"]), dq, TOL_GRAD)
+    check_close("dK", f64(out["dk"]), dk, TOL_GRAD)
+    check_close("dV", f64(out["dv"]), dv, TOL_GRAD)
+    # and bit for bit what the explicit shift -> attention -> unshift route gives (dQ: up to its summation order)
+    ref = run_attention(w, inputs=inp)
+    for n in ("o", "lse", "dk", "dv"):
+        assert torch.equal(out[n], ref[n]), n
+    assert (out["dq"].float() - ref["dq"].float()).abs().max().item() <= 2.0 ** -7
+
+
+def test_interleaved_flag_is_refused_where_the_tiles_do_not_line_up():
+    for w in (SMALL[0], SMALL[1], synth.Workload("r7", 1, 448, 7, 64, 2, 1, 128, seed=1)):
+        p = problem_of(w, ug.FLAG_INTERLEAVED)
+        N = ug.unigist_total_len(p)
+        q = torch.zeros(w.batch, N, w.num_q_heads, w.head_dim, dtype=torch.bfloat16, device=DEV)
+        kv = torch.zeros(w.batch, N, w.num_kv_heads, w.head_dim, dtype=torch.bfloat16, device=DEV)
+        lse = torch.zeros(w.batch, w.num_q_heads, N, dtype=torch.float32, device=DEV)
+        with pytest.raises(ug.UnigistError):
+            ug.unigist_attn_fwd(p, q, kv, kv, torch.empty_like(q), lse)
 
 
 def test_forward_is_deterministic():
