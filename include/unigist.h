@@ -145,8 +145,9 @@ int32_t unigist_attn_bwd(const unigist_problem* p, const void* q, const void* k,
  * The cache is paged: k_cache, v_cache [num_blocks, Hkv, 64, D] device bf16;
  * block_table [B, max_blocks_per_seq] device int32 maps logical block -> physical block.
  *
- *  k, v != NULL: gather from the shifted tensors k, v [B,N,Hkv,D] into the pages named by the
- *      first ceil(L / 64) entries of each block_table row (read only).
+ *  k, v != NULL: gather from the shifted tensors k, v [B,N,Hkv,D] (interleaved tensors with
+ *      UNIGIST_FLAG_INTERLEAVED, for any s and r) into the pages named by the first ceil(L / 64)
+ *      entries of each block_table row (read only).
  *  k == v == NULL: compact IN PLACE a paged cache that holds the whole shifted sequence
  *      (logical position = shifted position; the first ceil(N / 64) entries of each row are
  *      valid and distinct).  The row is rewritten: entries [0, ceil(L/64)) are the compacted

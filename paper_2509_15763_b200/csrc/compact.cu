@@ -14,12 +14,12 @@ __host__ __device__ inline int kept_source(const Geom& g, int c) {
   return g.s + (g.T - g.k * g.r) + (c - g.s - g.n);
 }
 
-// src: shifted [B,N,Hkv,D] (vecs = D/8 16-byte vectors per head row) -> pages.
+// src: shifted (or interleaved) [B,N,Hkv,D] (vecs = D/8 16-byte vectors per head row) -> pages.
 __global__ void __launch_bounds__(256)
 compact_gather_kernel(Geom g, int B, int Hkv, int vecs, int L, const uint4* __restrict__ k,
                       const uint4* __restrict__ v, uint4* __restrict__ kc, uint4* __restrict__ vc,
                       int num_blocks, const int32_t* __restrict__ table, int max_blocks,
-                      int32_t* __restrict__ seq_lens, int32_t* __restrict__ kept_idx) {
+                      int32_t* __restrict__ seq_lens, int32_t* __restrict__ kept_idx, int interleaved) {
   const long long per_tok = (long long)Hkv * vecs;
   const long long total = (long long)B * L * per_tok;
   for (long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x; e < total;
@@ -35,7 +35,8 @@ compact_gather_kernel(Geom g, int B, int Hkv, int vecs, int L, const uint4* __re
     }
     const int blk = table[(long long)b * max_blocks + c / PG];
     if (blk < 0 || blk >= num_blocks) continue;  // never write outside the cache
-    const long long so = (((long long)b * g.N + src) * Hkv + hk) * vecs + vec;
+    const int src_row = interleaved ? shift_perm(g, src) : src;  // k, v given in interleaved order
+    const long long so = (((long long)b * g.N + src_row) * Hkv + hk) * vecs + vec;
     const long long d = (((long long)blk * Hkv + hk) * PG + c % PG) * vecs + vec;
     kc[d] = __ldg(k + so);
     vc[d] = __ldg(v + so);
@@ -117,7 +118,7 @@ int32_t launch_compact_gather(const Geom& g, const unigist_problem& p, const voi
     KernelScope ks("compact_gather_kernel", st);
     compact_gather_kernel<<<grid_for(total), 256, 0, st>>>(
         g, p.batch, p.num_kv_heads, vecs, L, (const uint4*)k, (const uint4*)v, (uint4*)kc, (uint4*)vc,
-        num_blocks, table, max_blocks, seq_lens, kept_idx);
+        num_blocks, table, max_blocks, seq_lens, kept_idx, (p.flags & UNIGIST_FLAG_INTERLEAVED) ? 1 : 0);
   }
   return check_launch("compaction gather kernel");
 }

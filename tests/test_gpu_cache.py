@@ -31,9 +31,12 @@ COMPACT_CASES = [
 
 
 @pytest.mark.parametrize("B,s,T,r,W,Hkv,D", COMPACT_CASES)
-@pytest.mark.parametrize("mode", ["gather", "inplace"])
+@pytest.mark.parametrize("mode", ["gather", "gather_interleaved", "inplace"])
 def test_compaction_matches_oracle(B, s, T, r, W, Hkv, D, mode):
-    p = ug.Problem(B, T, r, W, Hkv, Hkv, D, num_sinks=s)
+    interleaved = mode == "gather_interleaved"  # K, V handed over in interleaved order (UNIGIST_FLAG_INTERLEAVED)
+    if interleaved:
+        mode = "gather"
+    p = ug.Problem(B, T, r, W, Hkv, Hkv, D, num_sinks=s, flags=ug.FLAG_INTERLEAVED if interleaved else 0)
     N, L = ug.unigist_total_len(p), ug.unigist_compact_len(p)
     k_units = oracle.window_units(W, r)
     kept = oracle.kept_set(s, T, r, k_units)              # interleaved indices, cache order
@@ -59,7 +62,11 @@ def test_compaction_matches_oracle(B, s, T, r, W, Hkv, D, mode):
     kept_idx = torch.full((B, L), -1, dtype=torch.int32, device=DEV)
     ws = torch.empty(max(ug.unigist_workspace_bytes(p, ug.OP_COMPACT), 16), dtype=torch.uint8, device=DEV)
     if mode == "gather":
-        ug.unigist_kv_compact(p, k_sh.to(DEV), v_sh.to(DEV), kc_d, vc_d, table_d, lens, kept_idx, ws)
+        src_k, src_v = k_sh, v_sh
+        if interleaved:  # the same tokens, in the order of Eq. 2
+            src_k, src_v = k_sh[:, torch.from_numpy(up).long()], v_sh[:, torch.from_numpy(up).long()]
+        ug.unigist_kv_compact(p, src_k.contiguous().to(DEV), src_v.contiguous().to(DEV), kc_d, vc_d, table_d, lens,
+                              kept_idx, ws)
     else:
         ug.unigist_kv_compact(p, None, None, kc_d, vc_d, table_d, lens, kept_idx, ws)
     torch.cuda.synchronize()
