@@ -283,6 +283,22 @@ def bench_decode(dev, iters=20):
             "l2_policy": "K+V (2.4 GB) exceed L2, every call streams from HBM"}
 
 
+def reduce_over_ranks(dist, times_ms, device):
+    """Replicas share nothing on the data path; the job's time is that of the slowest rank.
+    -> the element-wise MAX of `times_ms` over all ranks (the list itself without a process group)."""
+    import torch
+
+    t = torch.tensor(list(times_ms), dtype=torch.float64, device=device)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return t.tolist()
+
+
+def job_value(world, flop_per_replica_step, steps, total_ms):
+    """Whole-job effective TFLOP/s: every rank did `steps` steps of its own replica in `total_ms`."""
+    return world * flop_per_replica_step * steps / (total_ms * 1e-3) / 1e12
+
+
 def run_ours(args, w):
     import torch
 
@@ -367,18 +383,15 @@ def run_ours(args, w):
     barrier()
     e2e_ms = e0.elapsed_time(e1)
 
-    t = torch.tensor([total_ms, e2e_ms], dtype=torch.float64, device=dev)
-    if dist:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    total_ms, e2e_ms = t.tolist()
+    total_ms, e2e_ms = reduce_over_ranks(dist, [total_ms, e2e_ms], dev)
     if rank != 0:
         if dist:
             dist.destroy_process_group()
         return
 
     peaks = measured_peaks()
-    value = world * path.flops * args.steps / (total_ms * 1e-3) / 1e12
-    e2e_value = world * path.flops * args.steps / (e2e_ms * 1e-3) / 1e12
+    value = job_value(world, path.flops, args.steps, total_ms)
+    e2e_value = job_value(world, path.flops, args.steps, e2e_ms)
     attn = {k: v for k, v in per_kernel.items() if k in KERNEL_FLOP_PER_PAIR_D}
     top = max(attn, key=lambda k: attn[k][1])
     cnt, tot = attn[top]
