@@ -218,9 +218,7 @@ int32_t unigist_attn_fwd(const unigist_problem* p, const void* q, const void* k,
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || !aligned16(lse))
     return fail(UNIGIST_ERR_ALIGNMENT, "tensor pointers must be 16-byte aligned");
   if (int32_t rc = check_interleaved(p, g)) return rc;
-  // Tensor-core path for sequences without sinks; the CUDA-core kernels cover sink prefixes.
-  if (g.s == 0) return launch_fwd_sm100(g, *p, scale, q, k, v, o, lse, (cudaStream_t)stream);
-  return launch_fwd_simt(g, *p, scale, q, k, v, o, lse, (cudaStream_t)stream);
+  return launch_fwd_sm100(g, *p, scale, q, k, v, o, lse, (cudaStream_t)stream);
 }
 
 int32_t unigist_device_status(void) {

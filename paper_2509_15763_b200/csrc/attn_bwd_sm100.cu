@@ -1047,7 +1047,7 @@ attn_bwd_fused_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const 
     if (ok && n_iter > 0) ok = mbar_wait_warp(bar_final, 0);
     if (ok) {
       tc_fence_after();
-      const long long tok = (long long)b * g.N + seg_row_to_token(g, interleaved != 0, key_is_raw, key_valid ? key : key_a);
+      const long long tok = (long long)b * g.N + seg_row_to_token(g, interleaved != 0, key_is_raw ? kSegRaw : kSegGist, key_valid ? key : key_a);
       // this warp stores columns [64 hf, 64 hf + 64) of dK and of dV
 #pragma unroll
       for (int which = 0; which < 2; ++which) {
@@ -1147,10 +1147,10 @@ int32_t launch_bwd_sm100(const Geom& g, const unigist_problem& p, float scale, c
   const long long first[2] = {g.s, (long long)g.s + g.T}, len[2] = {g.T, g.n};
   for (int sgm = 0; sgm < 2; ++sgm) {
     if (fused) {  // 128-row tile maps that read shifted or interleaved tensors
-      if (int32_t rc = encode_tile_map(&mq[sgm], q, D, Hq, B, g.s, g.T, g.r, il, sgm == 0)) return rc;
-      if (int32_t rc = encode_tile_map(&md[sgm], do_src, D, Hq, B, g.s, g.T, g.r, il, sgm == 0)) return rc;
-      if (int32_t rc = encode_tile_map(&mk[sgm], k, D, Hkv, B, g.s, g.T, g.r, il, sgm == 0)) return rc;
-      if (int32_t rc = encode_tile_map(&mv[sgm], v, D, Hkv, B, g.s, g.T, g.r, il, sgm == 0)) return rc;
+      if (int32_t rc = encode_tile_map(&mq[sgm], q, D, Hq, B, g.s, g.T, g.r, il, sgm == 0 ? kSegRaw : kSegGist)) return rc;
+      if (int32_t rc = encode_tile_map(&md[sgm], do_src, D, Hq, B, g.s, g.T, g.r, il, sgm == 0 ? kSegRaw : kSegGist)) return rc;
+      if (int32_t rc = encode_tile_map(&mk[sgm], k, D, Hkv, B, g.s, g.T, g.r, il, sgm == 0 ? kSegRaw : kSegGist)) return rc;
+      if (int32_t rc = encode_tile_map(&mv[sgm], v, D, Hkv, B, g.s, g.T, g.r, il, sgm == 0 ? kSegRaw : kSegGist)) return rc;
       continue;
     }
     if (int32_t rc = encode_segment_map(&mq[sgm], q, D, Hq, g.N, B, first[sgm], len[sgm], 128)) return rc;

@@ -56,81 +56,89 @@ struct FwdSmem {
   static constexpr int kBytes = kXchOff + 2 * kSplit * BM * 4 + 1024 /*align*/;
 };
 
-// One query stream: a 128-row tile of one head, with the key-tile interval it can see.
+// One query stream: a 128-row tile of one head, with the key tiles it can see in each segment.
 struct Stream {
   bool valid;
   int h, row_a, row_b;      // head; first / last row inside the segment
   RowIv iv_a, iv_b;         // visible intervals of the first / last row
-  int raw_lo, raw_hi, n_gist;  // raw key tiles [raw_lo, raw_hi], gist key tiles [0, n_gist)
-  __device__ bool sees(bool is_raw, int idx) const {
-    return valid && (is_raw ? (idx >= raw_lo && idx <= raw_hi) : idx < n_gist);
+  int n_sink;               // sink key tiles [0, n_sink)
+  int raw_lo, raw_hi;       // raw key tiles [raw_lo, raw_hi] (none if raw_hi < raw_lo)
+  int n_gist;               // gist key tiles [0, n_gist)
+  __device__ bool sees(int seg, int idx) const {
+    if (!valid) return false;
+    if (seg == kSegRaw) return idx >= raw_lo && idx <= raw_hi;
+    return idx < (seg == kSegGist ? n_gist : n_sink);
   }
 };
 
-__device__ Stream make_stream(const Geom& g, bool valid, int h, int qt, bool q_is_raw) {
+__device__ Stream make_stream(const Geom& g, bool valid, int h, int qt, int qseg) {
   Stream s;
   s.valid = valid;
   s.h = h;
-  const int seg_len = q_is_raw ? g.T : g.n;
-  const int seg_base = q_is_raw ? g.s : g.s + g.T;
   s.row_a = qt * BM;
-  s.row_b = min(s.row_a + BM - 1, seg_len - 1);
+  s.row_b = min(s.row_a + BM - 1, seg_len(g, qseg) - 1);
   if (!valid) {
     s.row_a = s.row_b = 0;
   }
-  s.iv_a = row_intervals(g, seg_base + s.row_a);
-  s.iv_b = row_intervals(g, seg_base + s.row_b);
+  s.iv_a = row_intervals(g, seg_base(g, qseg) + s.row_a);
+  s.iv_b = row_intervals(g, seg_base(g, qseg) + s.row_b);
+  s.n_sink = s.iv_b.hi_sink >= 0 ? s.iv_b.hi_sink / BN + 1 : 0;
   s.raw_lo = s.iv_a.lo_raw / BN;
-  s.raw_hi = s.iv_b.hi_raw / BN;
+  s.raw_hi = s.iv_b.hi_raw >= 0 ? s.iv_b.hi_raw / BN : -1;
   s.n_gist = s.iv_b.hi_gist >= 0 ? s.iv_b.hi_gist / BN + 1 : 0;
   return s;
 }
 
-// Key tiles the block visits: the union of its streams' intervals; `n_first` tiles of the query
-// rows' own segment in descending order from `first_hi`, then `n_second` tiles of the other
-// segment ascending from `second_lo`.
+// Key tiles the block visits: the union of its streams' tiles, in three runs.  First the query rows' own
+// segment downwards from the tile that holds the diagonal (every row sees itself there, so the running
+// maximum is finite from a stream's first tile on), then the other segments upwards.
 struct TileSeq {
-  int n_first, first_hi, n_second, second_lo;
-  bool first_is_raw;
-  __device__ int count() const { return n_first + n_second; }
-  __device__ void at(int j, bool& is_raw, int& idx) const {
-    if (j < n_first) {
-      is_raw = first_is_raw;
-      idx = first_hi - j;
+  int seg[3], cnt[3], start[3];  // run i: cnt[i] tiles of segment seg[i]; run 0 counts down from start[0]
+  __device__ int count() const { return cnt[0] + cnt[1] + cnt[2]; }
+  __device__ void at(int j, int& sg, int& idx) const {
+    if (j < cnt[0]) {
+      sg = seg[0];
+      idx = start[0] - j;
+    } else if (j < cnt[0] + cnt[1]) {
+      sg = seg[1];
+      idx = start[1] + (j - cnt[0]);
     } else {
-      is_raw = !first_is_raw;
-      idx = second_lo + (j - n_first);
+      sg = seg[2];
+      idx = start[2] + (j - cnt[0] - cnt[1]);
     }
   }
 };
 
-__device__ TileSeq make_tile_seq(const Stream& a, const Stream& b, bool q_is_raw) {
-  int raw_lo, raw_hi, n_gist;
+__device__ TileSeq make_tile_seq(const Stream& a, const Stream& b, int qseg) {
+  int n_sink, raw_lo, raw_hi, n_gist;
   if (a.valid && b.valid) {
+    n_sink = max(a.n_sink, b.n_sink);
     raw_lo = min(a.raw_lo, b.raw_lo);
     raw_hi = max(a.raw_hi, b.raw_hi);
     n_gist = max(a.n_gist, b.n_gist);
   } else {
     const Stream& s = a.valid ? a : b;
+    n_sink = s.n_sink;
     raw_lo = s.raw_lo;
     raw_hi = s.raw_hi;
     n_gist = s.n_gist;
   }
-  const int n_raw = raw_hi - raw_lo + 1;
-  TileSeq s;
-  s.first_is_raw = q_is_raw;
-  if (q_is_raw) {
-    s.n_first = n_raw;
-    s.first_hi = raw_hi;
-    s.n_second = n_gist;
-    s.second_lo = 0;
-  } else {
-    s.n_first = n_gist;
-    s.first_hi = n_gist - 1;
-    s.n_second = n_raw;
-    s.second_lo = raw_lo;
+  const int n_raw = raw_hi >= raw_lo ? raw_hi - raw_lo + 1 : 0;
+  TileSeq t;
+  if (qseg == kSegRaw) {
+    t.seg[0] = kSegRaw, t.cnt[0] = n_raw, t.start[0] = raw_hi;
+    t.seg[1] = kSegGist, t.cnt[1] = n_gist, t.start[1] = 0;
+    t.seg[2] = kSegSink, t.cnt[2] = n_sink, t.start[2] = 0;
+  } else if (qseg == kSegGist) {
+    t.seg[0] = kSegGist, t.cnt[0] = n_gist, t.start[0] = n_gist - 1;
+    t.seg[1] = kSegRaw, t.cnt[1] = n_raw, t.start[1] = raw_lo;
+    t.seg[2] = kSegSink, t.cnt[2] = n_sink, t.start[2] = 0;
+  } else {  // sink queries see sinks only
+    t.seg[0] = kSegSink, t.cnt[0] = n_sink, t.start[0] = n_sink - 1;
+    t.seg[1] = kSegRaw, t.cnt[1] = 0, t.start[1] = 0;
+    t.seg[2] = kSegGist, t.cnt[2] = 0, t.start[2] = 0;
   }
-  return s;
+  return t;
 }
 
 __device__ __forceinline__ float max3(float a, float b, float c) {
@@ -205,12 +213,13 @@ __device__ __forceinline__ float row_exp(const uint32_t (&sc)[kCols], uint32_t t
 
 template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
-attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const __grid_constant__ CUtensorMap tm_q_gist,
+attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_sink, const __grid_constant__ CUtensorMap tm_q_raw,
+                      const __grid_constant__ CUtensorMap tm_q_gist, const __grid_constant__ CUtensorMap tm_k_sink,
                       const __grid_constant__ CUtensorMap tm_k_raw, const __grid_constant__ CUtensorMap tm_k_gist,
-                      const __grid_constant__ CUtensorMap tm_v_raw, const __grid_constant__ CUtensorMap tm_v_gist,
-                      Geom g, int Hq, int Hkv, float scale_log2, __nv_bfloat16* __restrict__ o,
-                      float* __restrict__ lse, int n_raw_units, int n_raw_qt, int n_gist_qt, int pair_heads,
-                      int interleaved) {
+                      const __grid_constant__ CUtensorMap tm_v_sink, const __grid_constant__ CUtensorMap tm_v_raw,
+                      const __grid_constant__ CUtensorMap tm_v_gist, Geom g, int Hq, int Hkv, float scale_log2,
+                      __nv_bfloat16* __restrict__ o, float* __restrict__ lse, int n_sink_units, int n_raw_units,
+                      int pair_heads, int interleaved) {
   using SM = FwdSmem<D>;
   extern __shared__ unsigned char smem_dyn[];
   const uint32_t base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
@@ -227,12 +236,12 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const __grid
 
   const int warp = threadIdx.x >> 5;
   const int b = blockIdx.z;
-  // heaviest units first: gist units from the end, then raw units from the end
+  // heaviest units first: gist units from the end, then raw units from the end, sink units last
   const int u_lin = gridDim.x - 1 - blockIdx.x;
-  const bool q_is_raw = u_lin < n_raw_units;
-  const int u = q_is_raw ? u_lin : u_lin - n_raw_units;
-  const int n_qt = q_is_raw ? n_raw_qt : n_gist_qt;
-  const int seg_base = q_is_raw ? g.s : g.s + g.T;  // shifted position of the segment's row 0
+  const int qseg = u_lin < n_sink_units ? kSegSink : (u_lin < n_sink_units + n_raw_units ? kSegRaw : kSegGist);
+  const int u = u_lin - (qseg == kSegSink ? 0 : (qseg == kSegRaw ? n_sink_units : n_sink_units + n_raw_units));
+  const int n_qt = (seg_len(g, qseg) + BM - 1) / BM;
+  const int q_seg_base = seg_base(g, qseg);  // shifted position of the segment's row 0
   int qt[2], hh[2];
   bool sv[2];
   if (pair_heads) {
@@ -248,8 +257,8 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const __grid
     sv[1] = qt[1] < n_qt;
   }
   const int hk = hh[0] / (Hq / Hkv);  // both streams share the KV head
-  const Stream str0 = make_stream(g, sv[0], hh[0], qt[0], q_is_raw), str1 = make_stream(g, sv[1], hh[1], qt[1], q_is_raw);
-  const TileSeq seq = make_tile_seq(str0, str1, q_is_raw);
+  const Stream str0 = make_stream(g, sv[0], hh[0], qt[0], qseg), str1 = make_stream(g, sv[1], hh[1], qt[1], qseg);
+  const TileSeq seq = make_tile_seq(str0, str1, qseg);
   const int nt = seq.count();
 
   if (threadIdx.x == 0) {
@@ -277,20 +286,20 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const __grid
     // ------------------------------------------------------------ TMA producer
     if (elect_one()) {
       // tile coordinate: its first unit (a raw tile of an interleaved tensor spans 128 / r gist units)
-      auto first_unit = [&](bool is_raw, int row0) { return interleaved && is_raw ? row0 / g.r : row0; };
-      const CUtensorMap* mq = q_is_raw ? &tm_q_raw : &tm_q_gist;
+      auto first_unit = [&](int sg, int row0) { return interleaved && sg == kSegRaw ? row0 / g.r : row0; };
+      const CUtensorMap* mq = qseg == kSegRaw ? &tm_q_raw : (qseg == kSegGist ? &tm_q_gist : &tm_q_sink);
       mbar_arrive_expect_tx(bar_q, (sv[1] ? 2 : 1) * SM::kTile);
       for (int i = 0; i < 2; ++i) {
         if (!sv[i]) continue;
 #pragma unroll
         for (int sl = 0; sl < D / 64; ++sl)
-          tma_load_5d(sQ[i] + sl * SM::kSlab, mq, bar_q, sl * 64, hh[i], 0, first_unit(q_is_raw, qt[i] * BM), b);
+          tma_load_5d(sQ[i] + sl * SM::kSlab, mq, bar_q, sl * 64, hh[i], 0, first_unit(qseg, qt[i] * BM), b);
       }
       for (int t = 0; t < 2 * nt && ok; ++t) {  // item t: K tile of step t/2 (even t) or its V tile (odd t)
-        bool is_raw;
-        int idx;
-        seq.at(t >> 1, is_raw, idx);
-        const CUtensorMap* m = (t & 1) ? (is_raw ? &tm_v_raw : &tm_v_gist) : (is_raw ? &tm_k_raw : &tm_k_gist);
+        int sg, idx;
+        seq.at(t >> 1, sg, idx);
+        const CUtensorMap* m = (t & 1) ? (sg == kSegRaw ? &tm_v_raw : (sg == kSegGist ? &tm_v_gist : &tm_v_sink))
+                                       : (sg == kSegRaw ? &tm_k_raw : (sg == kSegGist ? &tm_k_gist : &tm_k_sink));
         const int slot = t % kStages, use = t / kStages;
         if (use > 0) ok = mbar_wait(bar_empty + 8 * slot, (use - 1) & 1);
         if (!ok) break;
@@ -298,7 +307,7 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const __grid
 #pragma unroll
         for (int sl = 0; sl < D / 64; ++sl)
           tma_load_5d(ring + slot * SM::kTile + sl * SM::kSlab, m, bar_full + 8 * slot, sl * 64, hk, 0,
-                      first_unit(is_raw, idx * BN), b);
+                      first_unit(sg, idx * BN), b);
       }
       if (!ok) atomicExch(&g_fwd_timeout, 1u);
     }
@@ -334,30 +343,29 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const __grid
       };
       auto slot_of = [&](int t) { return t % kStages; };
       auto wait_full = [&](int t) { return mbar_wait(bar_full + 8 * slot_of(t), (t / kStages) & 1); };
-      bool is_raw, nx_raw = false;
-      int idx, nx_idx = 0;
+      int sg, nx_sg = 0, idx, nx_idx = 0;
       ok = mbar_wait(bar_q, 0);
       if (ok && nt > 0) {
-        seq.at(0, is_raw, idx);
+        seq.at(0, sg, idx);
         ok = wait_full(0);
         if (ok) {
           tc_fence_after();
-          if (str0.sees(is_raw, idx)) issue_s(0, ring + slot_of(0) * SM::kTile);
-          if (str1.sees(is_raw, idx)) issue_s(1, ring + slot_of(0) * SM::kTile);
+          if (str0.sees(sg, idx)) issue_s(0, ring + slot_of(0) * SM::kTile);
+          if (str1.sees(sg, idx)) issue_s(1, ring + slot_of(0) * SM::kTile);
           umma_commit(bar_empty + 8 * slot_of(0));
         }
       }
       for (int j = 0; j < nt && ok; ++j) {
-        seq.at(j, is_raw, idx);
+        seq.at(j, sg, idx);
         const bool has_next = j + 1 < nt;
-        if (has_next) seq.at(j + 1, nx_raw, nx_idx);
+        if (has_next) seq.at(j + 1, nx_sg, nx_idx);
         const int tv = 2 * j + 1, tk = 2 * j + 2;
         ok = wait_full(tv);
         if (!ok) break;
 #pragma unroll
         for (int i = 0; i < 2; ++i) {
           const Stream& si = i ? str1 : str0;
-          if (si.sees(is_raw, idx)) {
+          if (si.sees(sg, idx)) {
             ok = mbar_wait(bar_p[i], n_pv[i] & 1);
             if (!ok) break;
             tc_fence_after();
@@ -370,7 +378,7 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const __grid
               if (!ok) break;
               tc_fence_after();
             }
-            if (si.sees(nx_raw, nx_idx)) issue_s(i, ring + slot_of(tk) * SM::kTile);
+            if (si.sees(nx_sg, nx_idx)) issue_s(i, ring + slot_of(tk) * SM::kTile);
             if (i == 1) umma_commit(bar_empty + 8 * slot_of(tk));
           }
         }
@@ -389,21 +397,24 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const __grid
     if (me.valid) {
       const int r_in_tile = (warp & 3) * 32 + (threadIdx.x & 31);
       const int row = min(me.row_a + r_in_tile, me.row_b);
-      const RowIv my = row_intervals(g, seg_base + row);
+      const RowIv my = row_intervals(g, q_seg_base + row);
       const uint32_t lane_base = static_cast<uint32_t>((warp & 3) * 32) << 16;
       const uint32_t tS = tmem + i * 128 + lane_base, tO = tmem + 256 + i * 128 + lane_base + part * (D / kSplit);
       float m_run = -INFINITY, l_run = 0.f;
       int cnt = 0;
 
       for (int j = 0; j < nt && ok; ++j) {
-        bool is_raw;
-        int idx;
-        seq.at(j, is_raw, idx);
-        if (!me.sees(is_raw, idx)) continue;
+        int sg, idx;
+        seq.at(j, sg, idx);
+        if (!me.sees(sg, idx)) continue;
         const int col0 = idx * BN;
         bool full;
         int lo, hi;  // visible columns of this row, relative to the tile
-        if (is_raw) {
+        if (sg == kSegSink) {
+          full = col0 + BN - 1 <= me.iv_a.hi_sink;
+          lo = -part * kCols;
+          hi = my.hi_sink - col0 - part * kCols;
+        } else if (sg == kSegRaw) {
           full = col0 >= me.iv_b.lo_raw && col0 + BN - 1 <= me.iv_a.hi_raw;
           lo = my.lo_raw - col0 - part * kCols;
           hi = my.hi_raw - col0 - part * kCols;
@@ -468,7 +479,7 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const __grid
         }
         const float inv_l = 1.f / l_run;
         const bool valid = me.row_a + r_in_tile <= me.row_b;
-        const long long tok = (long long)b * g.N + seg_row_to_token(g, interleaved != 0, q_is_raw, me.row_a + r_in_tile);
+        const long long tok = (long long)b * g.N + seg_row_to_token(g, interleaved != 0, qseg, me.row_a + r_in_tile);
         __nv_bfloat16* orow = o + (tok * Hq + me.h) * D + part * (D / kSplit);
 #pragma unroll
         for (int c = 0; c < D / kSplit / 32; ++c) {
@@ -488,7 +499,7 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const __grid
           }
         }
         if (valid && part == 0)
-          lse[((long long)b * Hq + me.h) * g.N + seg_base + me.row_a + r_in_tile] =
+          lse[((long long)b * Hq + me.h) * g.N + q_seg_base + me.row_a + r_in_tile] =
               (m_run + log2f(l_run)) * 0.6931471805599453f;
       } else {
         atomicExch(&g_fwd_timeout, 1u);
@@ -553,13 +564,19 @@ int32_t encode_segment_map_f32(CUtensorMap* map, const void* base, int D, int H,
 }
 
 int32_t encode_tile_map(CUtensorMap* map, const void* base, int D, int H, int B, int s, int T, int r,
-                        bool interleaved, bool raw_segment) {
+                        bool interleaved, int segment) {
+  const bool raw_segment = segment == kSegRaw;
   EncodeFn encode;
   if (int32_t rc = get_encode_fn(&encode)) return rc;
   const long long n = T / r, N = (long long)s + T + n;
   const cuuint64_t row_bytes = (cuuint64_t)H * D * 2;
   long long first_row, units, unit_rows, unit_stride_rows;
-  if (!interleaved) {
+  if (segment == kSegSink) {  // the sinks are a prefix in either order; a tensor map cannot be empty
+    first_row = 0;
+    units = s > 0 ? s : 1;
+    unit_rows = 1;
+    unit_stride_rows = 1;
+  } else if (!interleaved) {
     first_row = raw_segment ? s : (long long)s + T;
     units = raw_segment ? T : n;
     unit_rows = 1;
@@ -605,29 +622,30 @@ int32_t encode_map_2d_bf16(CUtensorMap* map, const void* base, long long rows, i
 int32_t launch_fwd_sm100(const Geom& g, const unigist_problem& p, float scale, const void* q, const void* k,
                          const void* v, void* o, float* lse, cudaStream_t st) {
   const int D = p.head_dim, Hq = p.num_q_heads, Hkv = p.num_kv_heads, B = p.batch;
-  CUtensorMap mq_raw, mq_gist, mk_raw, mk_gist, mv_raw, mv_gist;
+  CUtensorMap mq[3], mk[3], mv[3];  // per segment: sinks, raw, gists
   const bool il = (p.flags & UNIGIST_FLAG_INTERLEAVED) != 0;
-  if (int32_t rc = encode_tile_map(&mq_raw, q, D, Hq, B, g.s, g.T, g.r, il, true)) return rc;
-  if (int32_t rc = encode_tile_map(&mq_gist, q, D, Hq, B, g.s, g.T, g.r, il, false)) return rc;
-  if (int32_t rc = encode_tile_map(&mk_raw, k, D, Hkv, B, g.s, g.T, g.r, il, true)) return rc;
-  if (int32_t rc = encode_tile_map(&mk_gist, k, D, Hkv, B, g.s, g.T, g.r, il, false)) return rc;
-  if (int32_t rc = encode_tile_map(&mv_raw, v, D, Hkv, B, g.s, g.T, g.r, il, true)) return rc;
-  if (int32_t rc = encode_tile_map(&mv_gist, v, D, Hkv, B, g.s, g.T, g.r, il, false)) return rc;
-  const int n_raw_qt = (g.T + BM - 1) / BM, n_gist_qt = (g.n + BM - 1) / BM;
+  for (int sg = 0; sg < 3; ++sg) {
+    if (int32_t rc = encode_tile_map(&mq[sg], q, D, Hq, B, g.s, g.T, g.r, il, sg)) return rc;
+    if (int32_t rc = encode_tile_map(&mk[sg], k, D, Hkv, B, g.s, g.T, g.r, il, sg)) return rc;
+    if (int32_t rc = encode_tile_map(&mv[sg], v, D, Hkv, B, g.s, g.T, g.r, il, sg)) return rc;
+  }
+  const int n_sink_qt = (g.s + BM - 1) / BM, n_raw_qt = (g.T + BM - 1) / BM, n_gist_qt = (g.n + BM - 1) / BM;
   // Two streams per block: neighbouring heads of a KV group when the group size is even,
   // otherwise neighbouring query tiles of one head.
   const int pair_heads = (Hq / Hkv) % 2 == 0 ? 1 : 0;
+  const int n_sink_units = pair_heads ? n_sink_qt : (n_sink_qt + 1) / 2;
   const int n_raw_units = pair_heads ? n_raw_qt : (n_raw_qt + 1) / 2;
   const int n_gist_units = pair_heads ? n_gist_qt : (n_gist_qt + 1) / 2;
-  dim3 grid(n_raw_units + n_gist_units, pair_heads ? Hq / 2 : Hq, B);
+  dim3 grid(n_sink_units + n_raw_units + n_gist_units, pair_heads ? Hq / 2 : Hq, B);
   const float scale_log2 = scale * 1.4426950408889634f;
   auto go = [&](auto kern, size_t smem) -> int32_t {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return fail(UNIGIST_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
     {
       KernelScope ks("attn_fwd_sm100_kernel", st);
-      kern<<<grid, kThreads, smem, st>>>(mq_raw, mq_gist, mk_raw, mk_gist, mv_raw, mv_gist, g, Hq, Hkv, scale_log2,
-                                         (__nv_bfloat16*)o, lse, n_raw_units, n_raw_qt, n_gist_qt, pair_heads, il ? 1 : 0);
+      kern<<<grid, kThreads, smem, st>>>(mq[0], mq[1], mq[2], mk[0], mk[1], mk[2], mv[0], mv[1], mv[2], g, Hq, Hkv,
+                                         scale_log2, (__nv_bfloat16*)o, lse, n_sink_units, n_raw_units, pair_heads,
+                                         il ? 1 : 0);
     }
     return check_launch("tcgen05 forward kernel");
   };

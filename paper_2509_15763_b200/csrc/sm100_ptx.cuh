@@ -241,12 +241,12 @@ int32_t encode_segment_map(CUtensorMap* map, const void* base, int D, int H, lon
 
 // 128-row tile maps over one segment of a [B, N, H, D] bf16 tensor with five dimensions
 // (D, H, row in unit, unit, B), so that one kernel reads shifted and interleaved tensors alike:
-//   shifted:           unit = row of the segment, one row per unit;         tile = 128 units
+//   sinks, or shifted: unit = row of the segment, one row per unit;         tile = 128 units
 //   interleaved raw:   unit = gist unit (r raw rows, stride r + 1 rows);    tile = 128 / r units x r rows
 //   interleaved gist:  unit = gist unit, its one gist row;                  tile = 128 units
 // A tile starts at coordinates (d, h, 0, first unit, b); units past the segment read as zero.
 int32_t encode_tile_map(CUtensorMap* map, const void* base, int D, int H, int B, int s, int T, int r,
-                        bool interleaved, bool raw_segment);
+                        bool interleaved, int segment /* kSegSink, kSegRaw, kSegGist */);
 
 // The same for an fp32 tensor, box = box_cols x 1 x box_rows x 1, no swizzle (rows of the box are
 // box_cols * 4 contiguous bytes in shared memory).  Used for reductions into the tensor.

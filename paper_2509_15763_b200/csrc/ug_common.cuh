@@ -75,11 +75,17 @@ __host__ __device__ inline int unshift_perm(const Geom& g, int t) {
   return p == g.r ? g.s + g.T + u : g.s + u * g.r + p;
 }
 
-// Row of a [B, N, H, D] tensor that holds row `row` of the raw (is_raw) or gist segment: in shifted
-// order, or in interleaved order (Eq. 2) when the caller's tensors were never shifted.
-__host__ __device__ inline int seg_row_to_token(const Geom& g, bool interleaved, bool is_raw, int row) {
-  if (!interleaved) return (is_raw ? g.s : g.s + g.T) + row;
-  return is_raw ? g.s + row + row / g.r : g.s + row * (g.r + 1) + g.r;
+// Row of a [B, N, H, D] tensor that holds row `row` of a segment: in shifted order, or in
+// interleaved order (Eq. 2) when the caller's tensors were never shifted.
+// The three segments of the shifted order.
+enum { kSegSink = 0, kSegRaw = 1, kSegGist = 2 };
+__host__ __device__ inline int seg_len(const Geom& g, int seg) { return seg == kSegRaw ? g.T : (seg == kSegGist ? g.n : g.s); }
+__host__ __device__ inline int seg_base(const Geom& g, int seg) {  // shifted position of the segment's row 0
+  return seg == kSegRaw ? g.s : (seg == kSegGist ? g.s + g.T : 0);
+}
+__host__ __device__ inline int seg_row_to_token(const Geom& g, bool interleaved, int seg, int row) {
+  if (!interleaved || seg == kSegSink) return seg_base(g, seg) + row;
+  return seg == kSegRaw ? g.s + row + row / g.r : g.s + row * (g.r + 1) + g.r;
 }
 
 // Host side helpers (api.cu).
