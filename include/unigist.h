@@ -57,8 +57,8 @@ typedef enum {
  * the loads (a raw tile is r rows of each of 128 / r consecutive gist units, a gist tile is one row per
  * unit) and outputs are stored at their interleaved row, so no separate shift / unshift pass is needed.
  * lse stays in shifted order (it is the tensor the backward reads back).  Supported when ratio divides
- * 128, head_dim is 128 and there are no sinks; otherwise the calls return UNIGIST_ERR_UNSUPPORTED and
- * the caller uses unigist_gist_shift / unigist_gist_unshift.
+ * 128 and head_dim is 128; otherwise the calls return UNIGIST_ERR_UNSUPPORTED and the caller uses
+ * unigist_gist_shift / unigist_gist_unshift.
  */
 #define UNIGIST_FLAG_INTERLEAVED 2u
 

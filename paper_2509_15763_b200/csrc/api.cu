@@ -93,11 +93,11 @@ static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 // UNIGIST_FLAG_INTERLEAVED needs the tile addressing of the tensor-core kernels for head_dim 128.
 int32_t check_interleaved(const unigist_problem* p, const Geom& g) {
   if (!(p->flags & UNIGIST_FLAG_INTERLEAVED)) return UNIGIST_OK;
-  if (g.s != 0 || p->head_dim != 128 || 128 % g.r != 0)
+  if (p->head_dim != 128 || 128 % g.r != 0)
     return fail(UNIGIST_ERR_UNSUPPORTED,
-                "interleaved tensors need no sinks, head_dim 128 and a ratio that divides 128 "
-                "(got s = %d, D = %d, r = %d): shift the tensors with unigist_gist_shift instead",
-                g.s, p->head_dim, g.r);
+                "interleaved tensors need head_dim 128 and a ratio that divides 128 (got D = %d, r = %d): "
+                "shift the tensors with unigist_gist_shift instead",
+                p->head_dim, g.r);
   return UNIGIST_OK;
 }
 
@@ -149,8 +149,8 @@ size_t unigist_workspace_bytes(const unigist_problem* p, int32_t op) {
       size_t b = align_up((size_t)p->batch * p->num_q_heads * g.N * sizeof(float), 256);
       if (p->flags & UNIGIST_FLAG_DOUT_FP32)
         b += align_up((size_t)p->batch * g.N * p->num_q_heads * p->head_dim * 2, 256);
-      // fp32 dQ accumulator of the fused tensor-core backward (head_dim 128, no sinks)
-      if (p->head_dim == 128 && g.s == 0)
+      // fp32 dQ accumulator of the fused tensor-core backward (head_dim 128)
+      if (p->head_dim == 128)
         b += align_up((size_t)p->batch * g.N * p->num_q_heads * p->head_dim * sizeof(float), 256);
       return b;
     }
@@ -250,7 +250,9 @@ int32_t unigist_attn_bwd(const unigist_problem* p, const void* q, const void* k,
   if (!workspace || ws_bytes < need)
     return fail(UNIGIST_ERR_WORKSPACE, "backward needs %zu bytes of workspace, got %zu", need,
                 ws_bytes);
-  if (g.s == 0)
+  // Tensor cores: the fused kernel for head_dim 128 (sinks included), the two-kernel path for head_dim 64
+  // without sinks; the CUDA-core kernels cover head_dim 64 with a sink prefix.
+  if (p->head_dim == 128 || g.s == 0)
     return launch_bwd_sm100(g, *p, scale, q, k, v, o, lse, d_o, dq, dk, dv, workspace, (cudaStream_t)stream);
   return launch_bwd_simt(g, *p, scale, q, k, v, o, lse, d_o, dq, dk, dv, (float*)workspace,
                          (cudaStream_t)stream);

@@ -668,6 +668,22 @@ __device__ __forceinline__ void fused_p_chunk(const uint32_t (&v)[32], const flo
   }
 }
 
+// Query rows of segment qseg (numbered inside it, inclusive) that see key `key` of segment kseg:
+// Eq. 3 read column-wise, sinks included.  An empty interval has lo > hi.
+__device__ __forceinline__ void key_q_interval3(const Geom& g, int kseg, int key, bool key_valid, int qseg, int& lo,
+                                                int& hi) {
+  lo = 1;
+  hi = 0;
+  if (!key_valid) return;
+  if (kseg == kSegSink) {  // a sink is seen by the sinks from itself on and by every raw and gist query
+    lo = qseg == kSegSink ? key : 0;
+    hi = seg_len(g, qseg) - 1;
+    return;
+  }
+  if (qseg == kSegSink) return;  // sink queries see sinks only
+  key_q_interval(g, kseg == kSegRaw, key, true, qseg == kSegRaw, lo, hi);
+}
+
 struct FuSmem {
   static constexpr int kSlab = 128 * 128;    // [128 rows x 64 bf16]
   static constexpr int kTile = 2 * kSlab;    // [128 x 128] bf16
@@ -680,14 +696,17 @@ struct FuSmem {
 };
 
 __global__ void __launch_bounds__(kFuThreads, 1)
-attn_bwd_fused_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const __grid_constant__ CUtensorMap tm_q_gist,
+attn_bwd_fused_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_sink, const __grid_constant__ CUtensorMap tm_q_raw,
+                            const __grid_constant__ CUtensorMap tm_q_gist, const __grid_constant__ CUtensorMap tm_do_sink,
                             const __grid_constant__ CUtensorMap tm_do_raw, const __grid_constant__ CUtensorMap tm_do_gist,
-                            const __grid_constant__ CUtensorMap tm_k_raw, const __grid_constant__ CUtensorMap tm_k_gist,
+                            const __grid_constant__ CUtensorMap tm_k_sink, const __grid_constant__ CUtensorMap tm_k_raw,
+                            const __grid_constant__ CUtensorMap tm_k_gist, const __grid_constant__ CUtensorMap tm_v_sink,
                             const __grid_constant__ CUtensorMap tm_v_raw, const __grid_constant__ CUtensorMap tm_v_gist,
-                            const __grid_constant__ CUtensorMap tm_dq_raw, const __grid_constant__ CUtensorMap tm_dq_gist,
-                            Geom g, int Hq, int Hkv, float scale, const float* __restrict__ lse,
-                            const float* __restrict__ delta,
-                            __nv_bfloat16* __restrict__ dk, __nv_bfloat16* __restrict__ dv, int n_gist_kt, int interleaved) {
+                            const __grid_constant__ CUtensorMap tm_dq_sink, const __grid_constant__ CUtensorMap tm_dq_raw,
+                            const __grid_constant__ CUtensorMap tm_dq_gist, Geom g, int Hq, int Hkv, float scale,
+                            const float* __restrict__ lse, const float* __restrict__ delta,
+                            __nv_bfloat16* __restrict__ dk, __nv_bfloat16* __restrict__ dv, int n_sink_kt, int n_gist_kt,
+                            int interleaved) {
   using SM = FuSmem;
   constexpr int D = 128;
   extern __shared__ unsigned char smem_dyn[];
@@ -709,27 +728,28 @@ attn_bwd_fused_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const 
   volatile uint32_t* tmem_slot_ptr = reinterpret_cast<volatile uint32_t*>(gen + SM::kOffBars + 136);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  // blockIdx.x = key tile rank * Hkv + KV head.  Gist key tiles are seen by every later query: they are
-  // the heaviest and come first, for all KV heads, before any raw key tile.
+  // blockIdx.x = key tile rank * Hkv + KV head.  Sink and gist key tiles are seen by every later query:
+  // they are the heaviest and come first, for all KV heads, before any raw key tile.
   const int hk = blockIdx.x % Hkv, rank = blockIdx.x / Hkv, b = blockIdx.z, G = Hq / Hkv;
-  const bool key_is_raw = rank >= n_gist_kt;
-  const int kt = key_is_raw ? rank - n_gist_kt : rank;
-  const int key_seg_len = key_is_raw ? g.T : g.n;
-  const int key_seg_base = key_is_raw ? g.s : g.s + g.T;
+  const int kseg = rank < n_sink_kt ? kSegSink : (rank < n_sink_kt + n_gist_kt ? kSegGist : kSegRaw);
+  const int kt = rank - (kseg == kSegSink ? 0 : (kseg == kSegGist ? n_sink_kt : n_sink_kt + n_gist_kt));
+  const int key_seg_len = seg_len(g, kseg);
   const int key_a = kt * 128, key_b = min(key_a + 127, key_seg_len - 1);
   const bool key_tile_whole = key_a + 127 <= key_seg_len - 1;
 
-  // query tiles that see this key tile, per query segment
-  int a_lo, a_hi, b_lo, b_hi, c_lo, c_hi, d_lo, d_hi;
-  key_q_interval(g, key_is_raw, key_a, true, true, a_lo, a_hi);   // first key vs raw queries
-  key_q_interval(g, key_is_raw, key_b, true, true, b_lo, b_hi);   // last key vs raw queries
-  key_q_interval(g, key_is_raw, key_a, true, false, c_lo, c_hi);  // first key vs gist queries
-  key_q_interval(g, key_is_raw, key_b, true, false, d_lo, d_hi);  // last key vs gist queries
-  const int n_raw_q = b_hi >= a_lo ? b_hi / 128 - a_lo / 128 + 1 : 0;
-  const int rq_lo = a_lo / 128;
-  const int n_gist_q = d_hi >= c_lo ? d_hi / 128 - c_lo / 128 + 1 : 0;
-  const int gq_lo = c_lo / 128;
-  const int n_iter = (n_raw_q + n_gist_q) * G;
+  // query tiles that see this key tile, per query segment: [first tile, count], and the bounds inside
+  // which a tile is "full" (seen by the last key from t_lo on, by the first key up to t_hi)
+  int lo_a, hi_a, lo_b, hi_b;
+  key_q_interval3(g, kseg, key_a, true, kSegRaw, lo_a, hi_a);
+  key_q_interval3(g, kseg, key_b, true, kSegRaw, lo_b, hi_b);
+  const int n_raw_q = hi_b >= lo_a ? hi_b / 128 - lo_a / 128 + 1 : 0, rq_lo = lo_a / 128, raw_t_lo = lo_b, raw_t_hi = hi_a;
+  key_q_interval3(g, kseg, key_a, true, kSegGist, lo_a, hi_a);
+  key_q_interval3(g, kseg, key_b, true, kSegGist, lo_b, hi_b);
+  const int n_gist_q = hi_b >= lo_a ? hi_b / 128 - lo_a / 128 + 1 : 0, gq_lo = lo_a / 128, gist_t_lo = lo_b, gist_t_hi = hi_a;
+  key_q_interval3(g, kseg, key_a, true, kSegSink, lo_a, hi_a);
+  key_q_interval3(g, kseg, key_b, true, kSegSink, lo_b, hi_b);
+  const int n_sink_q = hi_b >= lo_a ? hi_b / 128 - lo_a / 128 + 1 : 0, sq_lo = lo_a / 128, sink_t_lo = lo_b, sink_t_hi = hi_a;
+  const int n_iter = (n_raw_q + n_gist_q + n_sink_q) * G;
 
   if (threadIdx.x == 0) {
     mbar_init(bar_kv, 1);
@@ -757,14 +777,22 @@ attn_bwd_fused_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const 
   const uint32_t t_dK = tmem, t_dV = tmem + 128, t_S = tmem + 256, t_dP = tmem + 384;
   bool ok = true;
 
-  // Step order: raw query tiles from the last one down, then gist query tiles from the last one down, the
+  // Step order: raw query tiles from the last one down, then gist query tiles, then sink query tiles, the
   // G heads of a tile back to back.  Every key tile's visible range ends at the last tile of a segment, so
   // thread blocks that run side by side walk the same Q / dO / dQ tiles at the same time and share them in L2.
-  auto tile_of = [&](int it, bool& q_is_raw, int& qt, int& head) {
+  auto tile_of = [&](int it, int& qseg, int& qt, int& head) {
     const int t = it / G;
     head = hk * G + (it - t * G);
-    q_is_raw = t < n_raw_q;
-    qt = q_is_raw ? rq_lo + (n_raw_q - 1 - t) : gq_lo + (n_gist_q - 1 - (t - n_raw_q));
+    if (t < n_raw_q) {
+      qseg = kSegRaw;
+      qt = rq_lo + (n_raw_q - 1 - t);
+    } else if (t < n_raw_q + n_gist_q) {
+      qseg = kSegGist;
+      qt = gq_lo + (n_gist_q - 1 - (t - n_raw_q));
+    } else {
+      qseg = kSegSink;
+      qt = sq_lo + (n_sink_q - 1 - (t - n_raw_q - n_gist_q));
+    }
   };
 
   if (warp >= 16) {
@@ -772,24 +800,23 @@ attn_bwd_fused_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const 
     if (warp == kFuTmaWarp) {
       // ---------------------------------------------------------- producer: K, V once; Q, dO, LSE, Delta per step
       // tile coordinate: its first unit (a raw tile of an interleaved tensor spans 128 / r gist units)
-      auto first_unit = [&](bool is_raw, int row0) { return interleaved && is_raw ? row0 / g.r : row0; };
+      auto first_unit = [&](int sg, int row0) { return interleaved && sg == kSegRaw ? row0 / g.r : row0; };
       if (lane == 0) {
         mbar_arrive_expect_tx(bar_kv, 2 * SM::kTile);
-        const CUtensorMap* mk = key_is_raw ? &tm_k_raw : &tm_k_gist;
-        const CUtensorMap* mv = key_is_raw ? &tm_v_raw : &tm_v_gist;
+        const CUtensorMap* mk = kseg == kSegRaw ? &tm_k_raw : (kseg == kSegGist ? &tm_k_gist : &tm_k_sink);
+        const CUtensorMap* mv = kseg == kSegRaw ? &tm_v_raw : (kseg == kSegGist ? &tm_v_gist : &tm_v_sink);
 #pragma unroll
         for (int sl = 0; sl < 2; ++sl) {
-          tma_load_5d(sK + sl * SM::kSlab, mk, bar_kv, sl * 64, hk, 0, first_unit(key_is_raw, key_a), b);
-          tma_load_5d(sV + sl * SM::kSlab, mv, bar_kv, sl * 64, hk, 0, first_unit(key_is_raw, key_a), b);
+          tma_load_5d(sK + sl * SM::kSlab, mk, bar_kv, sl * 64, hk, 0, first_unit(kseg, key_a), b);
+          tma_load_5d(sV + sl * SM::kSlab, mv, bar_kv, sl * 64, hk, 0, first_unit(kseg, key_a), b);
         }
       }
       // LSE (in log2 units) and Delta of the step's 128 query rows, 4 rows per lane, fetched one step ahead
       float st_l[4], st_d[4];
       auto fetch_stats = [&](int it) {
-        bool q_is_raw;
-        int qt, head;
-        tile_of(it, q_is_raw, qt, head);
-        const int q_seg_len = q_is_raw ? g.T : g.n, q_seg_base = q_is_raw ? g.s : g.s + g.T;
+        int qseg, qt, head;
+        tile_of(it, qseg, qt, head);
+        const int q_seg_len = seg_len(g, qseg), q_seg_base = seg_base(g, qseg);
         const long long row_base = ((long long)b * Hq + head) * g.N + q_seg_base;
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
@@ -803,9 +830,8 @@ attn_bwd_fused_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const 
       if (n_iter > 0) fetch_stats(0);
       for (int it = 0; it < n_iter; ++it) {
         const int st = it & 1;
-        bool q_is_raw;
-        int qt, head;
-        tile_of(it, q_is_raw, qt, head);
+        int qseg, qt, head;
+        tile_of(it, qseg, qt, head);
         if (it >= 2) ok = mbar_wait_warp(empty_q0 + 8 * st, ((it >> 1) - 1) & 1);
         if (!ok) break;
         float* ls = stats + st * 256;
@@ -817,21 +843,21 @@ attn_bwd_fused_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const 
         __syncwarp();
         if (lane == 0) {
           mbar_arrive_expect_tx(full_q0 + 8 * st, SM::kTile);
-          const CUtensorMap* mq = q_is_raw ? &tm_q_raw : &tm_q_gist;
+          const CUtensorMap* mq = qseg == kSegRaw ? &tm_q_raw : (qseg == kSegGist ? &tm_q_gist : &tm_q_sink);
 #pragma unroll
           for (int sl = 0; sl < 2; ++sl)
             tma_load_5d(sQ0 + st * SM::kTile + sl * SM::kSlab, mq, full_q0 + 8 * st, sl * 64, head, 0,
-                        first_unit(q_is_raw, qt * 128), b);
+                        first_unit(qseg, qt * 128), b);
         }
         if (it + 1 < n_iter) fetch_stats(it + 1);
         if (it >= 1) ok = mbar_wait_warp(empty_do, (it - 1) & 1);  // one dO buffer: free once dV of the step before is done
         if (!ok) break;
         if (lane == 0) {
           mbar_arrive_expect_tx(full_do, SM::kTile);
-          const CUtensorMap* md = q_is_raw ? &tm_do_raw : &tm_do_gist;
+          const CUtensorMap* md = qseg == kSegRaw ? &tm_do_raw : (qseg == kSegGist ? &tm_do_gist : &tm_do_sink);
 #pragma unroll
           for (int sl = 0; sl < 2; ++sl)
-            tma_load_5d(sDO + sl * SM::kSlab, md, full_do, sl * 64, head, 0, first_unit(q_is_raw, qt * 128), b);
+            tma_load_5d(sDO + sl * SM::kSlab, md, full_do, sl * 64, head, 0, first_unit(qseg, qt * 128), b);
         }
         __syncwarp();
       }
@@ -933,11 +959,10 @@ attn_bwd_fused_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const 
     float* stage_gen = reinterpret_cast<float*>(gen + SM::kOffStage) + (warp - 8) * 1024 + lane;
     const uint32_t stage_sh = base + SM::kOffStage + (warp - 8) * 4096;
     for (int it = 0; it < n_iter && ok; ++it) {
-      bool q_is_raw;
-      int qt, head;
-      tile_of(it, q_is_raw, qt, head);
-      const CUtensorMap* mdq = q_is_raw ? &tm_dq_raw : &tm_dq_gist;
-      const int nq = (q_is_raw ? g.T : g.n) - qt * 128;  // rows of this tile inside the segment (may exceed 128)
+      int qseg, qt, head;
+      tile_of(it, qseg, qt, head);
+      const CUtensorMap* mdq = qseg == kSegRaw ? &tm_dq_raw : (qseg == kSegGist ? &tm_dq_gist : &tm_dq_sink);
+      const int nq = seg_len(g, qseg) - qt * 128;  // rows of this tile inside the segment (may exceed 128)
       ok = mbar_wait_warp(bar_dQ, it & 1);
       if (!ok) break;
       tc_fence_after();
@@ -975,24 +1000,26 @@ attn_bwd_fused_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const 
     const bool key_valid = key <= key_b;
     const uint32_t lane_base = static_cast<uint32_t>(qd * 32) << 16;
     const float scale_log2 = scale * kLog2e;
-    int my_lo_r, my_hi_r, my_lo_g, my_hi_g;  // queries that see this key: raw segment, gist segment
-    key_q_interval(g, key_is_raw, key, key_valid, true, my_lo_r, my_hi_r);
-    key_q_interval(g, key_is_raw, key, key_valid, false, my_lo_g, my_hi_g);
+    int my_lo_r, my_hi_r, my_lo_g, my_hi_g, my_lo_s, my_hi_s;  // queries that see this key, per query segment
+    key_q_interval3(g, kseg, key, key_valid, kSegRaw, my_lo_r, my_hi_r);
+    key_q_interval3(g, kseg, key, key_valid, kSegGist, my_lo_g, my_hi_g);
+    key_q_interval3(g, kseg, key, key_valid, kSegSink, my_lo_s, my_hi_s);
     // this thread's row of the dS^T tile in shared memory: slab hf, row krow, 16-byte chunks swizzled by row
     unsigned char* ds_row = gen + SM::kOffDS + hf * SM::kSlab + krow * 128;
     const int swz = krow & 7;
 
     for (int it = 0; it < n_iter && ok; ++it) {
       const int st = it & 1;
-      bool q_is_raw;
-      int qt, head;
-      tile_of(it, q_is_raw, qt, head);
-      const int q0 = qt * 128, q_seg_len = q_is_raw ? g.T : g.n;
+      int qseg, qt, head;
+      tile_of(it, qseg, qt, head);
+      const int q0 = qt * 128, q_seg_len = seg_len(g, qseg);
       const int qb = min(q0 + 127, q_seg_len - 1);
       // full: every (query, key) pair of the tile is visible -> no mask arithmetic
-      const int t_lo = q_is_raw ? b_lo : d_lo, t_hi = q_is_raw ? a_hi : c_hi;
+      const int t_lo = qseg == kSegRaw ? raw_t_lo : (qseg == kSegGist ? gist_t_lo : sink_t_lo);
+      const int t_hi = qseg == kSegRaw ? raw_t_hi : (qseg == kSegGist ? gist_t_hi : sink_t_hi);
       const bool full = key_tile_whole && q0 >= t_lo && qb <= t_hi;
-      const int lo = (q_is_raw ? my_lo_r : my_lo_g) - q0 - 64 * hf, hi = (q_is_raw ? my_hi_r : my_hi_g) - q0 - 64 * hf;
+      const int lo = (qseg == kSegRaw ? my_lo_r : (qseg == kSegGist ? my_lo_g : my_lo_s)) - q0 - 64 * hf;
+      const int hi = (qseg == kSegRaw ? my_hi_r : (qseg == kSegGist ? my_hi_g : my_hi_s)) - q0 - 64 * hf;
       const float* ls = stats + st * 256 + 64 * hf;
       const float* dl = ls + 128;
       ok = mbar_wait_warp(full_q0 + 8 * st, (it >> 1) & 1) && mbar_wait_warp(bar_S, it & 1);
@@ -1047,7 +1074,7 @@ attn_bwd_fused_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const 
     if (ok && n_iter > 0) ok = mbar_wait_warp(bar_final, 0);
     if (ok) {
       tc_fence_after();
-      const long long tok = (long long)b * g.N + seg_row_to_token(g, interleaved != 0, key_is_raw ? kSegRaw : kSegGist, key_valid ? key : key_a);
+      const long long tok = (long long)b * g.N + seg_row_to_token(g, interleaved != 0, kseg, key_valid ? key : key_a);
       // this warp stores columns [64 hf, 64 hf + 64) of dK and of dV
 #pragma unroll
       for (int which = 0; which < 2; ++which) {
@@ -1146,13 +1173,7 @@ int32_t launch_bwd_sm100(const Geom& g, const unigist_problem& p, float scale, c
   CUtensorMap mq[2], md[2], mk[2], mv[2], mk64[2], mv64[2];
   const long long first[2] = {g.s, (long long)g.s + g.T}, len[2] = {g.T, g.n};
   for (int sgm = 0; sgm < 2; ++sgm) {
-    if (fused) {  // 128-row tile maps that read shifted or interleaved tensors
-      if (int32_t rc = encode_tile_map(&mq[sgm], q, D, Hq, B, g.s, g.T, g.r, il, sgm == 0 ? kSegRaw : kSegGist)) return rc;
-      if (int32_t rc = encode_tile_map(&md[sgm], do_src, D, Hq, B, g.s, g.T, g.r, il, sgm == 0 ? kSegRaw : kSegGist)) return rc;
-      if (int32_t rc = encode_tile_map(&mk[sgm], k, D, Hkv, B, g.s, g.T, g.r, il, sgm == 0 ? kSegRaw : kSegGist)) return rc;
-      if (int32_t rc = encode_tile_map(&mv[sgm], v, D, Hkv, B, g.s, g.T, g.r, il, sgm == 0 ? kSegRaw : kSegGist)) return rc;
-      continue;
-    }
+    if (fused) continue;
     if (int32_t rc = encode_segment_map(&mq[sgm], q, D, Hq, g.N, B, first[sgm], len[sgm], 128)) return rc;
     if (int32_t rc = encode_segment_map(&md[sgm], do_src, D, Hq, g.N, B, first[sgm], len[sgm], 128)) return rc;
     if (int32_t rc = encode_segment_map(&mk[sgm], k, D, Hkv, g.N, B, first[sgm], len[sgm], 128)) return rc;
@@ -1192,17 +1213,26 @@ int32_t launch_bwd_sm100(const Geom& g, const unigist_problem& p, float scale, c
     if (int32_t rc = go_kv(attn_bwd_dkdv_sm100_kernel<128>, KvSmem<128>::kBytes)) return rc;
     return go_q(attn_bwd_dq_sm100_kernel<128>, DqSmem<128>::kBytes);
   }
-  CUtensorMap mdq[2];
-  for (int sgm = 0; sgm < 2; ++sgm)
-    if (int32_t rc = encode_segment_map_f32(&mdq[sgm], dq32, D, Hq, g.N, B, first[sgm], len[sgm], 32, 32)) return rc;
+  // 128-row tile maps per segment (sinks, raw, gists) that read shifted or interleaved tensors, and
+  // reduction maps over the fp32 dQ tensor (always shifted)
+  CUtensorMap fq[3], fdo[3], fk[3], fv[3], mdq[3];
+  for (int sg = 0; sg < 3; ++sg) {
+    if (int32_t rc = encode_tile_map(&fq[sg], q, D, Hq, B, g.s, g.T, g.r, il, sg)) return rc;
+    if (int32_t rc = encode_tile_map(&fdo[sg], do_src, D, Hq, B, g.s, g.T, g.r, il, sg)) return rc;
+    if (int32_t rc = encode_tile_map(&fk[sg], k, D, Hkv, B, g.s, g.T, g.r, il, sg)) return rc;
+    if (int32_t rc = encode_tile_map(&fv[sg], v, D, Hkv, B, g.s, g.T, g.r, il, sg)) return rc;
+    const int rows = seg_len(g, sg) > 0 ? seg_len(g, sg) : 1;  // a tensor map cannot be empty
+    if (int32_t rc = encode_segment_map_f32(&mdq[sg], dq32, D, Hq, g.N, B, seg_base(g, sg), rows, 32, 32)) return rc;
+  }
+  const int n_sink_t = (g.s + 127) / 128;
   cudaError_t e = cudaFuncSetAttribute(attn_bwd_fused_sm100_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        FuSmem::kBytes);
   if (e != cudaSuccess) return fail(UNIGIST_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
   {
     KernelScope ks("attn_bwd_fused_sm100_kernel", st);
-    attn_bwd_fused_sm100_kernel<<<dim3((n_raw_t + n_gist_t) * Hkv, 1, B), kFuThreads, FuSmem::kBytes, st>>>(
-        mq[0], mq[1], md[0], md[1], mk[0], mk[1], mv[0], mv[1], mdq[0], mdq[1], g, Hq, Hkv, scale, lse, delta,
-        (__nv_bfloat16*)dk, (__nv_bfloat16*)dv, n_gist_t, il ? 1 : 0);
+    attn_bwd_fused_sm100_kernel<<<dim3((n_sink_t + n_raw_t + n_gist_t) * Hkv, 1, B), kFuThreads, FuSmem::kBytes, st>>>(
+        fq[0], fq[1], fq[2], fdo[0], fdo[1], fdo[2], fk[0], fk[1], fk[2], fv[0], fv[1], fv[2], mdq[0], mdq[1], mdq[2], g,
+        Hq, Hkv, scale, lse, delta, (__nv_bfloat16*)dk, (__nv_bfloat16*)dv, n_sink_t, n_gist_t, il ? 1 : 0);
   }
   if (int32_t rc = check_launch("tcgen05 fused backward kernel")) return rc;
   {

@@ -66,6 +66,10 @@ SMALL = [
     synth.Workload("ragged_group3_128", 1, 777, 7, 77, 6, 2, 128, seed=110),
     synth.Workload("ragged_64", 2, 1000, 8, 200, 4, 2, 64, seed=111),
     synth.Workload("tiny_window_128", 1, 2048, 16, 16, 2, 1, 128, seed=112),
+    # sink prefixes on the tensor-core paths: one full sink tile (the paper's default 128), several ragged ones
+    synth.Workload("sinks_128", 1, 1024, 8, 128, 4, 2, 128, num_sinks=128, seed=113),
+    synth.Workload("sinks_300", 2, 640, 4, 64, 2, 2, 128, num_sinks=300, seed=114),
+    synth.Workload("sinks_64_d64", 1, 512, 8, 64, 2, 1, 64, num_sinks=64, seed=115),
 ]
 
 
@@ -86,7 +90,7 @@ def test_attention_matches_oracle(w):
     check_close("dV", f64(out["dv"]), dv, TOL_GRAD)
 
 
-INTERLEAVED = [w for w in SMALL if w.num_sinks == 0 and w.head_dim == 128 and 128 % w.ratio == 0]
+INTERLEAVED = [w for w in SMALL if w.head_dim == 128 and 128 % w.ratio == 0]
 
 
 @pytest.mark.parametrize("w", INTERLEAVED, ids=lambda w: w.name)
@@ -97,10 +101,10 @@ def test_interleaved_tensors_match_oracle(w):
     k = oracle.window_units(w.window, w.ratio)
     scale = w.head_dim ** -0.5
     q, kk, v, do = (f64(inp[n]) for n in ("q", "k", "v", "dout"))
-    o, lse = oracle.attn_fwd(0, w.raw_len, w.ratio, k, scale, q, kk, v)
+    o, lse = oracle.attn_fwd(w.num_sinks, w.raw_len, w.ratio, k, scale, q, kk, v)
     check_close("O", f64(out["o"]), o, TOL_O_MAX, TOL_O_MEAN)
     check_close("LSE", f64(out["lse"]), lse, TOL_LSE)
-    dq, dk, dv = oracle.attn_bwd(0, w.raw_len, w.ratio, k, scale, q, kk, v, do)
+    dq, dk, dv = oracle.attn_bwd(w.num_sinks, w.raw_len, w.ratio, k, scale, q, kk, v, do)
     check_close("dQ", f64(out["dq"]), dq, TOL_GRAD)
     check_close("dK", f64(out["dk"]), dk, TOL_GRAD)
     check_close("dV", f64(out["dv"]), dv, TOL_GRAD)
@@ -112,7 +116,7 @@ def test_interleaved_tensors_match_oracle(w):
 
 
 def test_interleaved_flag_is_refused_where_the_tiles_do_not_line_up():
-    for w in (SMALL[0], SMALL[1], synth.Workload("r7", 1, 448, 7, 64, 2, 1, 128, seed=1)):
+    for w in (SMALL[0], synth.Workload("r7", 1, 448, 7, 64, 2, 1, 128, seed=1)):
         p = problem_of(w, ug.FLAG_INTERLEAVED)
         N = ug.unigist_total_len(p)
         q = torch.zeros(w.batch, N, w.num_q_heads, w.head_dim, dtype=torch.bfloat16, device=DEV)
