@@ -127,11 +127,12 @@ def oracle_sample(w, seconds_hint: float = 20.0):
     scale = w.head_dim ** -0.5
     t0 = time.perf_counter()
     oracle.attn_fwd_slice(ws.num_sinks, T_s, w.ratio, ku, scale, q, k, v)
-    oracle.attn_bwd_slice(ws.num_sinks, T_s, w.ratio, ku, scale, q, k, v, do)
+    if not w.forward_only:
+        oracle.attn_bwd_slice(ws.num_sinks, T_s, w.ratio, ku, scale, q, k, v, do)
     dt = time.perf_counter() - t0
     pairs = oracle.count_pairs(ws.num_sinks, T_s, w.ratio, ku)
-    flops = 14.0 * w.head_dim * pairs * G
-    desc = (f"oracle fwd+bwd of one KV group ({G} query heads) over the first {T_s} raw tokens "
+    flops = (4.0 if w.forward_only else 14.0) * w.head_dim * pairs * G
+    desc = (f"oracle {'fwd' if w.forward_only else 'fwd+bwd'} of one KV group ({G} query heads) over the first {T_s} raw tokens "
             f"(N={ws.total_len}) of {w.name}, {pairs} visible pairs per head")
     return flops / dt / 1e12, oracle.num_threads(), desc, dt
 
@@ -176,7 +177,7 @@ class Path_:
         p = self.p
         self.N = ug.unigist_total_len(p)
         self.pairs = ug.unigist_visible_pairs(p)
-        host = synth.attention_inputs(w)
+        host = synth.attention_inputs(w, with_grad=not w.forward_only)
         self.host_in = {k: v.pin_memory() for k, v in host.items()}
         self.inter = {k: v.to(dev) for k, v in host.items()}                      # interleaved inputs
         self.sh = {k: torch.empty_like(v) for k, v in self.inter.items()}         # shifted inputs
@@ -185,7 +186,8 @@ class Path_:
         self.dq_s, self.dk_s, self.dv_s = (torch.empty_like(self.sh[n]) for n in ("q", "k", "v"))
         self.out = {"o": torch.empty_like(self.o_s), "dq": torch.empty_like(self.dq_s),
                     "dk": torch.empty_like(self.dk_s), "dv": torch.empty_like(self.dv_s)}
-        self.host_out = {k: torch.empty(v.shape, dtype=v.dtype).pin_memory() for k, v in self.out.items()}
+        self.host_out = {k: torch.empty(v.shape, dtype=v.dtype).pin_memory() for k, v in self.out.items()
+                         if k == "o" or not w.forward_only}
         self.ws = torch.empty(max(16, ug.unigist_workspace_bytes(p, ug.OP_BWD)), dtype=torch.uint8, device=dev)
         L = ug.unigist_compact_len(p)
         self.nb = -(-(L + 1) // ug.PAGE_TOKENS)
@@ -198,11 +200,12 @@ class Path_:
         self.qd = torch.empty(w.batch, w.num_q_heads, w.head_dim, dtype=torch.bfloat16, device=dev)
         self.od = torch.empty_like(self.qd)
         self.host_od = torch.empty(self.od.shape, dtype=self.od.dtype).pin_memory()
-        self.wsd = torch.empty(ug.unigist_decode_workspace_bytes(w.batch, w.num_q_heads, w.num_kv_heads,
-                                                                 w.head_dim, self.nb), dtype=torch.uint8, device=dev)
-        self.flops = 14.0 * w.head_dim * self.pairs * w.num_q_heads * w.batch
+        self.wsd = torch.empty(max(16, ug.unigist_decode_workspace_bytes(w.batch, w.num_q_heads, w.num_kv_heads,
+                                                                         w.head_dim, self.nb)),
+                               dtype=torch.uint8, device=dev)
+        self.flops = (4.0 if w.forward_only else 14.0) * w.head_dim * self.pairs * w.num_q_heads * w.batch
         # the gist shift as tile addressing inside the attention kernels (no shift / unshift launches)
-        self.fused_shift = w.num_sinks == 0 and w.head_dim == 128 and 128 % w.ratio == 0
+        self.fused_shift = w.head_dim == 128 and 128 % w.ratio == 0
         self.p_il = ug.Problem(w.batch, w.raw_len, w.ratio, w.window, w.num_q_heads, w.num_kv_heads, w.head_dim,
                                num_sinks=w.num_sinks, flags=ug.FLAG_INTERLEAVED)
 
@@ -215,30 +218,36 @@ class Path_:
         """Interleaved tensors in, interleaved results out: the shift is done by the kernels' tile loads."""
         ug, p, x, out = self.ug, self.p_il, self.inter, self.out
         ug.unigist_attn_fwd(p, x["q"], x["k"], x["v"], out["o"], self.lse)
-        ug.unigist_attn_bwd(p, x["q"], x["k"], x["v"], out["o"], self.lse, x["dout"], out["dq"], out["dk"], out["dv"],
-                            self.ws)
+        if not self.w.forward_only:
+            ug.unigist_attn_bwd(p, x["q"], x["k"], x["v"], out["o"], self.lse, x["dout"], out["dq"], out["dk"],
+                                out["dv"], self.ws)
         ug.unigist_kv_compact(p, x["k"], x["v"], self.kc, self.vc, self.table, self.lens)
         self.qd.copy_(x["q"][:, -1])  # the last token (the last gist) in either order
-        ug.unigist_decode(self.qd, self.kc, self.vc, self.table, self.lens, self.od, None, self.wsd)
+        if self.w.head_dim == 128:  # the decode kernel is written for head_dim 128
+            ug.unigist_decode(self.qd, self.kc, self.vc, self.table, self.lens, self.od, None, self.wsd)
 
     def step_explicit(self):
         ug, p = self.ug, self.p
-        for n in ("q", "k", "v", "dout"):
+        for n in self.inter:
             ug.unigist_gist_shift(p, self.inter[n], self.sh[n])
         ug.unigist_attn_fwd(p, self.sh["q"], self.sh["k"], self.sh["v"], self.o_s, self.lse)
-        ug.unigist_attn_bwd(p, self.sh["q"], self.sh["k"], self.sh["v"], self.o_s, self.lse, self.sh["dout"],
-                            self.dq_s, self.dk_s, self.dv_s, self.ws)
-        for n, t in (("o", self.o_s), ("dq", self.dq_s), ("dk", self.dk_s), ("dv", self.dv_s)):
+        outs = [("o", self.o_s)]
+        if not self.w.forward_only:
+            ug.unigist_attn_bwd(p, self.sh["q"], self.sh["k"], self.sh["v"], self.o_s, self.lse, self.sh["dout"],
+                                self.dq_s, self.dk_s, self.dv_s, self.ws)
+            outs += [("dq", self.dq_s), ("dk", self.dk_s), ("dv", self.dv_s)]
+        for n, t in outs:
             ug.unigist_gist_unshift(p, t, self.out[n])
         ug.unigist_kv_compact(p, self.sh["k"], self.sh["v"], self.kc, self.vc, self.table, self.lens)
         self.qd.copy_(self.sh["q"][:, -1])
-        ug.unigist_decode(self.qd, self.kc, self.vc, self.table, self.lens, self.od, None, self.wsd)
+        if self.w.head_dim == 128:  # the decode kernel is written for head_dim 128
+            ug.unigist_decode(self.qd, self.kc, self.vc, self.table, self.lens, self.od, None, self.wsd)
 
     def e2e_step(self):
-        for n in ("q", "k", "v", "dout"):
+        for n in self.inter:
             self.inter[n].copy_(self.host_in[n], non_blocking=True)
         self.step()
-        for n in self.out:
+        for n in self.host_out:
             self.host_out[n].copy_(self.out[n], non_blocking=True)
         self.host_od.copy_(self.od, non_blocking=True)
 

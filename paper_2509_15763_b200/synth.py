@@ -31,6 +31,7 @@ class Workload:
     num_sinks: int = 0
     k_scale: float = 1.0
     seed: int = BASE_SEED
+    forward_only: bool = False  # the workload is a prefill: no backward pass
 
     @property
     def num_gists(self) -> int:
@@ -50,8 +51,18 @@ WORKLOADS = {
     "llama8b_layer": Workload("llama8b_layer", 1, 16384, 8, 1024, 32, 8, 128,
                               k_scale=0.5, seed=BASE_SEED + 1),
     "train_batch": Workload("train_batch", 4, 32768, 4, 2048, 32, 8, 128, seed=BASE_SEED + 2),
-    "long_prefill": Workload("long_prefill", 1, 131072, 16, 4096, 32, 8, 128, seed=BASE_SEED + 3),
+    "long_prefill": Workload("long_prefill", 1, 131072, 16, 4096, 32, 8, 128, seed=BASE_SEED + 3,
+                             forward_only=True),
 }
+
+# The shapes of the paper's own speed table (appendix): one attention layer, batch 1, 32 heads (MHA),
+# head_dim 128, 16K to 128K raw tokens, ratio 4 or 8, with the main experiments' 128 sinks and
+# 128-token window.  Context for the numbers the paper prints, not one of the five workloads above.
+for _i, _ctx in enumerate((16, 32, 64, 128)):
+    for _r in (4, 8):
+        _name = f"table4_{_ctx}k_r{_r}"
+        WORKLOADS[_name] = Workload(_name, 1, _ctx * 1024, _r, 128, 32, 32, 128, num_sinks=128,
+                                    seed=BASE_SEED + 10 + 2 * _i + (_r == 8))
 
 
 @dataclass(frozen=True)
