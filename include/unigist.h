@@ -199,7 +199,7 @@ int32_t unigist_kernel_timing_get(int32_t index, char* name, int32_t cap, float*
  * allocate any.  (The paper has no counterpart; this exists for deployment.)  Typical cases: a
  * plugin called from inside an inference server that has already claimed the whole GPU for its
  * own memory pool, so a cudaMalloc from the plugin would fail or stall the device; or a decode
- * loop with a hard latency budget, where an allocation's implicit device-wide synchronisation is
+ * loop with a hard latency limit, where an allocation's implicit device-wide synchronisation is
  * not acceptable.
  *
  * Same arguments and results as unigist_decode, minus workspace / ws_bytes.  The split-KV

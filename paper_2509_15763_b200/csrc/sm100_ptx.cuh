@@ -48,12 +48,12 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 }
 // Waits for the phase with the given parity to complete.  Gives up after about a second of
 // SM clock and returns false, so a protocol error ends the kernel instead of hanging the GPU.
-constexpr long long kWaitBudgetCycles = 2000000000LL;
+constexpr long long kWaitLimitCycles = 2000000000LL;
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   while (!mbar_try_wait(bar, parity)) {
-    if (clock64() - t0 > kWaitBudgetCycles) return false;
+    if (clock64() - t0 > kWaitLimitCycles) return false;
   }
   return true;
 }

@@ -45,7 +45,7 @@ class Workload:
         return replace(self, **kw)
 
 
-# The five workloads of the build's baseline description.
+# The five benchmark workloads.
 WORKLOADS = {
     "tiny": Workload("tiny", 1, 448, 7, 64, 1, 1, 64, seed=BASE_SEED + 0),
     "llama8b_layer": Workload("llama8b_layer", 1, 16384, 8, 1024, 32, 8, 128,
