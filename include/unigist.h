@@ -132,7 +132,11 @@ int32_t unigist_attn_fwd(const unigist_problem* p, const void* q, const void* k,
  *   dQ = scale dS K, dK = scale dS^T Q;  dK, dV summed over the query heads of a KV head.
  * q, k, v, o, lse as in the forward; d_o [B,N,Hq,D] device bf16 (fp32 with
  * UNIGIST_FLAG_DOUT_FP32); dq [B,N,Hq,D], dk, dv [B,N,Hkv,D] device bf16, all shifted.
- * dK/dV are accumulated without atomics: each key tile is owned by one thread block.
+ * dK/dV are accumulated without atomics: each key tile is owned by one thread block, so they are the
+ * same bit for bit from run to run.  For head_dim 128 dQ is the sum, over the key tiles that see a query
+ * tile, of fp32 partial tiles reduced into the workspace in whatever order the blocks arrive: its last bit
+ * may differ between runs.  workspace: unigist_workspace_bytes(p, UNIGIST_OP_BWD) bytes (Delta, a bf16
+ * copy of an fp32 dO, and for head_dim 128 the fp32 dQ accumulator), 16-byte aligned.
  */
 int32_t unigist_attn_bwd(const unigist_problem* p, const void* q, const void* k, const void* v,
                          const void* o, const float* lse, const void* d_o, void* dq, void* dk,
