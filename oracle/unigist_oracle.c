@@ -24,6 +24,14 @@
  * differences for the backward pass, brute-force "visible to any future
  * token" for compaction, decode == row of the full forward.
  *
+ * Two readings of the paper are encoded here that no pin can settle, because
+ * the paper prints no worked example for them (parity unpinned against the
+ * authors' own implementation; every function is pinned against the paper's
+ * equations as listed above): a window given as W raw tokens means
+ * k = ceil(W / r) previous gist units (rounded up when r does not divide W),
+ * and sink tokens belong to no gist unit, attend causally among themselves and
+ * are seen by every later token.
+ *
  * Functions take one (batch, KV-head) slice at a time: G query heads share
  * one K/V head (grouped-query attention, q head h uses kv head h / G).
  */
