@@ -38,6 +38,35 @@ def test_host_geometry_matches_oracle(s, T, r, W):
     assert ug.unigist_compact_len(p) == len(oracle.kept_set(s, T, r, k))
 
 
+@pytest.mark.parametrize("s,T,r", [(0, 448, 7), (5, 64, 4), (128, 1024, 8), (0, 16, 16), (3, 9, 1), (2, 6, 3)])
+def test_host_layout_matches_oracle(s, T, r):
+    """on_device = 0: the index arrays are computed on the host (closed form) and must equal the oracle's,
+    which walks Eq. 2 token by token."""
+    import numpy as np
+    import torch
+
+    p = ug.Problem(1, T, r, 64, 1, 1, 64, num_sinks=s)
+    N = ug.unigist_total_len(p)
+    sp, up, pos = (torch.full((N,), -1, dtype=torch.int32) for _ in range(3))
+    ug.unigist_layout(p, sp, up, pos)
+    a, b, c = oracle.layout(s, T, r)
+    assert np.array_equal(sp.numpy(), a) and np.array_equal(up.numpy(), b) and np.array_equal(pos.numpy(), c)
+
+
+def test_interleaved_flag_is_validated_on_the_host():
+    lib = binding.lib()
+    buf = ctypes.create_string_buffer(1 << 16)
+    a = ctypes.addressof(buf)
+    a += (-a) % 16
+    for prob in (ug.Problem(1, 448, 7, 64, 2, 1, 128, flags=ug.FLAG_INTERLEAVED),     # 7 does not divide 128
+                 ug.Problem(1, 64, 8, 64, 2, 1, 64, flags=ug.FLAG_INTERLEAVED)):       # head_dim 64
+        p = prob.c()
+        before = ug.unigist_launch_count()
+        rc = lib.unigist_attn_fwd(ctypes.byref(p), a, a, a, a, ctypes.cast(a, ctypes.POINTER(ctypes.c_float)), None, 0,
+                                  None)
+        assert rc == 5 and ug.unigist_launch_count() == before   # UNIGIST_ERR_UNSUPPORTED, nothing launched
+
+
 def test_malformed_problems_are_rejected():
     bad = [ug.Problem(1, 10, 3, 4, 1, 1, 64), ug.Problem(1, 16, 4, 4, 3, 2, 64),
            ug.Problem(1, 16, 4, 4, 1, 1, 96), ug.Problem(0, 16, 4, 4, 1, 1, 64),
