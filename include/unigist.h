@@ -167,6 +167,28 @@ int32_t unigist_kv_compact(const unigist_problem* p, const void* k, const void* 
                            int32_t max_blocks_per_seq, int32_t* seq_lens, int32_t* kept_idx,
                            void* workspace, size_t ws_bytes, void* stream);
 
+/*
+ * Chunk-wise prefill (Section 4.3: "re-adopt the chunk-wise scheme and encode each chunk with our kernel").
+ * The prompt of p->raw_len raw tokens is fed in chunks of whole gist units; the chunk of unit_count units
+ * that starts at unit unit_begin attends to what the paged cache holds -- the sinks, the gists of units
+ * [0, unit_begin) and the raw tokens of the last min(k, unit_begin) units, in the cache order of
+ * unigist_kv_compact -- and to itself under Eq. 3; its outputs equal the corresponding rows of the one-pass
+ * forward over the whole prompt.  Afterwards the cache holds the state after unit_begin + unit_count units
+ * (seq_lens updated), ready for the next chunk or for unigist_decode.
+ *
+ * q [B, Nc, Hq, D], k, v [B, Nc, Hkv, D], o [B, Nc, Hq, D] device bf16, lse [B, Hq, Nc] device fp32: the
+ * chunk's own tokens in shifted CHUNK order [sinks (only when unit_begin == 0) | unit_count * r raw |
+ * unit_count gists], Nc = that many rows.  k_cache, v_cache, block_table, seq_lens as in unigist_kv_compact;
+ * for unit_begin > 0 the cache must be in the state a previous chunk (or unigist_kv_compact of the first
+ * unit_begin units) left it in.  block_table needs entries for the cache after the chunk.
+ * workspace: unigist_prefill_workspace_bytes() bytes (a dense copy of the keys and values the chunk sees).
+ */
+size_t unigist_prefill_workspace_bytes(const unigist_problem* p, int32_t unit_begin, int32_t unit_count);
+int32_t unigist_prefill_chunk(const unigist_problem* p, int32_t unit_begin, int32_t unit_count, const void* q,
+                              const void* k, const void* v, void* k_cache, void* v_cache, int32_t num_blocks,
+                              int32_t* block_table, int32_t max_blocks_per_seq, int32_t* seq_lens, void* o, float* lse,
+                              void* workspace, size_t ws_bytes, void* stream);
+
 /* Scratch for unigist_decode (split-KV partial results). */
 size_t unigist_decode_workspace_bytes(int32_t num_seqs, int32_t num_q_heads, int32_t num_kv_heads,
                                       int32_t head_dim, int32_t max_blocks_per_seq);

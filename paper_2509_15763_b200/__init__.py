@@ -4,5 +4,5 @@ from .binding import (DECODE_STATIC_SCRATCH_BYTES, FLAG_DOUT_FP32, FLAG_INTERLEA
                       unigist_decode_static, unigist_decode_workspace_bytes, unigist_device_status, unigist_gist_shift, unigist_gist_unshift,
                       unigist_kernel_timing, unigist_kernel_timing_count,
                       unigist_kernel_timing_get, unigist_kv_compact, unigist_last_error_string, unigist_launch_count,
-                      unigist_layout, unigist_total_len, unigist_visible_pairs, unigist_window_units,
+                      unigist_layout, unigist_prefill_chunk, unigist_prefill_workspace_bytes, unigist_total_len, unigist_visible_pairs, unigist_window_units,
                       unigist_workspace_bytes)

@@ -26,7 +26,7 @@ SYMBOLS = [
     "unigist_attn_fwd", "unigist_attn_bwd", "unigist_kv_compact", "unigist_decode_workspace_bytes",
     "unigist_decode", "unigist_launch_count", "unigist_last_error_string",
     "unigist_kernel_timing", "unigist_kernel_timing_count", "unigist_kernel_timing_get",
-    "unigist_device_status", "unigist_decode_static",
+    "unigist_device_status", "unigist_decode_static", "unigist_prefill_workspace_bytes", "unigist_prefill_chunk",
 ]
 
 
@@ -88,6 +88,8 @@ def lib() -> ctypes.CDLL:
             "unigist_attn_bwd": (i32, [P] + [vp] * 10 + [sz, vp]),
             "unigist_kv_compact": (i32, [P, vp, vp, vp, vp, i32, vp, i32, vp, vp, vp, sz, vp]),
             "unigist_decode_workspace_bytes": (sz, [i32] * 5),
+            "unigist_prefill_workspace_bytes": (sz, [P, i32, i32]),
+            "unigist_prefill_chunk": (i32, [P, i32, i32, vp, vp, vp, vp, vp, i32, vp, i32, vp, vp, vp, vp, sz, vp]),
             "unigist_decode": (i32, [i32, i32, i32, i32, f32, vp, vp, vp, i32, vp, i32, vp, vp, vp, vp, sz, vp]),
             "unigist_kernel_timing": (i32, [i32]),
             "unigist_kernel_timing_count": (i32, []),
@@ -236,6 +238,19 @@ def unigist_kv_compact(p: Problem, k, v, k_cache, v_cache, block_table, seq_lens
                                     _ptr(seq_lens), _ptr(kept_idx), _ptr(workspace),
                                     0 if workspace is None else workspace.numel() * workspace.element_size(),
                                     _stream(stream)))
+
+
+def unigist_prefill_workspace_bytes(p: Problem, unit_begin: int, unit_count: int) -> int:
+    return lib().unigist_prefill_workspace_bytes(ctypes.byref(p.c()), unit_begin, unit_count)
+
+
+def unigist_prefill_chunk(p: Problem, unit_begin: int, unit_count: int, q, k, v, k_cache, v_cache, block_table,
+                          seq_lens, o, lse, workspace, stream=None):
+    _dev(q, k, v, k_cache, v_cache, block_table, seq_lens, o, lse, workspace)
+    _check(lib().unigist_prefill_chunk(ctypes.byref(p.c()), unit_begin, unit_count, _ptr(q), _ptr(k), _ptr(v),
+                                       _ptr(k_cache), _ptr(v_cache), k_cache.shape[0], _ptr(block_table),
+                                       block_table.shape[1], _ptr(seq_lens), _ptr(o), _ptr(lse), _ptr(workspace),
+                                       workspace.numel() * workspace.element_size(), _stream(stream)))
 
 
 def unigist_decode_workspace_bytes(num_seqs, num_q_heads, num_kv_heads, head_dim, max_blocks_per_seq) -> int:

@@ -83,6 +83,7 @@ int32_t check_problem(const unigist_problem* p, Geom* g, float* scale) {
     g->N = (int)N;
     const int64_t k = ((int64_t)p->window + p->ratio - 1) / p->ratio;
     g->k = (int)(k < n ? k : n);
+    g->uoff = 0;
   }
   if (scale) *scale = p->softmax_scale > 0.f ? p->softmax_scale : 1.0f / sqrtf((float)p->head_dim);
   return UNIGIST_OK;
@@ -287,6 +288,47 @@ int32_t unigist_kv_compact(const unigist_problem* p, const void* k, const void* 
   }
   return launch_compact_inplace(g, *p, kc, vc, num_blocks, table, max_blocks, seq_lens, kept_idx,
                                 edit_only ? nullptr : workspace, (cudaStream_t)stream);
+}
+
+static int32_t check_chunk(const unigist_problem* p, const Geom& g, int32_t u0, int32_t c) {
+  if (u0 < 0 || c < 1 || (int64_t)u0 + c > g.n)
+    return fail(UNIGIST_ERR_INVALID_ARG, "chunk of %d units from unit %d does not fit the %d units of the prompt", c, u0,
+                g.n);
+  (void)p;
+  return UNIGIST_OK;
+}
+
+size_t unigist_prefill_workspace_bytes(const unigist_problem* p, int32_t unit_begin, int32_t unit_count) {
+  Geom g;
+  if (check_problem(p, &g, nullptr) != UNIGIST_OK || check_chunk(p, g, unit_begin, unit_count) != UNIGIST_OK) return 0;
+  const int64_t w_units = unit_begin < g.k ? unit_begin : g.k;
+  const int64_t n_ctx = (int64_t)g.s + (w_units + unit_count) * g.r + unit_begin + unit_count;
+  return align_up(2 * (size_t)p->batch * n_ctx * p->num_kv_heads * p->head_dim * 2, 256);
+}
+
+int32_t unigist_prefill_chunk(const unigist_problem* p, int32_t unit_begin, int32_t unit_count, const void* q,
+                              const void* k, const void* v, void* kc, void* vc, int32_t num_blocks, int32_t* table,
+                              int32_t max_blocks, int32_t* seq_lens, void* o, float* lse, void* workspace,
+                              size_t ws_bytes, void* stream) {
+  Geom g;
+  float scale;
+  if (int32_t rc = check_problem(p, &g, &scale)) return rc;
+  if (int32_t rc = check_chunk(p, g, unit_begin, unit_count)) return rc;
+  if (!q || !k || !v || !kc || !vc || !table || !seq_lens || !o || !lse)
+    return fail(UNIGIST_ERR_INVALID_ARG, "a pointer is NULL");
+  const void* ptrs[] = {q, k, v, kc, vc, o, lse, workspace};
+  for (const void* x : ptrs)
+    if (!aligned16(x)) return fail(UNIGIST_ERR_ALIGNMENT, "tensor pointers must be 16-byte aligned");
+  const size_t need = unigist_prefill_workspace_bytes(p, unit_begin, unit_count);
+  if (!workspace || ws_bytes < need)
+    return fail(UNIGIST_ERR_WORKSPACE, "this chunk needs %zu bytes of workspace, got %zu", need, ws_bytes);
+  const int64_t kept = (int64_t)g.s + unit_begin + unit_count +
+                       (int64_t)(g.k < unit_begin + unit_count ? g.k : unit_begin + unit_count) * g.r;
+  if (num_blocks < 1 || (int64_t)max_blocks * UNIGIST_PAGE_TOKENS < kept)
+    return fail(UNIGIST_ERR_SHAPE, "block table has %d entries per sequence, the cache after this chunk needs %lld tokens",
+                max_blocks, (long long)kept);
+  return launch_prefill_chunk(*p, g, scale, unit_begin, unit_count, q, k, v, kc, vc, num_blocks, table, max_blocks,
+                              seq_lens, o, lse, workspace, (cudaStream_t)stream);
 }
 
 size_t unigist_decode_workspace_bytes(int32_t S, int32_t Hq, int32_t Hkv, int32_t D,

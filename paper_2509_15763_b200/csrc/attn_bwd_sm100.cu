@@ -1217,10 +1217,10 @@ int32_t launch_bwd_sm100(const Geom& g, const unigist_problem& p, float scale, c
   // reduction maps over the fp32 dQ tensor (always shifted)
   CUtensorMap fq[3], fdo[3], fk[3], fv[3], mdq[3];
   for (int sg = 0; sg < 3; ++sg) {
-    if (int32_t rc = encode_tile_map(&fq[sg], q, D, Hq, B, g.s, g.T, g.r, il, sg)) return rc;
-    if (int32_t rc = encode_tile_map(&fdo[sg], do_src, D, Hq, B, g.s, g.T, g.r, il, sg)) return rc;
-    if (int32_t rc = encode_tile_map(&fk[sg], k, D, Hkv, B, g.s, g.T, g.r, il, sg)) return rc;
-    if (int32_t rc = encode_tile_map(&fv[sg], v, D, Hkv, B, g.s, g.T, g.r, il, sg)) return rc;
+    if (int32_t rc = encode_tile_map(&fq[sg], q, D, Hq, B, g.s, g.T, g.r, g.n, il, sg)) return rc;
+    if (int32_t rc = encode_tile_map(&fdo[sg], do_src, D, Hq, B, g.s, g.T, g.r, g.n, il, sg)) return rc;
+    if (int32_t rc = encode_tile_map(&fk[sg], k, D, Hkv, B, g.s, g.T, g.r, g.n, il, sg)) return rc;
+    if (int32_t rc = encode_tile_map(&fv[sg], v, D, Hkv, B, g.s, g.T, g.r, g.n, il, sg)) return rc;
     const int rows = seg_len(g, sg) > 0 ? seg_len(g, sg) : 1;  // a tensor map cannot be empty
     if (int32_t rc = encode_segment_map_f32(&mdq[sg], dq32, D, Hq, g.N, B, seg_base(g, sg), rows, 32, 32)) return rc;
   }

@@ -71,11 +71,11 @@ struct Stream {
   }
 };
 
-__device__ Stream make_stream(const Geom& g, bool valid, int h, int qt, int qseg) {
+__device__ Stream make_stream(const Geom& g, bool valid, int h, int qt, int qseg, int q_off) {
   Stream s;
   s.valid = valid;
   s.h = h;
-  s.row_a = qt * BM;
+  s.row_a = q_off + qt * BM;  // rows are numbered inside the key segment; the queries may start at q_off
   s.row_b = min(s.row_a + BM - 1, seg_len(g, qseg) - 1);
   if (!valid) {
     s.row_a = s.row_b = 0;
@@ -219,7 +219,7 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_sink, const __gri
                       const __grid_constant__ CUtensorMap tm_v_sink, const __grid_constant__ CUtensorMap tm_v_raw,
                       const __grid_constant__ CUtensorMap tm_v_gist, Geom g, int Hq, int Hkv, float scale_log2,
                       __nv_bfloat16* __restrict__ o, float* __restrict__ lse, int n_sink_units, int n_raw_units,
-                      int pair_heads, int interleaved) {
+                      int pair_heads, int interleaved, QueryRows qr) {
   using SM = FwdSmem<D>;
   extern __shared__ unsigned char smem_dyn[];
   const uint32_t base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
@@ -240,7 +240,8 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_sink, const __gri
   const int u_lin = gridDim.x - 1 - blockIdx.x;
   const int qseg = u_lin < n_sink_units ? kSegSink : (u_lin < n_sink_units + n_raw_units ? kSegRaw : kSegGist);
   const int u = u_lin - (qseg == kSegSink ? 0 : (qseg == kSegRaw ? n_sink_units : n_sink_units + n_raw_units));
-  const int n_qt = (seg_len(g, qseg) + BM - 1) / BM;
+  const int q_off = qr.off[qseg];  // first query row of the segment (0 unless this is a prefill chunk)
+  const int n_qt = (seg_len(g, qseg) - q_off + BM - 1) / BM;
   const int q_seg_base = seg_base(g, qseg);  // shifted position of the segment's row 0
   int qt[2], hh[2];
   bool sv[2];
@@ -257,7 +258,8 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_sink, const __gri
     sv[1] = qt[1] < n_qt;
   }
   const int hk = hh[0] / (Hq / Hkv);  // both streams share the KV head
-  const Stream str0 = make_stream(g, sv[0], hh[0], qt[0], qseg), str1 = make_stream(g, sv[1], hh[1], qt[1], qseg);
+  const Stream str0 = make_stream(g, sv[0], hh[0], qt[0], qseg, q_off),
+               str1 = make_stream(g, sv[1], hh[1], qt[1], qseg, q_off);
   const TileSeq seq = make_tile_seq(str0, str1, qseg);
   const int nt = seq.count();
 
@@ -479,7 +481,9 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_sink, const __gri
         }
         const float inv_l = 1.f / l_run;
         const bool valid = me.row_a + r_in_tile <= me.row_b;
-        const long long tok = (long long)b * g.N + seg_row_to_token(g, interleaved != 0, qseg, me.row_a + r_in_tile);
+        const int out_row = interleaved ? seg_row_to_token(g, true, qseg, me.row_a + r_in_tile)
+                                        : qr.out_base[qseg] + (me.row_a + r_in_tile - q_off);
+        const long long tok = (long long)b * qr.n_out + out_row;
         __nv_bfloat16* orow = o + (tok * Hq + me.h) * D + part * (D / kSplit);
 #pragma unroll
         for (int c = 0; c < D / kSplit / 32; ++c) {
@@ -499,7 +503,7 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_sink, const __gri
           }
         }
         if (valid && part == 0)
-          lse[((long long)b * Hq + me.h) * g.N + q_seg_base + me.row_a + r_in_tile] =
+          lse[((long long)b * Hq + me.h) * qr.n_out + qr.out_base[qseg] + (me.row_a + r_in_tile - q_off)] =
               (m_run + log2f(l_run)) * 0.6931471805599453f;
       } else {
         atomicExch(&g_fwd_timeout, 1u);
@@ -563,12 +567,12 @@ int32_t encode_segment_map_f32(CUtensorMap* map, const void* base, int D, int H,
   return encode_map(map, base, D, H, N, B, seg_first_row, seg_rows, box_cols, box_rows, 4);
 }
 
-int32_t encode_tile_map(CUtensorMap* map, const void* base, int D, int H, int B, int s, int T, int r,
+int32_t encode_tile_map(CUtensorMap* map, const void* base, int D, int H, int B, int s, int T, int r, int n_gists,
                         bool interleaved, int segment) {
   const bool raw_segment = segment == kSegRaw;
   EncodeFn encode;
   if (int32_t rc = get_encode_fn(&encode)) return rc;
-  const long long n = T / r, N = (long long)s + T + n;
+  const long long n = n_gists, N = (long long)s + T + n;
   const cuuint64_t row_bytes = (cuuint64_t)H * D * 2;
   long long first_row, units, unit_rows, unit_stride_rows;
   if (segment == kSegSink) {  // the sinks are a prefix in either order; a tensor map cannot be empty
@@ -620,16 +624,25 @@ int32_t encode_map_2d_bf16(CUtensorMap* map, const void* base, long long rows, i
 }
 
 int32_t launch_fwd_sm100(const Geom& g, const unigist_problem& p, float scale, const void* q, const void* k,
-                         const void* v, void* o, float* lse, cudaStream_t st) {
+                         const void* v, void* o, float* lse, cudaStream_t st, const QueryRows* chunk) {
   const int D = p.head_dim, Hq = p.num_q_heads, Hkv = p.num_kv_heads, B = p.batch;
   CUtensorMap mq[3], mk[3], mv[3];  // per segment: sinks, raw, gists
-  const bool il = (p.flags & UNIGIST_FLAG_INTERLEAVED) != 0;
-  for (int sg = 0; sg < 3; ++sg) {
-    if (int32_t rc = encode_tile_map(&mq[sg], q, D, Hq, B, g.s, g.T, g.r, il, sg)) return rc;
-    if (int32_t rc = encode_tile_map(&mk[sg], k, D, Hkv, B, g.s, g.T, g.r, il, sg)) return rc;
-    if (int32_t rc = encode_tile_map(&mv[sg], v, D, Hkv, B, g.s, g.T, g.r, il, sg)) return rc;
+  const bool il = (p.flags & UNIGIST_FLAG_INTERLEAVED) != 0 && !chunk;
+  QueryRows qr;
+  if (chunk) {
+    qr = *chunk;
+  } else {
+    for (int sg = 0; sg < 3; ++sg) qr.off[sg] = 0, qr.out_base[sg] = seg_base(g, sg);
+    qr.n_out = g.N;
   }
-  const int n_sink_qt = (g.s + BM - 1) / BM, n_raw_qt = (g.T + BM - 1) / BM, n_gist_qt = (g.n + BM - 1) / BM;
+  // the Q tensor holds the query rows only: the tail of each segment from qr.off on
+  const int sq = g.s - qr.off[kSegSink], Tq = g.T - qr.off[kSegRaw], nq = g.n - qr.off[kSegGist];
+  for (int sg = 0; sg < 3; ++sg) {
+    if (int32_t rc = encode_tile_map(&mq[sg], q, D, Hq, B, sq, Tq, g.r, nq, il, sg)) return rc;
+    if (int32_t rc = encode_tile_map(&mk[sg], k, D, Hkv, B, g.s, g.T, g.r, g.n, il, sg)) return rc;
+    if (int32_t rc = encode_tile_map(&mv[sg], v, D, Hkv, B, g.s, g.T, g.r, g.n, il, sg)) return rc;
+  }
+  const int n_sink_qt = (sq + BM - 1) / BM, n_raw_qt = (Tq + BM - 1) / BM, n_gist_qt = (nq + BM - 1) / BM;
   // Two streams per block: neighbouring heads of a KV group when the group size is even,
   // otherwise neighbouring query tiles of one head.
   const int pair_heads = (Hq / Hkv) % 2 == 0 ? 1 : 0;
@@ -645,7 +658,7 @@ int32_t launch_fwd_sm100(const Geom& g, const unigist_problem& p, float scale, c
       KernelScope ks("attn_fwd_sm100_kernel", st);
       kern<<<grid, kThreads, smem, st>>>(mq[0], mq[1], mq[2], mk[0], mk[1], mk[2], mv[0], mv[1], mv[2], g, Hq, Hkv,
                                          scale_log2, (__nv_bfloat16*)o, lse, n_sink_units, n_raw_units, pair_heads,
-                                         il ? 1 : 0);
+                                         il ? 1 : 0, qr);
     }
     return check_launch("tcgen05 forward kernel");
   };

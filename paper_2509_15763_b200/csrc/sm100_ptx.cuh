@@ -245,7 +245,7 @@ int32_t encode_segment_map(CUtensorMap* map, const void* base, int D, int H, lon
 //   interleaved raw:   unit = gist unit (r raw rows, stride r + 1 rows);    tile = 128 / r units x r rows
 //   interleaved gist:  unit = gist unit, its one gist row;                  tile = 128 units
 // A tile starts at coordinates (d, h, 0, first unit, b); units past the segment read as zero.
-int32_t encode_tile_map(CUtensorMap* map, const void* base, int D, int H, int B, int s, int T, int r,
+int32_t encode_tile_map(CUtensorMap* map, const void* base, int D, int H, int B, int s, int T, int r, int n_gists,
                         bool interleaved, int segment /* kSegSink, kSegRaw, kSegGist */);
 
 // The same for an fp32 tensor, box = box_cols x 1 x box_rows x 1, no swizzle (rows of the box are

@@ -12,6 +12,10 @@ namespace ug {
 // Geometry of one sequence.  Shifted order = [sinks | raw | gists] (Section 4.2).
 struct Geom {
   int s, T, r, k, n, N;  // k is clamped to n
+  // Gist number of raw unit 0.  0 for a whole sequence.  In chunk-wise prefill (Section 4.3) the raw
+  // segment holds only the units still in the cache plus the new chunk, while the gist segment holds
+  // every gist so far: raw unit u then belongs to gist number u + uoff, and n = T / r + uoff.
+  int uoff;
 };
 
 // Columns a query row may see, per segment, numbered inside the segment and inclusive
@@ -37,14 +41,15 @@ __host__ __device__ inline RowIv row_intervals(const Geom& g, int sigma) {
     v.hi_sink = g.s - 1;
     v.lo_raw = u0 * g.r;
     v.hi_raw = i;
-    v.hi_gist = u - 1;
-  } else {  // gist query u: its own unit's raw tokens and itself
-    const int u = sigma - g.s - g.T;
+    v.hi_gist = u + g.uoff - 1;
+  } else {  // gist query: its own unit's raw tokens and itself
+    const int ug = sigma - g.s - g.T;  // gist number
+    const int u = ug - g.uoff;         // its raw unit inside the raw segment (>= 0 for every gist that is a query)
     const int u0 = u > g.k ? u - g.k : 0;
     v.hi_sink = g.s - 1;
     v.lo_raw = u0 * g.r;
     v.hi_raw = (u + 1) * g.r - 1;
-    v.hi_gist = u;
+    v.hi_gist = ug;
   }
   return v;
 }
@@ -110,8 +115,16 @@ int32_t launch_shift(const Geom& g, int B, const void* src, void* dst, size_t ro
                      bool inverse, cudaStream_t st);
 int32_t launch_fwd_simt(const Geom& g, const unigist_problem& p, float scale, const void* q,
                         const void* k, const void* v, void* o, float* lse, cudaStream_t st);
+// Where the query rows of a forward call sit.  A whole-sequence call has queries for every row
+// (off = 0, out_base = the segments' shifted positions, n_out = N); a prefill chunk has queries only for
+// the tail of each segment: query row j of segment sg is row off[sg] + j of that segment, and its
+// output goes to token out_base[sg] + j of an [B, n_out, Hq, D] tensor.
+struct QueryRows {
+  int off[3], out_base[3], n_out;
+};
 int32_t launch_fwd_sm100(const Geom& g, const unigist_problem& p, float scale, const void* q,
-                         const void* k, const void* v, void* o, float* lse, cudaStream_t st);
+                         const void* k, const void* v, void* o, float* lse, cudaStream_t st,
+                         const QueryRows* chunk = nullptr);
 int32_t fwd_sm100_take_timeout(bool* timed_out);
 int32_t launch_bwd_sm100(const Geom& g, const unigist_problem& p, float scale, const void* q,
                          const void* k, const void* v, const void* o, const float* lse,
@@ -132,6 +145,9 @@ int32_t launch_compact_inplace(const Geom& g, const unigist_problem& p, void* kc
 int32_t launch_decode(int S, int Hq, int Hkv, int D, float scale, const void* q, const void* kc,
                       const void* vc, int num_blocks, const int32_t* table, int max_blocks,
                       const int32_t* seq_lens, void* o, float* lse, void* ws, cudaStream_t st);
+int32_t launch_prefill_chunk(const unigist_problem& p, const Geom& g_full, float scale, int u0, int c, const void* q,
+                             const void* k, const void* v, void* kc, void* vc, int num_blocks, int32_t* table,
+                             int max_blocks, int32_t* seq_lens, void* o, float* lse, void* workspace, cudaStream_t st);
 int decode_num_splits(int S, int Hkv, int max_blocks);
 int32_t decode_take_timeout(bool* timed_out);
 
