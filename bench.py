@@ -308,6 +308,47 @@ def job_value(world, flop_per_replica_step, steps, total_ms):
     return world * flop_per_replica_step * steps / (total_ms * 1e-3) / 1e12
 
 
+def bench_chunked_prefill(path, chunk_units, iters=3):
+    """The prefill workload fed in chunks of `chunk_units` gist units through unigist_prefill_chunk: each
+    chunk attends to the compressed paged cache and advances it.  -> dict for the JSON line."""
+    import torch
+
+    ug, w, dev = path.ug, path.w, path.dev
+    p, r, s, n = path.p, w.ratio, w.num_sinks, w.num_gists
+    chunk_units = min(chunk_units, n)
+    starts = list(range(0, n, chunk_units))
+    chunks = []
+    for u0 in starts:  # the chunk's tokens in shifted chunk order [sinks | raw | gists], sliced before timing
+        c = min(chunk_units, n - u0)
+        ar = torch.arange(u0, u0 + c, device=dev)
+        raw = (s + ar[:, None] * (r + 1) + torch.arange(r, device=dev)[None, :]).reshape(-1)
+        gist = s + ar * (r + 1) + r
+        idx = torch.cat(([torch.arange(s, device=dev)] if u0 == 0 else []) + [raw, gist])
+        chunks.append((u0, c, *(path.inter[k][:, idx].contiguous() for k in ("q", "k", "v"))))
+    o = [torch.empty_like(c[2]) for c in chunks]
+    lse = [torch.empty(w.batch, w.num_q_heads, c[2].shape[1], dtype=torch.float32, device=dev) for c in chunks]
+    ws = torch.empty(max(ug.unigist_prefill_workspace_bytes(p, u0, c) for u0, c, *_ in chunks), dtype=torch.uint8,
+                     device=dev)
+
+    def run():
+        for i, (u0, c, q, k, v) in enumerate(chunks):
+            ug.unigist_prefill_chunk(p, u0, c, q, k, v, path.kc, path.vc, path.table, path.lens, o[i], lse[i], ws)
+
+    run()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(iters):
+        run()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / iters
+    flops = 4.0 * w.head_dim * path.pairs * w.num_q_heads * w.batch
+    return {"chunk_units": chunk_units, "chunk_raw_tokens": chunk_units * r, "chunks": len(chunks), "ms": ms,
+            "value": flops / (ms * 1e-3) / 1e12, "unit": UNIT,
+            "note": "whole prompt through unigist_prefill_chunk: context gather + forward + cache advance per chunk"}
+
+
 def run_ours(args, w):
     import torch
 
@@ -436,6 +477,7 @@ def run_ours(args, w):
         "cpu_baseline": {"value": cpu_tf, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc},
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": path.h2d_bytes(),
                 "d2h_bytes_per_step": path.d2h_bytes()},
+        "chunked_prefill": bench_chunked_prefill(path, 1024) if w.forward_only else None,
         "explicit_shift_step": None if explicit_ms is None else {
             "ms_per_step": explicit_ms, "value": path.flops / (explicit_ms * 1e-3) / 1e12, "unit": UNIT,
             "note": "the same step with 4 shift and 4 unshift launches around shifted-order attention calls"},
