@@ -45,11 +45,11 @@ NCU_TRAFFIC_BYTES = {
 # FLOP per visible pair per query head that each attention kernel performs algorithmically,
 # in units of head_dim (a QK^T- or PV-shaped product is 2 * D FLOP per pair).
 KERNEL_FLOP_PER_PAIR_D = {
-    "fwd_simt_kernel": 4, "bwd_dq_simt_kernel": 6, "bwd_dkdv_simt_kernel": 8,
+    "bwd_dq_simt_kernel": 6, "bwd_dkdv_simt_kernel": 8,
     "attn_fwd_sm100_kernel": 4, "attn_bwd_dq_sm100_kernel": 6, "attn_bwd_dkdv_sm100_kernel": 8,
     "attn_bwd_fused_sm100_kernel": 10,
 }
-CUDA_CORE_KERNELS = {"fwd_simt_kernel", "bwd_dq_simt_kernel", "bwd_dkdv_simt_kernel"}
+CUDA_CORE_KERNELS = {"bwd_dq_simt_kernel", "bwd_dkdv_simt_kernel"}
 
 
 def measured_peaks():

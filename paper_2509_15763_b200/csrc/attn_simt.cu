@@ -1,7 +1,8 @@
-// CUDA-core (no tensor core) gist-masked attention: forward, dQ and dK/dV kernels on 64x64 tiles
-// of the SHIFTED sequence.  This is the general path: any s, T, r, W, head_dim 64 or 128, tiles
-// may straddle the sink / raw / gist segments because the mask is evaluated per element from
-// the closed-form row intervals.  Tiles with no visible pair are skipped without being read.
+// CUDA-core (no tensor core) backward of the gist-masked attention: dQ and dK/dV kernels on 64x64
+// tiles of the SHIFTED sequence.  The general path (any s, T, r, W, head_dim 64 or 128; tiles may
+// straddle the sink / raw / gist segments because the mask is evaluated per element from the
+// closed-form row intervals; tiles with no visible pair are skipped without being read), used for the
+// one case the tensor-core backward does not cover: head_dim 64 with a sink prefix.
 #include "ug_common.cuh"
 
 namespace ug {
@@ -161,96 +162,6 @@ __device__ __forceinline__ void store_rows_bf16(__nv_bfloat16* base, long long r
       pk.x = *reinterpret_cast<uint32_t*>(&lo);
       pk.y = *reinterpret_cast<uint32_t*>(&hi);
       *reinterpret_cast<uint2*>(base + (long long)(row0 + rr) * row_stride + tx * 4 + 64 * h) = pk;
-    }
-  }
-}
-
-// ---------------------------------------------------------------- forward
-template <int D>
-__global__ void __launch_bounds__(256)
-fwd_simt_kernel(Geom g, int Hq, int Hkv, float scale, const __nv_bfloat16* __restrict__ q,
-                const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restrict__ v,
-                __nv_bfloat16* __restrict__ o, float* __restrict__ lse) {
-  constexpr int LD = D + 4;
-  extern __shared__ __align__(16) float smem[];
-  float* Qs = smem;
-  float* Ks = Qs + TS * LD;
-  float* Vs = Ks + TS * LD;
-  float* Ss = Vs + TS * LD;
-  const int ntiles = (g.N + TS - 1) / TS;
-  const int qt = ntiles - 1 - blockIdx.x;  // heavy (late) tiles first
-  const int h = blockIdx.y, b = blockIdx.z, hk = h / (Hq / Hkv);
-  const int ty = threadIdx.x / 16, tx = threadIdx.x % 16;
-  const int row0 = qt * TS, nrows = min(TS, g.N - row0);
-  const long long qs = (long long)Hq * D, ks = (long long)Hkv * D;
-  const __nv_bfloat16* qb = q + ((long long)b * g.N * Hq + h) * D;
-  const __nv_bfloat16* kb = k + ((long long)b * g.N * Hkv + hk) * D;
-  const __nv_bfloat16* vb = v + ((long long)b * g.N * Hkv + hk) * D;
-  load_tile_bf16<D>(Qs, qb, qs, row0, nrows);
-
-  RowIv iv[4];
-  float m[4], l[4];
-  float4 acc[4][D / 64];
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    iv[i] = row_intervals(g, min(row0 + ty + 16 * i, g.N - 1));
-    m[i] = -INFINITY;
-    l[i] = 0.f;
-#pragma unroll
-    for (int hh = 0; hh < D / 64; ++hh) acc[i][hh] = make_float4(0.f, 0.f, 0.f, 0.f);
-  }
-  for (int kt = 0; kt < ntiles; ++kt) {
-    const int col0 = kt * TS, ncols = min(TS, g.N - col0);
-    if (!tile_any_visible(g, row0, row0 + nrows - 1, col0, col0 + ncols - 1)) continue;
-    __syncthreads();  // previous tile's readers are done
-    load_tile_bf16<D>(Ks, kb, ks, col0, ncols);
-    load_tile_bf16<D>(Vs, vb, ks, col0, ncols);
-    __syncthreads();
-    float sc[4][4] = {};
-    gemm_nt<D>(Qs, Ks, sc, ty, tx);
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      float mx = -INFINITY;
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        const int col = col0 + tx + 16 * j;
-        const bool ok = col < g.N && visible(g, iv[i], col);
-        sc[i][j] = ok ? sc[i][j] * scale : -INFINITY;
-        mx = fmaxf(mx, sc[i][j]);
-      }
-      mx = group16_max(mx);
-      const float mn = fmaxf(m[i], mx);
-      const float f = (mn == -INFINITY) ? 1.f : __expf(m[i] - mn);  // m = -inf -> exp(-inf) = 0
-      float ps = 0.f;
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        const float p = (mn == -INFINITY) ? 0.f : __expf(sc[i][j] - mn);
-        ps += p;
-        Ss[(ty + 16 * i) * LDS_ + tx + 16 * j] = p;
-      }
-      ps = group16_sum(ps);
-      l[i] = l[i] * f + ps;
-      m[i] = mn;
-#pragma unroll
-      for (int hh = 0; hh < D / 64; ++hh) {
-        acc[i][hh].x *= f;
-        acc[i][hh].y *= f;
-        acc[i][hh].z *= f;
-        acc[i][hh].w *= f;
-      }
-    }
-    __syncthreads();
-    gemm_nn<D>(Ss, Vs, acc, ty, tx);
-  }
-  float inv[4];
-#pragma unroll
-  for (int i = 0; i < 4; ++i) inv[i] = 1.f / l[i];
-  store_rows_bf16<D>(o + ((long long)b * g.N * Hq + h) * D, qs, row0, nrows, acc, inv, ty, tx);
-  if (tx == 0) {
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      const int rr = ty + 16 * i;
-      if (rr < nrows) lse[((long long)b * Hq + h) * g.N + row0 + rr] = m[i] + logf(l[i]);
     }
   }
 }
@@ -440,24 +351,6 @@ int32_t set_smem(K kernel, size_t bytes) {
 }
 
 }  // namespace
-
-int32_t launch_fwd_simt(const Geom& g, const unigist_problem& p, float scale, const void* q,
-                        const void* k, const void* v, void* o, float* lse, cudaStream_t st) {
-  const int ntiles = (g.N + TS - 1) / TS;
-  dim3 grid(ntiles, p.num_q_heads, p.batch);
-  auto go = [&](auto kern, int D) -> int32_t {
-    const size_t smem = (size_t)(3 * TS * (D + 4) + TS * LDS_) * sizeof(float);
-    if (int32_t rc = set_smem(kern, smem)) return rc;
-    {
-      KernelScope ks("fwd_simt_kernel", st);
-      kern<<<grid, 256, smem, st>>>(g, p.num_q_heads, p.num_kv_heads, scale, (const __nv_bfloat16*)q,
-                                    (const __nv_bfloat16*)k, (const __nv_bfloat16*)v,
-                                    (__nv_bfloat16*)o, lse);
-    }
-    return check_launch("forward kernel");
-  };
-  return p.head_dim == 64 ? go(fwd_simt_kernel<64>, 64) : go(fwd_simt_kernel<128>, 128);
-}
 
 int32_t launch_bwd_simt(const Geom& g, const unigist_problem& p, float scale, const void* q,
                         const void* k, const void* v, const void* o, const float* lse,

@@ -113,8 +113,6 @@ inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
 int32_t launch_layout(const Geom& g, int32_t* sp, int32_t* up, int32_t* pos, cudaStream_t st);
 int32_t launch_shift(const Geom& g, int B, const void* src, void* dst, size_t row_bytes,
                      bool inverse, cudaStream_t st);
-int32_t launch_fwd_simt(const Geom& g, const unigist_problem& p, float scale, const void* q,
-                        const void* k, const void* v, void* o, float* lse, cudaStream_t st);
 // Where the query rows of a forward call sit.  A whole-sequence call has queries for every row
 // (off = 0, out_base = the segments' shifted positions, n_out = N); a prefill chunk has queries only for
 // the tail of each segment: query row j of segment sg is row off[sg] + j of that segment, and its
