@@ -189,6 +189,38 @@ int32_t unigist_prefill_chunk(const unigist_problem* p, int32_t unit_begin, int3
                               int32_t* block_table, int32_t max_blocks_per_seq, int32_t* seq_lens, void* o, float* lse,
                               void* workspace, size_t ws_bytes, void* stream);
 
+/*
+ * Cache maintenance while decoding (Section 4.3: raw tokens outside the local window "can be safely discarded
+ * at each compression point").  The sequence grows token by token: r raw tokens, then their gist, and so on.
+ * unigist_cache_append writes one new token's K / V rows (k_new, v_new [B, Hkv, D] device bf16) into every
+ * sequence's cache.  A gist (is_gist = 1, after exactly r raw tokens) still attends to the k + 1 units of the
+ * window; the first raw token after it (is_gist = 0) opens a new unit, at which point the oldest unit's r
+ * raw tokens are seen by no one any more: their slots are freed and reused by the new unit's raw tokens.
+ * No entry ever moves; the cache occupies slots [0, seq_lens[b]) in an order that becomes arbitrary (attention
+ * does not care), grows by one slot per gist unit, and after every append its live slots hold exactly the
+ * tokens the new token sees.  p->raw_len is not used as a bound here.
+ *
+ * state: unigist_cache_state_bytes(p) bytes of device memory owned by the caller; unigist_cache_state_init
+ * sets it up for caches in the order unigist_kv_compact / unigist_prefill_chunk leave them in after
+ * units_done whole units (0 with an empty or sinks-only cache).  Misuse (a gist before its unit is
+ * complete, a raw token after it, a block table that is too short) sets state[b * ints + 4] != 0 and
+ * leaves the cache unchanged.
+ *
+ * Between the first raw token of a unit and its last, up to r - 1 freed slots inside [0, seq_lens[b]) still
+ * hold the evicted tokens; unigist_decode_step is unigist_decode (one query per sequence, p->batch sequences,
+ * shapes and scale from p) that leaves those slots, listed in `state`, out of the attention.  Use it for
+ * every query of a loop that maintains its cache with unigist_cache_append.
+ */
+size_t unigist_cache_state_bytes(const unigist_problem* p);
+int32_t unigist_cache_state_init(const unigist_problem* p, int32_t units_done, int32_t* state, void* stream);
+int32_t unigist_cache_append(const unigist_problem* p, const void* k_new, const void* v_new, int32_t is_gist,
+                             void* k_cache, void* v_cache, int32_t num_blocks, const int32_t* block_table,
+                             int32_t max_blocks_per_seq, int32_t* seq_lens, int32_t* state, void* stream);
+int32_t unigist_decode_step(const unigist_problem* p, const void* q, const void* k_cache, const void* v_cache,
+                            int32_t num_blocks, const int32_t* block_table, int32_t max_blocks_per_seq,
+                            const int32_t* seq_lens, const int32_t* state, void* o, float* lse, void* workspace,
+                            size_t ws_bytes, void* stream);
+
 /* Scratch for unigist_decode (split-KV partial results). */
 size_t unigist_decode_workspace_bytes(int32_t num_seqs, int32_t num_q_heads, int32_t num_kv_heads,
                                       int32_t head_dim, int32_t max_blocks_per_seq);

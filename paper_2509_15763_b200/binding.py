@@ -27,6 +27,7 @@ SYMBOLS = [
     "unigist_decode", "unigist_launch_count", "unigist_last_error_string",
     "unigist_kernel_timing", "unigist_kernel_timing_count", "unigist_kernel_timing_get",
     "unigist_device_status", "unigist_decode_static", "unigist_prefill_workspace_bytes", "unigist_prefill_chunk",
+    "unigist_cache_state_bytes", "unigist_cache_state_init", "unigist_cache_append", "unigist_decode_step",
 ]
 
 
@@ -89,6 +90,10 @@ def lib() -> ctypes.CDLL:
             "unigist_kv_compact": (i32, [P, vp, vp, vp, vp, i32, vp, i32, vp, vp, vp, sz, vp]),
             "unigist_decode_workspace_bytes": (sz, [i32] * 5),
             "unigist_prefill_workspace_bytes": (sz, [P, i32, i32]),
+            "unigist_cache_state_bytes": (sz, [P]),
+            "unigist_cache_state_init": (i32, [P, i32, vp, vp]),
+            "unigist_cache_append": (i32, [P, vp, vp, i32, vp, vp, i32, vp, i32, vp, vp, vp]),
+            "unigist_decode_step": (i32, [P, vp, vp, vp, i32, vp, i32, vp, vp, vp, vp, vp, sz, vp]),
             "unigist_prefill_chunk": (i32, [P, i32, i32, vp, vp, vp, vp, vp, i32, vp, i32, vp, vp, vp, vp, sz, vp]),
             "unigist_decode": (i32, [i32, i32, i32, i32, f32, vp, vp, vp, i32, vp, i32, vp, vp, vp, vp, sz, vp]),
             "unigist_kernel_timing": (i32, [i32]),
@@ -251,6 +256,33 @@ def unigist_prefill_chunk(p: Problem, unit_begin: int, unit_count: int, q, k, v,
                                        _ptr(k_cache), _ptr(v_cache), k_cache.shape[0], _ptr(block_table),
                                        block_table.shape[1], _ptr(seq_lens), _ptr(o), _ptr(lse), _ptr(workspace),
                                        workspace.numel() * workspace.element_size(), _stream(stream)))
+
+
+def unigist_cache_state_bytes(p: Problem) -> int:
+    return lib().unigist_cache_state_bytes(ctypes.byref(p.c()))
+
+
+def unigist_cache_state_init(p: Problem, units_done: int, state, stream=None):
+    _dev(state)
+    _check(lib().unigist_cache_state_init(ctypes.byref(p.c()), units_done, _ptr(state), _stream(stream)))
+
+
+def unigist_cache_append(p: Problem, k_new, v_new, is_gist: bool, k_cache, v_cache, block_table, seq_lens, state,
+                         stream=None):
+    _dev(k_new, v_new, k_cache, v_cache, block_table, seq_lens, state)
+    _check(lib().unigist_cache_append(ctypes.byref(p.c()), _ptr(k_new), _ptr(v_new), int(bool(is_gist)),
+                                      _ptr(k_cache), _ptr(v_cache), k_cache.shape[0], _ptr(block_table),
+                                      block_table.shape[1], _ptr(seq_lens), _ptr(state), _stream(stream)))
+
+
+def unigist_decode_step(p: Problem, q, k_cache, v_cache, block_table, seq_lens, state, o, lse=None, workspace=None,
+                        stream=None):
+    _dev(q, k_cache, v_cache, block_table, seq_lens, state, o, lse, workspace)
+    _check(lib().unigist_decode_step(ctypes.byref(p.c()), _ptr(q), _ptr(k_cache), _ptr(v_cache), k_cache.shape[0],
+                                     _ptr(block_table), block_table.shape[1], _ptr(seq_lens), _ptr(state), _ptr(o),
+                                     _ptr(lse), _ptr(workspace),
+                                     0 if workspace is None else workspace.numel() * workspace.element_size(),
+                                     _stream(stream)))
 
 
 def unigist_decode_workspace_bytes(num_seqs, num_q_heads, num_kv_heads, head_dim, max_blocks_per_seq) -> int:

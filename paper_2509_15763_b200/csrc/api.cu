@@ -331,6 +331,40 @@ int32_t unigist_prefill_chunk(const unigist_problem* p, int32_t unit_begin, int3
                               seq_lens, o, lse, workspace, (cudaStream_t)stream);
 }
 
+size_t unigist_cache_state_bytes(const unigist_problem* p) {
+  Geom g;
+  if (check_problem(p, &g, nullptr) != UNIGIST_OK) return 0;
+  return align_up(cache_state_bytes(p->batch, g.r, unigist_window_units(p)), 256);
+}
+
+// The window of a growing sequence is k = ceil(W / r) units, not clamped by the prompt's length.
+static Geom decode_geom(const unigist_problem* p, const Geom& g) {
+  Geom d = g;
+  d.k = (int)(((int64_t)p->window + p->ratio - 1) / p->ratio);
+  return d;
+}
+
+int32_t unigist_cache_state_init(const unigist_problem* p, int32_t units_done, int32_t* state, void* stream) {
+  Geom g;
+  if (int32_t rc = check_problem(p, &g, nullptr)) return rc;
+  if (!state || units_done < 0) return fail(UNIGIST_ERR_INVALID_ARG, "state is NULL or units_done < 0");
+  return launch_cache_state_init(decode_geom(p, g), p->batch, units_done, state, (cudaStream_t)stream);
+}
+
+int32_t unigist_cache_append(const unigist_problem* p, const void* k_new, const void* v_new, int32_t is_gist, void* kc,
+                             void* vc, int32_t num_blocks, const int32_t* table, int32_t max_blocks, int32_t* seq_lens,
+                             int32_t* state, void* stream) {
+  Geom g;
+  if (int32_t rc = check_problem(p, &g, nullptr)) return rc;
+  if (!k_new || !v_new || !kc || !vc || !table || !seq_lens || !state)
+    return fail(UNIGIST_ERR_INVALID_ARG, "a pointer is NULL");
+  if (!aligned16(k_new) || !aligned16(v_new) || !aligned16(kc) || !aligned16(vc))
+    return fail(UNIGIST_ERR_ALIGNMENT, "tensor pointers must be 16-byte aligned");
+  if (num_blocks < 1 || max_blocks < 1) return fail(UNIGIST_ERR_INVALID_ARG, "the cache has no blocks");
+  return launch_cache_append(decode_geom(p, g), *p, is_gist != 0, k_new, v_new, kc, vc, num_blocks, table, max_blocks,
+                             seq_lens, state, (cudaStream_t)stream);
+}
+
 size_t unigist_decode_workspace_bytes(int32_t S, int32_t Hq, int32_t Hkv, int32_t D,
                                       int32_t max_blocks) {
   if (S < 1 || Hq < 1 || Hkv < 1 || D < 1 || max_blocks < 1) return 0;
@@ -359,6 +393,28 @@ int32_t unigist_decode(int32_t S, int32_t Hq, int32_t Hkv, int32_t D, float soft
     return fail(UNIGIST_ERR_WORKSPACE, "decode needs %zu bytes of workspace, got %zu", need, ws_bytes);
   return launch_decode(S, Hq, Hkv, D, scale, q, kc, vc, num_blocks, table, max_blocks, seq_lens, o,
                        lse, workspace, (cudaStream_t)stream);
+}
+
+int32_t unigist_decode_step(const unigist_problem* p, const void* q, const void* kc, const void* vc, int32_t num_blocks,
+                            const int32_t* table, int32_t max_blocks, const int32_t* seq_lens, const int32_t* state,
+                            void* o, float* lse, void* workspace, size_t ws_bytes, void* stream) {
+  Geom g;
+  float scale;
+  if (int32_t rc = check_problem(p, &g, &scale)) return rc;
+  const int S = p->batch, Hq = p->num_q_heads, Hkv = p->num_kv_heads, D = p->head_dim;
+  if (max_blocks < 1 || num_blocks < 1) return fail(UNIGIST_ERR_INVALID_ARG, "the cache has no blocks");
+  if (D != 128) return fail(UNIGIST_ERR_SHAPE, "decode supports head_dim 128, got %d", D);
+  if (Hq / Hkv > 8) return fail(UNIGIST_ERR_UNSUPPORTED, "decode supports at most 8 query heads per KV head");
+  if (!q || !kc || !vc || !table || !seq_lens || !state || !o) return fail(UNIGIST_ERR_INVALID_ARG, "a pointer is NULL");
+  if (!aligned16(q) || !aligned16(kc) || !aligned16(vc) || !aligned16(o) || !aligned16(workspace))
+    return fail(UNIGIST_ERR_ALIGNMENT, "tensor pointers must be 16-byte aligned");
+  const size_t need = unigist_decode_workspace_bytes(S, Hq, Hkv, D, max_blocks);
+  if (!workspace || ws_bytes < need)
+    return fail(UNIGIST_ERR_WORKSPACE, "decode needs %zu bytes of workspace, got %zu", need, ws_bytes);
+  int stride = 0, free_off = 0;
+  cache_state_layout(g.r, decode_geom(p, g).k, &stride, &free_off);
+  return launch_decode(S, Hq, Hkv, D, scale, q, kc, vc, num_blocks, table, max_blocks, seq_lens, o, lse, workspace,
+                       (cudaStream_t)stream, state, stride, free_off);
 }
 
 int32_t unigist_kernel_timing(int32_t enable) {

@@ -65,7 +65,8 @@ __global__ void __launch_bounds__(THREADS, 2)
 decode_split_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v, int Hq,
                     int Hkv, int G, float scale_log2, const __nv_bfloat16* __restrict__ q, int num_blocks,
                     const int32_t* __restrict__ table, int max_blocks, const int32_t* __restrict__ seq_lens,
-                    int splits, int blocks_per_split, float* __restrict__ part) {
+                    int splits, int blocks_per_split, float* __restrict__ part, const int32_t* __restrict__ holes,
+                    int holes_stride, int holes_off) {
   extern __shared__ unsigned char smem_dyn[];
   const uint32_t base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
   unsigned char* gen = smem_dyn + (base - smem_u32(smem_dyn));
@@ -144,6 +145,16 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
       if (!ok) break;
       const uint32_t sK = base + st * STAGE_BYTES, sV = sK + PAGE_BYTES;
       const int nvalid = min(PG, len - (b0 + i) * PG);
+      // cache slots that were freed and not yet reused (a decoding loop's eviction list) hold stale tokens
+      unsigned long long hole_bits = 0ull;
+      if (holes) {
+        const int32_t* hs = holes + (long long)seq * holes_stride;
+        const int nh = hs[2];
+        for (int h2 = 0; h2 < nh; ++h2) {
+          const int pos = hs[holes_off + h2] - (b0 + i) * PG;
+          if (pos >= 0 && pos < PG) hole_bits |= 1ull << pos;
+        }
+      }
       // S = Q K^T: 8 token tiles of 8, fp32
       float s[8][4];
 #pragma unroll
@@ -165,20 +176,22 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
 #pragma unroll
       for (int nt = 0; nt < 8; ++nt) {
         const int tok = 8 * nt + 2 * qc;
-        s[nt][0] = tok < nvalid ? s[nt][0] * scale_log2 : -INFINITY;
-        s[nt][1] = tok + 1 < nvalid ? s[nt][1] * scale_log2 : -INFINITY;
+        s[nt][0] = (tok < nvalid && !((hole_bits >> tok) & 1ull)) ? s[nt][0] * scale_log2 : -INFINITY;
+        s[nt][1] = (tok + 1 < nvalid && !((hole_bits >> (tok + 1)) & 1ull)) ? s[nt][1] * scale_log2 : -INFINITY;
         mx = fmaxf(mx, fmaxf(s[nt][0], s[nt][1]));
       }
       mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
       mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
-      const float m_new = fmaxf(m_run, mx);  // finite: token 0 of a page is always valid
-      const float f = ex2(m_run - m_new);
+      const float m_new = fmaxf(m_run, mx);
+      // (a page of nothing but freed slots leaves the maximum at -inf: keep the exponent arguments finite)
+      const float f = m_new == -INFINITY ? 1.f : ex2(m_run - m_new);
       m_run = m_new;
       float ps = 0.f;
       uint32_t pa[8];  // P as bf16 pairs: pa[nt] = tokens 8 nt + 2 qc + {0, 1} of row g
 #pragma unroll
       for (int nt = 0; nt < 8; ++nt) {
-        const float p0 = ex2(s[nt][0] - m_new), p1 = ex2(s[nt][1] - m_new);
+        const float p0 = m_new == -INFINITY ? 0.f : ex2(s[nt][0] - m_new);
+        const float p1 = m_new == -INFINITY ? 0.f : ex2(s[nt][1] - m_new);
         ps += p0 + p1;
         pa[nt] = pack_bf16(p0, p1);
       }
@@ -288,7 +301,8 @@ int decode_num_splits(int S, int Hkv, int max_blocks) {
 
 int32_t launch_decode(int S, int Hq, int Hkv, int D, float scale, const void* q, const void* kc,
                       const void* vc, int num_blocks, const int32_t* table, int max_blocks,
-                      const int32_t* seq_lens, void* o, float* lse, void* ws, cudaStream_t st) {
+                      const int32_t* seq_lens, void* o, float* lse, void* ws, cudaStream_t st, const int32_t* holes,
+                      int holes_stride, int holes_off) {
   (void)D;
   const int G = Hq / Hkv;
   if (G < 1 || G > 8) return fail(UNIGIST_ERR_UNSUPPORTED, "decode supports 1 to 8 query heads per KV head, got %d", G);
@@ -306,7 +320,7 @@ int32_t launch_decode(int S, int Hq, int Hkv, int D, float scale, const void* q,
     KernelScope ks("decode_split_kernel", st);
     decode_split_kernel<<<dim3(splits, Hkv, S), THREADS, DecSmem::kBytes, st>>>(
         mk, mv, Hq, Hkv, G, scale * LOG2E, (const __nv_bfloat16*)q, num_blocks, table, max_blocks, seq_lens, splits, bps,
-        (float*)ws);
+        (float*)ws, holes, holes_stride, holes_off);
   }
   if (int32_t rc = check_launch("decode split kernel")) return rc;
   {

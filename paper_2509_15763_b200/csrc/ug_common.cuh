@@ -142,10 +142,17 @@ int32_t launch_compact_inplace(const Geom& g, const unigist_problem& p, void* kc
                                int32_t* kept_idx, void* ws, cudaStream_t st);
 int32_t launch_decode(int S, int Hq, int Hkv, int D, float scale, const void* q, const void* kc,
                       const void* vc, int num_blocks, const int32_t* table, int max_blocks,
-                      const int32_t* seq_lens, void* o, float* lse, void* ws, cudaStream_t st);
+                      const int32_t* seq_lens, void* o, float* lse, void* ws, cudaStream_t st,
+                      const int32_t* holes = nullptr, int holes_stride = 0, int holes_off = 0);
 int32_t launch_prefill_chunk(const unigist_problem& p, const Geom& g_full, float scale, int u0, int c, const void* q,
                              const void* k, const void* v, void* kc, void* vc, int num_blocks, int32_t* table,
                              int max_blocks, int32_t* seq_lens, void* o, float* lse, void* workspace, cudaStream_t st);
+size_t cache_state_bytes(int B, int r, int k);
+void cache_state_layout(int r, int k, int* stride_ints, int* free_list_off);
+int32_t launch_cache_state_init(const Geom& g, int B, int units_done, int32_t* state, cudaStream_t st);
+int32_t launch_cache_append(const Geom& g, const unigist_problem& p, int is_gist, const void* k_new, const void* v_new,
+                            void* kc, void* vc, int num_blocks, const int32_t* table, int max_blocks,
+                            int32_t* seq_lens, int32_t* state, cudaStream_t st);
 int decode_num_splits(int S, int Hkv, int max_blocks);
 int32_t decode_take_timeout(bool* timed_out);
 
