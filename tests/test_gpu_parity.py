@@ -144,11 +144,16 @@ def _sample_rows(N, rng, blocks=6, width=16):
     return np.array(rows, dtype=np.int64)
 
 
-@pytest.mark.parametrize("name,backward", [("llama8b_layer", True), ("train_batch", True),
-                                           ("long_prefill", False)])
-def test_full_size_sampled(name, backward):
+@pytest.mark.parametrize("name,backward,route", [("llama8b_layer", True, "explicit"), ("train_batch", True, "explicit"),
+                                                 ("long_prefill", False, "explicit"),
+                                                 # the route bench.py times: interleaved tensors, no shift launches
+                                                 ("llama8b_layer", True, "interleaved"),
+                                                 ("train_batch", True, "interleaved"),
+                                                 ("long_prefill", False, "interleaved"),
+                                                 ("table4_16k_r8", True, "interleaved")])
+def test_full_size_sampled(name, backward, route):
     w = synth.WORKLOADS[name]
-    out = run_attention(w, backward=backward)
+    out = run_attention(w, backward=backward) if route == "explicit" else run_attention_interleaved(w, backward=backward)
     inp = out["inputs"]
     s, T, r = w.num_sinks, w.raw_len, w.ratio
     k = oracle.window_units(w.window, r)
@@ -166,7 +171,7 @@ def test_full_size_sampled(name, backward):
         check_close(f"LSE rows {r0}", lse_gpu[:, r0:r0 + 16].T, lse, TOL_LSE)
     # no row anywhere was left unwritten
     assert torch.isfinite(out["lse_shifted"]).all()
-    assert torch.isfinite(out["o_shifted"].float()).all()
+    assert torch.isfinite(out["o_shifted" if route == "explicit" else "o"].float()).all()
     if not backward:
         return
     do = f64(inp["dout"][b, :, hs])
@@ -178,5 +183,5 @@ def test_full_size_sampled(name, backward):
     check_close("dQ rows", f64(out["dq"][b, rows][:, hs]), dq, TOL_GRAD)
     check_close("dK keys", f64(out["dk"][b, keys, hk]), dk, TOL_GRAD)
     check_close("dV keys", f64(out["dv"][b, keys, hk]), dv, TOL_GRAD)
-    for n in ("dq_shifted", "dk_shifted", "dv_shifted"):
-        assert torch.isfinite(out[n].float()).all(), n
+    for n in ("dq", "dk", "dv"):
+        assert torch.isfinite(out[n + "_shifted" if route == "explicit" else n].float()).all(), n
