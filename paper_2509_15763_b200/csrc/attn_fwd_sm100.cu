@@ -11,12 +11,16 @@
 //   TMA:      K, V tiles -> shared memory (128-byte swizzle), one tensor map per segment so a tile
 //             never straddles segments and rows past a segment's end read as zero.
 //   tcgen05:  S = Q K^T into TMEM (fp32);   O += P V with P (bf16) read from TMEM.
-//   softmax:  one warpgroup per stream, one query row per thread: row max, lazy rescale of O,
-//             exp2, row sum, P -> TMEM.  Only tiles classified "partial" evaluate the mask.
+//   softmax:  one warpgroup per stream, one query row per thread.  One pass over the 128 scores of
+//             the row takes 2^(s - m) against the RUNNING maximum m, the row sum and the tile's own
+//             maximum together; only when some row's maximum outgrew m by more than the lazy-rescale
+//             threshold (always checked, seldom true after the first tile) is O rescaled and the
+//             pass repeated.  Only tiles classified "partial" evaluate the mask (hidden scores are
+//             set to -inf before the pass).
 // The MMA issue order PV0(j), S0(j+1), PV1(j), S1(j+1) lets one stream's softmax run under the
 // other stream's matrix products.
-// Roles: one softmax warpgroup per stream (kSplit = 1: a thread owns a whole query row and keeps its
-// 128 scores of a tile in registers; kSplit = 2: two threads share a row), then one more warpgroup
+// Roles: one softmax warpgroup per stream (a thread owns a whole query row and keeps its 128 scores
+// of a tile in registers), then one more warpgroup
 // with the TMA producer warp and the MMA issuer / TMEM owner warp, which hands most of its registers
 // to the softmax warpgroups.  TMEM: S0 | S1 | O0 | O1, 128 columns each.
 #include "sm100_ptx.cuh"
@@ -30,16 +34,18 @@ using namespace sm100;
 constexpr int BM = 128;  // query rows per tile
 constexpr int BN = 128;  // keys per tile
 constexpr int kStages = 4;  // ring slots; K and V tiles alternate through them
-constexpr int kSplit = 1;              // threads per query row: each takes BN / kSplit score columns
-constexpr int kCols = BN / kSplit;     // score columns per thread and tile
-constexpr int kSmWarps = 8 * kSplit;   // softmax warps: 2 streams x kSplit column parts x 4 lane quarters
+constexpr int kCols = BN;     // score columns per thread and tile
+constexpr int kSmWarps = 8;   // softmax warps: 2 streams x 4 lane quarters
+#ifndef UG_EMU_NUM
+#define UG_EMU_NUM 2
+#endif
 constexpr int kTmaWarp = kSmWarps, kMmaWarp = kSmWarps + 1;
 constexpr int kThreads = (kSmWarps + 4) * 32;  // the last warpgroup: TMA warp, MMA warp, 2 idle warps
 constexpr uint32_t kTmemCols = 512;
 // Register split after launch: the softmax warpgroups grow, the last warpgroup shrinks.  The total must not exceed what the block was launched with, or the growing
 // warpgroups would wait forever.
-constexpr int kRegsLaunch = kSplit == 1 ? 168 : 96;  // 65536 / kThreads, rounded down to a multiple of 8
-constexpr int kRegsSoftmax = kSplit == 1 ? 216 : 104, kRegsOther = kSplit == 1 ? 72 : 64;
+constexpr int kRegsLaunch = 168;  // 65536 / kThreads, rounded down to a multiple of 8
+constexpr int kRegsSoftmax = 216, kRegsOther = 72;
 static_assert(kThreads * (kRegsLaunch + 8) > 65536 && kThreads * kRegsLaunch <= 65536, "kRegsLaunch is stale");
 static_assert((kSmWarps / 4) * kRegsSoftmax + kRegsOther <= (kSmWarps / 4 + 1) * kRegsLaunch,
               "register split exceeds the block's allocation");
@@ -52,8 +58,7 @@ struct FwdSmem {
   static constexpr int kSlab = BM * 128;          // bytes of one [128 rows x 64 bf16] slab
   static constexpr int kTile = kSlab * (D / 64);  // bytes of one [128 x D] tile
   static constexpr int kBarOff = (2 + kStages) * kTile;
-  static constexpr int kXchOff = kBarOff + 256;  // [2 streams][kSplit][128 rows] fp32 exchange slots
-  static constexpr int kBytes = kXchOff + 2 * kSplit * BM * 4 + 1024 /*align*/;
+  static constexpr int kBytes = kBarOff + 256 + 1024 /*align*/;
 };
 
 // One query stream: a 128-row tile of one head, with the key tiles it can see in each segment.
@@ -153,61 +158,71 @@ __device__ __forceinline__ uint32_t chunk_mask(int lo, int hi, int c) {
   return a > b ? 0u : ((0xffffffffu >> (31 - b)) & (0xffffffffu << a));
 }
 
-// Row maximum of the raw scores of one tile; kMasked: only columns [lo, hi] count.
-template <bool kMasked>
-__device__ __forceinline__ float row_max(const uint32_t (&sc)[kCols], int lo, int hi) {
-  float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
+// Hidden columns (outside [lo, hi]) of a row of raw scores become -inf.
+__device__ __forceinline__ void mask_row(uint32_t (&sc)[kCols], int lo, int hi) {
 #pragma unroll
   for (int c = 0; c < kCols / 32; ++c) {
-    if (kMasked) {
-      const uint32_t bits = chunk_mask(lo, hi, c);
+    const uint32_t bits = chunk_mask(lo, hi, c);
 #pragma unroll
-      for (int e = 0; e < 32; e += 2) {
-        const float x0 = (bits >> e) & 1u ? __uint_as_float(sc[c * 32 + e]) : -INFINITY;
-        const float x1 = (bits >> (e + 1)) & 1u ? __uint_as_float(sc[c * 32 + e + 1]) : -INFINITY;
-        if (e & 2) m1 = max3(m1, x0, x1); else m0 = max3(m0, x0, x1);
-      }
-    } else {
+    for (int e = 0; e < 32; ++e) sc[c * 32 + e] = (bits >> e) & 1u ? sc[c * 32 + e] : 0xff800000u;
+  }
+}
+
+// Row maximum of the raw scores of one tile.
+__device__ __forceinline__ float row_max(const uint32_t (&sc)[kCols]) {
+  float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
 #pragma unroll
-      for (int e = 0; e < 32; e += 8) {
-        m0 = max3(m0, __uint_as_float(sc[c * 32 + e]), __uint_as_float(sc[c * 32 + e + 1]));
-        m1 = max3(m1, __uint_as_float(sc[c * 32 + e + 2]), __uint_as_float(sc[c * 32 + e + 3]));
-        m2 = max3(m2, __uint_as_float(sc[c * 32 + e + 4]), __uint_as_float(sc[c * 32 + e + 5]));
-        m3 = max3(m3, __uint_as_float(sc[c * 32 + e + 6]), __uint_as_float(sc[c * 32 + e + 7]));
-      }
-    }
+  for (int e = 0; e < kCols; e += 8) {
+    m0 = max3(m0, __uint_as_float(sc[e]), __uint_as_float(sc[e + 1]));
+    m1 = max3(m1, __uint_as_float(sc[e + 2]), __uint_as_float(sc[e + 3]));
+    m2 = max3(m2, __uint_as_float(sc[e + 4]), __uint_as_float(sc[e + 5]));
+    m3 = max3(m3, __uint_as_float(sc[e + 6]), __uint_as_float(sc[e + 7]));
   }
   return fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
 }
 
-// p = 2^(s * scale_log2 - m) for one row of a tile, written to TMEM as bf16 pairs; returns the row sum.
-template <bool kMasked>
-__device__ __forceinline__ float row_exp(const uint32_t (&sc)[kCols], uint32_t t_p, float scale_log2, float m, int lo,
-                                         int hi) {
-  float l0 = 0.f, l1 = 0.f, l2 = 0.f, l3 = 0.f;
+// One pass over a row of raw scores: p = 2^(s * scale_log2 - m) written to TMEM as bf16 pairs; returns the
+// row sum and leaves the maximum raw score in mx.  m must be finite; a score of -inf gives p = 0 (or about
+// 2^-126 where the exponential is taken on the FMA pipe).  The special-function unit (16 exponentials per
+// clock and SM) bounds this loop, so kEmuNum of every kEmuDen column pairs go to the FMA pipe (ex2_fma2)
+// and the maximum rides along on the ALU pipe.
+constexpr int kEmuNum = UG_EMU_NUM, kEmuDen = 8;
+__device__ __forceinline__ float row_exp(const uint32_t (&sc)[kCols], uint32_t t_p, float scale_log2, float m, float& mx) {
+  uint64_t l01 = f32x2(0.f, 0.f), l23 = l01;
+  const uint64_t scale2 = f32x2(scale_log2, scale_log2), negm2 = f32x2(-m, -m);
+  float m0 = -INFINITY, m1 = -INFINITY;
 #pragma unroll
   for (int c = 0; c < kCols / 32; ++c) {
-    uint32_t bits = 0xffffffffu;
-    if (kMasked) bits = chunk_mask(lo, hi, c);
     uint32_t pk[16];
 #pragma unroll
     for (int e = 0; e < 32; e += 4) {
+      const int i0 = c * 32 + e;
       float x[4];
 #pragma unroll
-      for (int t = 0; t < 4; ++t) {
-        x[t] = fmaf(__uint_as_float(sc[c * 32 + e + t]), scale_log2, -m);
-        if (kMasked) x[t] = (bits >> (e + t)) & 1u ? x[t] : -INFINITY;
-        x[t] = ex2(x[t]);
+      for (int q = 0; q < 2; ++q) {
+        const int pair = i0 / 2 + q;
+        f32x2_split(fma2(f32x2(__uint_as_float(sc[i0 + 2 * q]), __uint_as_float(sc[i0 + 2 * q + 1])), scale2, negm2),
+                    x[2 * q], x[2 * q + 1]);
+        if ((pair * kEmuNum) % kEmuDen < kEmuNum) {
+          ex2_fma2(x[2 * q], x[2 * q + 1]);
+        } else {
+          x[2 * q] = ex2(x[2 * q]);
+          x[2 * q + 1] = ex2(x[2 * q + 1]);
+        }
       }
-      l0 += x[0];
-      l1 += x[1];
-      l2 += x[2];
-      l3 += x[3];
+      m0 = max3(m0, __uint_as_float(sc[i0]), __uint_as_float(sc[i0 + 1]));
+      m1 = max3(m1, __uint_as_float(sc[i0 + 2]), __uint_as_float(sc[i0 + 3]));
+      l01 = add2(l01, f32x2(x[0], x[1]));
+      l23 = add2(l23, f32x2(x[2], x[3]));
       pk[e / 2] = pack_bf16(x[0], x[1]);
       pk[e / 2 + 1] = pack_bf16(x[2], x[3]);
     }
     tmem_st(t_p + c * 16, pk);
   }
+  mx = fmaxf(m0, m1);
+  float l0, l1, l2, l3;
+  f32x2_split(l01, l0, l1);
+  f32x2_split(l23, l2, l3);
   return (l0 + l1) + (l2 + l3);
 }
 
@@ -268,7 +283,7 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_sink, const __gri
     mbar_init(bar_o, 1);
     for (int i = 0; i < 2; ++i) {
       mbar_init(bar_s[i], 1);
-      mbar_init(bar_p[i], 128 * kSplit);
+      mbar_init(bar_p[i], 128);
     }
     for (int i = 0; i < kStages; ++i) {
       mbar_init(bar_full + 8 * i, 1);
@@ -392,16 +407,14 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_sink, const __gri
   } else {
     reg_alloc<kRegsSoftmax>();
     // ------------------------------------------------------------ softmax + epilogue (one row per thread)
-    const int i = warp / (4 * kSplit);  // stream
-    const int part = (warp >> 2) % kSplit;  // which BN / kSplit columns of the row
-    float* xch = reinterpret_cast<float*>(gen_base + SM::kXchOff) + i * kSplit * BM;
+    const int i = warp / 4;  // stream
     const Stream me = i ? str1 : str0;
     if (me.valid) {
       const int r_in_tile = (warp & 3) * 32 + (threadIdx.x & 31);
       const int row = min(me.row_a + r_in_tile, me.row_b);
       const RowIv my = row_intervals(g, q_seg_base + row);
       const uint32_t lane_base = static_cast<uint32_t>((warp & 3) * 32) << 16;
-      const uint32_t tS = tmem + i * 128 + lane_base, tO = tmem + 256 + i * 128 + lane_base + part * (D / kSplit);
+      const uint32_t tS = tmem + i * 128 + lane_base, tO = tmem + 256 + i * 128 + lane_base;
       float m_run = -INFINITY, l_run = 0.f;
       int cnt = 0;
 
@@ -414,16 +427,16 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_sink, const __gri
         int lo, hi;  // visible columns of this row, relative to the tile
         if (sg == kSegSink) {
           full = col0 + BN - 1 <= me.iv_a.hi_sink;
-          lo = -part * kCols;
-          hi = my.hi_sink - col0 - part * kCols;
+          lo = 0;
+          hi = my.hi_sink - col0;
         } else if (sg == kSegRaw) {
           full = col0 >= me.iv_b.lo_raw && col0 + BN - 1 <= me.iv_a.hi_raw;
-          lo = my.lo_raw - col0 - part * kCols;
-          hi = my.hi_raw - col0 - part * kCols;
+          lo = my.lo_raw - col0;
+          hi = my.hi_raw - col0;
         } else {
           full = col0 + BN - 1 <= me.iv_a.hi_gist;
-          lo = -part * kCols;
-          hi = my.hi_gist - col0 - part * kCols;
+          lo = 0;
+          hi = my.hi_gist - col0;
         }
         ok = mbar_wait_warp(bar_s[i], cnt & 1);
         if (!ok) break;
@@ -432,25 +445,29 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_sink, const __gri
         // the whole score row of this tile sits in registers between the two passes
         uint32_t sc[kCols];
 #pragma unroll
-        for (int c = 0; c < kCols / 32; ++c) tmem_ld32(tS + part * kCols + c * 32, sc + c * 32);
+        for (int c = 0; c < kCols / 32; ++c) tmem_ld32(tS + c * 32, sc + c * 32);
         tmem_wait_ld();
-        float mx = full ? row_max<false>(sc, lo, hi) : row_max<true>(sc, lo, hi);
-        if (kSplit > 1) {  // the threads that share a row agree on its maximum
-          xch[part * BM + r_in_tile] = mx;
-          named_barrier_sync(1 + i, 128 * kSplit);
-#pragma unroll
-          for (int q = 0; q < kSplit; ++q) mx = fmaxf(mx, xch[q * BM + r_in_tile]);
-        }
-        const float mx_s = mx * scale_log2;
-        const bool need = mx_s > m_run + kRescaleThreshold;  // also true for the first visible tile
-        if (__any_sync(0xffffffffu, need)) {
+        if (!full) mask_row(sc, lo, hi);
+        // the first tile has no running maximum to go by: take its own first
+        if (cnt == 0) m_run = row_max(sc) * scale_log2;
+        float tile_sum;
+        for (int pass = 0; pass < 2; ++pass) {
+          // p = 2^(s * scale_log2 - m) against the running maximum, row sum, bf16 P into TMEM (over the first
+          // 64 columns of S), and the tile's own maximum
+          float mx;
+          tile_sum = row_exp(sc, tS, scale_log2, m_run == -INFINITY ? 0.f : m_run, mx);
+          const float mx_s = mx * scale_log2;
+          const bool need = mx_s > m_run + kRescaleThreshold;
+          if (!__any_sync(0xffffffffu, need)) break;
+          // some row of this warp outgrew its running maximum: rescale and take the pass again
           const float m_new = need ? mx_s : m_run;
           const float f = need ? ex2(m_run - m_new) : 1.f;  // m_run = -inf gives 0
           l_run *= f;
           m_run = m_new;
+          tmem_wait_st();
           if (cnt > 0) {  // S of this step complete implies the previous PV complete: O is stable here
 #pragma unroll
-            for (int c = 0; c < D / kSplit / 32; ++c) {
+            for (int c = 0; c < D / 32; ++c) {
               uint32_t v[32];
               tmem_ld(tO + c * 32, v);
               tmem_wait_ld();
@@ -460,9 +477,6 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_sink, const __gri
             }
           }
         }
-        // p = 2^(s * scale_log2 - m), row sum, bf16 P into TMEM (over the first 64 columns of S)
-        const float tile_sum = full ? row_exp<false>(sc, tS + part * (kCols / 2), scale_log2, m_run, lo, hi)
-                                    : row_exp<true>(sc, tS + part * (kCols / 2), scale_log2, m_run, lo, hi);
         l_run += tile_sum;
         tmem_wait_st();
         tc_fence_before();
@@ -472,21 +486,14 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_sink, const __gri
       if (ok) ok = mbar_wait_warp(bar_o, 0);
       if (ok) {
         tc_fence_after();
-        if (kSplit > 1) {  // row sum = sum of the parts (no thread reads a max slot any more: all P are consumed)
-          xch[part * BM + r_in_tile] = l_run;
-          named_barrier_sync(1 + i, 128 * kSplit);
-          l_run = 0.f;
-#pragma unroll
-          for (int q = 0; q < kSplit; ++q) l_run += xch[q * BM + r_in_tile];
-        }
         const float inv_l = 1.f / l_run;
         const bool valid = me.row_a + r_in_tile <= me.row_b;
         const int out_row = interleaved ? seg_row_to_token(g, true, qseg, me.row_a + r_in_tile)
                                         : qr.out_base[qseg] + (me.row_a + r_in_tile - q_off);
         const long long tok = (long long)b * qr.n_out + out_row;
-        __nv_bfloat16* orow = o + (tok * Hq + me.h) * D + part * (D / kSplit);
+        __nv_bfloat16* orow = o + (tok * Hq + me.h) * D;
 #pragma unroll
-        for (int c = 0; c < D / kSplit / 32; ++c) {
+        for (int c = 0; c < D / 32; ++c) {
           uint32_t v[32];
           tmem_ld(tO + c * 32, v);
           tmem_wait_ld();
@@ -502,7 +509,7 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_sink, const __gri
             }
           }
         }
-        if (valid && part == 0)
+        if (valid)
           lse[((long long)b * Hq + me.h) * qr.n_out + qr.out_base[qseg] + (me.row_a + r_in_tile - q_off)] =
               (m_run + log2f(l_run)) * 0.6931471805599453f;
       } else {

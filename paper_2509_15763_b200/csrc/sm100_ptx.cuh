@@ -214,6 +214,48 @@ __device__ __forceinline__ float ex2(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
+// Two fp32 lanes in one 64-bit register for the packed fp32 arithmetic of sm_100 (add / fma .f32x2).
+__device__ __forceinline__ uint64_t f32x2(float lo, float hi) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void f32x2_split(uint64_t v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+  uint64_t r;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
+__device__ __forceinline__ uint64_t sub2(uint64_t a, uint64_t b) {
+  uint64_t r;
+  asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t r;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+  return r;
+}
+// 2^x for two values on the FMA pipe instead of the special-function unit: x = n + f with n = round(x)
+// (taken from the low mantissa bits of x + 1.5 * 2^23), a cubic for 2^f on [-0.5, 0.5] (minimax in relative
+// error, 7.5e-5: well inside the bf16 rounding of the probabilities), n added to the exponent field.
+// Inputs below -126 give a value near 2^-126 instead of 0; inputs must stay below 128.
+__device__ __forceinline__ void ex2_fma2(float& x0, float& x1) {
+  const uint64_t magic = f32x2(12582912.f, 12582912.f);
+  const uint64_t x = f32x2(fmaxf(x0, -126.f), fmaxf(x1, -126.f));
+  const uint64_t t = add2(x, magic);
+  const uint64_t f = sub2(x, sub2(t, magic));
+  uint64_t p = fma2(f, f32x2(0.0551716685f, 0.0551716685f), f32x2(0.242611125f, 0.242611125f));
+  p = fma2(p, f, f32x2(0.693260968f, 0.693260968f));
+  p = fma2(p, f, f32x2(0.999928057f, 0.999928057f));
+  float t0, t1, p0, p1;
+  f32x2_split(t, t0, t1);
+  f32x2_split(p, p0, p1);
+  x0 = __uint_as_float(__float_as_uint(p0) + (__float_as_uint(t0) << 23));
+  x1 = __uint_as_float(__float_as_uint(p1) + (__float_as_uint(t1) << 23));
+}
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   uint32_t r;
   asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
