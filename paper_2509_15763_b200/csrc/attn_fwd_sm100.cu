@@ -181,18 +181,20 @@ __device__ __forceinline__ float row_max(const uint32_t (&sc)[kCols]) {
   return fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
 }
 
-// One pass over a row of raw scores: p = 2^(s * scale_log2 - m) written to TMEM as bf16 pairs; returns the
-// row sum and leaves the maximum raw score in mx.  m must be finite; a score of -inf gives p = 0 (or about
-// 2^-126 where the exponential is taken on the FMA pipe).  The special-function unit (16 exponentials per
-// clock and SM) bounds this loop, so kEmuNum of every kEmuDen column pairs go to the FMA pipe (ex2_fma2)
-// and the maximum rides along on the ALU pipe.
+// Half a pass over a row of raw scores (columns 64 * kHalf .. + 63): p = 2^(s * scale_log2 - m) written to
+// TMEM as bf16 pairs; returns the sum of the half row.  The first half also leaves the maximum raw score of
+// the WHOLE row in mx, so that the caller knows whether m still serves before it hands any of P over.
+// m must be finite; a score of -inf gives p = 0 (or about 2^-126 where the exponential is taken on the FMA
+// pipe).  The special-function unit (16 exponentials per clock and SM) bounds this loop, so kEmuNum of every
+// kEmuDen column pairs go to the FMA pipe (ex2_fma2) and the maximum rides along on the ALU pipe.
 constexpr int kEmuNum = UG_EMU_NUM, kEmuDen = 8;
+template <int kHalf>
 __device__ __forceinline__ float row_exp(const uint32_t (&sc)[kCols], uint32_t t_p, float scale_log2, float m, float& mx) {
   uint64_t l01 = f32x2(0.f, 0.f), l23 = l01;
   const uint64_t scale2 = f32x2(scale_log2, scale_log2), negm2 = f32x2(-m, -m);
   float m0 = -INFINITY, m1 = -INFINITY;
 #pragma unroll
-  for (int c = 0; c < kCols / 32; ++c) {
+  for (int c = kHalf * (kCols / 64); c < (kHalf + 1) * (kCols / 64); ++c) {
     uint32_t pk[16];
 #pragma unroll
     for (int e = 0; e < 32; e += 4) {
@@ -210,8 +212,13 @@ __device__ __forceinline__ float row_exp(const uint32_t (&sc)[kCols], uint32_t t
           x[2 * q + 1] = ex2(x[2 * q + 1]);
         }
       }
-      m0 = max3(m0, __uint_as_float(sc[i0]), __uint_as_float(sc[i0 + 1]));
-      m1 = max3(m1, __uint_as_float(sc[i0 + 2]), __uint_as_float(sc[i0 + 3]));
+      if (kHalf == 0) {  // the maximum of both halves: 8 columns per 4 exponentials
+        const int j0 = 2 * i0;
+        m0 = max3(m0, __uint_as_float(sc[j0]), __uint_as_float(sc[j0 + 1]));
+        m1 = max3(m1, __uint_as_float(sc[j0 + 2]), __uint_as_float(sc[j0 + 3]));
+        m0 = max3(m0, __uint_as_float(sc[j0 + 4]), __uint_as_float(sc[j0 + 5]));
+        m1 = max3(m1, __uint_as_float(sc[j0 + 6]), __uint_as_float(sc[j0 + 7]));
+      }
       l01 = add2(l01, f32x2(x[0], x[1]));
       l23 = add2(l23, f32x2(x[2], x[3]));
       pk[e / 2] = pack_bf16(x[0], x[1]);
@@ -219,7 +226,7 @@ __device__ __forceinline__ float row_exp(const uint32_t (&sc)[kCols], uint32_t t
     }
     tmem_st(t_p + c * 16, pk);
   }
-  mx = fmaxf(m0, m1);
+  if (kHalf == 0) mx = fmaxf(m0, m1);
   float l0, l1, l2, l3;
   f32x2_split(l01, l0, l1);
   f32x2_split(l23, l2, l3);
@@ -242,7 +249,8 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_sink, const __gri
   const uint32_t ring = base + 2 * SM::kTile;
   const uint32_t bars = base + SM::kBarOff;
   const uint32_t bar_q = bars, bar_o = bars + 8;
-  const uint32_t bar_s[2] = {bars + 16, bars + 24}, bar_p[2] = {bars + 32, bars + 40};
+  const uint32_t bar_s[2] = {bars + 16, bars + 24}, bar_p[2] = {bars + 32, bars + 40};  // bar_p: first half of P stored
+  const uint32_t bar_p2[2] = {bars + 64 + 16 * kStages, bars + 72 + 16 * kStages};          // second half of P stored
   const uint32_t bar_full = bars + 48, bar_empty = bars + 48 + 8 * kStages;  // arrays of kStages
   const uint32_t tmem_slot = bars + 48 + 16 * kStages;
   unsigned char* gen_base = smem_dyn + (base - smem_u32(smem_dyn));
@@ -284,6 +292,7 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_sink, const __gri
     for (int i = 0; i < 2; ++i) {
       mbar_init(bar_s[i], 1);
       mbar_init(bar_p[i], 128);
+      mbar_init(bar_p2[i], 128);
     }
     for (int i = 0; i < kStages; ++i) {
       mbar_init(bar_full + 8 * i, 1);
@@ -348,15 +357,16 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_sink, const __gri
         umma_commit(bar_s[i]);
         ++n_s[i];
       };
-      auto issue_pv = [&](int i, uint32_t sV) {
+      auto issue_pv = [&](int i, uint32_t sV, int half) {  // the k steps of one half of the keys of the tile
         // V tile is MN-major: 16 keys = 2048 B per k step, 64-column groups SM::kSlab apart
         const uint32_t v_lo = smem_desc_lo(sV, SM::kSlab);
 #pragma unroll
-        for (int kk = 0; kk < BN / 16; ++kk) {
+        for (int k4 = 0; k4 < BN / 32; ++k4) {
+          const int kk = half * (BN / 32) + k4;
           umma_ts(tmem + 256 + i * 128, tmem + i * 128 + kk * 8, smem_desc_join(v_lo + kk * (2048 >> 4), kHi),
                   idesc_pv, (n_pv[i] > 0 || kk > 0) ? 1u : 0u);
         }
-        ++n_pv[i];
+        n_pv[i] += half;
       };
       auto slot_of = [&](int t) { return t % kStages; };
       auto wait_full = [&](int t) { return mbar_wait(bar_full + 8 * slot_of(t), (t / kStages) & 1); };
@@ -383,10 +393,15 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_sink, const __gri
         for (int i = 0; i < 2; ++i) {
           const Stream& si = i ? str1 : str0;
           if (si.sees(sg, idx)) {
+            // the first half of P is handed over while the softmax still works on the second
             ok = mbar_wait(bar_p[i], n_pv[i] & 1);
             if (!ok) break;
             tc_fence_after();
-            issue_pv(i, ring + slot_of(tv) * SM::kTile);
+            issue_pv(i, ring + slot_of(tv) * SM::kTile, 0);
+            ok = mbar_wait(bar_p2[i], n_pv[i] & 1);
+            if (!ok) break;
+            tc_fence_after();
+            issue_pv(i, ring + slot_of(tv) * SM::kTile, 1);
           }
           if (i == 1) umma_commit(bar_empty + 8 * slot_of(tv));
           if (has_next) {
@@ -452,14 +467,14 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_sink, const __gri
         if (cnt == 0) m_run = row_max(sc) * scale_log2;
         float tile_sum;
         for (int pass = 0; pass < 2; ++pass) {
-          // p = 2^(s * scale_log2 - m) against the running maximum, row sum, bf16 P into TMEM (over the first
-          // 64 columns of S), and the tile's own maximum
+          // first half of the row: p = 2^(s * scale_log2 - m) against the running maximum, bf16 P into TMEM
+          // (over the first 64 columns of S), and the whole row's own maximum
           float mx;
-          tile_sum = row_exp(sc, tS, scale_log2, m_run == -INFINITY ? 0.f : m_run, mx);
+          tile_sum = row_exp<0>(sc, tS, scale_log2, m_run == -INFINITY ? 0.f : m_run, mx);
           const float mx_s = mx * scale_log2;
           const bool need = mx_s > m_run + kRescaleThreshold;
           if (!__any_sync(0xffffffffu, need)) break;
-          // some row of this warp outgrew its running maximum: rescale and take the pass again
+          // some row of this warp outgrew its running maximum: rescale and take the half again
           const float m_new = need ? mx_s : m_run;
           const float f = need ? ex2(m_run - m_new) : 1.f;  // m_run = -inf gives 0
           l_run *= f;
@@ -477,10 +492,16 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_sink, const __gri
             }
           }
         }
-        l_run += tile_sum;
+        // hand the first half of P over, so that its part of P V runs under the second half's exponentials
         tmem_wait_st();
         tc_fence_before();
         mbar_arrive(bar_p[i]);
+        float unused;
+        tile_sum += row_exp<1>(sc, tS, scale_log2, m_run == -INFINITY ? 0.f : m_run, unused);
+        l_run += tile_sum;
+        tmem_wait_st();
+        tc_fence_before();
+        mbar_arrive(bar_p2[i]);
         ++cnt;
       }
       if (ok) ok = mbar_wait_warp(bar_o, 0);
