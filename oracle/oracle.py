@@ -226,3 +226,26 @@ def decode(scale, q, k_list, v_list):
             o[i, h * G:(h + 1) * G] = a
             lse[i, h * G:(h + 1) * G] = b
     return o, lse
+
+
+def rope(x, pos_ids, theta_base):
+    """Rotary position embedding with the aligned position ids (Section 4.1, step 3).
+
+    x [N, H, D] in interleaved order, pos_ids [N] (from layout()).  The paper fixes the ids, not
+    the rotary convention; this is the one of the Llama models it trains: feature j < D/2 pairs
+    with feature j + D/2, and the pair of token t is rotated by the angle
+    pos_ids[t] * theta_base^(-2 j / D):
+        y[j]       = x[j] cos - x[j + D/2] sin
+        y[j + D/2] = x[j + D/2] cos + x[j] sin
+    """
+    x = np.asarray(x, np.float64)
+    N, H, D = x.shape
+    half = D // 2
+    y = np.empty_like(x)
+    for t in range(N):
+        for j in range(half):
+            ang = float(pos_ids[t]) * float(theta_base) ** (-2.0 * j / D)
+            c, s_ = np.cos(ang), np.sin(ang)
+            y[t, :, j] = x[t, :, j] * c - x[t, :, j + half] * s_
+            y[t, :, j + half] = x[t, :, j + half] * c + x[t, :, j] * s_
+    return y
