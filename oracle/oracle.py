@@ -249,3 +249,61 @@ def rope(x, pos_ids, theta_base):
             y[t, :, j] = x[t, :, j] * c - x[t, :, j + half] * s_
             y[t, :, j + half] = x[t, :, j + half] * c + x[t, :, j] * s_
     return y
+
+
+def docs_mask(s, doc_T, r, k) -> np.ndarray:
+    """Mask of a packed sample under cross-document masking (Section 5.1; documents padded to a
+    multiple of r, appendix on training data): token i of document a sees token j of document b
+    iff a == b and Eq. 3 holds inside that document (each document restarts its sinks, units and
+    window).  Interleaved order, documents one after another.  [N_total, N_total] bool."""
+    doc_of, local = [], []
+    for d, T in enumerate(doc_T):
+        n = total_len(s, T, r)
+        doc_of += [d] * n
+        local += list(range(n))
+    n_tot = len(doc_of)
+    m = np.zeros((n_tot, n_tot), bool)
+    for i in range(n_tot):
+        for j in range(n_tot):
+            m[i, j] = doc_of[i] == doc_of[j] and visible(local[i], local[j], s, r, k)
+    return m
+
+
+def docs_attn_fwd(s, doc_T, r, k, scale, q, kk, v):
+    """Dense softmax attention under docs_mask: q [N,Hq,D], kk/v [N,Hkv,D] (interleaved, packed)
+    -> o [N,Hq,D], lse [Hq,N].  The plain definition, O(N^2): small cases only."""
+    q, kk, v = _c64(q), _c64(kk), _c64(v)
+    N, Hq, D = q.shape
+    G = Hq // kk.shape[1]
+    m = docs_mask(s, doc_T, r, k)
+    o = np.empty((N, Hq, D))
+    lse = np.empty((Hq, N))
+    for h in range(Hq):
+        sc = scale * (q[:, h] @ kk[:, h // G].T)
+        sc = np.where(m, sc, -np.inf)
+        mx = sc.max(axis=1, keepdims=True)
+        e = np.exp(sc - mx)
+        l = e.sum(axis=1, keepdims=True)
+        o[:, h] = (e / l) @ v[:, h // G]
+        lse[h] = (mx + np.log(l))[:, 0]
+    return o, lse
+
+
+def docs_attn_bwd(s, doc_T, r, k, scale, q, kk, v, dout):
+    """Gradients of docs_attn_fwd's o with respect to q, kk, v for the cotangent dout (dense)."""
+    q, kk, v, dout = _c64(q), _c64(kk), _c64(v), _c64(dout)
+    N, Hq, D = q.shape
+    G = Hq // kk.shape[1]
+    m = docs_mask(s, doc_T, r, k)
+    dq, dk, dv = np.zeros_like(q), np.zeros_like(kk), np.zeros_like(v)
+    for h in range(Hq):
+        g = h // G
+        sc = np.where(m, scale * (q[:, h] @ kk[:, g].T), -np.inf)
+        p = np.exp(sc - sc.max(axis=1, keepdims=True))
+        p /= p.sum(axis=1, keepdims=True)
+        dv[:, g] += p.T @ dout[:, h]
+        dp = dout[:, h] @ v[:, g].T
+        ds = p * (dp - (p * dp).sum(axis=1, keepdims=True))
+        dq[:, h] = scale * (ds @ kk[:, g])
+        dk[:, g] += scale * (ds.T @ q[:, h])
+    return dq, dk, dv
