@@ -16,7 +16,7 @@
  *  - "Interleaved" order is Eq. 2's Z.  "Shifted" order is [sinks | raw | gists], each kind
  *    in its original order.  Attention calls take SHIFTED tensors.
  *  - Dense tensors are [batch, N, heads, head_dim], head_dim contiguous, bf16 unless stated,
- *    base pointers 16-byte aligned.  Query head h uses KV head h / (Hq / Hkv).
+ *    base pointers 16-byte aligned (the fp32 lse arrays: 4-byte).  Query head h uses KV head h / (Hq / Hkv).
  *  - Every pointer named "device" is memory of the current CUDA device; the CALLER owns every
  *    buffer, the library never allocates or frees device memory.  Scratch comes in through
  *    `workspace` (size from unigist_workspace_bytes / unigist_decode_workspace_bytes).
@@ -118,6 +118,23 @@ int32_t unigist_gist_unshift(const unigist_problem* p, const void* src, void* ds
                              int32_t elem_bytes, void* stream);
 
 /*
+ * Position-encoding alignment (Section 4.1, step 3) applied as a rotary embedding to a bf16
+ * [B, N, heads, D] device tensor in INTERLEAVED order: token t is rotated by its aligned position id
+ * (sinks and raw tokens count 0, 1, 2, ...; a gist takes the id of the raw token right after it, the
+ * last gist the id one past the last raw token), so distances between raw tokens are those of the
+ * sequence without gists.  The paper fixes the ids, not the rotary convention; this is the one of the
+ * Llama models it trains: feature j < D / 2 pairs with feature j + D / 2 and the pair turns by
+ * id * theta_base^(-2 j / D).  Angles are formed in fp64, the rotation in fp32, one rounding to bf16.
+ * flags = 0: dst has the order of src (dst == src, in place, is allowed).
+ * flags = UNIGIST_ROPE_TO_SHIFTED: dst is written in SHIFTED order (Section 4.2), i.e. the rotation is
+ * fused with unigist_gist_shift; src and dst must not overlap.
+ * Errors: INVALID_ARG (NULL, heads < 1, theta_base <= 1, unknown flag, overlap), ALIGNMENT, CUDA.
+ */
+#define UNIGIST_ROPE_TO_SHIFTED 1u
+int32_t unigist_rope(const unigist_problem* p, const void* src, void* dst, int32_t heads, float theta_base,
+                     uint32_t flags, void* stream);
+
+/*
  * Forward (Section 4.2 kernel; Eq. 3 mask): for each (b, head, row t)
  *   S_tj = scale * q_t . k_j over visible j,  LSE_t = log sum_j exp(S_tj),  O_t = softmax(S_t) V.
  * q [B,N,Hq,D], k, v [B,N,Hkv,D], o [B,N,Hq,D]: device bf16, SHIFTED order.
@@ -141,6 +158,28 @@ int32_t unigist_attn_fwd(const unigist_problem* p, const void* q, const void* k,
 int32_t unigist_attn_bwd(const unigist_problem* p, const void* q, const void* k, const void* v,
                          const void* o, const float* lse, const void* d_o, void* dq, void* dk,
                          void* dv, void* workspace, size_t ws_bytes, void* stream);
+
+/*
+ * Cross-document masking (the training set-up of Section 5.1; every document of a packed sample is padded to a
+ * multiple of the ratio, Appendix "Training Data Processing"): attention is blocked across document
+ * boundaries and every document restarts its sinks, gist units and window, so a packed sample is a list of
+ * independent sequences.  doc_raw_len (HOST pointer, num_docs entries) gives each document's raw length T_d, a
+ * multiple of ratio; p->batch must be 1 and p->raw_len is ignored.  Tensors are [N_total, heads, D] device
+ * tensors with N_total = sum_d (s + T_d + T_d / r) rows: document d owns the rows from the sum of the earlier
+ * documents' lengths on, in shifted order inside its block (interleaved with UNIGIST_FLAG_INTERLEAVED).
+ * lse holds one [Hq, N_d] block per document (shifted order), document d's block starting at float
+ * Hq * (first row of d).  Consecutive documents of equal length run as one batched launch; the launches follow
+ * one another on `stream` and share the workspace (unigist_docs_workspace_bytes: the largest any of them needs).
+ * Errors as for unigist_attn_fwd / unigist_attn_bwd, raised before the first launch where the list is malformed.
+ */
+int64_t unigist_docs_total_len(const unigist_problem* p, int32_t num_docs, const int32_t* doc_raw_len);
+size_t unigist_docs_workspace_bytes(const unigist_problem* p, int32_t op, int32_t num_docs, const int32_t* doc_raw_len);
+int32_t unigist_attn_fwd_docs(const unigist_problem* p, int32_t num_docs, const int32_t* doc_raw_len, const void* q,
+                              const void* k, const void* v, void* o, float* lse, void* workspace, size_t ws_bytes,
+                              void* stream);
+int32_t unigist_attn_bwd_docs(const unigist_problem* p, int32_t num_docs, const int32_t* doc_raw_len, const void* q,
+                              const void* k, const void* v, const void* o, const float* lse, const void* d_o, void* dq,
+                              void* dk, void* dv, void* workspace, size_t ws_bytes, void* stream);
 
 /*
  * KV compaction (Section 4.3): after the last gist of a T-token prefix, keep the sinks, all n

@@ -28,6 +28,8 @@ SYMBOLS = [
     "unigist_kernel_timing", "unigist_kernel_timing_count", "unigist_kernel_timing_get",
     "unigist_device_status", "unigist_decode_static", "unigist_prefill_workspace_bytes", "unigist_prefill_chunk",
     "unigist_cache_state_bytes", "unigist_cache_state_init", "unigist_cache_append", "unigist_decode_step",
+    "unigist_rope", "unigist_docs_total_len", "unigist_docs_workspace_bytes", "unigist_attn_fwd_docs",
+    "unigist_attn_bwd_docs",
 ]
 
 
@@ -85,6 +87,11 @@ def lib() -> ctypes.CDLL:
             "unigist_layout": (i32, [P, vp, vp, vp, i32, vp]),
             "unigist_gist_shift": (i32, [P, vp, vp, i32, i32, vp]),
             "unigist_gist_unshift": (i32, [P, vp, vp, i32, i32, vp]),
+            "unigist_rope": (i32, [P, vp, vp, i32, f32, ctypes.c_uint32, vp]),
+            "unigist_docs_total_len": (i64, [P, i32, vp]),
+            "unigist_docs_workspace_bytes": (sz, [P, i32, i32, vp]),
+            "unigist_attn_fwd_docs": (i32, [P, i32, vp] + [vp] * 6 + [sz, vp]),
+            "unigist_attn_bwd_docs": (i32, [P, i32, vp] + [vp] * 10 + [sz, vp]),
             "unigist_attn_fwd": (i32, [P, vp, vp, vp, vp, vp, vp, sz, vp]),
             "unigist_attn_bwd": (i32, [P] + [vp] * 10 + [sz, vp]),
             "unigist_kv_compact": (i32, [P, vp, vp, vp, vp, i32, vp, i32, vp, vp, vp, sz, vp]),
@@ -218,6 +225,42 @@ def unigist_gist_unshift(p: Problem, src, dst, stream=None):
     _dev(src, dst)
     _check(lib().unigist_gist_unshift(ctypes.byref(p.c()), _ptr(src), _ptr(dst), src.shape[2],
                                       src.element_size(), _stream(stream)))
+
+
+def _doc_array(doc_raw_len):
+    return (ctypes.c_int32 * len(doc_raw_len))(*[int(t) for t in doc_raw_len])
+
+
+def unigist_docs_total_len(p: Problem, doc_raw_len) -> int:
+    return int(lib().unigist_docs_total_len(ctypes.byref(p.c()), len(doc_raw_len), _doc_array(doc_raw_len)))
+
+
+def unigist_docs_workspace_bytes(p: Problem, op: int, doc_raw_len) -> int:
+    return int(lib().unigist_docs_workspace_bytes(ctypes.byref(p.c()), op, len(doc_raw_len), _doc_array(doc_raw_len)))
+
+
+def unigist_attn_fwd_docs(p: Problem, doc_raw_len, q, k, v, o, lse, workspace=None, stream=None):
+    _dev(q, k, v, o, lse, workspace)
+    _check(lib().unigist_attn_fwd_docs(ctypes.byref(p.c()), len(doc_raw_len), _doc_array(doc_raw_len), _ptr(q), _ptr(k),
+                                       _ptr(v), _ptr(o), _ptr(lse), _ptr(workspace),
+                                       0 if workspace is None else workspace.numel() * workspace.element_size(),
+                                       _stream(stream)))
+
+
+def unigist_attn_bwd_docs(p: Problem, doc_raw_len, q, k, v, o, lse, d_o, dq, dk, dv, workspace, stream=None):
+    _dev(q, k, v, o, lse, d_o, dq, dk, dv, workspace)
+    _check(lib().unigist_attn_bwd_docs(ctypes.byref(p.c()), len(doc_raw_len), _doc_array(doc_raw_len), _ptr(q), _ptr(k),
+                                       _ptr(v), _ptr(o), _ptr(lse), _ptr(d_o), _ptr(dq), _ptr(dk), _ptr(dv),
+                                       _ptr(workspace), workspace.numel() * workspace.element_size(), _stream(stream)))
+
+
+ROPE_TO_SHIFTED = 1
+
+
+def unigist_rope(p: Problem, src, dst, theta_base: float, flags: int = 0, stream=None):
+    _dev(src, dst)
+    _check(lib().unigist_rope(ctypes.byref(p.c()), _ptr(src), _ptr(dst), src.shape[2], float(theta_base), flags,
+                              _stream(stream)))
 
 
 def unigist_attn_fwd(p: Problem, q, k, v, o, lse, workspace=None, stream=None):

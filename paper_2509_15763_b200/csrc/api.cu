@@ -208,6 +208,23 @@ int32_t unigist_gist_unshift(const unigist_problem* p, const void* src, void* ds
   return shift_common(p, src, dst, heads, elem_bytes, stream, true);
 }
 
+int32_t unigist_rope(const unigist_problem* p, const void* src, void* dst, int32_t heads, float theta_base,
+                     uint32_t flags, void* stream) {
+  Geom g;
+  if (int32_t rc = check_problem(p, &g, nullptr)) return rc;
+  if (!src || !dst) return fail(UNIGIST_ERR_INVALID_ARG, "src/dst is NULL");
+  if (heads < 1 || !(theta_base > 1.f) || (flags & ~UNIGIST_ROPE_TO_SHIFTED))
+    return fail(UNIGIST_ERR_INVALID_ARG, "heads must be >= 1, theta_base > 1, flags 0 or UNIGIST_ROPE_TO_SHIFTED");
+  if (!aligned16(src) || !aligned16(dst)) return fail(UNIGIST_ERR_ALIGNMENT, "pointers must be 16-byte aligned");
+  const bool to_shifted = (flags & UNIGIST_ROPE_TO_SHIFTED) != 0;
+  const char* a = (const char*)src;
+  const char* b = (const char*)dst;
+  const size_t tot = (size_t)heads * p->head_dim * 2 * g.N * p->batch;
+  if ((to_shifted || a != b) && a < b + tot && b < a + tot)
+    return fail(UNIGIST_ERR_INVALID_ARG, "src and dst overlap (in place is allowed only without the shift)");
+  return launch_rope(g, p->batch, heads, p->head_dim, theta_base, to_shifted, src, dst, (cudaStream_t)stream);
+}
+
 int32_t unigist_attn_fwd(const unigist_problem* p, const void* q, const void* k, const void* v,
                          void* o, float* lse, void* workspace, size_t ws_bytes, void* stream) {
   Geom g;
@@ -216,8 +233,8 @@ int32_t unigist_attn_fwd(const unigist_problem* p, const void* q, const void* k,
   (void)workspace;
   (void)ws_bytes;
   if (!q || !k || !v || !o || !lse) return fail(UNIGIST_ERR_INVALID_ARG, "a tensor is NULL");
-  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || !aligned16(lse))
-    return fail(UNIGIST_ERR_ALIGNMENT, "tensor pointers must be 16-byte aligned");
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || (reinterpret_cast<uintptr_t>(lse) & 3))
+    return fail(UNIGIST_ERR_ALIGNMENT, "tensor pointers must be 16-byte aligned (lse: 4-byte)");
   if (int32_t rc = check_interleaved(p, g)) return rc;
   return launch_fwd_sm100(g, *p, scale, q, k, v, o, lse, (cudaStream_t)stream);
 }
@@ -243,9 +260,10 @@ int32_t unigist_attn_bwd(const unigist_problem* p, const void* q, const void* k,
   if (int32_t rc = check_problem(p, &g, &scale)) return rc;
   if (!q || !k || !v || !o || !lse || !d_o || !dq || !dk || !dv)
     return fail(UNIGIST_ERR_INVALID_ARG, "a tensor is NULL");
-  const void* ptrs[] = {q, k, v, o, lse, d_o, dq, dk, dv, workspace};
+  const void* ptrs[] = {q, k, v, o, d_o, dq, dk, dv, workspace};
   for (const void* x : ptrs)
     if (!aligned16(x)) return fail(UNIGIST_ERR_ALIGNMENT, "tensor pointers must be 16-byte aligned");
+  if (reinterpret_cast<uintptr_t>(lse) & 3) return fail(UNIGIST_ERR_ALIGNMENT, "lse must be 4-byte aligned");
   if (int32_t rc = check_interleaved(p, g)) return rc;
   const size_t need = unigist_workspace_bytes(p, UNIGIST_OP_BWD);
   if (!workspace || ws_bytes < need)
@@ -257,6 +275,90 @@ int32_t unigist_attn_bwd(const unigist_problem* p, const void* q, const void* k,
     return launch_bwd_sm100(g, *p, scale, q, k, v, o, lse, d_o, dq, dk, dv, workspace, (cudaStream_t)stream);
   return launch_bwd_simt(g, *p, scale, q, k, v, o, lse, d_o, dq, dk, dv, (float*)workspace,
                          (cudaStream_t)stream);
+}
+
+// ---- cross-document masking: a packed sample is a list of independent sequences -------------------------------
+
+extern "C++" {
+namespace {
+
+// Checks the document list; fills the problem of a run of `count` equal documents starting at doc `first`.
+int32_t check_docs(const unigist_problem* p, int32_t num_docs, const int32_t* doc_raw_len) {
+  if (!p || !doc_raw_len || num_docs < 1) return fail(UNIGIST_ERR_INVALID_ARG, "document list is NULL or empty");
+  if (p->batch != 1) return fail(UNIGIST_ERR_INVALID_ARG, "a packed sample has batch 1 (append the documents of more samples to the list)");
+  for (int32_t d = 0; d < num_docs; ++d) {
+    unigist_problem one = *p;
+    one.raw_len = doc_raw_len[d];
+    if (int32_t rc = check_problem(&one, nullptr, nullptr)) return rc;
+  }
+  return UNIGIST_OK;
+}
+
+// Calls fn(problem of the run, first token row of the run) for every run of consecutive documents of equal length.
+template <typename Fn>
+int32_t for_each_doc_run(const unigist_problem* p, int32_t num_docs, const int32_t* doc_raw_len, Fn fn) {
+  int64_t base = 0;
+  for (int32_t d = 0; d < num_docs;) {
+    int32_t e = d + 1;
+    while (e < num_docs && doc_raw_len[e] == doc_raw_len[d]) ++e;
+    unigist_problem run = *p;
+    run.raw_len = doc_raw_len[d];
+    run.batch = e - d;
+    const int64_t n_doc = (int64_t)run.num_sinks + run.raw_len + run.raw_len / run.ratio;
+    if (int32_t rc = fn(run, base)) return rc;
+    base += n_doc * run.batch;
+    d = e;
+  }
+  return UNIGIST_OK;
+}
+
+}  // namespace
+}  // extern "C++"
+
+int64_t unigist_docs_total_len(const unigist_problem* p, int32_t num_docs, const int32_t* doc_raw_len) {
+  if (check_docs(p, num_docs, doc_raw_len) != UNIGIST_OK) return -1;
+  int64_t tot = 0;
+  for (int32_t d = 0; d < num_docs; ++d) tot += (int64_t)p->num_sinks + doc_raw_len[d] + doc_raw_len[d] / p->ratio;
+  return tot;
+}
+
+size_t unigist_docs_workspace_bytes(const unigist_problem* p, int32_t op, int32_t num_docs, const int32_t* doc_raw_len) {
+  if (check_docs(p, num_docs, doc_raw_len) != UNIGIST_OK) return 0;
+  size_t need = 0;
+  for_each_doc_run(p, num_docs, doc_raw_len, [&](const unigist_problem& run, int64_t) {
+    const size_t b = unigist_workspace_bytes(&run, op);
+    need = b > need ? b : need;
+    return (int32_t)UNIGIST_OK;
+  });
+  return need;
+}
+
+int32_t unigist_attn_fwd_docs(const unigist_problem* p, int32_t num_docs, const int32_t* doc_raw_len, const void* q,
+                              const void* k, const void* v, void* o, float* lse, void* workspace, size_t ws_bytes,
+                              void* stream) {
+  if (int32_t rc = check_docs(p, num_docs, doc_raw_len)) return rc;
+  if (!q || !k || !v || !o || !lse) return fail(UNIGIST_ERR_INVALID_ARG, "a tensor is NULL");
+  const size_t rq = (size_t)p->num_q_heads * p->head_dim * 2, rk = (size_t)p->num_kv_heads * p->head_dim * 2;
+  return for_each_doc_run(p, num_docs, doc_raw_len, [&](const unigist_problem& run, int64_t base) {
+    return unigist_attn_fwd(&run, (const char*)q + base * rq, (const char*)k + base * rk, (const char*)v + base * rk,
+                            (char*)o + base * rq, lse + base * p->num_q_heads, workspace, ws_bytes, stream);
+  });
+}
+
+int32_t unigist_attn_bwd_docs(const unigist_problem* p, int32_t num_docs, const int32_t* doc_raw_len, const void* q,
+                              const void* k, const void* v, const void* o, const float* lse, const void* d_o, void* dq,
+                              void* dk, void* dv, void* workspace, size_t ws_bytes, void* stream) {
+  if (int32_t rc = check_docs(p, num_docs, doc_raw_len)) return rc;
+  if (!q || !k || !v || !o || !lse || !d_o || !dq || !dk || !dv) return fail(UNIGIST_ERR_INVALID_ARG, "a tensor is NULL");
+  const size_t rq = (size_t)p->num_q_heads * p->head_dim * 2, rk = (size_t)p->num_kv_heads * p->head_dim * 2;
+  const size_t rdo = (p->flags & UNIGIST_FLAG_DOUT_FP32) ? 2 * rq : rq;
+  // one stream: the runs follow one another, so they share the workspace
+  return for_each_doc_run(p, num_docs, doc_raw_len, [&](const unigist_problem& run, int64_t base) {
+    return unigist_attn_bwd(&run, (const char*)q + base * rq, (const char*)k + base * rk, (const char*)v + base * rk,
+                            (const char*)o + base * rq, lse + base * p->num_q_heads, (const char*)d_o + base * rdo,
+                            (char*)dq + base * rq, (char*)dk + base * rk, (char*)dv + base * rk, workspace, ws_bytes,
+                            stream);
+  });
 }
 
 int32_t unigist_kv_compact(const unigist_problem* p, const void* k, const void* v, void* kc,

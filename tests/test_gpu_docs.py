@@ -1,0 +1,90 @@
+"""Cross-document masking (Section 5.1): packed documents through the library against the dense oracle."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2509_15763_b200 as ug
+from oracle import oracle
+from gpu_util import TOL_GRAD, TOL_LSE, TOL_O_MAX, TOL_O_MEAN, check_close, f64
+
+pytestmark = pytest.mark.gpu
+
+CASES = [
+    # s, r, W, doc_T, Hq, Hkv, D, interleaved
+    (0, 4, 8, [256, 64, 64, 132], 4, 2, 128, False),   # a run of two equal documents, a ragged one
+    (0, 4, 8, [256, 64, 64, 132], 4, 2, 128, True),
+    (8, 8, 16, [40, 304, 8], 2, 1, 128, False),         # sinks in every document; a one-unit document
+    (8, 8, 16, [40, 304, 8], 2, 1, 128, True),
+    (0, 2, 4, [66, 130], 2, 2, 64, False),              # head_dim 64 (two-kernel backward)
+]
+
+
+def _packed_inputs(n_tot, Hq, Hkv, D, seed):
+    g = torch.Generator().manual_seed(seed)
+    mk = lambda h: torch.randn(n_tot, h, D, generator=g).to(torch.bfloat16)
+    return mk(Hq), mk(Hkv), mk(Hkv), mk(Hq)
+
+
+@pytest.mark.parametrize("case", CASES)
+def test_docs_match_oracle(case):
+    s, r, W, doc_T, Hq, Hkv, D, il = case
+    k_units = (W + r - 1) // r
+    p = ug.Problem(1, doc_T[0], r, W, Hq, Hkv, D, num_sinks=s, flags=ug.FLAG_INTERLEAVED if il else 0)
+    n_tot = ug.unigist_docs_total_len(p, doc_T)
+    assert n_tot == sum(oracle.total_len(s, T, r) for T in doc_T)
+    q, k, v, do = _packed_inputs(n_tot, Hq, Hkv, D, 77 + len(doc_T) + s)  # interleaved order, packed
+    scale = 1.0 / np.sqrt(D)
+    o_ref, lse_ref = oracle.docs_attn_fwd(s, doc_T, r, k_units, scale, f64(q), f64(k), f64(v))
+    dq_ref, dk_ref, dv_ref = oracle.docs_attn_bwd(s, doc_T, r, k_units, scale, f64(q), f64(k), f64(v), f64(do))
+
+    # per-document shift permutation of the packed rows (shifted position -> interleaved row)
+    perm, base = [], 0
+    for T in doc_T:
+        sp, _, _ = oracle.layout(s, T, r)
+        perm.append(base + sp.astype(np.int64))
+        base += len(sp)
+    perm = torch.from_numpy(np.concatenate(perm))
+    dev = torch.device("cuda:0")
+    to_lib = (lambda t: t.to(dev)) if il else (lambda t: t[perm].contiguous().to(dev))
+    qd, kd, vd, dod = to_lib(q), to_lib(k), to_lib(v), to_lib(do)
+    o = torch.full_like(qd, float("nan"))
+    lse = torch.full((Hq * n_tot,), float("nan"), device=dev)
+    ug.unigist_attn_fwd_docs(p, doc_T, qd, kd, vd, o, lse)
+    ws = torch.empty(max(ug.unigist_docs_workspace_bytes(p, ug.OP_BWD, doc_T), 16), dtype=torch.uint8, device=dev)
+    dq, dk, dv = (torch.full_like(t, float("nan")) for t in (qd, kd, vd))
+    ug.unigist_attn_bwd_docs(p, doc_T, qd, kd, vd, o, lse, dod, dq, dk, dv, ws)
+    ug.unigist_device_status()
+
+    def from_lib(t):  # back to interleaved packed order on the host
+        t = t.cpu()
+        if il:
+            return t
+        out = torch.empty_like(t)
+        out[perm] = t
+        return out
+
+    check_close("o", f64(from_lib(o)), o_ref, TOL_O_MAX, TOL_O_MEAN)
+    # lse: one [Hq, N_d] block per document, shifted order inside
+    lse_h = lse.cpu().double().numpy()
+    base = 0
+    for T in doc_T:
+        sp, _, _ = oracle.layout(s, T, r)
+        n = len(sp)
+        blk = lse_h[Hq * base: Hq * (base + n)].reshape(Hq, n)
+        check_close("lse", blk, lse_ref[:, base + sp], TOL_LSE)
+        base += n
+    check_close("dq", f64(from_lib(dq)), dq_ref, TOL_GRAD)
+    check_close("dk", f64(from_lib(dk)), dk_ref, TOL_GRAD)
+    check_close("dv", f64(from_lib(dv)), dv_ref, TOL_GRAD)
+
+
+def test_docs_reject_bad_lists():
+    p = ug.Problem(1, 16, 4, 8, 2, 2, 128)
+    x = torch.zeros(64, 2, 128, dtype=torch.bfloat16, device="cuda")
+    lse = torch.zeros(2 * 64, device="cuda")
+    with pytest.raises(ug.UnigistError):
+        ug.unigist_attn_fwd_docs(p, [16, 6], x, x, x, x, lse)  # 6 is not a multiple of the ratio
+    assert ug.unigist_docs_total_len(p, [16, 6]) == -1
+    p2 = ug.Problem(2, 16, 4, 8, 2, 2, 128)
+    with pytest.raises(ug.UnigistError):
+        ug.unigist_attn_fwd_docs(p2, [16], x, x, x, x, lse)  # batch must be 1
