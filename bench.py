@@ -349,6 +349,65 @@ def bench_chunked_prefill(path, chunk_units, iters=3):
             "note": "whole prompt through unigist_prefill_chunk: context gather + forward + cache advance per chunk"}
 
 
+def bench_rope_and_docs(path, iters=3):
+    """Two side measurements on the workload's own tensors: the rotary embedding with aligned position ids
+    fused with the gist shift (HBM-bound), and the attention step under cross-document masking, with the
+    sample cut into documents of T/2, T/4, ... raw tokens.  -> (rope dict, cross_doc dict)."""
+    import torch
+
+    ug, w, dev, p = path.ug, path.w, path.dev, path.p
+
+    def timed(fn):
+        fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(iters):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / iters
+
+    x, y = path.inter["q"], path.sh["q"]
+    ms = timed(lambda: ug.unigist_rope(p, x, y, 500000.0, ug.ROPE_TO_SHIFTED))
+    nbytes = 2 * x.numel() * x.element_size()
+    rope = {"ms": ms, "gbs": nbytes / (ms * 1e-3) / 1e9, "bytes": nbytes,
+            "note": "unigist_rope on Q, interleaved in, shifted out (read + write once)"}
+    if w.batch != 1 or w.forward_only or not path.fused_shift:
+        return rope, None
+    # documents of T/2, T/4, ... raw tokens; what is left at 1024 tokens or fewer is the last document
+    doc_T, left = [], w.raw_len
+    while left > 0:
+        t = left if left <= 1024 else (left // 2) // w.ratio * w.ratio
+        doc_T.append(t)
+        left -= t
+    p1 = ug.Problem(1, doc_T[0], w.ratio, w.window, w.num_q_heads, w.num_kv_heads, w.head_dim, num_sinks=w.num_sinks,
+                    flags=ug.FLAG_INTERLEAVED)
+    n_tot = ug.unigist_docs_total_len(p1, doc_T)
+    q, k, v, do = (path.inter[n][0, :n_tot] for n in ("q", "k", "v", "dout"))
+    if n_tot > path.inter["q"].shape[1]:  # every document carries its own sinks: more rows than the one-document sample
+        pad = lambda t: torch.cat([t, t[: n_tot - t.shape[0]]])
+        q, k, v, do = pad(q), pad(k), pad(v), pad(do)
+    o, dq, dk, dv = torch.empty_like(q), torch.empty_like(q), torch.empty_like(k), torch.empty_like(v)
+    lse = torch.empty(w.num_q_heads * n_tot, dtype=torch.float32, device=dev)
+    ws = torch.empty(max(16, ug.unigist_docs_workspace_bytes(p1, ug.OP_BWD, doc_T)), dtype=torch.uint8, device=dev)
+
+    def run():
+        ug.unigist_attn_fwd_docs(p1, doc_T, q, k, v, o, lse)
+        ug.unigist_attn_bwd_docs(p1, doc_T, q, k, v, o, lse, do, dq, dk, dv, ws)
+
+    ms = timed(run)
+    pairs = 0
+    for t in doc_T:
+        pairs += ug.unigist_visible_pairs(ug.Problem(1, t, w.ratio, w.window, w.num_q_heads, w.num_kv_heads, w.head_dim,
+                                                     num_sinks=w.num_sinks))
+    flops = 14.0 * w.head_dim * pairs * w.num_q_heads
+    docs = {"doc_raw_len": doc_T, "ms": ms, "value": flops / (ms * 1e-3) / 1e12, "unit": UNIT,
+            "note": "forward + backward of the sample cut into documents (one batched launch set per run of equal "
+                    "documents, spread over the library's side streams)"}
+    return rope, docs
+
+
 def run_ours(args, w):
     import torch
 
@@ -419,6 +478,7 @@ def run_ours(args, w):
             ev2.append((e0, e1))
         torch.cuda.synchronize()
         explicit_ms = sum(a.elapsed_time(b) for a, b in ev2) / args.steps
+    rope_line, docs_line = bench_rope_and_docs(path) if rank == 0 and world == 1 else (None, None)
     barrier()
 
     # ---- end to end: host buffers in, host buffers out
@@ -478,6 +538,7 @@ def run_ours(args, w):
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": path.h2d_bytes(),
                 "d2h_bytes_per_step": path.d2h_bytes()},
         "chunked_prefill": bench_chunked_prefill(path, 1024) if w.forward_only else None,
+        "rope": rope_line, "cross_doc": docs_line,
         "explicit_shift_step": None if explicit_ms is None else {
             "ms_per_step": explicit_ms, "value": path.flops / (explicit_ms * 1e-3) / 1e12, "unit": UNIT,
             "note": "the same step with 4 shift and 4 unshift launches around shifted-order attention calls"},

@@ -294,22 +294,69 @@ int32_t check_docs(const unigist_problem* p, int32_t num_docs, const int32_t* do
   return UNIGIST_OK;
 }
 
-// Calls fn(problem of the run, first token row of the run) for every run of consecutive documents of equal length.
+// Calls fn(problem of the run, first token row of the run, index of the run) for every run of consecutive
+// documents of equal length.
 template <typename Fn>
 int32_t for_each_doc_run(const unigist_problem* p, int32_t num_docs, const int32_t* doc_raw_len, Fn fn) {
   int64_t base = 0;
-  for (int32_t d = 0; d < num_docs;) {
+  int32_t index = 0;
+  for (int32_t d = 0; d < num_docs; ++index) {
     int32_t e = d + 1;
     while (e < num_docs && doc_raw_len[e] == doc_raw_len[d]) ++e;
     unigist_problem run = *p;
     run.raw_len = doc_raw_len[d];
     run.batch = e - d;
     const int64_t n_doc = (int64_t)run.num_sinks + run.raw_len + run.raw_len / run.ratio;
-    if (int32_t rc = fn(run, base)) return rc;
+    if (int32_t rc = fn(run, base, index)) return rc;
     base += n_doc * run.batch;
     d = e;
   }
   return UNIGIST_OK;
+}
+
+// The runs of a packed sample are independent, and the short ones do not fill the GPU: they are spread over
+// a few side streams that fork from the caller's stream and join it again (events only; capturable in a graph).
+constexpr int kSideStreams = 3;
+struct DocStreams {
+  cudaStream_t side[kSideStreams];
+  cudaEvent_t fork, join[kSideStreams];
+  bool ok = false;
+  DocStreams() {
+    ok = cudaEventCreateWithFlags(&fork, cudaEventDisableTiming) == cudaSuccess;
+    for (int i = 0; i < kSideStreams && ok; ++i)
+      ok = cudaStreamCreateWithFlags(&side[i], cudaStreamNonBlocking) == cudaSuccess &&
+           cudaEventCreateWithFlags(&join[i], cudaEventDisableTiming) == cudaSuccess;
+  }
+};
+DocStreams& doc_streams() {
+  static DocStreams ds;  // created on first use, lives as long as the library
+  return ds;
+}
+
+// Runs fn(run problem, first row, run index, stream of the run) with run i on stream i mod (1 + kSideStreams),
+// stream 0 being the caller's.
+template <typename Fn>
+int32_t spread_doc_runs(const unigist_problem* p, int32_t num_docs, const int32_t* doc_raw_len, cudaStream_t st, Fn fn) {
+  DocStreams& ds = doc_streams();
+  if (!ds.ok) return fail(UNIGIST_ERR_CUDA, "could not create the side streams");
+  int32_t runs = 0;
+  for_each_doc_run(p, num_docs, doc_raw_len, [&](const unigist_problem&, int64_t, int32_t) { ++runs; return (int32_t)UNIGIST_OK; });
+  const int used = runs - 1 < kSideStreams ? runs - 1 : kSideStreams;
+  if (used > 0) {
+    if (cudaEventRecord(ds.fork, st) != cudaSuccess) return fail(UNIGIST_ERR_CUDA, "cudaEventRecord failed");
+    for (int i = 0; i < used; ++i)
+      if (cudaStreamWaitEvent(ds.side[i], ds.fork, 0) != cudaSuccess) return fail(UNIGIST_ERR_CUDA, "cudaStreamWaitEvent failed");
+  }
+  const int32_t rc = for_each_doc_run(p, num_docs, doc_raw_len, [&](const unigist_problem& run, int64_t base, int32_t i) {
+    const int lane = i % (1 + kSideStreams);
+    return fn(run, base, i, lane == 0 ? st : ds.side[lane - 1]);
+  });
+  // join even after an error, so that the caller's stream stays ordered after whatever was enqueued
+  for (int i = 0; i < used; ++i) {
+    if (cudaEventRecord(ds.join[i], ds.side[i]) != cudaSuccess || cudaStreamWaitEvent(st, ds.join[i], 0) != cudaSuccess)
+      return fail(UNIGIST_ERR_CUDA, "joining a side stream failed");
+  }
+  return rc;
 }
 
 }  // namespace
@@ -324,10 +371,9 @@ int64_t unigist_docs_total_len(const unigist_problem* p, int32_t num_docs, const
 
 size_t unigist_docs_workspace_bytes(const unigist_problem* p, int32_t op, int32_t num_docs, const int32_t* doc_raw_len) {
   if (check_docs(p, num_docs, doc_raw_len) != UNIGIST_OK) return 0;
-  size_t need = 0;
-  for_each_doc_run(p, num_docs, doc_raw_len, [&](const unigist_problem& run, int64_t) {
-    const size_t b = unigist_workspace_bytes(&run, op);
-    need = b > need ? b : need;
+  size_t need = 0;  // the runs work side by side: one slice each
+  for_each_doc_run(p, num_docs, doc_raw_len, [&](const unigist_problem& run, int64_t, int32_t) {
+    need += align_up(unigist_workspace_bytes(&run, op), 256);
     return (int32_t)UNIGIST_OK;
   });
   return need;
@@ -339,9 +385,10 @@ int32_t unigist_attn_fwd_docs(const unigist_problem* p, int32_t num_docs, const 
   if (int32_t rc = check_docs(p, num_docs, doc_raw_len)) return rc;
   if (!q || !k || !v || !o || !lse) return fail(UNIGIST_ERR_INVALID_ARG, "a tensor is NULL");
   const size_t rq = (size_t)p->num_q_heads * p->head_dim * 2, rk = (size_t)p->num_kv_heads * p->head_dim * 2;
-  return for_each_doc_run(p, num_docs, doc_raw_len, [&](const unigist_problem& run, int64_t base) {
+  return spread_doc_runs(p, num_docs, doc_raw_len, (cudaStream_t)stream,
+                         [&](const unigist_problem& run, int64_t base, int32_t, cudaStream_t st) {
     return unigist_attn_fwd(&run, (const char*)q + base * rq, (const char*)k + base * rk, (const char*)v + base * rk,
-                            (char*)o + base * rq, lse + base * p->num_q_heads, workspace, ws_bytes, stream);
+                            (char*)o + base * rq, lse + base * p->num_q_heads, workspace, ws_bytes, st);
   });
 }
 
@@ -352,12 +399,18 @@ int32_t unigist_attn_bwd_docs(const unigist_problem* p, int32_t num_docs, const 
   if (!q || !k || !v || !o || !lse || !d_o || !dq || !dk || !dv) return fail(UNIGIST_ERR_INVALID_ARG, "a tensor is NULL");
   const size_t rq = (size_t)p->num_q_heads * p->head_dim * 2, rk = (size_t)p->num_kv_heads * p->head_dim * 2;
   const size_t rdo = (p->flags & UNIGIST_FLAG_DOUT_FP32) ? 2 * rq : rq;
-  // one stream: the runs follow one another, so they share the workspace
-  return for_each_doc_run(p, num_docs, doc_raw_len, [&](const unigist_problem& run, int64_t base) {
+  if (!workspace || !aligned16(workspace) || ws_bytes < unigist_docs_workspace_bytes(p, UNIGIST_OP_BWD, num_docs, doc_raw_len))
+    return fail(UNIGIST_ERR_WORKSPACE, "backward over documents needs %zu bytes of 16-byte aligned workspace, got %zu",
+                unigist_docs_workspace_bytes(p, UNIGIST_OP_BWD, num_docs, doc_raw_len), ws_bytes);
+  size_t ws_off = 0;
+  return spread_doc_runs(p, num_docs, doc_raw_len, (cudaStream_t)stream,
+                         [&](const unigist_problem& run, int64_t base, int32_t, cudaStream_t st) {
+    const size_t mine = align_up(unigist_workspace_bytes(&run, UNIGIST_OP_BWD), 256);
+    char* ws = (char*)workspace + ws_off;
+    ws_off += mine;
     return unigist_attn_bwd(&run, (const char*)q + base * rq, (const char*)k + base * rk, (const char*)v + base * rk,
                             (const char*)o + base * rq, lse + base * p->num_q_heads, (const char*)d_o + base * rdo,
-                            (char*)dq + base * rq, (char*)dk + base * rk, (char*)dv + base * rk, workspace, ws_bytes,
-                            stream);
+                            (char*)dq + base * rq, (char*)dk + base * rk, (char*)dv + base * rk, ws, mine, st);
   });
 }
 

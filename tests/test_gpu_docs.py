@@ -16,6 +16,7 @@ CASES = [
     (8, 8, 16, [40, 304, 8], 2, 1, 128, False),         # sinks in every document; a one-unit document
     (8, 8, 16, [40, 304, 8], 2, 1, 128, True),
     (0, 2, 4, [66, 130], 2, 2, 64, False),              # head_dim 64 (two-kernel backward)
+    (0, 4, 8, [64, 128, 64, 192, 64, 256], 2, 2, 128, True),  # six runs: more than the library has streams
 ]
 
 
