@@ -64,6 +64,11 @@ for _i, _ctx in enumerate((16, 32, 64, 128)):
         WORKLOADS[_name] = Workload(_name, 1, _ctx * 1024, _r, 128, 32, 32, 128, num_sinks=128,
                                     seed=BASE_SEED + 10 + 2 * _i + (_r == 8))
 
+    # the table's "causal attention" row: plain causal attention over the same raw tokens, which is the
+    # method's own special case of a single gist unit (ratio = window = T, one gist at the very end, no sinks)
+    _name = f"table4_{_ctx}k_causal"
+    WORKLOADS[_name] = Workload(_name, 1, _ctx * 1024, _ctx * 1024, _ctx * 1024, 32, 32, 128, seed=BASE_SEED + 30 + _i)
+
 
 @dataclass(frozen=True)
 class DecodeWorkload:

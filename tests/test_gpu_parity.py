@@ -70,6 +70,9 @@ SMALL = [
     synth.Workload("sinks_128", 1, 1024, 8, 128, 4, 2, 128, num_sinks=128, seed=113),
     synth.Workload("sinks_300", 2, 640, 4, 64, 2, 2, 128, num_sinks=300, seed=114),
     synth.Workload("sinks_64_d64", 1, 512, 8, 64, 2, 1, 64, num_sinks=64, seed=115),
+    # gist units longer than a tile: plain causal attention as a single unit, and two-tile units with a one-unit window
+    synth.Workload("single_unit_causal", 1, 640, 640, 640, 2, 2, 128, seed=116),
+    synth.Workload("long_units", 2, 1024, 256, 256, 4, 2, 128, num_sinks=5, seed=117),
 ]
 
 
