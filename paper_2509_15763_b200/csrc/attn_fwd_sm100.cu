@@ -239,8 +239,9 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_sink, const __gri
                       const __grid_constant__ CUtensorMap tm_q_gist, const __grid_constant__ CUtensorMap tm_k_sink,
                       const __grid_constant__ CUtensorMap tm_k_raw, const __grid_constant__ CUtensorMap tm_k_gist,
                       const __grid_constant__ CUtensorMap tm_v_sink, const __grid_constant__ CUtensorMap tm_v_raw,
-                      const __grid_constant__ CUtensorMap tm_v_gist, Geom g, int Hq, int Hkv, float scale_log2,
-                      __nv_bfloat16* __restrict__ o, float* __restrict__ lse, int n_sink_units, int n_raw_units,
+                      const __grid_constant__ CUtensorMap tm_v_gist, const __grid_constant__ CUtensorMap tm_o_sink,
+                      const __grid_constant__ CUtensorMap tm_o_raw, const __grid_constant__ CUtensorMap tm_o_gist, Geom g,
+                      int Hq, int Hkv, float scale_log2, float* __restrict__ lse, int n_sink_units, int n_raw_units,
                       int pair_heads, int interleaved, QueryRows qr) {
   using SM = FwdSmem<D>;
   extern __shared__ unsigned char smem_dyn[];
@@ -280,12 +281,9 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_sink, const __gri
     sv[0] = true;
     sv[1] = qt[1] < n_qt;
   }
-  const int hk = hh[0] / (Hq / Hkv);  // both streams share the KV head
-  const Stream str0 = make_stream(g, sv[0], hh[0], qt[0], qseg, q_off),
-               str1 = make_stream(g, sv[1], hh[1], qt[1], qseg, q_off);
-  const TileSeq seq = make_tile_seq(str0, str1, qseg);
-  const int nt = seq.count();
 
+  // Barriers, tensor memory and the Q loads come before the rest of the index arithmetic, which then runs
+  // under the latency of those loads.
   if (threadIdx.x == 0) {
     mbar_init(bar_q, 1);
     mbar_init(bar_o, 1);
@@ -306,21 +304,29 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_sink, const __gri
   tc_fence_after();
   const uint32_t tmem = *tmem_slot_ptr;
   bool ok = true;
+  if (warp == kTmaWarp && elect_one()) {
+    // tile coordinate: its first unit (a raw tile of an interleaved tensor spans 128 / r gist units)
+    const CUtensorMap* mq = qseg == kSegRaw ? &tm_q_raw : (qseg == kSegGist ? &tm_q_gist : &tm_q_sink);
+    mbar_arrive_expect_tx(bar_q, (sv[1] ? 2 : 1) * SM::kTile);
+    for (int i = 0; i < 2; ++i) {
+      if (!sv[i]) continue;
+      const int row0 = qt[i] * BM;
+#pragma unroll
+      for (int sl = 0; sl < D / 64; ++sl)
+        tma_load_5d(sQ[i] + sl * SM::kSlab, mq, bar_q, sl * 64, hh[i], 0, interleaved && qseg == kSegRaw ? row0 / g.r : row0, b);
+    }
+  }
+  const int hk = hh[0] / (Hq / Hkv);  // both streams share the KV head
+  const Stream str0 = make_stream(g, sv[0], hh[0], qt[0], qseg, q_off),
+               str1 = make_stream(g, sv[1], hh[1], qt[1], qseg, q_off);
+  const TileSeq seq = make_tile_seq(str0, str1, qseg);
+  const int nt = seq.count();
   if (warp >= kSmWarps) {
     reg_dealloc<kRegsOther>();
   if (warp == kTmaWarp) {
     // ------------------------------------------------------------ TMA producer
     if (elect_one()) {
-      // tile coordinate: its first unit (a raw tile of an interleaved tensor spans 128 / r gist units)
       auto first_unit = [&](int sg, int row0) { return interleaved && sg == kSegRaw ? row0 / g.r : row0; };
-      const CUtensorMap* mq = qseg == kSegRaw ? &tm_q_raw : (qseg == kSegGist ? &tm_q_gist : &tm_q_sink);
-      mbar_arrive_expect_tx(bar_q, (sv[1] ? 2 : 1) * SM::kTile);
-      for (int i = 0; i < 2; ++i) {
-        if (!sv[i]) continue;
-#pragma unroll
-        for (int sl = 0; sl < D / 64; ++sl)
-          tma_load_5d(sQ[i] + sl * SM::kSlab, mq, bar_q, sl * 64, hh[i], 0, first_unit(qseg, qt[i] * BM), b);
-      }
       for (int t = 0; t < 2 * nt && ok; ++t) {  // item t: K tile of step t/2 (even t) or its V tile (odd t)
         int sg, idx;
         seq.at(t >> 1, sg, idx);
@@ -508,33 +514,46 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_sink, const __gri
       if (ok) {
         tc_fence_after();
         const float inv_l = 1.f / l_run;
-        const bool valid = me.row_a + r_in_tile <= me.row_b;
-        const int out_row = interleaved ? seg_row_to_token(g, true, qseg, me.row_a + r_in_tile)
-                                        : qr.out_base[qseg] + (me.row_a + r_in_tile - q_off);
-        const long long tok = (long long)b * qr.n_out + out_row;
-        __nv_bfloat16* orow = o + (tok * Hq + me.h) * D;
+        // O leaves through shared memory and TMA stores: a thread's row-wise 16-byte stores to global memory
+        // would touch 32 rows per warp instruction.  Every product has completed, so the stream's Q tile is free:
+        // the normalised rows go there in the tile layout of the loads (128-byte swizzle, one slab per 64 columns).
+        const uint32_t srow = sQ[i] + r_in_tile * 128;
+        uint32_t v[D];
+#pragma unroll
+        for (int c = 0; c < D / 32; ++c) tmem_ld32(tO + c * 32, v + c * 32);
+        tmem_wait_ld();
 #pragma unroll
         for (int c = 0; c < D / 32; ++c) {
-          uint32_t v[32];
-          tmem_ld(tO + c * 32, v);
-          tmem_wait_ld();
-          if (valid) {
 #pragma unroll
-            for (int e = 0; e < 32; e += 8) {
-              uint4 pk;
-              pk.x = pack_bf16(__uint_as_float(v[e]) * inv_l, __uint_as_float(v[e + 1]) * inv_l);
-              pk.y = pack_bf16(__uint_as_float(v[e + 2]) * inv_l, __uint_as_float(v[e + 3]) * inv_l);
-              pk.z = pack_bf16(__uint_as_float(v[e + 4]) * inv_l, __uint_as_float(v[e + 5]) * inv_l);
-              pk.w = pack_bf16(__uint_as_float(v[e + 6]) * inv_l, __uint_as_float(v[e + 7]) * inv_l);
-              *reinterpret_cast<uint4*>(orow + c * 32 + e) = pk;
-            }
+          for (int e0 = 0; e0 < 32; e0 += 8) {
+            const int e = c * 32 + e0;
+            uint4 pk;
+            pk.x = pack_bf16(__uint_as_float(v[e]) * inv_l, __uint_as_float(v[e + 1]) * inv_l);
+            pk.y = pack_bf16(__uint_as_float(v[e + 2]) * inv_l, __uint_as_float(v[e + 3]) * inv_l);
+            pk.z = pack_bf16(__uint_as_float(v[e + 4]) * inv_l, __uint_as_float(v[e + 5]) * inv_l);
+            pk.w = pack_bf16(__uint_as_float(v[e + 6]) * inv_l, __uint_as_float(v[e + 7]) * inv_l);
+            const int chunk = e / 8;  // 16-byte chunk of the row: slab chunk / 8, position (chunk % 8) ^ (row % 8)
+            st_shared_v4(srow + (chunk >> 3) * SM::kSlab + (((chunk & 7) ^ (r_in_tile & 7)) << 4), pk);
           }
         }
-        if (valid)
+        if (me.row_a + r_in_tile <= me.row_b)
           lse[((long long)b * Hq + me.h) * qr.n_out + qr.out_base[qseg] + (me.row_a + r_in_tile - q_off)] =
               (m_run + log2f(l_run)) * 0.6931471805599453f;
       } else {
         atomicExch(&g_fwd_timeout, 1u);
+      }
+      // all four warps of the stream get here, whatever their waits returned
+      fence_proxy_async_smem();
+      named_barrier_sync(1 + i, 128);
+      if (ok && (warp & 3) == 0 && elect_one()) {
+        // rows past the end of the segment lie outside the map and are not written
+        const CUtensorMap* mo = qseg == kSegRaw ? &tm_o_raw : (qseg == kSegGist ? &tm_o_gist : &tm_o_sink);
+        const int row0 = qt[i] * BM;
+#pragma unroll
+        for (int sl = 0; sl < D / 64; ++sl)
+          tma_store_5d(mo, sQ[i] + sl * SM::kSlab, sl * 64, me.h, 0, interleaved && qseg == kSegRaw ? row0 / g.r : row0, b);
+        bulk_commit_group();
+        bulk_wait_group_read0();  // shared memory must outlive the reads of the store
       }
     }
   }
@@ -654,7 +673,7 @@ int32_t encode_map_2d_bf16(CUtensorMap* map, const void* base, long long rows, i
 int32_t launch_fwd_sm100(const Geom& g, const unigist_problem& p, float scale, const void* q, const void* k,
                          const void* v, void* o, float* lse, cudaStream_t st, const QueryRows* chunk) {
   const int D = p.head_dim, Hq = p.num_q_heads, Hkv = p.num_kv_heads, B = p.batch;
-  CUtensorMap mq[3], mk[3], mv[3];  // per segment: sinks, raw, gists
+  CUtensorMap mq[3], mk[3], mv[3], mo[3];  // per segment: sinks, raw, gists (O has the geometry of Q)
   const bool il = (p.flags & UNIGIST_FLAG_INTERLEAVED) != 0 && !chunk;
   QueryRows qr;
   if (chunk) {
@@ -667,6 +686,7 @@ int32_t launch_fwd_sm100(const Geom& g, const unigist_problem& p, float scale, c
   const int sq = g.s - qr.off[kSegSink], Tq = g.T - qr.off[kSegRaw], nq = g.n - qr.off[kSegGist];
   for (int sg = 0; sg < 3; ++sg) {
     if (int32_t rc = encode_tile_map(&mq[sg], q, D, Hq, B, sq, Tq, g.r, nq, il, sg)) return rc;
+    if (int32_t rc = encode_tile_map(&mo[sg], o, D, Hq, B, sq, Tq, g.r, nq, il, sg)) return rc;
     if (int32_t rc = encode_tile_map(&mk[sg], k, D, Hkv, B, g.s, g.T, g.r, g.n, il, sg)) return rc;
     if (int32_t rc = encode_tile_map(&mv[sg], v, D, Hkv, B, g.s, g.T, g.r, g.n, il, sg)) return rc;
   }
@@ -684,8 +704,8 @@ int32_t launch_fwd_sm100(const Geom& g, const unigist_problem& p, float scale, c
     if (e != cudaSuccess) return fail(UNIGIST_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
     {
       KernelScope ks("attn_fwd_sm100_kernel", st);
-      kern<<<grid, kThreads, smem, st>>>(mq[0], mq[1], mq[2], mk[0], mk[1], mk[2], mv[0], mv[1], mv[2], g, Hq, Hkv,
-                                         scale_log2, (__nv_bfloat16*)o, lse, n_sink_units, n_raw_units, pair_heads,
+      kern<<<grid, kThreads, smem, st>>>(mq[0], mq[1], mq[2], mk[0], mk[1], mk[2], mv[0], mv[1], mv[2], mo[0], mo[1], mo[2], g,
+                                         Hq, Hkv, scale_log2, lse, n_sink_units, n_raw_units, pair_heads,
                                          il ? 1 : 0, qr);
     }
     return check_launch("tcgen05 forward kernel");
