@@ -76,7 +76,7 @@ struct Stream {
   }
 };
 
-__device__ Stream make_stream(const Geom& g, bool valid, int h, int qt, int qseg, int q_off) {
+__device__ Stream make_stream(const Geom& g, const FastDiv& rdiv, bool valid, int h, int qt, int qseg, int q_off) {
   Stream s;
   s.valid = valid;
   s.h = h;
@@ -85,8 +85,9 @@ __device__ Stream make_stream(const Geom& g, bool valid, int h, int qt, int qseg
   if (!valid) {
     s.row_a = s.row_b = 0;
   }
-  s.iv_a = row_intervals(g, seg_base(g, qseg) + s.row_a);
-  s.iv_b = row_intervals(g, seg_base(g, qseg) + s.row_b);
+  auto div_r = [&](int x) { return fdiv(rdiv, x); };
+  s.iv_a = row_intervals_with(g, seg_base(g, qseg) + s.row_a, div_r);
+  s.iv_b = row_intervals_with(g, seg_base(g, qseg) + s.row_b, div_r);
   s.n_sink = s.iv_b.hi_sink >= 0 ? s.iv_b.hi_sink / BN + 1 : 0;
   s.raw_lo = s.iv_a.lo_raw / BN;
   s.raw_hi = s.iv_b.hi_raw >= 0 ? s.iv_b.hi_raw / BN : -1;
@@ -241,7 +242,7 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_sink, const __gri
                       const __grid_constant__ CUtensorMap tm_v_sink, const __grid_constant__ CUtensorMap tm_v_raw,
                       const __grid_constant__ CUtensorMap tm_v_gist, const __grid_constant__ CUtensorMap tm_o_sink,
                       const __grid_constant__ CUtensorMap tm_o_raw, const __grid_constant__ CUtensorMap tm_o_gist, Geom g,
-                      int Hq, int Hkv, float scale_log2, float* __restrict__ lse, int n_sink_units, int n_raw_units,
+                      int Hq, FastDiv rdiv, FastDiv hkdiv, float scale_log2, float* __restrict__ lse, int n_sink_units, int n_raw_units,
                       int pair_heads, int interleaved, QueryRows qr) {
   using SM = FwdSmem<D>;
   extern __shared__ unsigned char smem_dyn[];
@@ -304,8 +305,10 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_sink, const __gri
   tc_fence_after();
   const uint32_t tmem = *tmem_slot_ptr;
   bool ok = true;
+  const int hk = fdiv(hkdiv, blockIdx.y);  // both streams share the KV head
+  // tile coordinate: its first unit (a raw tile of an interleaved tensor spans 128 / r gist units)
+  auto first_unit = [&](int sg, int row0) { return interleaved && sg == kSegRaw ? fdiv(rdiv, row0) : row0; };
   if (warp == kTmaWarp && elect_one()) {
-    // tile coordinate: its first unit (a raw tile of an interleaved tensor spans 128 / r gist units)
     const CUtensorMap* mq = qseg == kSegRaw ? &tm_q_raw : (qseg == kSegGist ? &tm_q_gist : &tm_q_sink);
     mbar_arrive_expect_tx(bar_q, (sv[1] ? 2 : 1) * SM::kTile);
     for (int i = 0; i < 2; ++i) {
@@ -313,12 +316,25 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_sink, const __gri
       const int row0 = qt[i] * BM;
 #pragma unroll
       for (int sl = 0; sl < D / 64; ++sl)
-        tma_load_5d(sQ[i] + sl * SM::kSlab, mq, bar_q, sl * 64, hh[i], 0, interleaved && qseg == kSegRaw ? row0 / g.r : row0, b);
+        tma_load_5d(sQ[i] + sl * SM::kSlab, mq, bar_q, sl * 64, hh[i], 0, first_unit(qseg, row0), b);
+    }
+    // The first key tile is the one with the diagonal of the later stream (every stream starts in its own
+    // segment, at its last row's tile): its K and V loads need none of the interval arithmetic below.
+    const int last = sv[1] ? 1 : 0;
+    const int idx0 = min(q_off + qt[last] * BM + BM - 1, seg_len(g, qseg) - 1) / BN;
+    const CUtensorMap* mk0 = qseg == kSegRaw ? &tm_k_raw : (qseg == kSegGist ? &tm_k_gist : &tm_k_sink);
+    const CUtensorMap* mv0 = qseg == kSegRaw ? &tm_v_raw : (qseg == kSegGist ? &tm_v_gist : &tm_v_sink);
+#pragma unroll
+    for (int t = 0; t < 2; ++t) {
+      mbar_arrive_expect_tx(bar_full + 8 * t, SM::kTile);
+#pragma unroll
+      for (int sl = 0; sl < D / 64; ++sl)
+        tma_load_5d(ring + t * SM::kTile + sl * SM::kSlab, t ? mv0 : mk0, bar_full + 8 * t, sl * 64, hk, 0,
+                    first_unit(qseg, idx0 * BN), b);
     }
   }
-  const int hk = hh[0] / (Hq / Hkv);  // both streams share the KV head
-  const Stream str0 = make_stream(g, sv[0], hh[0], qt[0], qseg, q_off),
-               str1 = make_stream(g, sv[1], hh[1], qt[1], qseg, q_off);
+  const Stream str0 = make_stream(g, rdiv, sv[0], hh[0], qt[0], qseg, q_off),
+               str1 = make_stream(g, rdiv, sv[1], hh[1], qt[1], qseg, q_off);
   const TileSeq seq = make_tile_seq(str0, str1, qseg);
   const int nt = seq.count();
   if (warp >= kSmWarps) {
@@ -326,8 +342,7 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_sink, const __gri
   if (warp == kTmaWarp) {
     // ------------------------------------------------------------ TMA producer
     if (elect_one()) {
-      auto first_unit = [&](int sg, int row0) { return interleaved && sg == kSegRaw ? row0 / g.r : row0; };
-      for (int t = 0; t < 2 * nt && ok; ++t) {  // item t: K tile of step t/2 (even t) or its V tile (odd t)
+      for (int t = 2; t < 2 * nt && ok; ++t) {  // item t: K tile of step t/2 (even t) or its V tile (odd t); 0, 1 are on their way
         int sg, idx;
         seq.at(t >> 1, sg, idx);
         const CUtensorMap* m = (t & 1) ? (sg == kSegRaw ? &tm_v_raw : (sg == kSegGist ? &tm_v_gist : &tm_v_sink))
@@ -551,7 +566,7 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_sink, const __gri
         const int row0 = qt[i] * BM;
 #pragma unroll
         for (int sl = 0; sl < D / 64; ++sl)
-          tma_store_5d(mo, sQ[i] + sl * SM::kSlab, sl * 64, me.h, 0, interleaved && qseg == kSegRaw ? row0 / g.r : row0, b);
+          tma_store_5d(mo, sQ[i] + sl * SM::kSlab, sl * 64, me.h, 0, first_unit(qseg, row0), b);
         bulk_commit_group();
         bulk_wait_group_read0();  // shared memory must outlive the reads of the store
       }
@@ -705,7 +720,7 @@ int32_t launch_fwd_sm100(const Geom& g, const unigist_problem& p, float scale, c
     {
       KernelScope ks("attn_fwd_sm100_kernel", st);
       kern<<<grid, kThreads, smem, st>>>(mq[0], mq[1], mq[2], mk[0], mk[1], mk[2], mv[0], mv[1], mv[2], mo[0], mo[1], mo[2], g,
-                                         Hq, Hkv, scale_log2, lse, n_sink_units, n_raw_units, pair_heads,
+                                         Hq, make_fastdiv(g.r), make_fastdiv(pair_heads ? (Hq / Hkv) / 2 : Hq / Hkv), scale_log2, lse, n_sink_units, n_raw_units, pair_heads,
                                          il ? 1 : 0, qr);
     }
     return check_launch("tcgen05 forward kernel");

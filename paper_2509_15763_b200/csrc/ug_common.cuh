@@ -27,7 +27,27 @@ struct RowIv {
   int hi_gist;  // gist columns [0, hi_gist]
 };
 
-__host__ __device__ inline RowIv row_intervals(const Geom& g, int sigma) {
+// Division of a non-negative int (< 2^31) by a divisor fixed on the host: n / d = (n * mul) >> sh with
+// sh = 31 + ceil(log2 d) and mul = ceil(2^sh / d), exact for every such n.  A runtime integer division costs a
+// few hundred clocks at the start of a block; this is one wide multiply and a shift.
+struct FastDiv {
+  uint32_t mul, sh;
+};
+inline FastDiv make_fastdiv(int d) {
+  int s = 0;
+  while ((1ll << s) < d) ++s;
+  FastDiv f;
+  f.sh = 31 + s;
+  f.mul = (uint32_t)(((1ull << f.sh) + (unsigned long long)d - 1) / (unsigned long long)d);
+  return f;
+}
+__host__ __device__ inline int fdiv(const FastDiv& f, int n) {
+  return (int)(((unsigned long long)(unsigned)n * f.mul) >> f.sh);
+}
+
+// div_r(x) = x / g.r for x >= 0.
+template <typename DivR>
+__host__ __device__ inline RowIv row_intervals_with(const Geom& g, int sigma, DivR div_r) {
   RowIv v;
   if (sigma < g.s) {  // sink query: earlier sinks only
     v.hi_sink = sigma;
@@ -36,7 +56,7 @@ __host__ __device__ inline RowIv row_intervals(const Geom& g, int sigma) {
     v.hi_gist = -1;
   } else if (sigma < g.s + g.T) {  // raw query i of unit u
     const int i = sigma - g.s;
-    const int u = i / g.r;
+    const int u = div_r(i);
     const int u0 = u > g.k ? u - g.k : 0;
     v.hi_sink = g.s - 1;
     v.lo_raw = u0 * g.r;
@@ -52,6 +72,9 @@ __host__ __device__ inline RowIv row_intervals(const Geom& g, int sigma) {
     v.hi_gist = ug;
   }
   return v;
+}
+__host__ __device__ inline RowIv row_intervals(const Geom& g, int sigma) {
+  return row_intervals_with(g, sigma, [&](int x) { return x / g.r; });
 }
 
 __host__ __device__ inline bool visible(const Geom& g, const RowIv& v, int col_sigma) {
