@@ -726,6 +726,8 @@ attn_bwd_fused_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_sink, const
   const uint32_t full_q0 = bars + 72, empty_q0 = bars + 88 /* + 8 * st */, full_do = bars + 104, empty_do = bars + 120;
   const uint32_t tmem_slot = bars + 136;
   volatile uint32_t* tmem_slot_ptr = reinterpret_cast<volatile uint32_t*>(gen + SM::kOffBars + 136);
+  // number of Q tiles whose load the producer has issued so far (a scheduling hint for the dQ read-out, see there)
+  volatile int* q_issued = reinterpret_cast<volatile int*>(gen + SM::kOffBars + 144);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   // blockIdx.x = key tile rank * Hkv + KV head.  Sink and gist key tiles are seen by every later query:
@@ -767,6 +769,7 @@ attn_bwd_fused_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_sink, const
     }
     mbar_init(full_do, 1);
     mbar_init(empty_do, 1);
+    *q_issued = 0;
     mbar_fence_init();
   }
   if (warp == kFuMmaWarp) tmem_alloc(tmem_slot, 512);
@@ -848,6 +851,7 @@ attn_bwd_fused_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_sink, const
           for (int sl = 0; sl < 2; ++sl)
             tma_load_5d(sQ0 + st * SM::kTile + sl * SM::kSlab, mq, full_q0 + 8 * st, sl * 64, head, 0,
                         first_unit(qseg, qt * 128), b);
+          *q_issued = it + 1;
         }
         if (it + 1 < n_iter) fetch_stats(it + 1);
         if (it >= 1) ok = mbar_wait_warp(empty_do, (it - 1) & 1);  // one dO buffer: free once dV of the step before is done
@@ -966,28 +970,38 @@ attn_bwd_fused_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_sink, const
       ok = mbar_wait_warp(bar_dQ, it & 1);
       if (!ok) break;
       tc_fence_after();
-#pragma unroll
-      for (int c = 0; c < 2; ++c) {
-        const int col0 = 64 * half + 32 * c;
-        uint32_t v[32];
-        tmem_ld32(t_dP + lane_base + col0, v);
-        tmem_wait_ld();
-        if (c == 1) {  // this warp's columns are in registers: they may be overwritten
-          tc_fence_before();
-          mbar_arrive_relaxed(bar_dQfree);
-        }
-        // the reduction issued before has finished reading the staging buffer
+      uint32_t v[32];
+      const int col0 = 64 * half;
+      auto stage_rows = [&]() {  // the reduction issued before has finished reading the staging buffer
         if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
         __syncwarp();
 #pragma unroll
         for (int e = 0; e < 32; ++e) stage_gen[e * 32] = __uint_as_float(v[e]);
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         __syncwarp();
-        if (lane == 0 && col0 < nq) {  // rows past the segment's end are clipped by the tensor map
-          tma_reduce_add_4d(mdq, stage_sh, qd * 32, head, qt * 128 + col0, b);
+      };
+      auto reduce_rows = [&](int c0) {
+        if (lane == 0 && c0 < nq) {  // rows past the segment's end are clipped by the tensor map
+          tma_reduce_add_4d(mdq, stage_sh, qd * 32, head, qt * 128 + c0, b);
           asm volatile("cp.async.bulk.commit_group;" ::: "memory");
         }
-      }
+      };
+      tmem_ld32(t_dP + lane_base + col0, v);
+      tmem_wait_ld();
+      stage_rows();  // the first 32 queries wait in the staging buffer
+      tmem_ld32(t_dP + lane_base + col0 + 32, v);
+      tmem_wait_ld();
+      tc_fence_before();  // this warp's columns are in registers or staged: they may be overwritten
+      mbar_arrive_relaxed(bar_dQfree);
+      // The TMA unit takes its work in order, and a step's 16 reduce-adds keep it busy for about 1200 clocks.
+      // The Q tile of step it + 2 can be loaded once dK of this step is done, a few hundred clocks from now, and
+      // S of that step waits for it: let that load go first.  A hint only: bounded, and no error if it runs out.
+      if (lane == 0 && it + 2 < n_iter)
+        for (int spin = 0; spin < 4096 && *q_issued < it + 3; ++spin) __nanosleep(20);
+      __syncwarp();
+      reduce_rows(col0);
+      stage_rows();
+      reduce_rows(col0 + 32);
     }
     if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
     if (!ok && lane == 0) atomicExch(&g_bwd_timeout, 1u);
