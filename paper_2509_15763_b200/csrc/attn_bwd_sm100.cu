@@ -643,7 +643,7 @@ attn_bwd_dq_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const __g
 constexpr bool kFusedBackward = true;
 constexpr int kFuThreads = 640;
 constexpr int kFuTmaWarp = 16, kFuMmaWarp = 17;
-constexpr int kFuRegsLaunch = 96, kFuRegsCompute = 144, kFuRegsReadout = 64, kFuRegsOther = 64;
+constexpr int kFuRegsLaunch = 96, kFuRegsCompute = 128, kFuRegsReadout = 80, kFuRegsOther = 64;
 static_assert(kFuThreads * kFuRegsLaunch <= 65536 && kFuThreads * (kFuRegsLaunch + 8) > 65536,
               "launch register count is stale");
 static_assert(2 * kFuRegsCompute + 2 * kFuRegsReadout + kFuRegsOther <= 5 * kFuRegsLaunch,
@@ -970,9 +970,16 @@ attn_bwd_fused_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_sink, const
       ok = mbar_wait_warp(bar_dQ, it & 1);
       if (!ok) break;
       tc_fence_after();
-      uint32_t v[32];
+      // both halves of this warp's 64 query columns into registers, then the dQ^T columns are free again: the
+      // MMA warp never waits for the staging buffer or for the TMA unit
+      uint32_t v0[32], v1[32];
       const int col0 = 64 * half;
-      auto stage_rows = [&]() {  // the reduction issued before has finished reading the staging buffer
+      tmem_ld32(t_dP + lane_base + col0, v0);
+      tmem_ld32(t_dP + lane_base + col0 + 32, v1);
+      tmem_wait_ld();
+      tc_fence_before();
+      mbar_arrive_relaxed(bar_dQfree);
+      auto stage_rows = [&](const uint32_t (&v)[32]) {  // the reduction issued before has finished reading the staging buffer
         if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
         __syncwarp();
 #pragma unroll
@@ -986,13 +993,7 @@ attn_bwd_fused_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_sink, const
           asm volatile("cp.async.bulk.commit_group;" ::: "memory");
         }
       };
-      tmem_ld32(t_dP + lane_base + col0, v);
-      tmem_wait_ld();
-      stage_rows();  // the first 32 queries wait in the staging buffer
-      tmem_ld32(t_dP + lane_base + col0 + 32, v);
-      tmem_wait_ld();
-      tc_fence_before();  // this warp's columns are in registers or staged: they may be overwritten
-      mbar_arrive_relaxed(bar_dQfree);
+      stage_rows(v0);
       // The TMA unit takes its work in order, and a step's 16 reduce-adds keep it busy for about 1200 clocks.
       // The Q tile of step it + 2 can be loaded once dK of this step is done, a few hundred clocks from now, and
       // S of that step waits for it: let that load go first.  A hint only: bounded, and no error if it runs out.
@@ -1000,7 +1001,7 @@ attn_bwd_fused_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_sink, const
         for (int spin = 0; spin < 4096 && *q_issued < it + 3; ++spin) __nanosleep(20);
       __syncwarp();
       reduce_rows(col0);
-      stage_rows();
+      stage_rows(v1);
       reduce_rows(col0 + 32);
     }
     if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
