@@ -89,3 +89,40 @@ def test_docs_reject_bad_lists():
     p2 = ug.Problem(2, 16, 4, 8, 2, 2, 128)
     with pytest.raises(ug.UnigistError):
         ug.unigist_attn_fwd_docs(p2, [16], x, x, x, x, lse)  # batch must be 1
+
+
+def test_docs_calls_can_be_captured_in_a_cuda_graph():
+    """The runs of a packed sample fork onto the library's side streams and join again by events only, so
+    the whole forward + backward is capturable; a replay gives what the eager calls gave."""
+    s, r, W, doc_T, Hq, Hkv, D = 0, 4, 8, [256, 128, 64, 64, 192], 4, 2, 128
+    p = ug.Problem(1, doc_T[0], r, W, Hq, Hkv, D, num_sinks=s, flags=ug.FLAG_INTERLEAVED)
+    n_tot = ug.unigist_docs_total_len(p, doc_T)
+    dev = torch.device("cuda:0")
+    q, k, v, do = (t.to(dev) for t in _packed_inputs(n_tot, Hq, Hkv, D, 5))
+    o = torch.empty_like(q)
+    lse = torch.empty(Hq * n_tot, device=dev)
+    dq, dk, dv = torch.empty_like(q), torch.empty_like(k), torch.empty_like(v)
+    ws = torch.empty(max(ug.unigist_docs_workspace_bytes(p, ug.OP_BWD, doc_T), 16), dtype=torch.uint8, device=dev)
+
+    def run():
+        ug.unigist_attn_fwd_docs(p, doc_T, q, k, v, o, lse)
+        ug.unigist_attn_bwd_docs(p, doc_T, q, k, v, o, lse, do, dq, dk, dv, ws)
+
+    run()  # eager: also creates the side streams outside the capture
+    torch.cuda.synchronize()
+    want = [t.clone() for t in (o, lse, dk, dv)]
+    want_dq = dq.clone()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            run()
+    for t in (o, lse, dq, dk, dv):
+        t.zero_()
+    graph.replay()
+    torch.cuda.synchronize()
+    ug.unigist_device_status()
+    for got, ref in zip((o, lse, dk, dv), want):
+        assert torch.equal(got, ref)
+    assert (dq.float() - want_dq.float()).abs().max().item() <= 2.0 ** -7  # dQ: up to its summation order
