@@ -1,4 +1,6 @@
 // C-ABI entry points: argument validation, error reporting, dispatch to the kernel launchers.
+#include <algorithm>
+#include <vector>
 #include <atomic>
 #include <cmath>
 #include <cstdarg>
@@ -347,10 +349,26 @@ int32_t spread_doc_runs(const unigist_problem* p, int32_t num_docs, const int32_
     for (int i = 0; i < used; ++i)
       if (cudaStreamWaitEvent(ds.side[i], ds.fork, 0) != cudaSuccess) return fail(UNIGIST_ERR_CUDA, "cudaStreamWaitEvent failed");
   }
-  const int32_t rc = for_each_doc_run(p, num_docs, doc_raw_len, [&](const unigist_problem& run, int64_t base, int32_t i) {
-    const int lane = i % (1 + kSideStreams);
-    return fn(run, base, i, lane == 0 ? st : ds.side[lane - 1]);
+  // longest runs first (their launches fill the GPU; the short ones then run in their tails), streams round robin
+  struct Run {
+    unigist_problem p;
+    int64_t base;
+    int32_t index;
+  };
+  std::vector<Run> order;
+  order.reserve(runs);
+  for_each_doc_run(p, num_docs, doc_raw_len, [&](const unigist_problem& run, int64_t base, int32_t i) {
+    order.push_back(Run{run, base, i});
+    return (int32_t)UNIGIST_OK;
   });
+  std::stable_sort(order.begin(), order.end(), [](const Run& a, const Run& b) {
+    return (int64_t)a.p.raw_len * a.p.batch > (int64_t)b.p.raw_len * b.p.batch;
+  });
+  int32_t rc = UNIGIST_OK;
+  for (size_t j = 0; j < order.size() && rc == UNIGIST_OK; ++j) {
+    const int lane = (int)(j % (1 + kSideStreams));
+    rc = fn(order[j].p, order[j].base, order[j].index, lane == 0 ? st : ds.side[lane - 1]);
+  }
   // join even after an error, so that the caller's stream stays ordered after whatever was enqueued
   for (int i = 0; i < used; ++i) {
     if (cudaEventRecord(ds.join[i], ds.side[i]) != cudaSuccess || cudaStreamWaitEvent(st, ds.join[i], 0) != cudaSuccess)
