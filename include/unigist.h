@@ -119,18 +119,25 @@ int32_t unigist_gist_unshift(const unigist_problem* p, const void* src, void* ds
 
 /*
  * Position-encoding alignment (Section 4.1, step 3) applied as a rotary embedding to a bf16
- * [B, N, heads, D] device tensor in INTERLEAVED order: token t is rotated by its aligned position id
+ * [B, N, heads, D] device tensor (INTERLEAVED order unless a flag says otherwise): token t is rotated by its aligned position id
  * (sinks and raw tokens count 0, 1, 2, ...; a gist takes the id of the raw token right after it, the
  * last gist the id one past the last raw token), so distances between raw tokens are those of the
  * sequence without gists.  The paper fixes the ids, not the rotary convention; this is the one of the
  * Llama models it trains: feature j < D / 2 pairs with feature j + D / 2 and the pair turns by
  * id * theta_base^(-2 j / D).  Angles are formed in fp64, the rotation in fp32, one rounding to bf16.
- * flags = 0: dst has the order of src (dst == src, in place, is allowed).
- * flags = UNIGIST_ROPE_TO_SHIFTED: dst is written in SHIFTED order (Section 4.2), i.e. the rotation is
- * fused with unigist_gist_shift; src and dst must not overlap.
+ * flags (a combination):
+ *   UNIGIST_ROPE_TO_SHIFTED    dst is written in SHIFTED order (Section 4.2): the rotation fused with
+ *                              unigist_gist_shift;
+ *   UNIGIST_ROPE_FROM_SHIFTED  src is in SHIFTED order (with both flags the tensor stays shifted; with this one
+ *                              alone the rotation is fused with unigist_gist_unshift);
+ *   UNIGIST_ROPE_INVERSE       rotate by the negative angle: the transpose of the rotation, which is what the
+ *                              backward pass applies to the gradient of a rotated tensor.
+ * Where src and dst have the same order, dst == src (in place) is allowed; otherwise they must not overlap.
  * Errors: INVALID_ARG (NULL, heads < 1, theta_base <= 1, unknown flag, overlap), ALIGNMENT, CUDA.
  */
 #define UNIGIST_ROPE_TO_SHIFTED 1u
+#define UNIGIST_ROPE_FROM_SHIFTED 2u
+#define UNIGIST_ROPE_INVERSE 4u
 int32_t unigist_rope(const unigist_problem* p, const void* src, void* dst, int32_t heads, float theta_base,
                      uint32_t flags, void* stream);
 

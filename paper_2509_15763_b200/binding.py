@@ -254,7 +254,7 @@ def unigist_attn_bwd_docs(p: Problem, doc_raw_len, q, k, v, o, lse, d_o, dq, dk,
                                        _ptr(workspace), workspace.numel() * workspace.element_size(), _stream(stream)))
 
 
-ROPE_TO_SHIFTED = 1
+ROPE_TO_SHIFTED, ROPE_FROM_SHIFTED, ROPE_INVERSE = 1, 2, 4
 
 
 def unigist_rope(p: Problem, src, dst, theta_base: float, flags: int = 0, stream=None):

@@ -215,16 +215,18 @@ int32_t unigist_rope(const unigist_problem* p, const void* src, void* dst, int32
   Geom g;
   if (int32_t rc = check_problem(p, &g, nullptr)) return rc;
   if (!src || !dst) return fail(UNIGIST_ERR_INVALID_ARG, "src/dst is NULL");
-  if (heads < 1 || !(theta_base > 1.f) || (flags & ~UNIGIST_ROPE_TO_SHIFTED))
-    return fail(UNIGIST_ERR_INVALID_ARG, "heads must be >= 1, theta_base > 1, flags 0 or UNIGIST_ROPE_TO_SHIFTED");
+  if (heads < 1 || !(theta_base > 1.f) || (flags & ~(UNIGIST_ROPE_TO_SHIFTED | UNIGIST_ROPE_FROM_SHIFTED | UNIGIST_ROPE_INVERSE)))
+    return fail(UNIGIST_ERR_INVALID_ARG, "heads must be >= 1, theta_base > 1, flags a combination of UNIGIST_ROPE_*");
   if (!aligned16(src) || !aligned16(dst)) return fail(UNIGIST_ERR_ALIGNMENT, "pointers must be 16-byte aligned");
-  const bool to_shifted = (flags & UNIGIST_ROPE_TO_SHIFTED) != 0;
+  const bool to_shifted = (flags & UNIGIST_ROPE_TO_SHIFTED) != 0, from_shifted = (flags & UNIGIST_ROPE_FROM_SHIFTED) != 0;
+  const bool same_order = to_shifted == from_shifted;  // a row is read and written at the same place
   const char* a = (const char*)src;
   const char* b = (const char*)dst;
   const size_t tot = (size_t)heads * p->head_dim * 2 * g.N * p->batch;
-  if ((to_shifted || a != b) && a < b + tot && b < a + tot)
-    return fail(UNIGIST_ERR_INVALID_ARG, "src and dst overlap (in place is allowed only without the shift)");
-  return launch_rope(g, p->batch, heads, p->head_dim, theta_base, to_shifted, src, dst, (cudaStream_t)stream);
+  if ((!same_order || a != b) && a < b + tot && b < a + tot)
+    return fail(UNIGIST_ERR_INVALID_ARG, "src and dst overlap (in place is allowed only where the order does not change)");
+  return launch_rope(g, p->batch, heads, p->head_dim, theta_base, to_shifted, from_shifted,
+                     (flags & UNIGIST_ROPE_INVERSE) != 0, src, dst, (cudaStream_t)stream);
 }
 
 int32_t unigist_attn_fwd(const unigist_problem* p, const void* q, const void* k, const void* v,

@@ -21,7 +21,7 @@ __device__ __forceinline__ int aligned_pos(const Geom& g, int t) {
 // for every head.
 template <int D>
 __global__ void __launch_bounds__(256)
-rope_kernel(Geom g, long long tokens, int heads, double log2_theta, int to_shifted,
+rope_kernel(Geom g, long long tokens, int heads, double log2_theta, int to_shifted, int from_shifted, int inverse,
             const __nv_bfloat16* __restrict__ src, __nv_bfloat16* __restrict__ dst) {
   constexpr int kLanesPerRow = D / 8, kRowsPerPass = 32 / kLanesPerRow;
   const int lane = threadIdx.x & 31;
@@ -41,9 +41,11 @@ rope_kernel(Geom g, long long tokens, int heads, double log2_theta, int to_shift
       double a = pos * inv_freq[e];
       a -= 6.283185307179586476925 * rint(a * 0.15915494309189533577);  // into [-pi, pi]
       sincosf((float)a, &sn[e], &cs[e]);
+      if (inverse) sn[e] = -sn[e];  // the transpose of the rotation: what the backward pass applies to a gradient
     }
-    const long long out_tk = b * g.N + (to_shifted ? unshift_perm(g, t) : t);
-    const __nv_bfloat16* s_tok = src + tk * heads * D;
+    const int sigma = (to_shifted | from_shifted) ? unshift_perm(g, t) : t;  // the token's shifted position
+    const long long out_tk = b * g.N + (to_shifted ? sigma : t);
+    const __nv_bfloat16* s_tok = src + (b * g.N + (from_shifted ? sigma : t)) * heads * D;
     __nv_bfloat16* d_tok = dst + out_tk * heads * D;
     for (int h0 = 0; h0 < heads; h0 += 2 * kRowsPerPass) {  // two passes in flight
       uint2 lo[2], hi[2];
@@ -87,8 +89,8 @@ rope_kernel(Geom g, long long tokens, int heads, double log2_theta, int to_shift
 
 }  // namespace
 
-int32_t launch_rope(const Geom& g, int B, int heads, int D, float theta_base, bool to_shifted, const void* src,
-                    void* dst, cudaStream_t st) {
+int32_t launch_rope(const Geom& g, int B, int heads, int D, float theta_base, bool to_shifted, bool from_shifted,
+                    bool inverse, const void* src, void* dst, cudaStream_t st) {
   const long long tokens = (long long)B * g.N;
   const long long want = (tokens + 7) / 8;  // 8 warps per block
   const int blocks = (int)(want < 148 * 8 ? (want > 0 ? want : 1) : 148 * 8);
@@ -96,10 +98,10 @@ int32_t launch_rope(const Geom& g, int B, int heads, int D, float theta_base, bo
   {
     KernelScope ks("rope_kernel", st);
     if (D == 128)
-      rope_kernel<128><<<blocks, 256, 0, st>>>(g, tokens, heads, log2_theta, to_shifted ? 1 : 0,
+      rope_kernel<128><<<blocks, 256, 0, st>>>(g, tokens, heads, log2_theta, to_shifted ? 1 : 0, from_shifted ? 1 : 0, inverse ? 1 : 0,
                                                  (const __nv_bfloat16*)src, (__nv_bfloat16*)dst);
     else
-      rope_kernel<64><<<blocks, 256, 0, st>>>(g, tokens, heads, log2_theta, to_shifted ? 1 : 0,
+      rope_kernel<64><<<blocks, 256, 0, st>>>(g, tokens, heads, log2_theta, to_shifted ? 1 : 0, from_shifted ? 1 : 0, inverse ? 1 : 0,
                                                 (const __nv_bfloat16*)src, (__nv_bfloat16*)dst);
   }
   return check_launch("rope kernel");

@@ -134,8 +134,8 @@ inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
 
 // Kernel launchers (one per .cu file).
 int32_t launch_layout(const Geom& g, int32_t* sp, int32_t* up, int32_t* pos, cudaStream_t st);
-int32_t launch_rope(const Geom& g, int B, int heads, int D, float theta_base, bool to_shifted, const void* src,
-                    void* dst, cudaStream_t st);
+int32_t launch_rope(const Geom& g, int B, int heads, int D, float theta_base, bool to_shifted, bool from_shifted,
+                    bool inverse, const void* src, void* dst, cudaStream_t st);
 int32_t launch_shift(const Geom& g, int B, const void* src, void* dst, size_t row_bytes,
                      bool inverse, cudaStream_t st);
 // Where the query rows of a forward call sit.  A whole-sequence call has queries for every row

@@ -58,3 +58,38 @@ def test_rope_rejects_overlap_with_shift():
     x = torch.zeros(1, ug.unigist_total_len(p), 1, 128, dtype=torch.bfloat16, device="cuda")
     with pytest.raises(ug.UnigistError):
         ug.unigist_rope(p, x, x, 10000.0, ug.ROPE_TO_SHIFTED)
+
+
+def test_rope_inverse_and_shifted_source():
+    """The inverse flag is the transposed rotation (what a backward pass applies); a shifted source gives
+    the same rows as an interleaved one."""
+    s, T, r, H, D, B, theta = 3, 120, 4, 2, 128, 1, 500000.0
+    p = ug.Problem(batch=B, raw_len=T, num_sinks=s, ratio=r, window=r, num_q_heads=H, num_kv_heads=H, head_dim=D)
+    N = ug.unigist_total_len(p)
+    g = torch.Generator().manual_seed(9)
+    x = torch.randn(B, N, H, D, generator=g).to(torch.bfloat16)
+    dy = torch.randn(B, N, H, D, generator=g).to(torch.bfloat16)
+    sp, up, pos = oracle.layout(s, T, r)
+    xd, dyd = x.cuda(), dy.cuda()
+    # the transposed rotation against the oracle rotating by the negated ids
+    dx = torch.empty_like(dyd)
+    ug.unigist_rope(p, dyd, dx, theta, ug.ROPE_INVERSE)
+    want = oracle.rope(dy[0].double().numpy(), -pos.astype(np.int64), theta)
+    got = dx[0].cpu().double().numpy()
+    assert (np.abs(got - want) <= 2.0 ** -8 * np.maximum(np.abs(want), 1e-2) + 1e-6).all()
+    # <R x, dy> = <x, R^T dy> up to the bf16 rounding of the two results
+    y = torch.empty_like(xd)
+    ug.unigist_rope(p, xd, y, theta, 0)
+    lhs = (y.double() * dyd.double()).sum().item()
+    rhs = (xd.double() * dx.double()).sum().item()
+    assert abs(lhs - rhs) <= 2e-3 * (y.double().abs() * dyd.double().abs()).sum().item() ** 0.5 + 1e-2 * abs(lhs)
+    # shifted in, interleaved out (fused unshift), and shifted in, shifted out: the same rows as from interleaved input
+    xs = xd[:, torch.from_numpy(sp.astype(np.int64)).cuda()].contiguous()
+    a = torch.empty_like(xd)
+    ug.unigist_rope(p, xs, a, theta, ug.ROPE_FROM_SHIFTED)
+    assert torch.equal(a, y)
+    b = torch.empty_like(xd)
+    ug.unigist_rope(p, xs, b, theta, ug.ROPE_FROM_SHIFTED | ug.ROPE_TO_SHIFTED)
+    assert torch.equal(b, y[:, torch.from_numpy(sp.astype(np.int64)).cuda()])
+    ug.unigist_rope(p, xs, xs, theta, ug.ROPE_FROM_SHIFTED | ug.ROPE_TO_SHIFTED)  # in place: the order does not change
+    assert torch.equal(xs, b)

@@ -62,3 +62,13 @@ def test_gist_shares_the_angle_of_the_next_raw_token():
         g = u * (r + 1) + r
         assert np.allclose(y[g], y[g + 1])
     assert np.allclose(y[0], x[0])  # id 0: no rotation
+
+
+def test_negated_ids_undo_the_rotation():
+    # the rotation is orthogonal: rotating by the negated ids is its transpose and its inverse
+    s, T, r, D, H = 2, 12, 4, 8, 2
+    _, _, pos = oracle.layout(s, T, r)
+    x, dy = _rand((oracle.total_len(s, T, r), H, D), 5), _rand((oracle.total_len(s, T, r), H, D), 6)
+    y = oracle.rope(x, pos, 10000.0)
+    assert np.allclose(oracle.rope(y, -pos.astype(np.int64), 10000.0), x, atol=1e-12)
+    assert np.isclose((y * dy).sum(), (x * oracle.rope(dy, -pos.astype(np.int64), 10000.0)).sum())
