@@ -22,46 +22,69 @@ constexpr float kLog2e = 1.4426950408889634f;
 __device__ unsigned int g_bwd_timeout = 0;
 
 // ------------------------------------------------------------------------------------------------
-// Delta and dO conversion: one warp per (batch, token, head) row, 4 elements per lane and pass.
+// Delta and dO conversion: one warp per token.  The token's batch index and shifted position are worked out
+// once (the divisions cost more than a row's loads), then its Hq rows go by four at a time, all loads of the
+// four issued before the first use; 4 elements per lane and pass.
 template <bool kF32>
 __global__ void __launch_bounds__(256)
-bwd_prep_kernel(Geom g, int interleaved, int Hq, int D, long long rows, const void* __restrict__ d_o,
+bwd_prep_kernel(Geom g, int interleaved, int Hq, int D, long long tokens, const void* __restrict__ d_o,
                 const __nv_bfloat16* __restrict__ o, float* __restrict__ delta,
                 __nv_bfloat16* __restrict__ d_o_bf16, float* __restrict__ dq32) {
+  constexpr int kHeads = 4;  // rows in flight
   const int lane = threadIdx.x & 31;
   const long long warp = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const long long nwarps = ((long long)gridDim.x * blockDim.x) >> 5;
-  for (long long rw = warp; rw < rows; rw += nwarps) {  // rw = (b*N + t)*Hq + h
-    float acc = 0.f;
-    for (int d = lane * 4; d < D; d += 128) {
-      // the fused backward accumulates dQ into this fp32 buffer: start it at zero
-      if (dq32) __stcs(reinterpret_cast<float4*>(dq32 + rw * D + d), make_float4(0.f, 0.f, 0.f, 0.f));
-      uint2 dbits;  // 4 bf16 of dO
-      if (kF32) {
-        const float4 t = __ldcs(reinterpret_cast<const float4*>(reinterpret_cast<const float*>(d_o) + rw * D + d));
-        const __nv_bfloat162 lo = __floats2bfloat162_rn(t.x, t.y), hi = __floats2bfloat162_rn(t.z, t.w);
-        dbits.x = *reinterpret_cast<const uint32_t*>(&lo);
-        dbits.y = *reinterpret_cast<const uint32_t*>(&hi);
-        *reinterpret_cast<uint2*>(d_o_bf16 + rw * D + d) = dbits;
-      } else {
-        dbits = *reinterpret_cast<const uint2*>(reinterpret_cast<const __nv_bfloat16*>(d_o) + rw * D + d);
-      }
-      const uint2 obits = *reinterpret_cast<const uint2*>(o + rw * D + d);
-      // a bf16 is the high half of an fp32
-      acc += __uint_as_float(dbits.x << 16) * __uint_as_float(obits.x << 16) +
-             __uint_as_float(dbits.x & 0xffff0000u) * __uint_as_float(obits.x & 0xffff0000u) +
-             __uint_as_float(dbits.y << 16) * __uint_as_float(obits.y << 16) +
-             __uint_as_float(dbits.y & 0xffff0000u) * __uint_as_float(obits.y & 0xffff0000u);
-    }
+  for (long long tk = warp; tk < tokens; tk += nwarps) {  // tk = b * N + t
+    const long long b = tk / g.N;
+    const int t = (int)(tk - b * g.N);
+    // Delta is kept in shifted order, whatever the order of dO and O
+    float* delta_tok = delta + b * Hq * g.N + (interleaved ? unshift_perm(g, t) : t);
+    const long long row0 = tk * Hq;
+    for (int h0 = 0; h0 < Hq; h0 += kHeads) {
+      float acc[kHeads];
 #pragma unroll
-    for (int off = 16; off >= 1; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
-    if (lane == 0) {
-      const int h = (int)(rw % Hq);
-      const long long bt = rw / Hq;
-      const int t = (int)(bt % g.N);
-      const long long b = bt / g.N;
-      // Delta is kept in shifted order, whatever the order of dO and O
-      delta[(b * Hq + h) * g.N + (interleaved ? unshift_perm(g, t) : t)] = acc;
+      for (int u = 0; u < kHeads; ++u) acc[u] = 0.f;
+      for (int d = lane * 4; d < D; d += 128) {
+        uint2 dbits[kHeads], obits[kHeads];  // 4 bf16 of dO and of O
+#pragma unroll
+        for (int u = 0; u < kHeads; ++u) {
+          if (h0 + u >= Hq) continue;
+          const long long at = (row0 + h0 + u) * D + d;
+          if (kF32) {
+            const float4 x = __ldcs(reinterpret_cast<const float4*>(reinterpret_cast<const float*>(d_o) + at));
+            const __nv_bfloat162 lo = __floats2bfloat162_rn(x.x, x.y), hi = __floats2bfloat162_rn(x.z, x.w);
+            dbits[u].x = *reinterpret_cast<const uint32_t*>(&lo);
+            dbits[u].y = *reinterpret_cast<const uint32_t*>(&hi);
+          } else {
+            dbits[u] = *reinterpret_cast<const uint2*>(reinterpret_cast<const __nv_bfloat16*>(d_o) + at);
+          }
+          obits[u] = *reinterpret_cast<const uint2*>(o + at);
+        }
+#pragma unroll
+        for (int u = 0; u < kHeads; ++u) {
+          if (h0 + u >= Hq) continue;
+          const long long at = (row0 + h0 + u) * D + d;
+          // the fused backward accumulates dQ into this fp32 buffer: start it at zero
+          if (dq32) __stcs(reinterpret_cast<float4*>(dq32 + at), make_float4(0.f, 0.f, 0.f, 0.f));
+          if (kF32) *reinterpret_cast<uint2*>(d_o_bf16 + at) = dbits[u];
+          // a bf16 is the high half of an fp32
+          acc[u] += __uint_as_float(dbits[u].x << 16) * __uint_as_float(obits[u].x << 16) +
+                    __uint_as_float(dbits[u].x & 0xffff0000u) * __uint_as_float(obits[u].x & 0xffff0000u) +
+                    __uint_as_float(dbits[u].y << 16) * __uint_as_float(obits[u].y << 16) +
+                    __uint_as_float(dbits[u].y & 0xffff0000u) * __uint_as_float(obits[u].y & 0xffff0000u);
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < kHeads; ++u) {
+#pragma unroll
+        for (int off = 16; off >= 1; off >>= 1) acc[u] += __shfl_xor_sync(0xffffffffu, acc[u], off);
+      }
+      if (lane < kHeads && h0 + lane < Hq) {
+        float mine = acc[0];
+#pragma unroll
+        for (int u = 1; u < kHeads; ++u) mine = lane == u ? acc[u] : mine;
+        delta_tok[(long long)(h0 + lane) * g.N] = mine;
+      }
     }
   }
 }
@@ -1175,13 +1198,13 @@ int32_t launch_bwd_sm100(const Geom& g, const unigist_problem& p, float scale, c
   const bool fused = kFusedBackward && D == 128;  // head_dim 64 keeps the two-kernel path
   float* dq32 = fused ? reinterpret_cast<float*>(static_cast<char*>(workspace) + delta_bytes + do_bytes) : nullptr;
   {
-    const long long rows = (long long)B * g.N * Hq;
-    const int blocks = (int)((rows + 7) / 8 < 148 * 16 ? (rows + 7) / 8 : 148 * 16);
+    const long long tokens = (long long)B * g.N;
+    const int blocks = (int)((tokens + 7) / 8 < 148 * 16 ? (tokens + 7) / 8 : 148 * 16);
     KernelScope ks("bwd_prep_kernel", st);
     if (f32)
-      bwd_prep_kernel<true><<<blocks, 256, 0, st>>>(g, il ? 1 : 0, Hq, D, rows, d_o, (const __nv_bfloat16*)o, delta, do_bf16, dq32);
+      bwd_prep_kernel<true><<<blocks, 256, 0, st>>>(g, il ? 1 : 0, Hq, D, tokens, d_o, (const __nv_bfloat16*)o, delta, do_bf16, dq32);
     else
-      bwd_prep_kernel<false><<<blocks, 256, 0, st>>>(g, il ? 1 : 0, Hq, D, rows, d_o, (const __nv_bfloat16*)o, delta, nullptr, dq32);
+      bwd_prep_kernel<false><<<blocks, 256, 0, st>>>(g, il ? 1 : 0, Hq, D, tokens, d_o, (const __nv_bfloat16*)o, delta, nullptr, dq32);
   }
   if (int32_t rc = check_launch("backward prep kernel")) return rc;
 
