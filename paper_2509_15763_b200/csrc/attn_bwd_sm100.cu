@@ -729,7 +729,7 @@ attn_bwd_fused_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_sink, const
                             const __grid_constant__ CUtensorMap tm_dq_gist, Geom g, int Hq, int Hkv, float scale,
                             const float* __restrict__ lse, const float* __restrict__ delta,
                             __nv_bfloat16* __restrict__ dk, __nv_bfloat16* __restrict__ dv, int n_sink_kt, int n_gist_kt,
-                            int interleaved) {
+                            int interleaved, FastDiv gdiv, FastDiv rdiv) {
   using SM = FuSmem;
   constexpr int D = 128;
   extern __shared__ unsigned char smem_dyn[];
@@ -807,7 +807,7 @@ attn_bwd_fused_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_sink, const
   // G heads of a tile back to back.  Every key tile's visible range ends at the last tile of a segment, so
   // thread blocks that run side by side walk the same Q / dO / dQ tiles at the same time and share them in L2.
   auto tile_of = [&](int it, int& qseg, int& qt, int& head) {
-    const int t = it / G;
+    const int t = fdiv(gdiv, it);  // it / G: on the producer's path to every Q load
     head = hk * G + (it - t * G);
     if (t < n_raw_q) {
       qseg = kSegRaw;
@@ -826,7 +826,7 @@ attn_bwd_fused_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_sink, const
     if (warp == kFuTmaWarp) {
       // ---------------------------------------------------------- producer: K, V once; Q, dO, LSE, Delta per step
       // tile coordinate: its first unit (a raw tile of an interleaved tensor spans 128 / r gist units)
-      auto first_unit = [&](int sg, int row0) { return interleaved && sg == kSegRaw ? row0 / g.r : row0; };
+      auto first_unit = [&](int sg, int row0) { return interleaved && sg == kSegRaw ? fdiv(rdiv, row0) : row0; };
       if (lane == 0) {
         mbar_arrive_expect_tx(bar_kv, 2 * SM::kTile);
         const CUtensorMap* mk = kseg == kSegRaw ? &tm_k_raw : (kseg == kSegGist ? &tm_k_gist : &tm_k_sink);
@@ -1270,7 +1270,8 @@ int32_t launch_bwd_sm100(const Geom& g, const unigist_problem& p, float scale, c
     KernelScope ks("attn_bwd_fused_sm100_kernel", st);
     attn_bwd_fused_sm100_kernel<<<dim3((n_sink_t + n_raw_t + n_gist_t) * Hkv, 1, B), kFuThreads, FuSmem::kBytes, st>>>(
         fq[0], fq[1], fq[2], fdo[0], fdo[1], fdo[2], fk[0], fk[1], fk[2], fv[0], fv[1], fv[2], mdq[0], mdq[1], mdq[2], g,
-        Hq, Hkv, scale, lse, delta, (__nv_bfloat16*)dk, (__nv_bfloat16*)dv, n_sink_t, n_gist_t, il ? 1 : 0);
+        Hq, Hkv, scale, lse, delta, (__nv_bfloat16*)dk, (__nv_bfloat16*)dv, n_sink_t, n_gist_t, il ? 1 : 0, make_fastdiv(Hq / Hkv),
+        make_fastdiv(g.r));
   }
   if (int32_t rc = check_launch("tcgen05 fused backward kernel")) return rc;
   {
