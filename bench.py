@@ -38,8 +38,8 @@ UNIT = "TFLOP/s"
 # DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures
 # summarised under profiles/, keyed by (kernel, workload); None until a capture exists.
 NCU_TRAFFIC_BYTES = {
-    ("attn_fwd_sm100_kernel", "llama8b_layer"): 354265000,
-    ("attn_bwd_fused_sm100_kernel", "llama8b_layer"): 5058844000,
+    ("attn_fwd_sm100_kernel", "llama8b_layer"): 353900000,
+    ("attn_bwd_fused_sm100_kernel", "llama8b_layer"): 4827655000,
 }
 
 # FLOP per visible pair per query head that each attention kernel performs algorithmically,
