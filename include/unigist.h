@@ -179,6 +179,7 @@ int32_t unigist_attn_bwd(const unigist_problem* p, const void* q, const void* k,
  * over `stream` and three side streams of the library that fork from `stream` and join it again before the call
  * returns (events only, so the call can be captured in a CUDA graph); each run has its own slice of the
  * workspace (unigist_docs_workspace_bytes: the sum over the runs).
+ * The side streams are created at the first call, on the device current then: one process drives one GPU.
  * Errors as for unigist_attn_fwd / unigist_attn_bwd, raised before the first launch where the list is malformed.
  */
 int64_t unigist_docs_total_len(const unigist_problem* p, int32_t num_docs, const int32_t* doc_raw_len);
