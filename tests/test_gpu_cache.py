@@ -85,6 +85,57 @@ def test_compaction_matches_oracle(B, s, T, r, W, Hkv, D, mode):
         assert torch.equal(kc_d.cpu()[spare], kc[spare])
 
 
+@pytest.mark.parametrize("mode", ["gather_interleaved", "inplace"])
+def test_compaction_of_the_long_prefill_at_full_size(mode):
+    """The prefill workload's second half (Section 4.3): after the 131072-token prompt, the cache keeps the 8192
+    gists and the last 4096 raw tokens of 139264.  Both routes a caller has at that size: the gather out of the
+    interleaved K / V tensors (what the benchmark step does) and the in-place compaction of a paged cache that
+    holds the whole shifted sequence (every segment is page aligned: a block-table edit).  Indices bit-exact
+    against the oracle's brute-force kept set, pages byte-equal to the source rows."""
+    w = synth.WORKLOADS["long_prefill"]
+    s, T, r, Hkv, D = w.num_sinks, w.raw_len, w.ratio, w.num_kv_heads, w.head_dim
+    il = mode == "gather_interleaved"
+    p = ug.Problem(1, T, r, w.window, w.num_q_heads, Hkv, D, num_sinks=s, flags=ug.FLAG_INTERLEAVED if il else 0)
+    N, L = ug.unigist_total_len(p), ug.unigist_compact_len(p)
+    assert (N, L) == (139264, 12288)
+    kept = oracle.kept_set(s, T, r, oracle.window_units(w.window, r))  # interleaved indices, cache order
+    sp, up, _ = oracle.layout(s, T, r)
+    want_idx = torch.from_numpy(up[kept]).long()
+    assert len(kept) == L
+    g = torch.Generator().manual_seed(w.seed + 1000)
+    k_il = torch.randn(1, N, Hkv, D, generator=g).to(torch.bfloat16)  # interleaved order (Eq. 2)
+    v_il = torch.randn(1, N, Hkv, D, generator=g).to(torch.bfloat16)
+    k_sh, v_sh = k_il[:, torch.from_numpy(sp).long()], v_il[:, torch.from_numpy(sp).long()]
+    nbN, nbL = N // PG, L // PG
+    per_seq = nbL if il else nbN
+    nblocks = per_seq + 5
+    table = torch.randperm(nblocks, generator=g)[:per_seq].to(torch.int32).reshape(1, per_seq)
+    kc = torch.zeros(nblocks, Hkv, PG, D, dtype=torch.bfloat16)
+    vc = torch.zeros_like(kc)
+    if not il:  # the cache holds the whole shifted sequence, logical position = shifted position
+        for src, dst in ((k_sh, kc), (v_sh, vc)):
+            dst[table[0].long()] = src[0].reshape(nbN, PG, Hkv, D).permute(0, 2, 1, 3)
+    kc_d, vc_d, table_d = kc.to(DEV), vc.to(DEV), table.to(DEV)
+    lens = torch.zeros(1, dtype=torch.int32, device=DEV)
+    kept_idx = torch.full((1, L), -1, dtype=torch.int32, device=DEV)
+    before = ug.unigist_launch_count()
+    if il:
+        ug.unigist_kv_compact(p, k_il.to(DEV), v_il.to(DEV), kc_d, vc_d, table_d, lens, kept_idx)
+    else:
+        ug.unigist_kv_compact(p, None, None, kc_d, vc_d, table_d, lens, kept_idx)
+    torch.cuda.synchronize()
+    assert ug.unigist_launch_count() == before + 1
+    assert lens.cpu().tolist() == [L]
+    assert np.array_equal(kept_idx.cpu().numpy()[0], want_idx.numpy())
+    new_table = table_d.cpu()
+    assert sorted(new_table[0].tolist()) == sorted(table[0].tolist())  # a permutation of the row
+    for cache, src in ((kc_d, k_sh), (vc_d, v_sh)):
+        assert torch.equal(read_cache(cache.cpu(), new_table[0], L), src[0, want_idx])
+    if not il:  # no token moved: the cache bytes are what they were, and the freed blocks are listed after the kept ones
+        assert torch.equal(kc_d.cpu(), kc) and torch.equal(vc_d.cpu(), vc)
+        assert len(set(new_table[0, nbL:].tolist()) & set(new_table[0, :nbL].tolist())) == 0
+
+
 def run_decode(inp, lens=None):
     d = {k: v.to(DEV) for k, v in inp.items()}
     if lens is not None:
@@ -119,6 +170,17 @@ def test_decode_matches_oracle(S, Hq, Hkv, gists, window):
     lens = [max(1, w.seq_len - 13 * i) for i in range(S)]  # ragged lengths
     o, lse, lens = run_decode(inp, lens)
     check_decode(inp, o, lse, lens, range(S))
+
+
+def test_decode_of_an_empty_sequence_is_zero_not_nan():
+    """A padding slot of a decode batch (length 0) attends to nothing: O = 0 and LSE = -inf there, and the
+    other sequences of the batch are not disturbed."""
+    w = synth.DecodeWorkload("pad", 3, 200, 30, 8, 2, 128, seed=310)
+    inp = synth.decode_inputs(w, spare_blocks=1)
+    o, lse, lens = run_decode(inp, [w.seq_len, 0, 77])
+    assert torch.equal(o[1].float(), torch.zeros_like(o[1].float()))
+    assert torch.isinf(lse[1]).all() and (lse[1] < 0).all()
+    check_decode(inp, o, lse, lens, [0, 2])
 
 
 def test_decode_full_size_sampled():

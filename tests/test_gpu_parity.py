@@ -141,10 +141,26 @@ def test_forward_is_deterministic():
 
 
 # ------------------------------------------------------------------ full-size workloads, sampled outputs
-def _sample_rows(N, rng, blocks=6, width=16):
-    starts = [0, N - width] + list(rng.integers(0, N - width, size=blocks))
-    rows = sorted({int(s0) + i for s0 in starts for i in range(width)})
-    return np.array(rows, dtype=np.int64)
+def _edge_positions(s, T, r, k):
+    """SHIFTED positions of the rows / keys the 128-row tile kernels branch on: the first and last row of the first
+    tile of each segment, of the tile in which the window starts to clip (raw row (k + 1) r, gist k + 1), of a middle
+    tile and of the last tile, the rows on either side of the clipping point, a row inside a tile, and the sinks' ends."""
+    n = T // r
+    pos = set()
+
+    def tiles(base, length, first_clipped):
+        last_tile = (length - 1) // 128
+        for j in {0, min(first_clipped // 128, last_tile), last_tile // 2, last_tile}:
+            pos.update(base + x for x in (128 * j, min(128 * j + 127, length - 1)))
+        for x in (first_clipped - 1, first_clipped, length // 3 + 5):
+            if 0 <= x < length:
+                pos.add(base + x)
+
+    tiles(s, T, (k + 1) * r)      # raw rows: unit k + 1 is the first whose window no longer reaches unit 0
+    tiles(s + T, n, k + 1)        # gist rows
+    if s:
+        pos.update((0, s - 1))
+    return np.array(sorted(pos), dtype=np.int64)
 
 
 @pytest.mark.parametrize("name,backward,route", [("llama8b_layer", True, "explicit"), ("train_batch", True, "explicit"),
@@ -163,28 +179,40 @@ def test_full_size_sampled(name, backward, route):
     N, G = w.total_len, w.num_q_heads // w.num_kv_heads
     scale = w.head_dim ** -0.5
     rng = np.random.default_rng(w.seed)
-    b, hk = w.batch - 1, int(rng.integers(0, w.num_kv_heads))
-    hs = slice(hk * G, (hk + 1) * G)
-    q, kk, v = f64(inp["q"][b, :, hs]), f64(inp["k"][b, :, hk]), f64(inp["v"][b, :, hk])
-    # forward: blocks of rows, among them the first units, the window edge and the tail
-    o_gpu, lse_gpu = f64(out["o"][b, :, hs]), f64(out["lse"][b, hs])
-    for r0 in [0, (k + 1) * (r + 1) - 8, N // 2 + 3, N - 16]:
-        o, lse = oracle.attn_fwd_slice(s, T, r, k, scale, q, kk, v, r0, r0 + 16)
-        check_close(f"O rows {r0}", o_gpu[r0:r0 + 16], o, TOL_O_MAX, TOL_O_MEAN)
-        check_close(f"LSE rows {r0}", lse_gpu[:, r0:r0 + 16].T, lse, TOL_LSE)
+    sp, _, _ = oracle.layout(s, T, r)
+    edge = sp[_edge_positions(s, T, r, min(k, T // r))].astype(np.int64)  # interleaved indices of the edge rows
+    hk0 = int(rng.integers(0, w.num_kv_heads))
+    kv_heads = sorted({hk0, (hk0 + max(1, w.num_kv_heads // 2)) % w.num_kv_heads})
     # no row anywhere was left unwritten
     assert torch.isfinite(out["lse_shifted"]).all()
     assert torch.isfinite(out["o_shifted" if route == "explicit" else "o"].float()).all()
+    if backward:
+        for n in ("dq", "dk", "dv"):
+            assert torch.isfinite(out[n + "_shifted" if route == "explicit" else n].float()).all(), n
+    # forward: every batch index, two KV heads; the edge rows one by one and three blocks of 16 consecutive rows
+    for b in range(w.batch):
+        for hk in kv_heads:
+            hs = slice(hk * G, (hk + 1) * G)
+            q, kk, v = f64(inp["q"][b, :, hs]), f64(inp["k"][b, :, hk]), f64(inp["v"][b, :, hk])
+            o_gpu, lse_gpu = f64(out["o"][b, :, hs]), f64(out["lse"][b, hs])
+            blocks = [(int(t), int(t) + 1) for t in edge]
+            blocks += [(r0, r0 + 16) for r0 in (0, int(rng.integers(16, N - 32)), N - 16)]
+            for r0, r1 in blocks:
+                o, lse = oracle.attn_fwd_slice(s, T, r, k, scale, q, kk, v, r0, r1)
+                check_close(f"O b{b} hk{hk} rows {r0}:{r1}", o_gpu[r0:r1], o, TOL_O_MAX, TOL_O_MEAN if r1 - r0 > 1 else None)
+                check_close(f"LSE b{b} hk{hk} rows {r0}:{r1}", lse_gpu[:, r0:r1].T, lse, TOL_LSE)
     if not backward:
         return
-    do = f64(inp["dout"][b, :, hs])
-    rows = np.concatenate([np.arange(0, 8), np.arange(N // 3, N // 3 + 8), np.arange(N - 8, N)])
-    last_gist = N - 1
-    keys = np.array([0, 1, r, (r + 1) * 5 + 2, N // 2, N // 2 + 1, N - 2 - (r + 1) * 3,
-                     last_gist - 40 * (r + 1), last_gist, N - 2], dtype=np.int64)
-    dq, dk, dv = oracle.attn_bwd_sample(s, T, r, k, scale, q, kk, v, do, rows, keys)
-    check_close("dQ rows", f64(out["dq"][b, rows][:, hs]), dq, TOL_GRAD)
-    check_close("dK keys", f64(out["dk"][b, keys, hk]), dk, TOL_GRAD)
-    check_close("dV keys", f64(out["dv"][b, keys, hk]), dv, TOL_GRAD)
-    for n in ("dq", "dk", "dv"):
-        assert torch.isfinite(out[n + "_shifted" if route == "explicit" else n].float()).all(), n
+    # backward: first and last batch index, the same two KV heads; dQ of the edge rows, dK / dV of the edge keys (among
+    # them gist keys, which every later row sees: the oracle walks all rows of the slice)
+    keys = np.unique(np.concatenate([edge, [0, 1, r, N // 2, N - 2, N - 1]])).astype(np.int64)
+    rows = np.unique(np.concatenate([edge, np.arange(0, 8), np.arange(N - 8, N)])).astype(np.int64)
+    for b in sorted({0, w.batch - 1}):
+        for hk in kv_heads:
+            hs = slice(hk * G, (hk + 1) * G)
+            q, kk, v = f64(inp["q"][b, :, hs]), f64(inp["k"][b, :, hk]), f64(inp["v"][b, :, hk])
+            do = f64(inp["dout"][b, :, hs])
+            dq, dk, dv = oracle.attn_bwd_sample(s, T, r, k, scale, q, kk, v, do, rows, keys)
+            check_close(f"dQ rows b{b} hk{hk}", f64(out["dq"][b, rows][:, hs]), dq, TOL_GRAD)
+            check_close(f"dK keys b{b} hk{hk}", f64(out["dk"][b, keys, hk]), dk, TOL_GRAD)
+            check_close(f"dV keys b{b} hk{hk}", f64(out["dv"][b, keys, hk]), dv, TOL_GRAD)
