@@ -253,7 +253,7 @@ int32_t unigist_prefill_chunk(const unigist_problem* p, int32_t unit_begin, int3
  * sets it up for caches in the order unigist_kv_compact / unigist_prefill_chunk leave them in after
  * units_done whole units (0 with an empty or sinks-only cache).  Misuse (a gist before its unit is
  * complete, a raw token after it, a block table that is too short) sets state[b * ints + 4] != 0 and
- * leaves the cache unchanged.
+ * leaves the cache, seq_lens and the rest of the state unchanged.
  *
  * Between the first raw token of a unit and its last, up to r - 1 freed slots inside [0, seq_lens[b]) still
  * hold the evicted tokens; unigist_decode_step is unigist_decode (one query per sequence, p->batch sequences,
@@ -279,8 +279,9 @@ size_t unigist_decode_workspace_bytes(int32_t num_seqs, int32_t num_q_heads, int
  * query per sequence attends to ALL seq_lens[i] cache entries (what is left in a compacted
  * cache is visible by construction; the caller appends the new token's K/V first).
  * q, o [num_seqs, Hq, D] device bf16; k_cache, v_cache [num_blocks, Hkv, 64, D] device bf16;
- * block_table [num_seqs, max_blocks_per_seq], seq_lens [num_seqs] device int32 (>= 1);
- * lse [num_seqs, Hq] device fp32, nullable.  head_dim must be 128.
+ * block_table [num_seqs, max_blocks_per_seq], seq_lens [num_seqs] device int32 (>= 0);
+ * lse [num_seqs, Hq] device fp32, nullable.  head_dim must be 128, Hq / Hkv at most 8.
+ * A sequence with nothing to attend to (length 0: a padding slot of the batch) gets O = 0 and LSE = -inf.
  */
 int32_t unigist_decode(int32_t num_seqs, int32_t num_q_heads, int32_t num_kv_heads,
                        int32_t head_dim, float softmax_scale, const void* q, const void* k_cache,
@@ -309,7 +310,8 @@ int32_t unigist_kernel_timing_get(int32_t index, char* name, int32_t cap, float*
  * loop with a hard latency limit, where an allocation's implicit device-wide synchronisation is
  * not acceptable.
  *
- * Same arguments and results as unigist_decode, minus workspace / ws_bytes.  The split-KV
+ * Same arguments, same accepted shapes and bit-identical results as unigist_decode, minus workspace /
+ * ws_bytes.  The split-KV
  * partial results are kept in a fixed array of UNIGIST_DECODE_STATIC_SCRATCH_BYTES bytes that is
  * part of the library image: every GPU that loads the library holds that much global memory
  * until the process exits.  The call allocates and frees nothing.

@@ -54,7 +54,7 @@ def build(force: bool = False, verbose: bool = False) -> Path:
     if failed:
         raise RuntimeError("nvcc failed")
     tmp = LIB.with_suffix(f".tmp{os.getpid()}.so")
-    subprocess.check_call([nvcc, "-shared", "-o", str(tmp), *objs, "-lcudart_static", "-ldl", "-lpthread", "-lrt"])
+    subprocess.check_call([nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-shared", "-o", str(tmp), *objs, "-lcudart_static", "-ldl", "-lpthread", "-lrt"])
     os.replace(tmp, LIB)
     return LIB
 

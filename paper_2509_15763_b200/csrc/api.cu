@@ -24,6 +24,24 @@ int32_t fail(int32_t code, const char* fmt, ...) {
 
 void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
 
+int sm_count() {
+  constexpr int kMaxDevices = 64, kB200 = 148;
+  static std::atomic<int> cached[kMaxDevices];  // 0 = not asked yet
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
+    cudaGetLastError();  // a size query on a machine without a GPU is not an error of the caller's
+    return kB200;
+  }
+  int n = cached[dev].load(std::memory_order_relaxed);
+  if (n > 0) return n;
+  if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) {
+    cudaGetLastError();
+    return kB200;
+  }
+  cached[dev].store(n, std::memory_order_relaxed);
+  return n;
+}
+
 namespace {
 struct TimingRecord {
   const char* name;

@@ -1,13 +1,14 @@
-// Forward gist-masked attention on Blackwell tensor cores (tcgen05 + TMEM + TMA), no sinks.
+// Forward gist-masked attention on Blackwell tensor cores (tcgen05 + TMEM + TMA).
 //
-// The SHIFTED sequence is [raw (T) | gists (n)].  A thread block runs TWO query streams at once,
+// The SHIFTED sequence is [sinks (s) | raw (T) | gists (n)]; a tile never straddles two of these segments.
+// A thread block runs TWO query streams at once,
 // each a 128-row query tile of one query head: either the same tile of two neighbouring heads of
 // one KV group (when the group size is even: both streams then walk the same key tiles under the
 // same mask), or two neighbouring tiles of one head.  Both streams read the same K / V tiles, which
 // are loaded once into a ring in shared memory.  From the closed-form row intervals each stream
-// derives the interval of 128-key tiles that hold a visible pair; the block walks the union (own
-// segment first, downwards from the diagonal, then the other segment) and a stream skips the tiles
-// outside its own interval.  Masked-out tiles are never loaded.  Per key tile and stream:
+// derives, per segment, the interval of 128-key tiles that hold a visible pair; the block walks the union
+// (own segment first, downwards from the diagonal, then the other segments) and a stream skips the tiles
+// outside its own intervals.  Masked-out tiles are never loaded.  Per key tile and stream:
 //   TMA:      K, V tiles -> shared memory (128-byte swizzle), one tensor map per segment so a tile
 //             never straddles segments and rows past a segment's end read as zero.
 //   tcgen05:  S = Q K^T into TMEM (fp32);   O += P V with P (bf16) read from TMEM.
@@ -36,9 +37,6 @@ constexpr int BN = 128;  // keys per tile
 constexpr int kStages = 4;  // ring slots; K and V tiles alternate through them
 constexpr int kCols = BN;     // score columns per thread and tile
 constexpr int kSmWarps = 8;   // softmax warps: 2 streams x 4 lane quarters
-#ifndef UG_EMU_NUM
-#define UG_EMU_NUM 2
-#endif
 constexpr int kTmaWarp = kSmWarps, kMmaWarp = kSmWarps + 1;
 constexpr int kThreads = (kSmWarps + 4) * 32;  // the last warpgroup: TMA warp, MMA warp, 2 idle warps
 constexpr uint32_t kTmemCols = 512;
@@ -188,7 +186,7 @@ __device__ __forceinline__ float row_max(const uint32_t (&sc)[kCols]) {
 // m must be finite; a score of -inf gives p = 0 (or about 2^-126 where the exponential is taken on the FMA
 // pipe).  The special-function unit (16 exponentials per clock and SM) bounds this loop, so kEmuNum of every
 // kEmuDen column pairs go to the FMA pipe (ex2_fma2) and the maximum rides along on the ALU pipe.
-constexpr int kEmuNum = UG_EMU_NUM, kEmuDen = 8;
+constexpr int kEmuNum = 2, kEmuDen = 8;
 template <int kHalf>
 __device__ __forceinline__ float row_exp(const uint32_t (&sc)[kCols], uint32_t t_p, float scale_log2, float m, float& mx) {
   uint64_t l01 = f32x2(0.f, 0.f), l23 = l01;

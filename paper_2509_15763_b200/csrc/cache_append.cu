@@ -52,32 +52,37 @@ cache_append_kernel(int Hkv, int vecs, int r, int k, int is_gist, const uint4* _
       if (st[3] >= r) {
         st[4] = 1;  // a raw token after a complete unit: the gist is missing
       } else {
-        if (st[3] == 0 && st[1] > k * r) {
-          // a new unit opens while the window holds k + 1 earlier units: the oldest one is seen by no token
-          // from here on (its own window ended with the gist just before), so its r slots are free
-          for (int i = 0; i < r; ++i) freel[st[2]++] = ring[(st[0] + i) % cap];
-          st[0] = (st[0] + r) % cap;
-          st[1] -= r;
+        // a new unit opens while the window holds k + 1 earlier units: the oldest one is seen by no token
+        // from here on (its own window ended with the gist just before), so its r slots are free
+        const bool evicts = st[3] == 0 && st[1] > k * r;
+        if (!evicts && st[2] == 0 && seq_lens[b] >= max_blocks * PG) {
+          st[4] = 3;  // the block table is too short; nothing has changed
+        } else {
+          if (evicts) {
+            for (int i = 0; i < r; ++i) freel[st[2]++] = ring[(st[0] + i) % cap];
+            st[0] = (st[0] + r) % cap;
+            st[1] -= r;
+          }
+          if (st[2] > 0) slot = freel[--st[2]];
+          else slot = seq_lens[b]++;
+          ring[(st[0] + st[1]) % cap] = slot;
+          ++st[1];
+          ++st[3];
         }
-        if (st[2] > 0) slot = freel[--st[2]];
-        else slot = seq_lens[b]++;
-        ring[(st[0] + st[1]) % cap] = slot;
-        ++st[1];
-        ++st[3];
       }
     } else {
       if (st[3] != r) {
         st[4] = 2;  // a gist before its unit is complete
       } else {
         // the gist still attends to all k + 1 units of the window; eviction waits for the next raw token
-        if (st[2] > 0) slot = freel[--st[2]];
-        else slot = seq_lens[b]++;
-        st[3] = 0;
+        if (st[2] == 0 && seq_lens[b] >= max_blocks * PG) {
+          st[4] = 3;  // the block table is too short; nothing has changed
+        } else {
+          if (st[2] > 0) slot = freel[--st[2]];
+          else slot = seq_lens[b]++;
+          st[3] = 0;
+        }
       }
-    }
-    if (slot >= max_blocks * PG) {
-      st[4] = 3;  // the block table is too short
-      slot = -1;
     }
     slot_sh = slot;
   }

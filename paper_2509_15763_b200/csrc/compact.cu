@@ -103,7 +103,8 @@ compact_stage_kernel(Geom g, int B, int Hkv, int vecs, int L, uint4* __restrict_
 
 int grid_for(long long total) {
   long long want = (total + 255) / 256;
-  return (int)(want < 148 * 16 ? (want < 1 ? 1 : want) : 148 * 16);
+  const long long cap = (long long)sm_count() * 16;
+  return (int)(want < cap ? (want < 1 ? 1 : want) : cap);
 }
 
 }  // namespace

@@ -273,15 +273,16 @@ decode_combine_kernel(int splits, const float* __restrict__ part, __nv_bfloat16*
     L += w * base[i * (DD + 2) + DD + 1];
     acc += w * base[i * (DD + 2) + threadIdx.x];
   }
-  o[sh * DD + threadIdx.x] = __float2bfloat16_rn(acc / L);
-  if (lse && threadIdx.x == 0) lse[sh] = (M + log2f(L)) * 0.6931471805599453f;
+  // a sequence with nothing to attend to (length 0, or every slot freed): O = 0, LSE = -inf, not 0 / 0
+  o[sh * DD + threadIdx.x] = __float2bfloat16_rn(L > 0.f ? acc / L : 0.f);
+  if (lse && threadIdx.x == 0) lse[sh] = L > 0.f ? (M + log2f(L)) * 0.6931471805599453f : -INFINITY;
 }
 
 }  // namespace
 
-// Pick the split count that fills whole waves of 2 blocks per SM on 148 SMs.
+// Pick the split count that fills whole waves of 2 blocks per SM.
 int decode_num_splits(int S, int Hkv, int max_blocks) {
-  const long long slots = 148 * 2;
+  const long long slots = (long long)sm_count() * 2;
   const long long base = (long long)S * Hkv;
   int best = 1;
   double best_eff = -1.0;
@@ -386,9 +387,7 @@ extern "C" int32_t unigist_decode_static(int32_t S, int32_t Hq, int32_t Hkv, int
     return fail(UNIGIST_ERR_INVALID_ARG, "decode has a non-positive size");
   if (Hq % Hkv) return fail(UNIGIST_ERR_SHAPE, "num_q_heads %d is not a multiple of num_kv_heads %d", Hq, Hkv);
   if (D != 128) return fail(UNIGIST_ERR_SHAPE, "decode supports head_dim 128, got %d", D);
-  const int G = Hq / Hkv;
-  if (G != 1 && G != 2 && G != 4 && G != 8)
-    return fail(UNIGIST_ERR_UNSUPPORTED, "decode supports 1, 2, 4 or 8 query heads per KV head, got %d", G);
+  if (Hq / Hkv > 8) return fail(UNIGIST_ERR_UNSUPPORTED, "decode supports at most 8 query heads per KV head");
   if (!q || !kc || !vc || !table || !seq_lens || !o) return fail(UNIGIST_ERR_INVALID_ARG, "a pointer is NULL");
   if (!aligned16(q) || !aligned16(kc) || !aligned16(vc) || !aligned16(o))
     return fail(UNIGIST_ERR_ALIGNMENT, "tensor pointers must be 16-byte aligned");

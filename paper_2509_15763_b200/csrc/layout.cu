@@ -17,7 +17,7 @@ __global__ void layout_kernel(Geom g, int32_t* __restrict__ sp, int32_t* __restr
 int32_t launch_layout(const Geom& g, int32_t* sp, int32_t* up, int32_t* pos, cudaStream_t st) {
   const int threads = 256;
   int blocks = (g.N + threads - 1) / threads;
-  if (blocks > 148 * 8) blocks = 148 * 8;
+  if (blocks > sm_count() * 8) blocks = sm_count() * 8;
   {
     KernelScope ks("layout_kernel", st);
     layout_kernel<<<blocks, threads, 0, st>>>(g, sp, up, pos);
@@ -69,7 +69,8 @@ int32_t launch_shift(const Geom& g, int B, const void* src, void* dst, size_t ro
   const int vecs = (int)(row_bytes / 16);
   const long long rows = (long long)B * g.N;
   const long long want = (rows + 31) / 32;  // 8 warps x 4 rows per block and pass
-  const int blocks = (int)(want < 148 * 8 ? (want > 0 ? want : 1) : 148 * 8);
+  const long long cap = (long long)sm_count() * 8;
+  const int blocks = (int)(want < cap ? (want > 0 ? want : 1) : cap);
   {
     KernelScope ks(inverse ? "unshift_rows_kernel" : "shift_rows_kernel", st);
     if (inverse)

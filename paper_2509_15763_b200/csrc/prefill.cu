@@ -81,7 +81,8 @@ int32_t launch_prefill_chunk(const unigist_problem& p, const Geom& g_full, float
   {
     const long long total = (long long)B * gc.N * Hkv * vecs;
     const long long want = (total + 255) / 256;
-    const int blocks = (int)(want < 148 * 16 ? want : 148 * 16);
+    const long long cap = (long long)sm_count() * 16;
+    const int blocks = (int)(want < cap ? want : cap);
     KernelScope ks("prefill_gather_kernel", st);
     prefill_gather_kernel<<<blocks, 256, 0, st>>>(B, Hkv, vecs, s, u0, w0, c_raw, c, (const uint4*)kc, (const uint4*)vc,
                                                   num_blocks, table, max_blocks, (const uint4*)k, (const uint4*)v, k_ctx,

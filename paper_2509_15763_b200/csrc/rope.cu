@@ -93,7 +93,8 @@ int32_t launch_rope(const Geom& g, int B, int heads, int D, float theta_base, bo
                     bool inverse, const void* src, void* dst, cudaStream_t st) {
   const long long tokens = (long long)B * g.N;
   const long long want = (tokens + 7) / 8;  // 8 warps per block
-  const int blocks = (int)(want < 148 * 8 ? (want > 0 ? want : 1) : 148 * 8);
+  const long long cap = (long long)sm_count() * 8;
+  const int blocks = (int)(want < cap ? (want > 0 ? want : 1) : cap);
   const double log2_theta = log2((double)theta_base);
   {
     KernelScope ks("rope_kernel", st);

@@ -122,6 +122,9 @@ int32_t check_problem(const unigist_problem* p, Geom* g, float* scale);
 int32_t check_launch(const char* what);
 int32_t check_interleaved(const unigist_problem* p, const Geom& g);
 void count_launch(int n = 1);
+// Streaming multiprocessors of the current device (asked once per device); 148, the B200's count, when no
+// device can be asked (a size query on a machine without a GPU).
+int sm_count();
 // Records a CUDA event before and after the kernels launched in its scope when per-kernel
 // timing is switched on; also counts the launch.
 struct KernelScope {
