@@ -10,8 +10,12 @@ through tile maps that pick the raw rows or the gist row of each gist unit and s
 at interleaved rows; the step with explicit shift launches is timed too and reported beside it.  The headline value is the effective TFLOP/s of forward + backward
 counting only unmasked (visible) pairs: 14 * D * pairs * Hq * B FLOP per step / step time.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--only] [--impl reference]
 
+The headline workload is the largest forward + backward one that fits one GPU (`train_batch`: batch 4,
+32768 raw tokens, ratio 4, window 2048).  On one GPU the same run also times decode over the compressed
+cache and, with fewer steps, the one-layer and the long-prefill workloads; they are reported as extra
+keys (`decode`, `workloads`) of the one JSON line.
 With N > 1 (launched by torchrun) every rank runs an independent replica of the workload (the
 path has no exchange step); the value is the work of all ranks over the slowest rank's time.
 `--impl reference` times the fp64 CPU oracle on a bounded sample of the same workload.
@@ -35,21 +39,55 @@ if str(ROOT) not in sys.path:
 METRIC = "effective_tflops_fwd_bwd_unmasked"
 UNIT = "TFLOP/s"
 
-# DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures
-# summarised under profiles/, keyed by (kernel, workload); None until a capture exists.
-NCU_TRAFFIC_BYTES = {
-    ("attn_fwd_sm100_kernel", "llama8b_layer"): 353900000,
-    ("attn_bwd_fused_sm100_kernel", "llama8b_layer"): 4827655000,
-}
-
 # FLOP per visible pair per query head that each attention kernel performs algorithmically,
 # in units of head_dim (a QK^T- or PV-shaped product is 2 * D FLOP per pair).
 KERNEL_FLOP_PER_PAIR_D = {
-    "bwd_dq_simt_kernel": 6, "bwd_dkdv_simt_kernel": 8,
     "attn_fwd_sm100_kernel": 4, "attn_bwd_dq_sm100_kernel": 6, "attn_bwd_dkdv_sm100_kernel": 8,
     "attn_bwd_fused_sm100_kernel": 10,
 }
-CUDA_CORE_KERNELS = {"bwd_dq_simt_kernel", "bwd_dkdv_simt_kernel"}
+# The source files whose change makes a committed ncu capture of the kernel stale.
+KERNEL_SOURCES = {
+    "attn_fwd_sm100_kernel": ("attn_fwd_sm100.cu", "sm100_ptx.cuh", "ug_common.cuh"),
+    "attn_bwd_fused_sm100_kernel": ("attn_bwd_sm100.cu", "sm100_ptx.cuh", "ug_common.cuh"),
+    "attn_bwd_dkdv_sm100_kernel": ("attn_bwd_sm100.cu", "sm100_ptx.cuh", "ug_common.cuh"),
+    "attn_bwd_dq_sm100_kernel": ("attn_bwd_sm100.cu", "sm100_ptx.cuh", "ug_common.cuh"),
+    "decode_split_kernel": ("decode.cu", "sm100_ptx.cuh", "ug_common.cuh"),
+}
+HEADLINE = "train_batch"                       # the largest single-GPU forward + backward workload
+ALSO = ("llama8b_layer", "long_prefill")       # timed as well (fewer steps), reported under "workloads"
+
+
+def kernel_source_digest(kernel: str) -> str:
+    """Short sha256 over the sources that define `kernel` (what an ncu summary records)."""
+    import hashlib
+
+    h = hashlib.sha256()
+    for name in KERNEL_SOURCES[kernel]:
+        h.update((ROOT / "paper_2509_15763_b200" / "csrc" / name).read_bytes())
+    return h.hexdigest()[:16]
+
+
+def ncu_traffic(kernel: str, workload: str, batch: int):
+    """DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of `kernel` on `workload`, from the
+    committed ncu summary profiles/<kernel>_<workload>.md.  The summary states the batch size of the captured
+    slice (the traffic of these kernels grows in proportion to the batch: every batch index is an independent
+    set of thread blocks over its own tensors) and a digest of the kernel's sources.
+    -> (bytes scaled to `batch`, note); (None, why) without a capture or once the sources changed."""
+    import re
+
+    f = ROOT / "profiles" / f"{kernel}_{workload}.md"
+    if not f.exists():
+        return None, "no ncu capture committed for this kernel and workload"
+    text = f.read_text()
+    m_bytes = re.search(r"DRAM traffic per launch = ([0-9.eE+]+) bytes", text)
+    m_batch = re.search(r"captured batch: (\d+)", text)
+    m_src = re.search(r"kernel sources sha256: ([0-9a-f]+)", text)
+    if not (m_bytes and m_batch and m_src):
+        return None, f"{f.name} lacks the traffic, batch or source-digest line"
+    if kernel not in KERNEL_SOURCES or m_src.group(1) != kernel_source_digest(kernel):
+        return None, f"the kernel's sources changed since {f.name} was captured"
+    cap_b = int(m_batch.group(1))
+    return float(m_bytes.group(1)) * batch / cap_b, f"{f.name}: captured at batch {cap_b}, scaled x{batch / cap_b:g}"
 
 
 def measured_peaks():
@@ -137,6 +175,44 @@ def oracle_sample(w, seconds_hint: float = 20.0):
     return flops / dt / 1e12, oracle.num_threads(), desc, dt
 
 
+def oracle_decode_sample(num_seqs: int = 4):
+    """Time the oracle's decode (as it stands) on `num_seqs` of the 64 sequences of the decode workload, all
+    heads.  -> (GB/s of K+V, cores, description)."""
+    import torch
+
+    from oracle import oracle
+    from paper_2509_15763_b200 import synth
+
+    w = synth.DECODE_WORKLOADS["decode_cache"]
+    ws = synth.DecodeWorkload(w.name + "_sample", num_seqs, w.num_gists, w.window_raw, w.num_q_heads, w.num_kv_heads,
+                              w.head_dim, seed=w.seed)
+    d = synth.decode_inputs(ws)
+    f = lambda t: t.to(dtype=torch.float64).numpy()
+    view = lambda c, i: c[d["block_table"][i].long()].permute(0, 2, 1, 3).reshape(-1, c.shape[1], c.shape[3])[: ws.seq_len]
+    k_list = [f(view(d["k_cache"], i)) for i in range(num_seqs)]
+    v_list = [f(view(d["v_cache"], i)) for i in range(num_seqs)]
+    q = f(d["q"])
+    t0 = time.perf_counter()
+    oracle.decode(w.head_dim ** -0.5, q, k_list, v_list)
+    dt = time.perf_counter() - t0
+    nbytes = num_seqs * ws.seq_len * w.num_kv_heads * w.head_dim * 2 * 2  # the bf16 K and V the query attends to
+    desc = (f"oracle decode of {num_seqs} of the {w.num_seqs} sequences ({ws.seq_len} cache entries each, all "
+            f"{w.num_q_heads} query heads); the whole workload is {w.num_seqs // num_seqs}x this")
+    return nbytes / dt / 1e9, oracle.num_threads(), desc
+
+
+def pick_tensor_peak(peaks, clocks, timed_seconds):
+    """The measured bf16 rate the timed kernel is held against: the burst figure for a short region at full
+    clock, the sustained one for a region of a second or more or one the power cap held below full clock."""
+    sm, mx = clocks.get("sm_mhz"), clocks.get("sm_max_mhz")
+    capped = "sw_power_cap" in clocks.get("reasons", []) or (sm is not None and mx and sm < 0.9 * mx)
+    if capped or timed_seconds >= 1.0:
+        why = ("power cap active / SM clock below 0.9 of max during the timed region" if capped else
+               "timed region of a second or more")
+        return peaks["bf16_tflops_sustained"], f"{peaks['source']} sustained bf16 ({why})"
+    return peaks["bf16_tflops"], f"{peaks['source']} burst bf16 (timed region {timed_seconds:.2f} s at full clock)"
+
+
 def run_reference(args, w):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
@@ -165,7 +241,7 @@ def run_reference(args, w):
 class Path_:
     """Device buffers of one workload and the step that runs the whole path on them."""
 
-    def __init__(self, w, dev):
+    def __init__(self, w, dev, host_buffers=True):
         import torch
 
         import paper_2509_15763_b200 as ug
@@ -178,7 +254,7 @@ class Path_:
         self.N = ug.unigist_total_len(p)
         self.pairs = ug.unigist_visible_pairs(p)
         host = synth.attention_inputs(w, with_grad=not w.forward_only)
-        self.host_in = {k: v.pin_memory() for k, v in host.items()}
+        self.host_in = {k: v.pin_memory() for k, v in host.items()} if host_buffers else {}
         self.inter = {k: v.to(dev) for k, v in host.items()}                      # interleaved inputs
         self.sh = {k: torch.empty_like(v) for k, v in self.inter.items()}         # shifted inputs
         self.o_s = torch.empty_like(self.sh["q"])
@@ -187,7 +263,7 @@ class Path_:
         self.out = {"o": torch.empty_like(self.o_s), "dq": torch.empty_like(self.dq_s),
                     "dk": torch.empty_like(self.dk_s), "dv": torch.empty_like(self.dv_s)}
         self.host_out = {k: torch.empty(v.shape, dtype=v.dtype).pin_memory() for k, v in self.out.items()
-                         if k == "o" or not w.forward_only}
+                         if host_buffers and (k == "o" or not w.forward_only)}
         self.ws = torch.empty(max(16, ug.unigist_workspace_bytes(p, ug.OP_BWD)), dtype=torch.uint8, device=dev)
         L = ug.unigist_compact_len(p)
         self.nb = -(-(L + 1) // ug.PAGE_TOKENS)
@@ -295,7 +371,9 @@ class Path_:
 
 
 def bench_decode(dev, iters=20):
-    """Decode over the compressed-cache workload (64 sequences x 9216 cached tokens): GB/s of K+V."""
+    """Decode over the compressed-cache workload (64 sequences x 9216 cached tokens): GB/s of K+V.
+    The calls alternate between two independent copies of the cache (2.4 GB each), so nothing a call reads
+    can still sit in the 126 MB L2 from the call before."""
     import torch
 
     import paper_2509_15763_b200 as ug
@@ -303,18 +381,19 @@ def bench_decode(dev, iters=20):
 
     w = synth.DECODE_WORKLOADS["decode_cache"]
     d = {k: v.to(dev) for k, v in synth.decode_inputs(w).items()}
+    sets = [(d["k_cache"], d["v_cache"]), (d["k_cache"].clone(), d["v_cache"].clone())]
     ws = torch.empty(ug.unigist_decode_workspace_bytes(w.num_seqs, w.num_q_heads, w.num_kv_heads, w.head_dim,
                                                        d["block_table"].shape[1]), dtype=torch.uint8, device=dev)
     o = torch.empty_like(d["q"])
-    run = lambda: ug.unigist_decode(d["q"], d["k_cache"], d["v_cache"], d["block_table"], d["seq_lens"], o, None, ws)
-    for _ in range(3):
-        run()
+    run = lambda i: ug.unigist_decode(d["q"], sets[i & 1][0], sets[i & 1][1], d["block_table"], d["seq_lens"], o, None, ws)
+    for i in range(4):
+        run(i)
     torch.cuda.synchronize()
     ug.unigist_kernel_timing(True)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
-    for _ in range(iters):
-        run()
+    for i in range(iters):
+        run(i)
     e1.record()
     torch.cuda.synchronize()
     ms = e0.elapsed_time(e1) / iters
@@ -322,9 +401,11 @@ def bench_decode(dev, iters=20):
                 if ug.unigist_kernel_timing_get(i)[0] == "decode_split_kernel"]
     ug.unigist_kernel_timing(False)
     nbytes = w.num_seqs * w.seq_len * w.num_kv_heads * w.head_dim * 2 * 2
+    traffic, traffic_note = ncu_traffic("decode_split_kernel", w.name, 1)
     return {"workload": w.name, "kv_bytes": nbytes, "us_per_call": 1e3 * ms, "gbs": nbytes / (ms * 1e-3) / 1e9,
             "split_kernel_us": 1e3 * statistics.mean(split_ms), "split_kernel_gbs": nbytes / (statistics.mean(split_ms) * 1e-3) / 1e9,
-            "l2_policy": "K+V (2.4 GB) exceed L2, every call streams from HBM"}
+            "traffic": traffic, "traffic_source": traffic_note,
+            "l2_policy": "consecutive calls read two different copies of the cache (2.4 GB each, L2 is 126 MB)"}
 
 
 def reduce_over_ranks(dist, times_ms, device):
@@ -443,6 +524,92 @@ def bench_rope_and_docs(path, iters=3):
     return rope, docs
 
 
+def timed_steps(torch, ug, path, steps, flush, barrier, local):
+    """`steps` device-resident steps of `path`, L2 flushed before each, CUDA events around each step and (inside
+    the library) around each kernel.  -> (step times ms, {kernel: (launches, total ms)}, launches, clock summary)."""
+    ug.unigist_kernel_timing(True)
+    launches0 = ug.unigist_launch_count()
+    evs = []
+    barrier()
+    with ClockSampler(local) as clocks:
+        for _ in range(steps):
+            flush.fill_(1)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            path.step()
+            e1.record()
+            evs.append((e0, e1))
+        barrier()
+    launches = ug.unigist_launch_count() - launches0
+    per_kernel = {}
+    for i in range(ug.unigist_kernel_timing_count()):
+        name, ms = ug.unigist_kernel_timing_get(i)
+        cnt, tot = per_kernel.get(name, (0, 0.0))
+        per_kernel[name] = (cnt + 1, tot + ms)
+    ug.unigist_kernel_timing(False)
+    return [a.elapsed_time(b) for a, b in evs], per_kernel, launches, clocks.summary()
+
+
+def roofline_of(w, path, per_kernel, clocks, timed_seconds, peaks):
+    """The roofline object of the attention kernel with the largest share of the step."""
+    attn = {k: v for k, v in per_kernel.items() if k in KERNEL_FLOP_PER_PAIR_D}
+    top = max(attn, key=lambda k: attn[k][1])
+    cnt, tot = attn[top]
+    top_flops = KERNEL_FLOP_PER_PAIR_D[top] * w.head_dim * path.pairs * w.num_q_heads * w.batch
+    achieved = top_flops / (tot / cnt * 1e-3) / 1e12
+    peak, peak_src = pick_tensor_peak(peaks, clocks, timed_seconds)
+    traffic, traffic_note = ncu_traffic(top, w.name, w.batch)
+    sm, mx = clocks.get("sm_mhz"), clocks.get("sm_max_mhz")
+    return {"kernel": top, "bound": "tensor", "achieved": achieved, "peak": peak, "unit": UNIT, "frac": achieved / peak,
+            "peak_source": peak_src, "kernel_ms": tot / cnt, "algorithmic_flop_per_launch": top_flops,
+            "frac_of_burst": achieved / peaks["bf16_tflops"], "frac_of_sustained": achieved / peaks["bf16_tflops_sustained"],
+            "frac_of_nominal_2250": achieved / 2250.0,
+            # the same rate carried to the maximum SM clock: how much of the gap to the peak is the clock
+            "achieved_at_max_clock": achieved * mx / sm if sm and mx else None,
+            "traffic": traffic, "traffic_source": traffic_note}
+
+
+def kernel_shares(per_kernel):
+    total = sum(x[1] for x in per_kernel.values())
+    return {k: {"launches": c, "ms": round(m, 4), "share": round(m / total, 4)}
+            for k, (c, m) in sorted(per_kernel.items(), key=lambda kv: -kv[1][1])}
+
+
+def config_of(w, path, world):
+    return {"workload": w.name, "batch": w.batch, "raw_len": w.raw_len, "ratio": w.ratio, "window": w.window,
+            "q_heads": w.num_q_heads, "kv_heads": w.num_kv_heads, "head_dim": w.head_dim,
+            "total_len": path.N, "visible_pairs_per_head": path.pairs, "flop_per_step": path.flops,
+            "l2": "256 MB buffer written between timed steps", "parallelism": f"replicas x{world}",
+            "gist_shift": ("done by the attention kernels' tile loads and row-mapped stores on interleaved "
+                           "tensors (UNIGIST_FLAG_INTERLEAVED), no shift / unshift launch") if path.fused_shift
+            else "shift_rows_kernel / unshift_rows_kernel launches inside the step"}
+
+
+def side_workload(torch, ug, name, dev, steps, flush, barrier, local, peaks):
+    """One of the other workloads, device-resident timing only (rank 0, one GPU): a dict for the JSON line."""
+    from paper_2509_15763_b200 import synth
+
+    w = synth.WORKLOADS[name]
+    path = Path_(w, dev, host_buffers=False)
+    for _ in range(3):
+        path.step()
+    step_ms, per_kernel, _, clocks = timed_steps(torch, ug, path, steps, flush, barrier, local)
+    ms = sum(step_ms) / steps
+    out = {"config": config_of(w, path, 1), "steps": steps, "ms_per_step": ms,
+           "value": path.flops / (ms * 1e-3) / 1e12, "unit": UNIT,
+           "what": "forward only (prefill)" if w.forward_only else "forward + backward",
+           "pct_of_nominal_bf16_peak": 100.0 * path.flops / (ms * 1e-3) / 1e12 / 2250.0,
+           "roofline": roofline_of(w, path, per_kernel, clocks, sum(step_ms) * 1e-3, peaks),
+           "kernels": kernel_shares(per_kernel), "clocks": clocks}
+    if w.forward_only:
+        out["chunked_prefill"] = bench_chunked_prefill(path, 1024)
+    else:
+        out["rope"], out["cross_doc"] = bench_rope_and_docs(path)
+    del path
+    torch.cuda.empty_cache()
+    return out
+
+
 def run_ours(args, w):
     import torch
 
@@ -468,35 +635,16 @@ def run_ours(args, w):
             dist.barrier()
         torch.cuda.synchronize()
 
+    warmup = max(args.warmup, 3)
     path = Path_(w, dev)
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)  # > 126 MB L2
-    for _ in range(max(args.warmup, 3)):
+    for _ in range(warmup):
         path.step()
     barrier()
 
     # ---- device-resident timing
-    ug.unigist_kernel_timing(True)
-    launches0 = ug.unigist_launch_count()
-    evs = []
-    barrier()
-    with ClockSampler(local) as clocks:
-        for _ in range(args.steps):
-            flush.fill_(1)
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            e0.record()
-            path.step()
-            e1.record()
-            evs.append((e0, e1))
-        barrier()
-    launches = ug.unigist_launch_count() - launches0
-    step_ms = [a.elapsed_time(b) for a, b in evs]
+    step_ms, per_kernel, launches, clocks = timed_steps(torch, ug, path, args.steps, flush, barrier, local)
     total_ms = sum(step_ms)
-    per_kernel = {}
-    for i in range(ug.unigist_kernel_timing_count()):
-        name, ms = ug.unigist_kernel_timing_get(i)
-        cnt, tot = per_kernel.get(name, (0, 0.0))
-        per_kernel[name] = (cnt + 1, tot + ms)
-    ug.unigist_kernel_timing(False)
 
     # ---- the same step with the gist shift as separate launches (context for the fused number)
     explicit_ms = None
@@ -504,7 +652,7 @@ def run_ours(args, w):
         for _ in range(2):
             path.step_explicit()
         ev2 = []
-        for _ in range(args.steps):
+        for _ in range(min(args.steps, 5)):
             flush.fill_(1)
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             e0.record()
@@ -512,31 +660,7 @@ def run_ours(args, w):
             e1.record()
             ev2.append((e0, e1))
         torch.cuda.synchronize()
-        explicit_ms = sum(a.elapsed_time(b) for a, b in ev2) / args.steps
-    # ---- the same step replayed from a CUDA graph (the tensor maps are kernel arguments, so a captured step
-    # needs no host work at all); context for the launch gaps inside the eager number
-    graph_ms = None
-    if rank == 0 and world == 1:
-        side = torch.cuda.Stream()
-        side.wait_stream(torch.cuda.current_stream())
-        graph = torch.cuda.CUDAGraph()
-        with torch.cuda.stream(side):
-            path.step()
-            with torch.cuda.graph(graph, stream=side):
-                path.step()
-        torch.cuda.current_stream().wait_stream(side)
-        graph.replay()
-        ev3 = []
-        for _ in range(args.steps):
-            flush.fill_(1)
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            e0.record()
-            graph.replay()
-            e1.record()
-            ev3.append((e0, e1))
-        torch.cuda.synchronize()
-        graph_ms = sum(a.elapsed_time(b) for a, b in ev3) / args.steps
-    rope_line, docs_line = bench_rope_and_docs(path) if rank == 0 and world == 1 else (None, None)
+        explicit_ms = sum(a.elapsed_time(b) for a, b in ev2) / len(ev2)
     barrier()
 
     # ---- end to end: host buffers in, host buffers out
@@ -558,54 +682,47 @@ def run_ours(args, w):
     peaks = measured_peaks()
     value = job_value(world, path.flops, args.steps, total_ms)
     e2e_value = job_value(world, path.flops, args.steps, e2e_ms)
-    attn = {k: v for k, v in per_kernel.items() if k in KERNEL_FLOP_PER_PAIR_D}
-    top = max(attn, key=lambda k: attn[k][1])
-    cnt, tot = attn[top]
-    top_flops = KERNEL_FLOP_PER_PAIR_D[top] * w.head_dim * path.pairs * w.num_q_heads * w.batch
-    achieved = top_flops / (tot / cnt * 1e-3) / 1e12
-    if top in CUDA_CORE_KERNELS:
-        # fp32 FMA pipe: 148 SMs x 128 lanes x 2 FLOP x 1.965 GHz
-        bound, peak, peak_src = "alu", 148 * 128 * 2 * 1.965e9 / 1e12, "derived from unit counts and max clock"
-    else:
-        bound, peak, peak_src = "tensor", peaks["bf16_tflops_sustained"], peaks["source"] + " sustained bf16"
-    kernel_share = {k: {"launches": c, "ms": round(m, 4), "share": round(m / sum(x[1] for x in per_kernel.values()), 4)}
-                    for k, (c, m) in sorted(per_kernel.items(), key=lambda kv: -kv[1][1])}
-    decode = bench_decode(dev)
-    cpu_tf, cores, desc, _ = oracle_sample(w)
     line = {
-        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": warmup,
         "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": w.name, "batch": w.batch, "raw_len": w.raw_len, "ratio": w.ratio, "window": w.window,
-                   "q_heads": w.num_q_heads, "kv_heads": w.num_kv_heads, "head_dim": w.head_dim,
-                   "total_len": path.N, "visible_pairs_per_head": path.pairs, "flop_per_step": path.flops,
-                   "l2": "256 MB buffer written between timed steps", "parallelism": f"replicas x{world}",
-                   "gist_shift": ("done by the attention kernels' tile loads and row-mapped stores on interleaved "
-                                  "tensors (UNIGIST_FLAG_INTERLEAVED), no shift / unshift launch") if path.fused_shift
-                   else "shift_rows_kernel / unshift_rows_kernel launches inside the step"},
-        "roofline": {"kernel": top, "bound": bound, "achieved": achieved, "peak": peak, "unit": UNIT,
-                     "frac": achieved / peak, "peak_source": peak_src,
-                     "traffic": NCU_TRAFFIC_BYTES.get((top, w.name))},
+        "config": config_of(w, path, world),
+        "roofline": roofline_of(w, path, per_kernel, clocks, total_ms * 1e-3, peaks),
         "pct_of_nominal_bf16_peak": 100.0 * value / world / 2250.0,
-        "kernels": kernel_share,
-        "decode": dict(decode, frac_of_measured_hbm=decode["split_kernel_gbs"] / peaks["hbm_gbs"],
-                       frac_of_nominal_8tbs=decode["split_kernel_gbs"] / 8000.0),
-        "cpu_baseline": {"value": cpu_tf, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc},
+        "kernels": kernel_shares(per_kernel),
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": path.h2d_bytes(),
                 "d2h_bytes_per_step": path.d2h_bytes(), "ms_per_step": e2e_ms / args.steps,
                 "how": "every step copies its inputs from pinned host memory and its results back; the copies of "
                        "neighbouring steps run on two side streams under the kernels (two device buffer sets)"},
-        "chunked_prefill": bench_chunked_prefill(path, 1024) if w.forward_only else None,
-        "rope": rope_line, "cross_doc": docs_line,
-        "graph_step": None if graph_ms is None else {
-            "ms_per_step": graph_ms, "value": path.flops / (graph_ms * 1e-3) / 1e12, "unit": UNIT,
-            "note": "the timed step captured once in a CUDA graph and replayed"},
         "explicit_shift_step": None if explicit_ms is None else {
             "ms_per_step": explicit_ms, "value": path.flops / (explicit_ms * 1e-3) / 1e12, "unit": UNIT,
             "note": "the same step with 4 shift and 4 unshift launches around shifted-order attention calls"},
         "gpu_launches": launches,
-        "clocks": clocks.summary(),
+        "clocks": clocks,
+        # clock-normalised step: milliseconds x median SM MHz = thousands of SM cycles per step
+        "kcycles_per_step": None if not clocks.get("sm_mhz") else total_ms / args.steps * clocks["sm_mhz"],
     }
+    if w.forward_only:
+        line["chunked_prefill"] = bench_chunked_prefill(path, 1024)
+    elif world == 1:
+        line["rope"], line["cross_doc"] = bench_rope_and_docs(path)
+    del path
+    torch.cuda.empty_cache()
+    # ---- the metric's other parts (one GPU): decode over the compressed cache, and the other workloads
+    decode = bench_decode(dev)
+    line["decode"] = dict(decode, frac_of_measured_hbm=decode["split_kernel_gbs"] / peaks["hbm_gbs"],
+                          frac_of_nominal_8tbs=decode["split_kernel_gbs"] / 8000.0)
+    torch.cuda.empty_cache()
+    line["workloads"] = {}
+    if world == 1 and not args.only:
+        for name in ALSO:
+            if name != w.name:
+                line["workloads"][name] = side_workload(torch, ug, name, dev, min(args.steps, 5), flush, barrier, local, peaks)
+    cpu_tf, cores, desc, _ = oracle_sample(w)
+    line["cpu_baseline"] = {"value": cpu_tf, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc}
+    dec_gbs, dec_cores, dec_desc = oracle_decode_sample()
+    line["decode"]["cpu_baseline"] = {"value": dec_gbs, "unit": "GB/s", "cores": dec_cores, "kind": "oracle",
+                                      "sample": dec_desc}
     print(json.dumps(line))
     if dist:
         dist.destroy_process_group()
@@ -616,10 +733,11 @@ def main():
 
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="llama8b_layer", choices=sorted(synth.WORKLOADS))
+    ap.add_argument("--workload", default=HEADLINE, choices=sorted(synth.WORKLOADS))
+    ap.add_argument("--only", action="store_true", help="time the named workload alone, not the other workloads beside it")
     args = ap.parse_args()
     w = synth.WORKLOADS[args.workload]
     if args.impl == "reference":
