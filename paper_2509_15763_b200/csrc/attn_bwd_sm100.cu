@@ -1,7 +1,9 @@
-// Backward gist-masked attention on Blackwell tensor cores (tcgen05 + TMEM + TMA), no sinks.
-//
-// Three kernels on the SHIFTED sequence [raw (T) | gists (n)]:
-//   bwd_prep_kernel            Delta = rowsum(dO o O) (fp32) and, for an fp32 dO, its bf16 copy.
+// Backward gist-masked attention on Blackwell tensor cores (tcgen05 + TMEM + TMA) on the SHIFTED sequence
+// [sinks (s) | raw (T) | gists (n)]; a tile never straddles two of these segments.
+//   bwd_prep_kernel            Delta = rowsum(dO o O) (fp32) and, for an fp32 dO, its bf16 copy; zeroes the fp32
+//                              dQ accumulator of the fused kernel.
+// head_dim 128: attn_bwd_fused_sm100_kernel (described where it is defined) and dq_convert_kernel.
+// head_dim 64: two kernels (a 64-row dQ^T accumulator would halve the fused kernel's tensor throughput):
 //   attn_bwd_dkdv_sm100_kernel one thread block owns a 128-key tile of one KV head and walks every
 //                              128-query tile of every query head of the group that can see it:
 //                              S^T = K Q^T and dP^T = V dO^T (TMEM), P^T = exp2(S^T c - LSE),
@@ -662,8 +664,6 @@ attn_bwd_dq_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const __g
 // step i+1 and the dQ read-out of step i run under matrix products.
 // Warps: 0-7 compute (thread = key, 64 query columns each), 8-15 dQ read-out (two warps per TMEM lane
 // quarter, 64 query columns each, so the dQ^T columns are free again after two TMEM loads), 16 TMA, 17 MMA.
-// Which backward head_dim 128 takes: the fused kernel below, or the two kernels above.
-constexpr bool kFusedBackward = true;
 constexpr int kFuThreads = 640;
 constexpr int kFuTmaWarp = 16, kFuMmaWarp = 17;
 constexpr int kFuRegsLaunch = 96, kFuRegsCompute = 128, kFuRegsReadout = 80, kFuRegsOther = 64;
@@ -729,7 +729,7 @@ attn_bwd_fused_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_sink, const
                             const __grid_constant__ CUtensorMap tm_dq_gist, Geom g, int Hq, int Hkv, float scale,
                             const float* __restrict__ lse, const float* __restrict__ delta,
                             __nv_bfloat16* __restrict__ dk, __nv_bfloat16* __restrict__ dv, int n_sink_kt, int n_gist_kt,
-                            int interleaved, FastDiv gdiv, FastDiv rdiv) {
+                            int interleaved, FastDiv rdiv) {
   using SM = FuSmem;
   constexpr int D = 128;
   extern __shared__ unsigned char smem_dyn[];
@@ -803,12 +803,27 @@ attn_bwd_fused_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_sink, const
   const uint32_t t_dK = tmem, t_dV = tmem + 128, t_S = tmem + 256, t_dP = tmem + 384;
   bool ok = true;
 
-  // Step order: raw query tiles from the last one down, then gist query tiles, then sink query tiles, the
-  // G heads of a tile back to back.  Every key tile's visible range ends at the last tile of a segment, so
-  // thread blocks that run side by side walk the same Q / dO / dQ tiles at the same time and share them in L2.
-  auto tile_of = [&](int it, int& qseg, int& qt, int& head) {
-    const int t = fdiv(gdiv, it);  // it / G: on the producer's path to every Q load
-    head = hk * G + (it - t * G);
+  // Step order.  Tiles: raw query tiles from the last one down, then gist query tiles, then sink query tiles.
+  // A sink or gist key tile is seen up to the last tile of every segment, so the blocks of one KV head that start
+  // together walk the same tiles: with the G heads of a tile back to back they stay in step until each runs out,
+  // and share Q / dO / dQ lines in L2.  A raw key tile sees a window of query tiles that moves with the key tile:
+  // its neighbour is one tile behind, i.e. G steps with the heads innermost but a single step with the tiles
+  // innermost (head by head), which keeps the shared lines in L2 between the two uses.
+  const int n_tiles = n_raw_q + n_gist_q + n_sink_q;
+  const bool tiles_inner = kseg == kSegRaw;
+  struct StepIter {
+    int t, hd;  // tile index in the order above, head of the group
+  };
+  auto advance = [&](StepIter& x) {  // no division: the walk is sequential for every role
+    if (tiles_inner) {
+      if (++x.t == n_tiles) x.t = 0, ++x.hd;
+    } else {
+      if (++x.hd == G) x.hd = 0, ++x.t;
+    }
+  };
+  auto tile_of = [&](const StepIter& x, int& qseg, int& qt, int& head) {
+    const int t = x.t;
+    head = hk * G + x.hd;
     if (t < n_raw_q) {
       qseg = kSegRaw;
       qt = rq_lo + (n_raw_q - 1 - t);
@@ -839,9 +854,9 @@ attn_bwd_fused_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_sink, const
       }
       // LSE (in log2 units) and Delta of the step's 128 query rows, 4 rows per lane, fetched one step ahead
       float st_l[4], st_d[4];
-      auto fetch_stats = [&](int it) {
+      auto fetch_stats = [&](const StepIter& at) {
         int qseg, qt, head;
-        tile_of(it, qseg, qt, head);
+        tile_of(at, qseg, qt, head);
         const int q_seg_len = seg_len(g, qseg), q_seg_base = seg_base(g, qseg);
         const long long row_base = ((long long)b * Hq + head) * g.N + q_seg_base;
 #pragma unroll
@@ -853,11 +868,12 @@ attn_bwd_fused_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_sink, const
           st_d[i] = valid ? delta[row_base + row] : 0.f;
         }
       };
-      if (n_iter > 0) fetch_stats(0);
-      for (int it = 0; it < n_iter; ++it) {
+      StepIter cur{0, 0}, ahead{0, 0};
+      if (n_iter > 0) fetch_stats(ahead);
+      for (int it = 0; it < n_iter; ++it, advance(cur)) {
         const int st = it & 1;
         int qseg, qt, head;
-        tile_of(it, qseg, qt, head);
+        tile_of(cur, qseg, qt, head);
         if (it >= 2) ok = mbar_wait_warp(empty_q0 + 8 * st, ((it >> 1) - 1) & 1);
         if (!ok) break;
         float* ls = stats + st * 256;
@@ -876,7 +892,8 @@ attn_bwd_fused_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_sink, const
                         first_unit(qseg, qt * 128), b);
           *q_issued = it + 1;
         }
-        if (it + 1 < n_iter) fetch_stats(it + 1);
+        advance(ahead);
+        if (it + 1 < n_iter) fetch_stats(ahead);
         if (it >= 1) ok = mbar_wait_warp(empty_do, (it - 1) & 1);  // one dO buffer: free once dV of the step before is done
         if (!ok) break;
         if (lane == 0) {
@@ -985,9 +1002,10 @@ attn_bwd_fused_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_sink, const
     const uint32_t lane_base = static_cast<uint32_t>(qd * 32) << 16;
     float* stage_gen = reinterpret_cast<float*>(gen + SM::kOffStage) + (warp - 8) * 1024 + lane;
     const uint32_t stage_sh = base + SM::kOffStage + (warp - 8) * 4096;
-    for (int it = 0; it < n_iter && ok; ++it) {
+    StepIter cur{0, 0};
+    for (int it = 0; it < n_iter && ok; ++it, advance(cur)) {
       int qseg, qt, head;
-      tile_of(it, qseg, qt, head);
+      tile_of(cur, qseg, qt, head);
       const CUtensorMap* mdq = qseg == kSegRaw ? &tm_dq_raw : (qseg == kSegGist ? &tm_dq_gist : &tm_dq_sink);
       const int nq = seg_len(g, qseg) - qt * 128;  // rows of this tile inside the segment (may exceed 128)
       ok = mbar_wait_warp(bar_dQ, it & 1);
@@ -1046,10 +1064,11 @@ attn_bwd_fused_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_sink, const
     unsigned char* ds_row = gen + SM::kOffDS + hf * SM::kSlab + krow * 128;
     const int swz = krow & 7;
 
-    for (int it = 0; it < n_iter && ok; ++it) {
+    StepIter cur{0, 0};
+    for (int it = 0; it < n_iter && ok; ++it, advance(cur)) {
       const int st = it & 1;
       int qseg, qt, head;
-      tile_of(it, qseg, qt, head);
+      tile_of(cur, qseg, qt, head);
       const int q0 = qt * 128, q_seg_len = seg_len(g, qseg);
       const int qb = min(q0 + 127, q_seg_len - 1);
       // full: every (query, key) pair of the tile is visible -> no mask arithmetic
@@ -1195,11 +1214,11 @@ int32_t launch_bwd_sm100(const Geom& g, const unigist_problem& p, float scale, c
   __nv_bfloat16* do_bf16 = reinterpret_cast<__nv_bfloat16*>(static_cast<char*>(workspace) + delta_bytes);
   const void* do_src = f32 ? static_cast<const void*>(do_bf16) : d_o;
   const size_t do_bytes = f32 ? ((size_t)B * g.N * Hq * D * 2 + 255) / 256 * 256 : 0;
-  const bool fused = kFusedBackward && D == 128;  // head_dim 64 keeps the two-kernel path
+  const bool fused = D == 128;  // head_dim 64 takes the two-kernel path
   float* dq32 = fused ? reinterpret_cast<float*>(static_cast<char*>(workspace) + delta_bytes + do_bytes) : nullptr;
   {
     const long long tokens = (long long)B * g.N;
-    const int blocks = (int)((tokens + 7) / 8 < 148 * 16 ? (tokens + 7) / 8 : 148 * 16);
+    const int blocks = (int)((tokens + 7) / 8 < sm_count() * 16 ? (tokens + 7) / 8 : sm_count() * 16);
     KernelScope ks("bwd_prep_kernel", st);
     if (f32)
       bwd_prep_kernel<true><<<blocks, 256, 0, st>>>(g, il ? 1 : 0, Hq, D, tokens, d_o, (const __nv_bfloat16*)o, delta, do_bf16, dq32);
@@ -1243,13 +1262,9 @@ int32_t launch_bwd_sm100(const Geom& g, const unigist_problem& p, float scale, c
     }
     return check_launch("tcgen05 dQ kernel");
   };
-  if (!fused && D == 64) {
+  if (!fused) {
     if (int32_t rc = go_kv(attn_bwd_dkdv_sm100_kernel<64>, KvSmem<64>::kBytes)) return rc;
     return go_q(attn_bwd_dq_sm100_kernel<64>, DqSmem<64>::kBytes);
-  }
-  if (!fused) {
-    if (int32_t rc = go_kv(attn_bwd_dkdv_sm100_kernel<128>, KvSmem<128>::kBytes)) return rc;
-    return go_q(attn_bwd_dq_sm100_kernel<128>, DqSmem<128>::kBytes);
   }
   // 128-row tile maps per segment (sinks, raw, gists) that read shifted or interleaved tensors, and
   // reduction maps over the fp32 dQ tensor (always shifted)
@@ -1270,13 +1285,12 @@ int32_t launch_bwd_sm100(const Geom& g, const unigist_problem& p, float scale, c
     KernelScope ks("attn_bwd_fused_sm100_kernel", st);
     attn_bwd_fused_sm100_kernel<<<dim3((n_sink_t + n_raw_t + n_gist_t) * Hkv, 1, B), kFuThreads, FuSmem::kBytes, st>>>(
         fq[0], fq[1], fq[2], fdo[0], fdo[1], fdo[2], fk[0], fk[1], fk[2], fv[0], fv[1], fv[2], mdq[0], mdq[1], mdq[2], g,
-        Hq, Hkv, scale, lse, delta, (__nv_bfloat16*)dk, (__nv_bfloat16*)dv, n_sink_t, n_gist_t, il ? 1 : 0, make_fastdiv(Hq / Hkv),
-        make_fastdiv(g.r));
+        Hq, Hkv, scale, lse, delta, (__nv_bfloat16*)dk, (__nv_bfloat16*)dv, n_sink_t, n_gist_t, il ? 1 : 0, make_fastdiv(g.r));
   }
   if (int32_t rc = check_launch("tcgen05 fused backward kernel")) return rc;
   {
     const long long tokens = (long long)B * g.N;
-    const int blocks = (int)((tokens + 7) / 8 < 148 * 16 ? (tokens + 7) / 8 : 148 * 16);
+    const int blocks = (int)((tokens + 7) / 8 < sm_count() * 16 ? (tokens + 7) / 8 : sm_count() * 16);
     KernelScope ks("dq_convert_kernel", st);
     dq_convert_kernel<<<blocks, 256, 0, st>>>(g, il ? 1 : 0, Hq, tokens, dq32, (__nv_bfloat16*)dq, scale);
   }
