@@ -519,8 +519,8 @@ def bench_rope_and_docs(path, iters=3):
                                                      num_sinks=w.num_sinks))
     flops = 14.0 * w.head_dim * pairs * w.num_q_heads
     docs = {"doc_raw_len": doc_T, "ms": ms, "value": flops / (ms * 1e-3) / 1e12, "unit": UNIT,
-            "note": "forward + backward of the sample cut into documents (one batched launch set per run of equal "
-                    "documents, spread over the library's side streams)"}
+            "note": "forward + backward of the sample cut into documents of different lengths: one launch of each "
+                    "kernel for all of them (every block finds its document from its block index)"}
     return rope, docs
 
 
@@ -738,8 +738,12 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default=HEADLINE, choices=sorted(synth.WORKLOADS))
     ap.add_argument("--only", action="store_true", help="time the named workload alone, not the other workloads beside it")
+    ap.add_argument("--batch", type=int, default=0,
+                    help="run a slice of the workload with this batch size (what the ncu captures under profiles/ use)")
     args = ap.parse_args()
     w = synth.WORKLOADS[args.workload]
+    if args.batch > 0:
+        w = w.scaled(batch=args.batch)
     if args.impl == "reference":
         run_reference(args, w)
     else:

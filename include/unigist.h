@@ -175,11 +175,11 @@ int32_t unigist_attn_bwd(const unigist_problem* p, const void* q, const void* k,
  * tensors with N_total = sum_d (s + T_d + T_d / r) rows: document d owns the rows from the sum of the earlier
  * documents' lengths on, in shifted order inside its block (interleaved with UNIGIST_FLAG_INTERLEAVED).
  * lse holds one [Hq, N_d] block per document (shifted order), document d's block starting at float
- * Hq * (first row of d).  Consecutive documents of equal length run as one batched launch; the runs are spread
- * over `stream` and three side streams of the library that fork from `stream` and join it again before the call
- * returns (events only, so the call can be captured in a CUDA graph); each run has its own slice of the
- * workspace (unigist_docs_workspace_bytes: the sum over the runs).
- * The side streams are created at the first call, on the device current then: one process drives one GPU.
+ * Hq * (first row of d).  Consecutive documents of equal length form one launch unit (a batch); up to twelve
+ * units, of equal or different lengths, share ONE launch of each kernel (every thread block finds its document
+ * from its block index; the units' tensor maps travel as kernel parameters), a sample with more units takes one
+ * launch per twelve.  Everything is enqueued on `stream`.  For head_dim 64 the backward runs its two kernels once
+ * per unit.  workspace (backward only): unigist_docs_workspace_bytes bytes.
  * Errors as for unigist_attn_fwd / unigist_attn_bwd, raised before the first launch where the list is malformed.
  */
 int64_t unigist_docs_total_len(const unigist_problem* p, int32_t num_docs, const int32_t* doc_raw_len);

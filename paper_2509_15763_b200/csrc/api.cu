@@ -165,16 +165,11 @@ size_t unigist_workspace_bytes(const unigist_problem* p, int32_t op) {
   switch (op) {
     case UNIGIST_OP_FWD:
       return 0;
-    case UNIGIST_OP_BWD: {
-      // Delta [B,Hq,N] fp32, plus a bf16 copy of dO when it arrives as fp32.
-      size_t b = align_up((size_t)p->batch * p->num_q_heads * g.N * sizeof(float), 256);
-      if (p->flags & UNIGIST_FLAG_DOUT_FP32)
-        b += align_up((size_t)p->batch * g.N * p->num_q_heads * p->head_dim * 2, 256);
-      // fp32 dQ accumulator of the fused tensor-core backward (head_dim 128)
-      if (p->head_dim == 128)
-        b += align_up((size_t)p->batch * g.N * p->num_q_heads * p->head_dim * sizeof(float), 256);
-      return b;
-    }
+    case UNIGIST_OP_BWD:
+      // Delta [B,Hq,N] fp32, a bf16 copy of dO when it arrives as fp32, and for head_dim 128 the fp32 dQ
+      // accumulator of the fused tensor-core backward
+      return bwd_scratch_bytes((long long)p->batch * g.N, p->num_q_heads, p->head_dim,
+                               (p->flags & UNIGIST_FLAG_DOUT_FP32) != 0);
     case UNIGIST_OP_COMPACT: {
       const size_t L = (size_t)g.s + g.n + (size_t)g.k * g.r;
       return align_up(2 * (size_t)p->batch * L * p->num_kv_heads * p->head_dim * 2, 256);
@@ -291,12 +286,8 @@ int32_t unigist_attn_bwd(const unigist_problem* p, const void* q, const void* k,
   if (!workspace || ws_bytes < need)
     return fail(UNIGIST_ERR_WORKSPACE, "backward needs %zu bytes of workspace, got %zu", need,
                 ws_bytes);
-  // Tensor cores: the fused kernel for head_dim 128 (sinks included), the two-kernel path for head_dim 64
-  // without sinks; the CUDA-core kernels cover head_dim 64 with a sink prefix.
-  if (p->head_dim == 128 || g.s == 0)
-    return launch_bwd_sm100(g, *p, scale, q, k, v, o, lse, d_o, dq, dk, dv, workspace, (cudaStream_t)stream);
-  return launch_bwd_simt(g, *p, scale, q, k, v, o, lse, d_o, dq, dk, dv, (float*)workspace,
-                         (cudaStream_t)stream);
+  // the fused kernel for head_dim 128, the two-kernel path for head_dim 64; both on the tensor cores
+  return launch_bwd_sm100(g, *p, scale, q, k, v, o, lse, d_o, dq, dk, dv, workspace, (cudaStream_t)stream);
 }
 
 // ---- cross-document masking: a packed sample is a list of independent sequences -------------------------------
@@ -336,64 +327,21 @@ int32_t for_each_doc_run(const unigist_problem* p, int32_t num_docs, const int32
   return UNIGIST_OK;
 }
 
-// The runs of a packed sample are independent, and the short ones do not fill the GPU: they are spread over
-// a few side streams that fork from the caller's stream and join it again (events only; capturable in a graph).
-constexpr int kSideStreams = 3;
-struct DocStreams {
-  cudaStream_t side[kSideStreams];
-  cudaEvent_t fork, join[kSideStreams];
-  bool ok = false;
-  DocStreams() {
-    ok = cudaEventCreateWithFlags(&fork, cudaEventDisableTiming) == cudaSuccess;
-    for (int i = 0; i < kSideStreams && ok; ++i)
-      ok = cudaStreamCreateWithFlags(&side[i], cudaStreamNonBlocking) == cudaSuccess &&
-           cudaEventCreateWithFlags(&join[i], cudaEventDisableTiming) == cudaSuccess;
-  }
-};
-DocStreams& doc_streams() {
-  static DocStreams ds;  // created on first use, lives as long as the library
-  return ds;
-}
-
-// Runs fn(run problem, first row, run index, stream of the run) with run i on stream i mod (1 + kSideStreams),
-// stream 0 being the caller's.
-template <typename Fn>
-int32_t spread_doc_runs(const unigist_problem* p, int32_t num_docs, const int32_t* doc_raw_len, cudaStream_t st, Fn fn) {
-  DocStreams& ds = doc_streams();
-  if (!ds.ok) return fail(UNIGIST_ERR_CUDA, "could not create the side streams");
-  int32_t runs = 0;
-  for_each_doc_run(p, num_docs, doc_raw_len, [&](const unigist_problem&, int64_t, int32_t) { ++runs; return (int32_t)UNIGIST_OK; });
-  const int used = runs - 1 < kSideStreams ? runs - 1 : kSideStreams;
-  if (used > 0) {
-    if (cudaEventRecord(ds.fork, st) != cudaSuccess) return fail(UNIGIST_ERR_CUDA, "cudaEventRecord failed");
-    for (int i = 0; i < used; ++i)
-      if (cudaStreamWaitEvent(ds.side[i], ds.fork, 0) != cudaSuccess) return fail(UNIGIST_ERR_CUDA, "cudaStreamWaitEvent failed");
-  }
-  // longest runs first (their launches fill the GPU; the short ones then run in their tails), streams round robin
-  struct Run {
-    unigist_problem p;
-    int64_t base;
-    int32_t index;
-  };
-  std::vector<Run> order;
-  order.reserve(runs);
-  for_each_doc_run(p, num_docs, doc_raw_len, [&](const unigist_problem& run, int64_t base, int32_t i) {
-    order.push_back(Run{run, base, i});
+// The runs of a packed sample as launch units, in token order.
+int32_t doc_runs(const unigist_problem* p, int32_t num_docs, const int32_t* doc_raw_len, std::vector<SeqRun>* out,
+                 int64_t* tokens) {
+  out->clear();
+  int64_t end = 0;
+  int32_t rc = for_each_doc_run(p, num_docs, doc_raw_len, [&](const unigist_problem& run, int64_t base, int32_t) {
+    SeqRun r;
+    if (int32_t e = check_problem(&run, &r.g, nullptr)) return e;
+    r.batch = run.batch;
+    r.first_row = base;
+    out->push_back(r);
+    end = base + (int64_t)r.g.N * r.batch;
     return (int32_t)UNIGIST_OK;
   });
-  std::stable_sort(order.begin(), order.end(), [](const Run& a, const Run& b) {
-    return (int64_t)a.p.raw_len * a.p.batch > (int64_t)b.p.raw_len * b.p.batch;
-  });
-  int32_t rc = UNIGIST_OK;
-  for (size_t j = 0; j < order.size() && rc == UNIGIST_OK; ++j) {
-    const int lane = (int)(j % (1 + kSideStreams));
-    rc = fn(order[j].p, order[j].base, order[j].index, lane == 0 ? st : ds.side[lane - 1]);
-  }
-  // join even after an error, so that the caller's stream stays ordered after whatever was enqueued
-  for (int i = 0; i < used; ++i) {
-    if (cudaEventRecord(ds.join[i], ds.side[i]) != cudaSuccess || cudaStreamWaitEvent(st, ds.join[i], 0) != cudaSuccess)
-      return fail(UNIGIST_ERR_CUDA, "joining a side stream failed");
-  }
+  *tokens = end;
   return rc;
 }
 
@@ -409,7 +357,11 @@ int64_t unigist_docs_total_len(const unigist_problem* p, int32_t num_docs, const
 
 size_t unigist_docs_workspace_bytes(const unigist_problem* p, int32_t op, int32_t num_docs, const int32_t* doc_raw_len) {
   if (check_docs(p, num_docs, doc_raw_len) != UNIGIST_OK) return 0;
-  size_t need = 0;  // the runs work side by side: one slice each
+  if (op != UNIGIST_OP_BWD) return 0;
+  if (p->head_dim == 128)  // one scratch layout over all packed tokens
+    return bwd_scratch_bytes(unigist_docs_total_len(p, num_docs, doc_raw_len), p->num_q_heads, p->head_dim,
+                             (p->flags & UNIGIST_FLAG_DOUT_FP32) != 0);
+  size_t need = 0;  // head_dim 64: one launch set per run, each with its own slice
   for_each_doc_run(p, num_docs, doc_raw_len, [&](const unigist_problem& run, int64_t, int32_t) {
     need += align_up(unigist_workspace_bytes(&run, op), 256);
     return (int32_t)UNIGIST_OK;
@@ -420,14 +372,18 @@ size_t unigist_docs_workspace_bytes(const unigist_problem* p, int32_t op, int32_
 int32_t unigist_attn_fwd_docs(const unigist_problem* p, int32_t num_docs, const int32_t* doc_raw_len, const void* q,
                               const void* k, const void* v, void* o, float* lse, void* workspace, size_t ws_bytes,
                               void* stream) {
+  (void)workspace;
+  (void)ws_bytes;
   if (int32_t rc = check_docs(p, num_docs, doc_raw_len)) return rc;
   if (!q || !k || !v || !o || !lse) return fail(UNIGIST_ERR_INVALID_ARG, "a tensor is NULL");
-  const size_t rq = (size_t)p->num_q_heads * p->head_dim * 2, rk = (size_t)p->num_kv_heads * p->head_dim * 2;
-  return spread_doc_runs(p, num_docs, doc_raw_len, (cudaStream_t)stream,
-                         [&](const unigist_problem& run, int64_t base, int32_t, cudaStream_t st) {
-    return unigist_attn_fwd(&run, (const char*)q + base * rq, (const char*)k + base * rk, (const char*)v + base * rk,
-                            (char*)o + base * rq, lse + base * p->num_q_heads, workspace, ws_bytes, st);
-  });
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || (reinterpret_cast<uintptr_t>(lse) & 3))
+    return fail(UNIGIST_ERR_ALIGNMENT, "tensor pointers must be 16-byte aligned (lse: 4-byte)");
+  std::vector<SeqRun> runs;
+  int64_t tokens = 0;
+  if (int32_t rc = doc_runs(p, num_docs, doc_raw_len, &runs, &tokens)) return rc;
+  if (int32_t rc = check_interleaved(p, runs[0].g)) return rc;
+  const float scale = p->softmax_scale > 0.f ? p->softmax_scale : 1.0f / sqrtf((float)p->head_dim);
+  return launch_fwd_sm100_runs(runs.data(), (int)runs.size(), *p, scale, q, k, v, o, lse, (cudaStream_t)stream);
 }
 
 int32_t unigist_attn_bwd_docs(const unigist_problem* p, int32_t num_docs, const int32_t* doc_raw_len, const void* q,
@@ -435,20 +391,33 @@ int32_t unigist_attn_bwd_docs(const unigist_problem* p, int32_t num_docs, const 
                               void* dk, void* dv, void* workspace, size_t ws_bytes, void* stream) {
   if (int32_t rc = check_docs(p, num_docs, doc_raw_len)) return rc;
   if (!q || !k || !v || !o || !lse || !d_o || !dq || !dk || !dv) return fail(UNIGIST_ERR_INVALID_ARG, "a tensor is NULL");
+  const void* ptrs[] = {q, k, v, o, d_o, dq, dk, dv, workspace};
+  for (const void* x : ptrs)
+    if (!aligned16(x)) return fail(UNIGIST_ERR_ALIGNMENT, "tensor pointers must be 16-byte aligned");
+  if (reinterpret_cast<uintptr_t>(lse) & 3) return fail(UNIGIST_ERR_ALIGNMENT, "lse must be 4-byte aligned");
+  const size_t need = unigist_docs_workspace_bytes(p, UNIGIST_OP_BWD, num_docs, doc_raw_len);
+  if (!workspace || ws_bytes < need)
+    return fail(UNIGIST_ERR_WORKSPACE, "backward over documents needs %zu bytes of 16-byte aligned workspace, got %zu", need,
+                ws_bytes);
+  std::vector<SeqRun> runs;
+  int64_t tokens = 0;
+  if (int32_t rc = doc_runs(p, num_docs, doc_raw_len, &runs, &tokens)) return rc;
+  if (int32_t rc = check_interleaved(p, runs[0].g)) return rc;
+  const float scale = p->softmax_scale > 0.f ? p->softmax_scale : 1.0f / sqrtf((float)p->head_dim);
+  if (p->head_dim == 128)
+    return launch_bwd_sm100_runs(runs.data(), (int)runs.size(), tokens, *p, scale, q, k, v, o, lse, d_o, dq, dk, dv,
+                                 workspace, (cudaStream_t)stream);
+  // head_dim 64 (two kernels per run): the runs one after the other on the caller's stream
   const size_t rq = (size_t)p->num_q_heads * p->head_dim * 2, rk = (size_t)p->num_kv_heads * p->head_dim * 2;
   const size_t rdo = (p->flags & UNIGIST_FLAG_DOUT_FP32) ? 2 * rq : rq;
-  if (!workspace || !aligned16(workspace) || ws_bytes < unigist_docs_workspace_bytes(p, UNIGIST_OP_BWD, num_docs, doc_raw_len))
-    return fail(UNIGIST_ERR_WORKSPACE, "backward over documents needs %zu bytes of 16-byte aligned workspace, got %zu",
-                unigist_docs_workspace_bytes(p, UNIGIST_OP_BWD, num_docs, doc_raw_len), ws_bytes);
   size_t ws_off = 0;
-  return spread_doc_runs(p, num_docs, doc_raw_len, (cudaStream_t)stream,
-                         [&](const unigist_problem& run, int64_t base, int32_t, cudaStream_t st) {
+  return for_each_doc_run(p, num_docs, doc_raw_len, [&](const unigist_problem& run, int64_t base, int32_t) {
     const size_t mine = align_up(unigist_workspace_bytes(&run, UNIGIST_OP_BWD), 256);
     char* ws = (char*)workspace + ws_off;
     ws_off += mine;
     return unigist_attn_bwd(&run, (const char*)q + base * rq, (const char*)k + base * rk, (const char*)v + base * rk,
                             (const char*)o + base * rq, lse + base * p->num_q_heads, (const char*)d_o + base * rdo,
-                            (char*)dq + base * rq, (char*)dk + base * rk, (char*)dv + base * rk, ws, mine, st);
+                            (char*)dq + base * rq, (char*)dk + base * rk, (char*)dv + base * rk, ws, mine, stream);
   });
 }
 

@@ -12,6 +12,8 @@
 //   attn_bwd_dq_sm100_kernel   one thread block owns a 128-query tile of one query head and walks
 //                              the visible 64-key tiles: S, dP, dS as above, dQ += dS K in TMEM.
 // Tiles without a visible pair are never loaded; only "partial" tiles evaluate the mask.
+#include <algorithm>
+
 #include "sm100_ptx.cuh"
 #include "ug_common.cuh"
 
@@ -24,23 +26,43 @@ constexpr float kLog2e = 1.4426950408889634f;
 __device__ unsigned int g_bwd_timeout = 0;
 
 // ------------------------------------------------------------------------------------------------
+// A run of equal sequences as the per-token kernels see it: its geometry, its first packed token and its
+// [batch, Hq, N] block of Delta.  One problem is one run; a packed sample (cross-document masking) has several
+// and a warp finds its token's run by scanning the (at most twelve) first-token indices.
+struct TokRun {
+  Geom g;
+  long long tok_begin;
+  float* delta;
+};
+template <int kRuns>
+struct TokRuns {
+  TokRun run[kRuns];
+  int n;
+};
+
+
 // Delta and dO conversion: one warp per token.  The token's batch index and shifted position are worked out
 // once (the divisions cost more than a row's loads), then its Hq rows go by four at a time, all loads of the
 // four issued before the first use; 4 elements per lane and pass.
-template <bool kF32>
+template <bool kF32, int kRuns>
 __global__ void __launch_bounds__(256)
-bwd_prep_kernel(Geom g, int interleaved, int Hq, int D, long long tokens, const void* __restrict__ d_o,
-                const __nv_bfloat16* __restrict__ o, float* __restrict__ delta,
+bwd_prep_kernel(const __grid_constant__ TokRuns<kRuns> P, int interleaved, int Hq, int D, long long tokens,
+                const void* __restrict__ d_o, const __nv_bfloat16* __restrict__ o,
                 __nv_bfloat16* __restrict__ d_o_bf16, float* __restrict__ dq32) {
   constexpr int kHeads = 4;  // rows in flight
   const int lane = threadIdx.x & 31;
   const long long warp = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const long long nwarps = ((long long)gridDim.x * blockDim.x) >> 5;
-  for (long long tk = warp; tk < tokens; tk += nwarps) {  // tk = b * N + t
-    const long long b = tk / g.N;
-    const int t = (int)(tk - b * g.N);
+  for (long long tk = warp; tk < tokens; tk += nwarps) {  // tk = packed token index (run's first token + b * N + t)
+    int ri = 0;
+    if constexpr (kRuns > 1)
+      while (ri + 1 < P.n && tk >= P.run[ri + 1].tok_begin) ++ri;
+    const Geom g = P.run[ri].g;
+    const long long local = tk - P.run[ri].tok_begin;
+    const long long b = local / g.N;
+    const int t = (int)(local - b * g.N);
     // Delta is kept in shifted order, whatever the order of dO and O
-    float* delta_tok = delta + b * Hq * g.N + (interleaved ? unshift_perm(g, t) : t);
+    float* delta_tok = P.run[ri].delta + b * Hq * g.N + (interleaved ? unshift_perm(g, t) : t);
     const long long row0 = tk * Hq;
     for (int h0 = 0; h0 < Hq; h0 += kHeads) {
       float acc[kHeads];
@@ -120,6 +142,22 @@ __device__ __forceinline__ void key_q_interval(const Geom& g, bool key_is_raw, i
   }
 }
 
+// Query rows of segment qseg (numbered inside it, inclusive) that see key `key` of segment kseg:
+// Eq. 3 read column-wise, sinks included.  An empty interval has lo > hi.
+__device__ __forceinline__ void key_q_interval3(const Geom& g, int kseg, int key, bool key_valid, int qseg, int& lo,
+                                                int& hi) {
+  lo = 1;
+  hi = 0;
+  if (!key_valid) return;
+  if (kseg == kSegSink) {  // a sink is seen by the sinks from itself on and by every raw and gist query
+    lo = qseg == kSegSink ? key : 0;
+    hi = seg_len(g, qseg) - 1;
+    return;
+  }
+  if (qseg == kSegSink) return;  // sink queries see sinks only
+  key_q_interval(g, kseg == kSegRaw, key, true, qseg == kSegRaw, lo, hi);
+}
+
 // ------------------------------------------------------------------------------------------------
 // dK / dV kernel
 constexpr int KV_BM = 128;       // keys per block (TMEM lanes)
@@ -136,13 +174,15 @@ struct KvSmem {
 
 template <int D>
 __global__ void __launch_bounds__(kKvThreads, 1)
-attn_bwd_dkdv_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const __grid_constant__ CUtensorMap tm_q_gist,
+attn_bwd_dkdv_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_sink, const __grid_constant__ CUtensorMap tm_q_raw,
+                           const __grid_constant__ CUtensorMap tm_q_gist, const __grid_constant__ CUtensorMap tm_do_sink,
                            const __grid_constant__ CUtensorMap tm_do_raw, const __grid_constant__ CUtensorMap tm_do_gist,
-                           const __grid_constant__ CUtensorMap tm_k_raw, const __grid_constant__ CUtensorMap tm_k_gist,
+                           const __grid_constant__ CUtensorMap tm_k_sink, const __grid_constant__ CUtensorMap tm_k_raw,
+                           const __grid_constant__ CUtensorMap tm_k_gist, const __grid_constant__ CUtensorMap tm_v_sink,
                            const __grid_constant__ CUtensorMap tm_v_raw, const __grid_constant__ CUtensorMap tm_v_gist,
                            Geom g, int Hq, int Hkv, float scale, const float* __restrict__ lse,
                            const float* __restrict__ delta, __nv_bfloat16* __restrict__ dk,
-                           __nv_bfloat16* __restrict__ dv, int n_gist_kt) {
+                           __nv_bfloat16* __restrict__ dv, int n_sink_kt, int n_gist_kt) {
   using SM = KvSmem<D>;
   extern __shared__ unsigned char smem_dyn[];
   const uint32_t base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
@@ -159,25 +199,28 @@ attn_bwd_dkdv_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const _
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int hk = blockIdx.y, b = blockIdx.z, G = Hq / Hkv;
-  // gist key tiles are seen by every later query: heaviest, scheduled first
-  const bool key_is_raw = (int)blockIdx.x >= n_gist_kt;
-  const int kt = key_is_raw ? blockIdx.x - n_gist_kt : blockIdx.x;
-  const int key_seg_len = key_is_raw ? g.T : g.n;
-  const int key_seg_base = key_is_raw ? g.s : g.s + g.T;
+  // sink and gist key tiles are seen by every later query: heaviest, scheduled first
+  const int rank = blockIdx.x;
+  const int kseg = rank < n_sink_kt ? kSegSink : (rank < n_sink_kt + n_gist_kt ? kSegGist : kSegRaw);
+  const int kt = rank - (kseg == kSegSink ? 0 : (kseg == kSegGist ? n_sink_kt : n_sink_kt + n_gist_kt));
+  const int key_seg_len = seg_len(g, kseg);
+  const int key_seg_base = seg_base(g, kseg);
   const int key_a = kt * KV_BM, key_b = min(key_a + KV_BM - 1, key_seg_len - 1);
   const bool key_tile_whole = key_a + KV_BM - 1 <= key_seg_len - 1;
 
-  // query tiles that see this key tile: raw-segment tiles [rq_lo, rq_hi], gist-segment tiles [gq_lo, gq_hi]
-  int a_lo, a_hi, b_lo, b_hi, c_lo, c_hi, d_lo, d_hi;
-  key_q_interval(g, key_is_raw, key_a, true, true, a_lo, a_hi);   // first key vs raw queries
-  key_q_interval(g, key_is_raw, key_b, true, true, b_lo, b_hi);   // last key vs raw queries
-  key_q_interval(g, key_is_raw, key_a, true, false, c_lo, c_hi);  // first key vs gist queries
-  key_q_interval(g, key_is_raw, key_b, true, false, d_lo, d_hi);  // last key vs gist queries
-  const int n_raw_q = b_hi >= a_lo ? b_hi / KV_BN - a_lo / KV_BN + 1 : 0;
-  const int rq_lo = a_lo / KV_BN;
-  const int n_gist_q = d_hi >= c_lo ? d_hi / KV_BN - c_lo / KV_BN + 1 : 0;
-  const int gq_lo = c_lo / KV_BN;
-  const int n_iter = (n_raw_q + n_gist_q) * G;
+  // query tiles that see this key tile, per query segment: first tile and count, and the bounds inside which a
+  // tile is "full" (seen by the last key from t_lo on, by the first key up to t_hi)
+  int lo_a, hi_a, lo_b, hi_b;
+  key_q_interval3(g, kseg, key_a, true, kSegRaw, lo_a, hi_a);
+  key_q_interval3(g, kseg, key_b, true, kSegRaw, lo_b, hi_b);
+  const int n_raw_q = hi_b >= lo_a ? hi_b / KV_BN - lo_a / KV_BN + 1 : 0, rq_lo = lo_a / KV_BN, raw_t_lo = lo_b, raw_t_hi = hi_a;
+  key_q_interval3(g, kseg, key_a, true, kSegGist, lo_a, hi_a);
+  key_q_interval3(g, kseg, key_b, true, kSegGist, lo_b, hi_b);
+  const int n_gist_q = hi_b >= lo_a ? hi_b / KV_BN - lo_a / KV_BN + 1 : 0, gq_lo = lo_a / KV_BN, gist_t_lo = lo_b, gist_t_hi = hi_a;
+  key_q_interval3(g, kseg, key_a, true, kSegSink, lo_a, hi_a);
+  key_q_interval3(g, kseg, key_b, true, kSegSink, lo_b, hi_b);
+  const int n_sink_q = hi_b >= lo_a ? hi_b / KV_BN - lo_a / KV_BN + 1 : 0, sq_lo = lo_a / KV_BN, sink_t_lo = lo_b, sink_t_hi = hi_a;
+  const int n_iter = (n_raw_q + n_gist_q + n_sink_q) * G;
 
   if (threadIdx.x == 0) {
     mbar_init(bar_kv, 1);
@@ -200,19 +243,27 @@ attn_bwd_dkdv_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const _
   const uint32_t t_dK = tmem, t_dV = tmem + 128, t_A = tmem + 256, t_B = tmem + 384;
   bool ok = true;
 
-  auto tile_of = [&](int it, bool& q_is_raw, int& qt, int& head) {
+  auto tile_of = [&](int it, int& qseg, int& qt, int& head) {
     const int t = it / G;
     head = hk * G + (it - t * G);
-    q_is_raw = t < n_raw_q;
-    qt = q_is_raw ? rq_lo + t : gq_lo + (t - n_raw_q);
+    if (t < n_raw_q) {
+      qseg = kSegRaw;
+      qt = rq_lo + t;
+    } else if (t < n_raw_q + n_gist_q) {
+      qseg = kSegGist;
+      qt = gq_lo + (t - n_raw_q);
+    } else {
+      qseg = kSegSink;
+      qt = sq_lo + (t - n_raw_q - n_gist_q);
+    }
   };
 
   if (warp == 8) {
     // ------------------------------------------------------------ producer: K, V once; Q, dO, LSE, Delta per step
     if (lane == 0) {
       mbar_arrive_expect_tx(bar_kv, 2 * SM::kTile);
-      const CUtensorMap* mk = key_is_raw ? &tm_k_raw : &tm_k_gist;
-      const CUtensorMap* mv = key_is_raw ? &tm_v_raw : &tm_v_gist;
+      const CUtensorMap* mk = kseg == kSegRaw ? &tm_k_raw : (kseg == kSegGist ? &tm_k_gist : &tm_k_sink);
+      const CUtensorMap* mv = kseg == kSegRaw ? &tm_v_raw : (kseg == kSegGist ? &tm_v_gist : &tm_v_sink);
 #pragma unroll
       for (int sl = 0; sl < D / 64; ++sl) {
         tma_load_4d(sK + sl * SM::kSlab, mk, bar_kv, sl * 64, hk, key_a, b);
@@ -221,12 +272,11 @@ attn_bwd_dkdv_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const _
     }
     for (int it = 0; it < n_iter; ++it) {
       const int st = it & 1;
-      bool q_is_raw;
-      int qt, head;
-      tile_of(it, q_is_raw, qt, head);
+      int qseg, qt, head;
+      tile_of(it, qseg, qt, head);
       if (it >= 2) ok = mbar_wait_warp(bar_empty[st], ((it >> 1) - 1) & 1);
       if (!ok) break;
-      const int q_seg_len = q_is_raw ? g.T : g.n, q_seg_base = q_is_raw ? g.s : g.s + g.T;
+      const int q_seg_len = seg_len(g, qseg), q_seg_base = seg_base(g, qseg);
       float* ls = stats + st * 2 * KV_BN;
       const long long row_base = ((long long)b * Hq + head) * g.N + q_seg_base;
 #pragma unroll
@@ -240,8 +290,8 @@ attn_bwd_dkdv_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const _
       __syncwarp();
       if (lane == 0) {
         mbar_arrive_expect_tx(bar_full[st], 2 * SM::kTile);
-        const CUtensorMap* mq = q_is_raw ? &tm_q_raw : &tm_q_gist;
-        const CUtensorMap* md = q_is_raw ? &tm_do_raw : &tm_do_gist;
+        const CUtensorMap* mq = qseg == kSegRaw ? &tm_q_raw : (qseg == kSegGist ? &tm_q_gist : &tm_q_sink);
+        const CUtensorMap* md = qseg == kSegRaw ? &tm_do_raw : (qseg == kSegGist ? &tm_do_gist : &tm_do_sink);
 #pragma unroll
         for (int sl = 0; sl < D / 64; ++sl) {
           tma_load_4d(sQ[st] + sl * SM::kSlab, mq, bar_full[st], sl * 64, head, qt * KV_BN, b);
@@ -317,21 +367,23 @@ attn_bwd_dkdv_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const _
     const bool key_valid = key <= key_b;
     const uint32_t lane_base = static_cast<uint32_t>(qd * 32) << 16;
     const float scale_log2 = scale * kLog2e;
-    int my_lo[2], my_hi[2];  // [0]: vs raw queries, [1]: vs gist queries
-    key_q_interval(g, key_is_raw, key, key_valid, true, my_lo[0], my_hi[0]);
-    key_q_interval(g, key_is_raw, key, key_valid, false, my_lo[1], my_hi[1]);
+    int my_lo_r, my_hi_r, my_lo_g, my_hi_g, my_lo_s, my_hi_s;  // queries that see this key, per query segment
+    key_q_interval3(g, kseg, key, key_valid, kSegRaw, my_lo_r, my_hi_r);
+    key_q_interval3(g, kseg, key, key_valid, kSegGist, my_lo_g, my_hi_g);
+    key_q_interval3(g, kseg, key, key_valid, kSegSink, my_lo_s, my_hi_s);
 
     for (int it = 0; it < n_iter && ok; ++it) {
       const int st = it & 1;
-      bool q_is_raw;
-      int qt, head;
-      tile_of(it, q_is_raw, qt, head);
-      const int q0 = qt * KV_BN, q_seg_len = q_is_raw ? g.T : g.n;
+      int qseg, qt, head;
+      tile_of(it, qseg, qt, head);
+      const int q0 = qt * KV_BN, q_seg_len = seg_len(g, qseg);
       const int qb = min(q0 + KV_BN - 1, q_seg_len - 1);
       // full: every (query, key) pair of the tile is visible -> no mask arithmetic
-      const int t_lo = q_is_raw ? b_lo : d_lo, t_hi = q_is_raw ? a_hi : c_hi;
+      const int t_lo = qseg == kSegRaw ? raw_t_lo : (qseg == kSegGist ? gist_t_lo : sink_t_lo);
+      const int t_hi = qseg == kSegRaw ? raw_t_hi : (qseg == kSegGist ? gist_t_hi : sink_t_hi);
       const bool full = key_tile_whole && q0 >= t_lo && qb <= t_hi;
-      const int lo = my_lo[q_is_raw ? 0 : 1] - q0 - 64 * hf, hi = my_hi[q_is_raw ? 0 : 1] - q0 - 64 * hf;
+      const int lo = (qseg == kSegRaw ? my_lo_r : (qseg == kSegGist ? my_lo_g : my_lo_s)) - q0 - 64 * hf;
+      const int hi = (qseg == kSegRaw ? my_hi_r : (qseg == kSegGist ? my_hi_g : my_hi_s)) - q0 - 64 * hf;
       const float* ls = stats + st * 2 * KV_BN + 64 * hf;
       const float* dl = ls + KV_BN;
       ok = mbar_wait_warp(bar_full[st], (it >> 1) & 1) && mbar_wait_warp(bar_S, it & 1);
@@ -453,12 +505,14 @@ struct DqSmem {
 
 template <int D>
 __global__ void __launch_bounds__(kDqThreads, 2)
-attn_bwd_dq_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const __grid_constant__ CUtensorMap tm_q_gist,
+attn_bwd_dq_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_sink, const __grid_constant__ CUtensorMap tm_q_raw,
+                         const __grid_constant__ CUtensorMap tm_q_gist, const __grid_constant__ CUtensorMap tm_do_sink,
                          const __grid_constant__ CUtensorMap tm_do_raw, const __grid_constant__ CUtensorMap tm_do_gist,
-                         const __grid_constant__ CUtensorMap tm_k_raw, const __grid_constant__ CUtensorMap tm_k_gist,
+                         const __grid_constant__ CUtensorMap tm_k_sink, const __grid_constant__ CUtensorMap tm_k_raw,
+                         const __grid_constant__ CUtensorMap tm_k_gist, const __grid_constant__ CUtensorMap tm_v_sink,
                          const __grid_constant__ CUtensorMap tm_v_raw, const __grid_constant__ CUtensorMap tm_v_gist,
                          Geom g, int Hq, int Hkv, float scale, const float* __restrict__ lse,
-                         const float* __restrict__ delta, __nv_bfloat16* __restrict__ dq, int n_raw_qt) {
+                         const float* __restrict__ delta, __nv_bfloat16* __restrict__ dq, int n_sink_qt, int n_raw_qt) {
   using SM = DqSmem<D>;
   extern __shared__ unsigned char smem_dyn[];
   const uint32_t base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
@@ -472,17 +526,32 @@ attn_bwd_dq_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const __g
 
   const int warp = threadIdx.x >> 5;
   const int h = blockIdx.y, b = blockIdx.z, hk = h / (Hq / Hkv);
-  const int qt_lin = gridDim.x - 1 - blockIdx.x;  // heaviest tiles first
-  const bool q_is_raw = qt_lin < n_raw_qt;
-  const int qt = q_is_raw ? qt_lin : qt_lin - n_raw_qt;
-  const int seg_len = q_is_raw ? g.T : g.n;
-  const int seg_base = q_is_raw ? g.s : g.s + g.T;
-  const int row_a = qt * DQ_BM, row_b = min(row_a + DQ_BM - 1, seg_len - 1);
-  const RowIv iv_a = row_intervals(g, seg_base + row_a), iv_b = row_intervals(g, seg_base + row_b);
-  // visible 64-key tiles: raw tiles [raw_lo, raw_hi] then gist tiles [0, n_gist)
-  const int raw_lo = iv_a.lo_raw / DQ_BN, n_raw = iv_b.hi_raw / DQ_BN - raw_lo + 1;
+  // heaviest tiles first: gist query tiles from the end, then raw query tiles from the end, sink tiles last
+  const int qt_lin = gridDim.x - 1 - blockIdx.x;
+  const int qseg = qt_lin < n_sink_qt ? kSegSink : (qt_lin < n_sink_qt + n_raw_qt ? kSegRaw : kSegGist);
+  const int qt = qt_lin - (qseg == kSegSink ? 0 : (qseg == kSegRaw ? n_sink_qt : n_sink_qt + n_raw_qt));
+  const int q_len = seg_len(g, qseg);
+  const int q_base = seg_base(g, qseg);
+  const int row_a = qt * DQ_BM, row_b = min(row_a + DQ_BM - 1, q_len - 1);
+  const RowIv iv_a = row_intervals(g, q_base + row_a), iv_b = row_intervals(g, q_base + row_b);
+  // visible 64-key tiles: sink tiles [0, n_sink), raw tiles [raw_lo, raw_lo + n_raw), gist tiles [0, n_gist)
+  const int n_sink = iv_b.hi_sink >= 0 ? iv_b.hi_sink / DQ_BN + 1 : 0;
+  const int raw_lo = iv_a.lo_raw / DQ_BN, n_raw = iv_b.hi_raw >= iv_a.lo_raw ? iv_b.hi_raw / DQ_BN - raw_lo + 1 : 0;
   const int n_gist = iv_b.hi_gist >= 0 ? iv_b.hi_gist / DQ_BN + 1 : 0;
-  const int nt = n_raw + n_gist;
+  const int nt = n_sink + n_raw + n_gist;
+  // step j: its key segment and 64-key tile
+  auto key_tile = [&](int j, int& sg, int& idx) {
+    if (j < n_raw) {
+      sg = kSegRaw;
+      idx = raw_lo + j;
+    } else if (j < n_raw + n_gist) {
+      sg = kSegGist;
+      idx = j - n_raw;
+    } else {
+      sg = kSegSink;
+      idx = j - n_raw - n_gist;
+    }
+  };
 
   if (threadIdx.x == 0) {
     mbar_init(bar_q, 1);
@@ -504,18 +573,18 @@ attn_bwd_dq_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const __g
   if (warp == 4) {
     if (elect_one()) {
       mbar_arrive_expect_tx(bar_q, 2 * SM::kQTile);
-      const CUtensorMap* mq = q_is_raw ? &tm_q_raw : &tm_q_gist;
-      const CUtensorMap* md = q_is_raw ? &tm_do_raw : &tm_do_gist;
+      const CUtensorMap* mq = qseg == kSegRaw ? &tm_q_raw : (qseg == kSegGist ? &tm_q_gist : &tm_q_sink);
+      const CUtensorMap* md = qseg == kSegRaw ? &tm_do_raw : (qseg == kSegGist ? &tm_do_gist : &tm_do_sink);
 #pragma unroll
       for (int sl = 0; sl < D / 64; ++sl) {
         tma_load_4d(sQ + sl * SM::kQSlab, mq, bar_q, sl * 64, h, row_a, b);
         tma_load_4d(sDO + sl * SM::kQSlab, md, bar_q, sl * 64, h, row_a, b);
       }
       for (int j = 0; j < nt && ok; ++j) {
-        const bool is_raw = j < n_raw;
-        const int idx = is_raw ? raw_lo + j : j - n_raw;
-        const CUtensorMap* mk = is_raw ? &tm_k_raw : &tm_k_gist;
-        const CUtensorMap* mv = is_raw ? &tm_v_raw : &tm_v_gist;
+        int sg, idx;
+        key_tile(j, sg, idx);
+        const CUtensorMap* mk = sg == kSegRaw ? &tm_k_raw : (sg == kSegGist ? &tm_k_gist : &tm_k_sink);
+        const CUtensorMap* mv = sg == kSegRaw ? &tm_v_raw : (sg == kSegGist ? &tm_v_gist : &tm_v_sink);
         if (j > 0) ok = mbar_wait(bar_s, (j - 1) & 1);  // dP(j-1) done: V buffer free
         if (!ok) break;
         mbar_arrive_expect_tx(bar_v, SM::kKTile);
@@ -564,24 +633,29 @@ attn_bwd_dq_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const __g
     const int r_in_tile = threadIdx.x;
     const int row = min(row_a + r_in_tile, row_b);
     const bool valid = row_a + r_in_tile <= row_b;
-    const RowIv my = row_intervals(g, seg_base + row);
+    const RowIv my = row_intervals(g, q_base + row);
     const uint32_t lane_base = static_cast<uint32_t>(warp * 32) << 16;
     const float scale_log2 = scale * kLog2e;
-    const long long stat_idx = ((long long)b * Hq + h) * g.N + seg_base + row;
+    const long long stat_idx = ((long long)b * Hq + h) * g.N + q_base + row;
     const float lse2 = lse[stat_idx] * kLog2e, dl = delta[stat_idx];
     for (int j = 0; j < nt && ok; ++j) {
-      const bool is_raw = j < n_raw;
-      const int col0 = (is_raw ? raw_lo + j : j - n_raw) * DQ_BN;
+      int sg, idx;
+      key_tile(j, sg, idx);
+      const int col0 = idx * DQ_BN;
       bool full;
       int lo, hi;
-      if (is_raw) {
+      if (sg == kSegRaw) {
         full = col0 >= iv_b.lo_raw && col0 + DQ_BN - 1 <= iv_a.hi_raw;
         lo = my.lo_raw - col0;
         hi = my.hi_raw - col0;
-      } else {
+      } else if (sg == kSegGist) {
         full = col0 + DQ_BN - 1 <= iv_a.hi_gist;
         lo = 0;
         hi = my.hi_gist - col0;
+      } else {
+        full = col0 + DQ_BN - 1 <= iv_a.hi_sink;
+        lo = 0;
+        hi = my.hi_sink - col0;
       }
       ok = mbar_wait_warp(bar_s, j & 1);
       if (!ok) break;
@@ -615,7 +689,7 @@ attn_bwd_dq_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_raw, const __g
     if (ok) ok = mbar_wait_warp(bar_pv, (nt - 1) & 1);
     if (ok) {
       tc_fence_after();
-      const long long tok = (long long)b * g.N + seg_base + row_a + r_in_tile;
+      const long long tok = (long long)b * g.N + q_base + row_a + r_in_tile;
       __nv_bfloat16* drow = dq + (tok * Hq + h) * D;
 #pragma unroll
       for (int c = 0; c < D / 32; ++c) {
@@ -691,22 +765,6 @@ __device__ __forceinline__ void fused_p_chunk(const uint32_t (&v)[32], const flo
   }
 }
 
-// Query rows of segment qseg (numbered inside it, inclusive) that see key `key` of segment kseg:
-// Eq. 3 read column-wise, sinks included.  An empty interval has lo > hi.
-__device__ __forceinline__ void key_q_interval3(const Geom& g, int kseg, int key, bool key_valid, int qseg, int& lo,
-                                                int& hi) {
-  lo = 1;
-  hi = 0;
-  if (!key_valid) return;
-  if (kseg == kSegSink) {  // a sink is seen by the sinks from itself on and by every raw and gist query
-    lo = qseg == kSegSink ? key : 0;
-    hi = seg_len(g, qseg) - 1;
-    return;
-  }
-  if (qseg == kSegSink) return;  // sink queries see sinks only
-  key_q_interval(g, kseg == kSegRaw, key, true, qseg == kSegRaw, lo, hi);
-}
-
 struct FuSmem {
   static constexpr int kSlab = 128 * 128;    // [128 rows x 64 bf16]
   static constexpr int kTile = 2 * kSlab;    // [128 x 128] bf16
@@ -718,18 +776,49 @@ struct FuSmem {
   static constexpr int kBytes = 232448;  // all a block may have; the 1024-byte alignment slack comes out of it
 };
 
+// One launch unit of the fused backward: a batch of sequences of one geometry with its own tensor maps (one per
+// segment) and output pointers.  A call on one problem is one unit with a (blocks, 1, batch) grid; a packed
+// sample under cross-document masking is several units in ONE launch with a flat grid, and a block finds its
+// unit from the units' first block indices.
+struct alignas(64) BwdRun {
+  CUtensorMap q[3], dout[3], k[3], v[3], dq[3];
+  Geom g;
+  const float* lse;
+  const float* delta;
+  __nv_bfloat16* dk;
+  __nv_bfloat16* dv;
+  int n_sink_kt, n_gist_kt, n_raw_kt;
+  int cta_begin, plane;  // flat grid: first block of the unit; blocks per batch index
+  FastDiv heavy_div, raw_div, plane_div;
+};
+template <int kRuns>
+struct BwdRuns {
+  BwdRun run[kRuns];
+  int n;
+};
+constexpr int kMaxRunsPerLaunch = 12;  // 12 units are 24 KB of kernel parameters (the limit is 32 KB)
+
+template <int kRuns>
 __global__ void __launch_bounds__(kFuThreads, 1)
-attn_bwd_fused_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_sink, const __grid_constant__ CUtensorMap tm_q_raw,
-                            const __grid_constant__ CUtensorMap tm_q_gist, const __grid_constant__ CUtensorMap tm_do_sink,
-                            const __grid_constant__ CUtensorMap tm_do_raw, const __grid_constant__ CUtensorMap tm_do_gist,
-                            const __grid_constant__ CUtensorMap tm_k_sink, const __grid_constant__ CUtensorMap tm_k_raw,
-                            const __grid_constant__ CUtensorMap tm_k_gist, const __grid_constant__ CUtensorMap tm_v_sink,
-                            const __grid_constant__ CUtensorMap tm_v_raw, const __grid_constant__ CUtensorMap tm_v_gist,
-                            const __grid_constant__ CUtensorMap tm_dq_sink, const __grid_constant__ CUtensorMap tm_dq_raw,
-                            const __grid_constant__ CUtensorMap tm_dq_gist, Geom g, int Hq, int Hkv, float scale,
-                            const float* __restrict__ lse, const float* __restrict__ delta,
-                            __nv_bfloat16* __restrict__ dk, __nv_bfloat16* __restrict__ dv, int n_sink_kt, int n_gist_kt,
-                            int interleaved, FastDiv rdiv) {
+attn_bwd_fused_sm100_kernel(const __grid_constant__ BwdRuns<kRuns> P, int Hq, int Hkv, float scale, int interleaved,
+                            FastDiv rdiv) {
+  int ri = 0, bx, b;
+  if constexpr (kRuns == 1) {
+    bx = blockIdx.x, b = blockIdx.z;
+  } else {
+    const int c = blockIdx.x;
+    while (ri + 1 < P.n && c >= P.run[ri + 1].cta_begin) ++ri;
+    const int local = c - P.run[ri].cta_begin;
+    b = fdiv(P.run[ri].plane_div, local);
+    bx = local - b * P.run[ri].plane;
+  }
+  const BwdRun& R = P.run[ri];
+  const Geom g = R.g;
+  const float* __restrict__ lse = R.lse;
+  const float* __restrict__ delta = R.delta;
+  __nv_bfloat16* __restrict__ dk = R.dk;
+  __nv_bfloat16* __restrict__ dv = R.dv;
+  const int n_sink_kt = R.n_sink_kt, n_gist_kt = R.n_gist_kt, n_raw_kt = R.n_raw_kt;
   using SM = FuSmem;
   constexpr int D = 128;
   extern __shared__ unsigned char smem_dyn[];
@@ -753,9 +842,24 @@ attn_bwd_fused_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_sink, const
   volatile int* q_issued = reinterpret_cast<volatile int*>(gen + SM::kOffBars + 144);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  // blockIdx.x = key tile rank * Hkv + KV head.  Sink and gist key tiles are seen by every later query:
-  // they are the heaviest and come first, for all KV heads, before any raw key tile.
-  const int hk = blockIdx.x % Hkv, rank = blockIdx.x / Hkv, b = blockIdx.z, G = Hq / Hkv;
+  // Block order (the hardware starts blocks in the order of their index): sink and gist key tiles are seen by
+  // every later query, so they are the heaviest and come first, for all KV heads, before any raw key tile;
+  // inside each of the two classes the key tiles of ONE KV head are consecutive.  The blocks that run side by
+  // side then belong to one or two KV heads and walk the same Q / dO / dQ tiles at about the same time, so a
+  // tile comes from DRAM once and from L2 for every other block that needs it (with the KV heads interleaved
+  // instead, a head's sweep over its queries was repeated by every wave of its blocks: about 8 times the
+  // algorithmic DRAM traffic, and a fifth more time).
+  const int G = Hq / Hkv;
+  const int n_heavy_kt = n_sink_kt + n_gist_kt;
+  int hk, rank;
+  if (bx < n_heavy_kt * Hkv) {
+    hk = fdiv(R.heavy_div, bx);
+    rank = bx - hk * n_heavy_kt;
+  } else {
+    const int y = bx - n_heavy_kt * Hkv;
+    hk = fdiv(R.raw_div, y);
+    rank = n_heavy_kt + (y - hk * n_raw_kt);
+  }
   const int kseg = rank < n_sink_kt ? kSegSink : (rank < n_sink_kt + n_gist_kt ? kSegGist : kSegRaw);
   const int kt = rank - (kseg == kSegSink ? 0 : (kseg == kSegGist ? n_sink_kt : n_sink_kt + n_gist_kt));
   const int key_seg_len = seg_len(g, kseg);
@@ -844,8 +948,8 @@ attn_bwd_fused_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_sink, const
       auto first_unit = [&](int sg, int row0) { return interleaved && sg == kSegRaw ? fdiv(rdiv, row0) : row0; };
       if (lane == 0) {
         mbar_arrive_expect_tx(bar_kv, 2 * SM::kTile);
-        const CUtensorMap* mk = kseg == kSegRaw ? &tm_k_raw : (kseg == kSegGist ? &tm_k_gist : &tm_k_sink);
-        const CUtensorMap* mv = kseg == kSegRaw ? &tm_v_raw : (kseg == kSegGist ? &tm_v_gist : &tm_v_sink);
+        const CUtensorMap* mk = &R.k[kseg];
+        const CUtensorMap* mv = &R.v[kseg];
 #pragma unroll
         for (int sl = 0; sl < 2; ++sl) {
           tma_load_5d(sK + sl * SM::kSlab, mk, bar_kv, sl * 64, hk, 0, first_unit(kseg, key_a), b);
@@ -885,7 +989,7 @@ attn_bwd_fused_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_sink, const
         __syncwarp();
         if (lane == 0) {
           mbar_arrive_expect_tx(full_q0 + 8 * st, SM::kTile);
-          const CUtensorMap* mq = qseg == kSegRaw ? &tm_q_raw : (qseg == kSegGist ? &tm_q_gist : &tm_q_sink);
+          const CUtensorMap* mq = &R.q[qseg];
 #pragma unroll
           for (int sl = 0; sl < 2; ++sl)
             tma_load_5d(sQ0 + st * SM::kTile + sl * SM::kSlab, mq, full_q0 + 8 * st, sl * 64, head, 0,
@@ -898,7 +1002,7 @@ attn_bwd_fused_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_sink, const
         if (!ok) break;
         if (lane == 0) {
           mbar_arrive_expect_tx(full_do, SM::kTile);
-          const CUtensorMap* md = qseg == kSegRaw ? &tm_do_raw : (qseg == kSegGist ? &tm_do_gist : &tm_do_sink);
+          const CUtensorMap* md = &R.dout[qseg];
 #pragma unroll
           for (int sl = 0; sl < 2; ++sl)
             tma_load_5d(sDO + sl * SM::kSlab, md, full_do, sl * 64, head, 0, first_unit(qseg, qt * 128), b);
@@ -1006,7 +1110,7 @@ attn_bwd_fused_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_sink, const
     for (int it = 0; it < n_iter && ok; ++it, advance(cur)) {
       int qseg, qt, head;
       tile_of(cur, qseg, qt, head);
-      const CUtensorMap* mdq = qseg == kSegRaw ? &tm_dq_raw : (qseg == kSegGist ? &tm_dq_gist : &tm_dq_sink);
+      const CUtensorMap* mdq = &R.dq[qseg];
       const int nq = seg_len(g, qseg) - qt * 128;  // rows of this tile inside the segment (may exceed 128)
       ok = mbar_wait_warp(bar_dQ, it & 1);
       if (!ok) break;
@@ -1176,16 +1280,22 @@ attn_bwd_fused_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_sink, const
 
 // dQ (bf16) = scale * dQ accumulated in fp32 (shifted order, head_dim 128).  One warp per token: Hq rows of
 // 128 floats, 4 per lane; the bf16 row goes to the token's shifted or interleaved position.
+template <int kRuns>
 __global__ void __launch_bounds__(256)
-dq_convert_kernel(Geom g, int interleaved, int Hq, long long tokens, const float* __restrict__ src,
-                  __nv_bfloat16* __restrict__ dst, float scale) {
+dq_convert_kernel(const __grid_constant__ TokRuns<kRuns> P, int interleaved, int Hq, long long tokens,
+                  const float* __restrict__ src, __nv_bfloat16* __restrict__ dst, float scale) {
   const int lane = threadIdx.x & 31;
   const long long warp = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const long long nwarps = ((long long)gridDim.x * blockDim.x) >> 5;
-  for (long long tk = warp; tk < tokens; tk += nwarps) {  // tk = b * N + sigma
-    const long long b = tk / g.N;
-    const int sigma = (int)(tk - b * g.N);
-    const long long out_tk = b * g.N + (interleaved ? shift_perm(g, sigma) : sigma);
+  for (long long tk = warp; tk < tokens; tk += nwarps) {  // tk = packed token index, shifted order inside a sequence
+    int ri = 0;
+    if constexpr (kRuns > 1)
+      while (ri + 1 < P.n && tk >= P.run[ri + 1].tok_begin) ++ri;
+    const Geom g = P.run[ri].g;
+    const long long local = tk - P.run[ri].tok_begin;
+    const long long b = local / g.N;
+    const int sigma = (int)(local - b * g.N);
+    const long long out_tk = P.run[ri].tok_begin + b * g.N + (interleaved ? shift_perm(g, sigma) : sigma);
     const float4* s4 = reinterpret_cast<const float4*>(src + tk * Hq * 128) + lane;
     uint2* d2 = reinterpret_cast<uint2*>(dst + out_tk * Hq * 128) + lane;
     for (int h0 = 0; h0 < Hq; h0 += 4) {
@@ -1203,98 +1313,223 @@ dq_convert_kernel(Geom g, int interleaved, int Hq, long long tokens, const float
 
 }  // namespace
 
+namespace {
+
+size_t align256(size_t x) { return (x + 255) / 256 * 256; }
+
+// The backward's scratch for `tokens` packed tokens: Delta (fp32, per run a [batch, Hq, N] block that starts at
+// float Hq * first token), the bf16 copy of an fp32 dO, and for head_dim 128 the fp32 dQ accumulator.
+struct BwdScratch {
+  float* delta;
+  __nv_bfloat16* do_bf16;
+  float* dq32;
+};
+BwdScratch carve_scratch(void* workspace, long long tokens, int Hq, int D, bool f32) {
+  char* ws = static_cast<char*>(workspace);
+  BwdScratch sc;
+  sc.delta = reinterpret_cast<float*>(ws);
+  ws += align256((size_t)tokens * Hq * sizeof(float));
+  sc.do_bf16 = f32 ? reinterpret_cast<__nv_bfloat16*>(ws) : nullptr;
+  if (f32) ws += align256((size_t)tokens * Hq * D * 2);
+  sc.dq32 = D == 128 ? reinterpret_cast<float*>(ws) : nullptr;
+  return sc;
+}
+
+template <int kRuns>
+int32_t launch_prep(const TokRuns<kRuns>& T, const unigist_problem& p, long long tokens, const void* d_o, const void* o,
+                    const BwdScratch& sc, cudaStream_t st) {
+  const bool f32 = (p.flags & UNIGIST_FLAG_DOUT_FP32) != 0;
+  const int il = (p.flags & UNIGIST_FLAG_INTERLEAVED) ? 1 : 0;
+  const int blocks = (int)((tokens + 7) / 8 < sm_count() * 16 ? (tokens + 7) / 8 : sm_count() * 16);
+  {
+    KernelScope ks("bwd_prep_kernel", st);
+    if (f32)
+      bwd_prep_kernel<true, kRuns><<<blocks, 256, 0, st>>>(T, il, p.num_q_heads, p.head_dim, tokens, d_o,
+                                                           (const __nv_bfloat16*)o, sc.do_bf16, sc.dq32);
+    else
+      bwd_prep_kernel<false, kRuns><<<blocks, 256, 0, st>>>(T, il, p.num_q_heads, p.head_dim, tokens, d_o,
+                                                            (const __nv_bfloat16*)o, nullptr, sc.dq32);
+  }
+  return check_launch("backward prep kernel");
+}
+
+template <int kRuns>
+int32_t launch_convert(const TokRuns<kRuns>& T, const unigist_problem& p, long long tokens, const BwdScratch& sc, void* dq,
+                       float scale, cudaStream_t st) {
+  const int blocks = (int)((tokens + 7) / 8 < sm_count() * 16 ? (tokens + 7) / 8 : sm_count() * 16);
+  {
+    KernelScope ks("dq_convert_kernel", st);
+    dq_convert_kernel<kRuns><<<blocks, 256, 0, st>>>(T, (p.flags & UNIGIST_FLAG_INTERLEAVED) ? 1 : 0, p.num_q_heads, tokens,
+                                                     sc.dq32, (__nv_bfloat16*)dq, scale);
+  }
+  return check_launch("dQ convert kernel");
+}
+
+// Tensor maps and tile counts of one launch unit of the fused backward: `batch` sequences of geometry g whose
+// first rows are the given pointers.  128-row tile maps per segment (sinks, raw, gists) that read shifted or
+// interleaved tensors, and reduction maps over the fp32 dQ tensor (always shifted).
+int32_t fill_bwd_run(BwdRun* R, const Geom& g, const unigist_problem& p, int batch, const void* q, const void* do_src,
+                     const void* k, const void* v, float* dq32, const float* lse, const float* delta, void* dk, void* dv) {
+  const int D = p.head_dim, Hq = p.num_q_heads, Hkv = p.num_kv_heads;
+  const bool il = (p.flags & UNIGIST_FLAG_INTERLEAVED) != 0;
+  for (int sg = 0; sg < 3; ++sg) {
+    if (int32_t rc = encode_tile_map(&R->q[sg], q, D, Hq, batch, g.s, g.T, g.r, g.n, il, sg)) return rc;
+    if (int32_t rc = encode_tile_map(&R->dout[sg], do_src, D, Hq, batch, g.s, g.T, g.r, g.n, il, sg)) return rc;
+    if (int32_t rc = encode_tile_map(&R->k[sg], k, D, Hkv, batch, g.s, g.T, g.r, g.n, il, sg)) return rc;
+    if (int32_t rc = encode_tile_map(&R->v[sg], v, D, Hkv, batch, g.s, g.T, g.r, g.n, il, sg)) return rc;
+    const int rows = seg_len(g, sg) > 0 ? seg_len(g, sg) : 1;  // a tensor map cannot be empty
+    if (int32_t rc = encode_segment_map_f32(&R->dq[sg], dq32, D, Hq, g.N, batch, seg_base(g, sg), rows, 32, 32)) return rc;
+  }
+  R->g = g;
+  R->lse = lse;
+  R->delta = delta;
+  R->dk = static_cast<__nv_bfloat16*>(dk);
+  R->dv = static_cast<__nv_bfloat16*>(dv);
+  R->n_sink_kt = (g.s + 127) / 128;
+  R->n_gist_kt = (g.n + 127) / 128;
+  R->n_raw_kt = (g.T + 127) / 128;
+  R->plane = (R->n_sink_kt + R->n_gist_kt + R->n_raw_kt) * Hkv;
+  R->cta_begin = 0;
+  R->heavy_div = make_fastdiv(R->n_sink_kt + R->n_gist_kt);
+  R->raw_div = make_fastdiv(R->n_raw_kt);
+  R->plane_div = make_fastdiv(R->plane);
+  return UNIGIST_OK;
+}
+
+template <int kRuns>
+int32_t launch_fused(const BwdRuns<kRuns>& P, dim3 grid, const unigist_problem& p, float scale, cudaStream_t st) {
+  cudaError_t e = cudaFuncSetAttribute(attn_bwd_fused_sm100_kernel<kRuns>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       FuSmem::kBytes);
+  if (e != cudaSuccess) return fail(UNIGIST_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
+  {
+    KernelScope ks("attn_bwd_fused_sm100_kernel", st);
+    attn_bwd_fused_sm100_kernel<kRuns><<<grid, kFuThreads, FuSmem::kBytes, st>>>(
+        P, p.num_q_heads, p.num_kv_heads, scale, (p.flags & UNIGIST_FLAG_INTERLEAVED) ? 1 : 0, make_fastdiv(p.ratio));
+  }
+  return check_launch("tcgen05 fused backward kernel");
+}
+
+}  // namespace
+
+size_t bwd_scratch_bytes(long long tokens, int Hq, int D, bool dout_fp32) {
+  size_t b = align256((size_t)tokens * Hq * sizeof(float));
+  if (dout_fp32) b += align256((size_t)tokens * Hq * D * 2);
+  if (D == 128) b += align256((size_t)tokens * Hq * D * sizeof(float));
+  return b;
+}
+
 int32_t launch_bwd_sm100(const Geom& g, const unigist_problem& p, float scale, const void* q, const void* k,
                          const void* v, const void* o, const float* lse, const void* d_o, void* dq, void* dk,
                          void* dv, void* workspace, cudaStream_t st) {
   const int D = p.head_dim, Hq = p.num_q_heads, Hkv = p.num_kv_heads, B = p.batch;
   const bool f32 = (p.flags & UNIGIST_FLAG_DOUT_FP32) != 0;
-  const bool il = (p.flags & UNIGIST_FLAG_INTERLEAVED) != 0;
-  float* delta = static_cast<float*>(workspace);
-  const size_t delta_bytes = ((size_t)B * Hq * g.N * sizeof(float) + 255) / 256 * 256;
-  __nv_bfloat16* do_bf16 = reinterpret_cast<__nv_bfloat16*>(static_cast<char*>(workspace) + delta_bytes);
-  const void* do_src = f32 ? static_cast<const void*>(do_bf16) : d_o;
-  const size_t do_bytes = f32 ? ((size_t)B * g.N * Hq * D * 2 + 255) / 256 * 256 : 0;
+  const long long tokens = (long long)B * g.N;
+  const BwdScratch sc = carve_scratch(workspace, tokens, Hq, D, f32);
+  float* delta = sc.delta;
+  const void* do_src = f32 ? static_cast<const void*>(sc.do_bf16) : d_o;
   const bool fused = D == 128;  // head_dim 64 takes the two-kernel path
-  float* dq32 = fused ? reinterpret_cast<float*>(static_cast<char*>(workspace) + delta_bytes + do_bytes) : nullptr;
-  {
-    const long long tokens = (long long)B * g.N;
-    const int blocks = (int)((tokens + 7) / 8 < sm_count() * 16 ? (tokens + 7) / 8 : sm_count() * 16);
-    KernelScope ks("bwd_prep_kernel", st);
-    if (f32)
-      bwd_prep_kernel<true><<<blocks, 256, 0, st>>>(g, il ? 1 : 0, Hq, D, tokens, d_o, (const __nv_bfloat16*)o, delta, do_bf16, dq32);
-    else
-      bwd_prep_kernel<false><<<blocks, 256, 0, st>>>(g, il ? 1 : 0, Hq, D, tokens, d_o, (const __nv_bfloat16*)o, delta, nullptr, dq32);
-  }
-  if (int32_t rc = check_launch("backward prep kernel")) return rc;
+  TokRuns<1> T;
+  T.n = 1;
+  T.run[0].g = g;
+  T.run[0].tok_begin = 0;
+  T.run[0].delta = delta;
+  if (int32_t rc = launch_prep(T, p, tokens, d_o, o, sc, st)) return rc;
 
-  CUtensorMap mq[2], md[2], mk[2], mv[2], mk64[2], mv64[2];
-  const long long first[2] = {g.s, (long long)g.s + g.T}, len[2] = {g.T, g.n};
-  for (int sgm = 0; sgm < 2; ++sgm) {
-    if (fused) continue;
-    if (int32_t rc = encode_segment_map(&mq[sgm], q, D, Hq, g.N, B, first[sgm], len[sgm], 128)) return rc;
-    if (int32_t rc = encode_segment_map(&md[sgm], do_src, D, Hq, g.N, B, first[sgm], len[sgm], 128)) return rc;
-    if (int32_t rc = encode_segment_map(&mk[sgm], k, D, Hkv, g.N, B, first[sgm], len[sgm], 128)) return rc;
-    if (int32_t rc = encode_segment_map(&mv[sgm], v, D, Hkv, g.N, B, first[sgm], len[sgm], 128)) return rc;
-    if (int32_t rc = encode_segment_map(&mk64[sgm], k, D, Hkv, g.N, B, first[sgm], len[sgm], DQ_BN)) return rc;
-    if (int32_t rc = encode_segment_map(&mv64[sgm], v, D, Hkv, g.N, B, first[sgm], len[sgm], DQ_BN)) return rc;
-  }
-  const int n_raw_t = (g.T + 127) / 128, n_gist_t = (g.n + 127) / 128;
-
-  auto go_kv = [&](auto kern, size_t smem) -> int32_t {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  const int n_sink_t = (g.s + 127) / 128, n_raw_t = (g.T + 127) / 128, n_gist_t = (g.n + 127) / 128;
+  if (!fused) {
+    // head_dim 64: one map per segment (sinks, raw, gists; a tensor map cannot be empty) with 128-row boxes,
+    // and 64-row boxes over K and V for the dQ kernel
+    CUtensorMap mq[3], md[3], mk[3], mv[3], mk64[3], mv64[3];
+    for (int sg = 0; sg < 3; ++sg) {
+      const long long first = seg_base(g, sg), len = seg_len(g, sg) > 0 ? seg_len(g, sg) : 1;
+      if (int32_t rc = encode_segment_map(&mq[sg], q, D, Hq, g.N, B, first, len, 128)) return rc;
+      if (int32_t rc = encode_segment_map(&md[sg], do_src, D, Hq, g.N, B, first, len, 128)) return rc;
+      if (int32_t rc = encode_segment_map(&mk[sg], k, D, Hkv, g.N, B, first, len, 128)) return rc;
+      if (int32_t rc = encode_segment_map(&mv[sg], v, D, Hkv, g.N, B, first, len, 128)) return rc;
+      if (int32_t rc = encode_segment_map(&mk64[sg], k, D, Hkv, g.N, B, first, len, DQ_BN)) return rc;
+      if (int32_t rc = encode_segment_map(&mv64[sg], v, D, Hkv, g.N, B, first, len, DQ_BN)) return rc;
+    }
+    const int n_tiles = n_sink_t + n_raw_t + n_gist_t;
+    cudaError_t e = cudaFuncSetAttribute(attn_bwd_dkdv_sm100_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         KvSmem<64>::kBytes);
+    if (e == cudaSuccess)
+      e = cudaFuncSetAttribute(attn_bwd_dq_sm100_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, DqSmem<64>::kBytes);
     if (e != cudaSuccess) return fail(UNIGIST_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
     {
       KernelScope ks("attn_bwd_dkdv_sm100_kernel", st);
-      kern<<<dim3(n_raw_t + n_gist_t, Hkv, B), kKvThreads, smem, st>>>(
-          mq[0], mq[1], md[0], md[1], mk[0], mk[1], mv[0], mv[1], g, Hq, Hkv, scale, lse, delta,
-          (__nv_bfloat16*)dk, (__nv_bfloat16*)dv, n_gist_t);
+      attn_bwd_dkdv_sm100_kernel<64><<<dim3(n_tiles, Hkv, B), kKvThreads, KvSmem<64>::kBytes, st>>>(
+          mq[0], mq[1], mq[2], md[0], md[1], md[2], mk[0], mk[1], mk[2], mv[0], mv[1], mv[2], g, Hq, Hkv, scale, lse, delta,
+          (__nv_bfloat16*)dk, (__nv_bfloat16*)dv, n_sink_t, n_gist_t);
     }
-    return check_launch("tcgen05 dK/dV kernel");
-  };
-  auto go_q = [&](auto kern, size_t smem) -> int32_t {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return fail(UNIGIST_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
+    if (int32_t rc = check_launch("tcgen05 dK/dV kernel")) return rc;
     {
       KernelScope ks("attn_bwd_dq_sm100_kernel", st);
-      kern<<<dim3(n_raw_t + n_gist_t, Hq, B), kDqThreads, smem, st>>>(
-          mq[0], mq[1], md[0], md[1], mk64[0], mk64[1], mv64[0], mv64[1], g, Hq, Hkv, scale, lse, delta,
-          (__nv_bfloat16*)dq, n_raw_t);
+      attn_bwd_dq_sm100_kernel<64><<<dim3(n_tiles, Hq, B), kDqThreads, DqSmem<64>::kBytes, st>>>(
+          mq[0], mq[1], mq[2], md[0], md[1], md[2], mk64[0], mk64[1], mk64[2], mv64[0], mv64[1], mv64[2], g, Hq, Hkv, scale,
+          lse, delta, (__nv_bfloat16*)dq, n_sink_t, n_raw_t);
     }
     return check_launch("tcgen05 dQ kernel");
-  };
-  if (!fused) {
-    if (int32_t rc = go_kv(attn_bwd_dkdv_sm100_kernel<64>, KvSmem<64>::kBytes)) return rc;
-    return go_q(attn_bwd_dq_sm100_kernel<64>, DqSmem<64>::kBytes);
   }
-  // 128-row tile maps per segment (sinks, raw, gists) that read shifted or interleaved tensors, and
-  // reduction maps over the fp32 dQ tensor (always shifted)
-  CUtensorMap fq[3], fdo[3], fk[3], fv[3], mdq[3];
-  for (int sg = 0; sg < 3; ++sg) {
-    if (int32_t rc = encode_tile_map(&fq[sg], q, D, Hq, B, g.s, g.T, g.r, g.n, il, sg)) return rc;
-    if (int32_t rc = encode_tile_map(&fdo[sg], do_src, D, Hq, B, g.s, g.T, g.r, g.n, il, sg)) return rc;
-    if (int32_t rc = encode_tile_map(&fk[sg], k, D, Hkv, B, g.s, g.T, g.r, g.n, il, sg)) return rc;
-    if (int32_t rc = encode_tile_map(&fv[sg], v, D, Hkv, B, g.s, g.T, g.r, g.n, il, sg)) return rc;
-    const int rows = seg_len(g, sg) > 0 ? seg_len(g, sg) : 1;  // a tensor map cannot be empty
-    if (int32_t rc = encode_segment_map_f32(&mdq[sg], dq32, D, Hq, g.N, B, seg_base(g, sg), rows, 32, 32)) return rc;
+  BwdRuns<1> P;
+  P.n = 1;
+  if (int32_t rc = fill_bwd_run(&P.run[0], g, p, B, q, do_src, k, v, sc.dq32, lse, delta, dk, dv)) return rc;
+  if (int32_t rc = launch_fused(P, dim3(P.run[0].plane, 1, B), p, scale, st)) return rc;
+  return launch_convert(T, p, tokens, sc, dq, scale, st);
+}
+
+// Backward over a packed sample (head_dim 128): every run of equal documents is a launch unit; up to twelve
+// units share one launch of the prep, fused and convert kernels.
+int32_t launch_bwd_sm100_runs(const SeqRun* runs, int n_runs, long long tokens, const unigist_problem& p, float scale,
+                              const void* q, const void* k, const void* v, const void* o, const float* lse,
+                              const void* d_o, void* dq, void* dk, void* dv, void* workspace, cudaStream_t st) {
+  const int D = p.head_dim, Hq = p.num_q_heads, Hkv = p.num_kv_heads;
+  const bool f32 = (p.flags & UNIGIST_FLAG_DOUT_FP32) != 0;
+  const BwdScratch sc = carve_scratch(workspace, tokens, Hq, D, f32);
+  const void* do_src = f32 ? static_cast<const void*>(sc.do_bf16) : d_o;
+  const size_t rq = (size_t)Hq * D * 2, rk = (size_t)Hkv * D * 2;
+  for (int first = 0; first < n_runs; first += kMaxRunsPerLaunch) {
+    const int n = n_runs - first < kMaxRunsPerLaunch ? n_runs - first : kMaxRunsPerLaunch;
+    // the runs of one launch hold consecutive packed tokens [tok_lo, tok_hi)
+    const long long tok_lo = runs[first].first_row;
+    const long long tok_hi = runs[first + n - 1].first_row + (long long)runs[first + n - 1].g.N * runs[first + n - 1].batch;
+    TokRuns<kMaxRunsPerLaunch> T;
+    BwdRuns<kMaxRunsPerLaunch> P;
+    T.n = P.n = n;
+    // the per-token kernels scan the runs in token order; the fused kernel starts the longest run's blocks first
+    int order[kMaxRunsPerLaunch];
+    for (int i = 0; i < n; ++i) order[i] = i;
+    std::stable_sort(order, order + n, [&](int a, int b) {
+      return (long long)runs[first + a].g.N * runs[first + a].batch > (long long)runs[first + b].g.N * runs[first + b].batch;
+    });
+    long long ctas = 0;
+    for (int i = 0; i < n; ++i) {
+      const SeqRun& t = runs[first + i];
+      T.run[i].g = t.g;
+      T.run[i].tok_begin = t.first_row - tok_lo;
+      T.run[i].delta = sc.delta + t.first_row * Hq;
+      const SeqRun& r = runs[first + order[i]];
+      if (int32_t rc = fill_bwd_run(&P.run[i], r.g, p, r.batch, (const char*)q + r.first_row * rq,
+                                    (const char*)do_src + r.first_row * rq, (const char*)k + r.first_row * rk,
+                                    (const char*)v + r.first_row * rk, sc.dq32 + r.first_row * Hq * D,
+                                    lse + r.first_row * Hq, sc.delta + r.first_row * Hq, (char*)dk + r.first_row * rk,
+                                    (char*)dv + r.first_row * rk))
+        return rc;
+      P.run[i].cta_begin = (int)ctas;
+      ctas += (long long)P.run[i].plane * r.batch;
+      if (ctas > 0x7fffffffLL) return fail(UNIGIST_ERR_SHAPE, "packed sample too large for one grid");
+    }
+    for (int i = n; i < kMaxRunsPerLaunch; ++i) T.run[i] = T.run[0], P.run[i] = P.run[0];  // never selected
+    // the per-token kernels of this launch see the tensors from packed token tok_lo on
+    BwdScratch part = sc;
+    if (part.do_bf16) part.do_bf16 += tok_lo * Hq * D;
+    part.dq32 += tok_lo * Hq * D;
+    const size_t rdo = f32 ? 2 * rq : rq;
+    if (int32_t rc = launch_prep(T, p, tok_hi - tok_lo, (const char*)d_o + tok_lo * rdo, (const char*)o + tok_lo * rq, part, st))
+      return rc;
+    if (int32_t rc = launch_fused(P, dim3((unsigned)ctas, 1, 1), p, scale, st)) return rc;
+    if (int32_t rc = launch_convert(T, p, tok_hi - tok_lo, part, (char*)dq + tok_lo * rq, scale, st)) return rc;
   }
-  const int n_sink_t = (g.s + 127) / 128;
-  cudaError_t e = cudaFuncSetAttribute(attn_bwd_fused_sm100_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       FuSmem::kBytes);
-  if (e != cudaSuccess) return fail(UNIGIST_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
-  {
-    KernelScope ks("attn_bwd_fused_sm100_kernel", st);
-    attn_bwd_fused_sm100_kernel<<<dim3((n_sink_t + n_raw_t + n_gist_t) * Hkv, 1, B), kFuThreads, FuSmem::kBytes, st>>>(
-        fq[0], fq[1], fq[2], fdo[0], fdo[1], fdo[2], fk[0], fk[1], fk[2], fv[0], fv[1], fv[2], mdq[0], mdq[1], mdq[2], g,
-        Hq, Hkv, scale, lse, delta, (__nv_bfloat16*)dk, (__nv_bfloat16*)dv, n_sink_t, n_gist_t, il ? 1 : 0, make_fastdiv(g.r));
-  }
-  if (int32_t rc = check_launch("tcgen05 fused backward kernel")) return rc;
-  {
-    const long long tokens = (long long)B * g.N;
-    const int blocks = (int)((tokens + 7) / 8 < sm_count() * 16 ? (tokens + 7) / 8 : sm_count() * 16);
-    KernelScope ks("dq_convert_kernel", st);
-    dq_convert_kernel<<<blocks, 256, 0, st>>>(g, il ? 1 : 0, Hq, tokens, dq32, (__nv_bfloat16*)dq, scale);
-  }
-  return check_launch("dQ convert kernel");
+  return UNIGIST_OK;
 }
 
 int32_t bwd_sm100_take_timeout(bool* timed_out) {

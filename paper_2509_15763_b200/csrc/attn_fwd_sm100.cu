@@ -24,6 +24,8 @@
 // of a tile in registers), then one more warpgroup
 // with the TMA producer warp and the MMA issuer / TMEM owner warp, which hands most of its registers
 // to the softmax warpgroups.  TMEM: S0 | S1 | O0 | O1, 128 columns each.
+#include <algorithm>
+
 #include "sm100_ptx.cuh"
 #include "ug_common.cuh"
 
@@ -232,16 +234,49 @@ __device__ __forceinline__ float row_exp(const uint32_t (&sc)[kCols], uint32_t t
   return (l0 + l1) + (l2 + l3);
 }
 
-template <int D>
+// One launch unit: a batch of sequences of one geometry with its own tensor maps (one per segment, so that
+// tiles never straddle segments, ragged ends read as zero and stores past a segment's end are dropped).
+// A call on one problem is one unit with a (tiles, heads, batch) grid.  A packed sample under cross-document
+// masking (Section 5.1) is several units in ONE launch: the grid is flat and a block finds its unit from the
+// units' first block indices.
+struct alignas(64) FwdRun {
+  CUtensorMap q[3], k[3], v[3], o[3];
+  Geom g;
+  QueryRows qr;
+  float* lse;
+  int n_sink_units, n_raw_units, n_units;  // n_units: x extent of the unit's grid
+  int cta_begin;                           // flat grid: first block of the unit
+  int plane;                               // n_units * (y extent)
+  FastDiv units_div, plane_div;
+};
+template <int kRuns>
+struct FwdRuns {
+  FwdRun run[kRuns];
+  int n;
+};
+constexpr int kMaxRunsPerLaunch = 12;  // 12 units are 20 KB of kernel parameters (the limit is 32 KB)
+
+template <int D, int kRuns>
 __global__ void __launch_bounds__(kThreads, 1)
-attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_sink, const __grid_constant__ CUtensorMap tm_q_raw,
-                      const __grid_constant__ CUtensorMap tm_q_gist, const __grid_constant__ CUtensorMap tm_k_sink,
-                      const __grid_constant__ CUtensorMap tm_k_raw, const __grid_constant__ CUtensorMap tm_k_gist,
-                      const __grid_constant__ CUtensorMap tm_v_sink, const __grid_constant__ CUtensorMap tm_v_raw,
-                      const __grid_constant__ CUtensorMap tm_v_gist, const __grid_constant__ CUtensorMap tm_o_sink,
-                      const __grid_constant__ CUtensorMap tm_o_raw, const __grid_constant__ CUtensorMap tm_o_gist, Geom g,
-                      int Hq, FastDiv rdiv, FastDiv hkdiv, float scale_log2, float* __restrict__ lse, int n_sink_units, int n_raw_units,
-                      int pair_heads, int interleaved, QueryRows qr) {
+attn_fwd_sm100_kernel(const __grid_constant__ FwdRuns<kRuns> P, int Hq, FastDiv rdiv, FastDiv hkdiv, float scale_log2,
+                      int pair_heads, int interleaved) {
+  int ri = 0, bx, by, bz;
+  if constexpr (kRuns == 1) {
+    bx = blockIdx.x, by = blockIdx.y, bz = blockIdx.z;
+  } else {
+    const int c = blockIdx.x;
+    while (ri + 1 < P.n && c >= P.run[ri + 1].cta_begin) ++ri;
+    const int local = c - P.run[ri].cta_begin;
+    bz = fdiv(P.run[ri].plane_div, local);
+    const int rem = local - bz * P.run[ri].plane;
+    by = fdiv(P.run[ri].units_div, rem);
+    bx = rem - by * P.run[ri].n_units;
+  }
+  const FwdRun& R = P.run[ri];
+  const Geom g = R.g;
+  const QueryRows qr = R.qr;
+  float* __restrict__ lse = R.lse;
+  const int n_sink_units = R.n_sink_units, n_raw_units = R.n_raw_units;
   using SM = FwdSmem<D>;
   extern __shared__ unsigned char smem_dyn[];
   const uint32_t base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
@@ -258,9 +293,9 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_sink, const __gri
       reinterpret_cast<volatile uint32_t*>(gen_base + SM::kBarOff + 48 + 16 * kStages);
 
   const int warp = threadIdx.x >> 5;
-  const int b = blockIdx.z;
+  const int b = bz;
   // heaviest units first: gist units from the end, then raw units from the end, sink units last
-  const int u_lin = gridDim.x - 1 - blockIdx.x;
+  const int u_lin = R.n_units - 1 - bx;
   const int qseg = u_lin < n_sink_units ? kSegSink : (u_lin < n_sink_units + n_raw_units ? kSegRaw : kSegGist);
   const int u = u_lin - (qseg == kSegSink ? 0 : (qseg == kSegRaw ? n_sink_units : n_sink_units + n_raw_units));
   const int q_off = qr.off[qseg];  // first query row of the segment (0 unless this is a prefill chunk)
@@ -270,13 +305,13 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_sink, const __gri
   bool sv[2];
   if (pair_heads) {
     qt[0] = qt[1] = u;
-    hh[0] = 2 * blockIdx.y;
+    hh[0] = 2 * by;
     hh[1] = hh[0] + 1;
     sv[0] = sv[1] = true;
   } else {
     qt[0] = 2 * u;
     qt[1] = 2 * u + 1;
-    hh[0] = hh[1] = blockIdx.y;
+    hh[0] = hh[1] = by;
     sv[0] = true;
     sv[1] = qt[1] < n_qt;
   }
@@ -303,11 +338,11 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_sink, const __gri
   tc_fence_after();
   const uint32_t tmem = *tmem_slot_ptr;
   bool ok = true;
-  const int hk = fdiv(hkdiv, blockIdx.y);  // both streams share the KV head
+  const int hk = fdiv(hkdiv, by);  // both streams share the KV head
   // tile coordinate: its first unit (a raw tile of an interleaved tensor spans 128 / r gist units)
   auto first_unit = [&](int sg, int row0) { return interleaved && sg == kSegRaw ? fdiv(rdiv, row0) : row0; };
   if (warp == kTmaWarp && elect_one()) {
-    const CUtensorMap* mq = qseg == kSegRaw ? &tm_q_raw : (qseg == kSegGist ? &tm_q_gist : &tm_q_sink);
+    const CUtensorMap* mq = &R.q[qseg];
     mbar_arrive_expect_tx(bar_q, (sv[1] ? 2 : 1) * SM::kTile);
     for (int i = 0; i < 2; ++i) {
       if (!sv[i]) continue;
@@ -320,8 +355,8 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_sink, const __gri
     // segment, at its last row's tile): its K and V loads need none of the interval arithmetic below.
     const int last = sv[1] ? 1 : 0;
     const int idx0 = min(q_off + qt[last] * BM + BM - 1, seg_len(g, qseg) - 1) / BN;
-    const CUtensorMap* mk0 = qseg == kSegRaw ? &tm_k_raw : (qseg == kSegGist ? &tm_k_gist : &tm_k_sink);
-    const CUtensorMap* mv0 = qseg == kSegRaw ? &tm_v_raw : (qseg == kSegGist ? &tm_v_gist : &tm_v_sink);
+    const CUtensorMap* mk0 = &R.k[qseg];
+    const CUtensorMap* mv0 = &R.v[qseg];
 #pragma unroll
     for (int t = 0; t < 2; ++t) {
       mbar_arrive_expect_tx(bar_full + 8 * t, SM::kTile);
@@ -343,8 +378,7 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_sink, const __gri
       for (int t = 2; t < 2 * nt && ok; ++t) {  // item t: K tile of step t/2 (even t) or its V tile (odd t); 0, 1 are on their way
         int sg, idx;
         seq.at(t >> 1, sg, idx);
-        const CUtensorMap* m = (t & 1) ? (sg == kSegRaw ? &tm_v_raw : (sg == kSegGist ? &tm_v_gist : &tm_v_sink))
-                                       : (sg == kSegRaw ? &tm_k_raw : (sg == kSegGist ? &tm_k_gist : &tm_k_sink));
+        const CUtensorMap* m = (t & 1) ? &R.v[sg] : &R.k[sg];
         const int slot = t % kStages, use = t / kStages;
         if (use > 0) ok = mbar_wait(bar_empty + 8 * slot, (use - 1) & 1);
         if (!ok) break;
@@ -560,7 +594,7 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q_sink, const __gri
       named_barrier_sync(1 + i, 128);
       if (ok && (warp & 3) == 0 && elect_one()) {
         // rows past the end of the segment lie outside the map and are not written
-        const CUtensorMap* mo = qseg == kSegRaw ? &tm_o_raw : (qseg == kSegGist ? &tm_o_gist : &tm_o_sink);
+        const CUtensorMap* mo = &R.o[qseg];
         const int row0 = qt[i] * BM;
 #pragma unroll
         for (int sl = 0; sl < D / 64; ++sl)
@@ -683,47 +717,104 @@ int32_t encode_map_2d_bf16(CUtensorMap* map, const void* base, long long rows, i
   return UNIGIST_OK;
 }
 
-int32_t launch_fwd_sm100(const Geom& g, const unigist_problem& p, float scale, const void* q, const void* k,
-                         const void* v, void* o, float* lse, cudaStream_t st, const QueryRows* chunk) {
-  const int D = p.head_dim, Hq = p.num_q_heads, Hkv = p.num_kv_heads, B = p.batch;
-  CUtensorMap mq[3], mk[3], mv[3], mo[3];  // per segment: sinks, raw, gists (O has the geometry of Q)
-  const bool il = (p.flags & UNIGIST_FLAG_INTERLEAVED) != 0 && !chunk;
-  QueryRows qr;
+namespace {
+
+// Two streams per block: neighbouring heads of a KV group when the group size is even, otherwise
+// neighbouring query tiles of one head.
+int fwd_pair_heads(const unigist_problem& p) { return (p.num_q_heads / p.num_kv_heads) % 2 == 0 ? 1 : 0; }
+
+// Tensor maps and tile counts of one launch unit: `batch` sequences of geometry g whose first rows are
+// q, k, v, o (and lse).  With `chunk` the queries are the tail of each segment only (chunk-wise prefill).
+int32_t fill_fwd_run(FwdRun* R, const Geom& g, const unigist_problem& p, int batch, bool il, const void* q, const void* k,
+                     const void* v, void* o, float* lse, const QueryRows* chunk) {
+  const int D = p.head_dim, Hq = p.num_q_heads, Hkv = p.num_kv_heads;
   if (chunk) {
-    qr = *chunk;
+    R->qr = *chunk;
   } else {
-    for (int sg = 0; sg < 3; ++sg) qr.off[sg] = 0, qr.out_base[sg] = seg_base(g, sg);
-    qr.n_out = g.N;
+    for (int sg = 0; sg < 3; ++sg) R->qr.off[sg] = 0, R->qr.out_base[sg] = seg_base(g, sg);
+    R->qr.n_out = g.N;
   }
   // the Q tensor holds the query rows only: the tail of each segment from qr.off on
-  const int sq = g.s - qr.off[kSegSink], Tq = g.T - qr.off[kSegRaw], nq = g.n - qr.off[kSegGist];
-  for (int sg = 0; sg < 3; ++sg) {
-    if (int32_t rc = encode_tile_map(&mq[sg], q, D, Hq, B, sq, Tq, g.r, nq, il, sg)) return rc;
-    if (int32_t rc = encode_tile_map(&mo[sg], o, D, Hq, B, sq, Tq, g.r, nq, il, sg)) return rc;
-    if (int32_t rc = encode_tile_map(&mk[sg], k, D, Hkv, B, g.s, g.T, g.r, g.n, il, sg)) return rc;
-    if (int32_t rc = encode_tile_map(&mv[sg], v, D, Hkv, B, g.s, g.T, g.r, g.n, il, sg)) return rc;
+  const int sq = g.s - R->qr.off[kSegSink], Tq = g.T - R->qr.off[kSegRaw], nq = g.n - R->qr.off[kSegGist];
+  for (int sg = 0; sg < 3; ++sg) {  // per segment: sinks, raw, gists (O has the geometry of Q)
+    if (int32_t rc = encode_tile_map(&R->q[sg], q, D, Hq, batch, sq, Tq, g.r, nq, il, sg)) return rc;
+    if (int32_t rc = encode_tile_map(&R->o[sg], o, D, Hq, batch, sq, Tq, g.r, nq, il, sg)) return rc;
+    if (int32_t rc = encode_tile_map(&R->k[sg], k, D, Hkv, batch, g.s, g.T, g.r, g.n, il, sg)) return rc;
+    if (int32_t rc = encode_tile_map(&R->v[sg], v, D, Hkv, batch, g.s, g.T, g.r, g.n, il, sg)) return rc;
   }
   const int n_sink_qt = (sq + BM - 1) / BM, n_raw_qt = (Tq + BM - 1) / BM, n_gist_qt = (nq + BM - 1) / BM;
-  // Two streams per block: neighbouring heads of a KV group when the group size is even,
-  // otherwise neighbouring query tiles of one head.
-  const int pair_heads = (Hq / Hkv) % 2 == 0 ? 1 : 0;
-  const int n_sink_units = pair_heads ? n_sink_qt : (n_sink_qt + 1) / 2;
-  const int n_raw_units = pair_heads ? n_raw_qt : (n_raw_qt + 1) / 2;
-  const int n_gist_units = pair_heads ? n_gist_qt : (n_gist_qt + 1) / 2;
-  dim3 grid(n_sink_units + n_raw_units + n_gist_units, pair_heads ? Hq / 2 : Hq, B);
-  const float scale_log2 = scale * 1.4426950408889634f;
-  auto go = [&](auto kern, size_t smem) -> int32_t {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return fail(UNIGIST_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
-    {
-      KernelScope ks("attn_fwd_sm100_kernel", st);
-      kern<<<grid, kThreads, smem, st>>>(mq[0], mq[1], mq[2], mk[0], mk[1], mk[2], mv[0], mv[1], mv[2], mo[0], mo[1], mo[2], g,
-                                         Hq, make_fastdiv(g.r), make_fastdiv(pair_heads ? (Hq / Hkv) / 2 : Hq / Hkv), scale_log2, lse, n_sink_units, n_raw_units, pair_heads,
-                                         il ? 1 : 0, qr);
+  const int pair = fwd_pair_heads(p);
+  R->n_sink_units = pair ? n_sink_qt : (n_sink_qt + 1) / 2;
+  R->n_raw_units = pair ? n_raw_qt : (n_raw_qt + 1) / 2;
+  const int n_gist_units = pair ? n_gist_qt : (n_gist_qt + 1) / 2;
+  R->n_units = R->n_sink_units + R->n_raw_units + n_gist_units;
+  R->g = g;
+  R->lse = lse;
+  const int ydim = pair ? Hq / 2 : Hq;
+  R->plane = R->n_units * ydim;
+  R->units_div = make_fastdiv(R->n_units);
+  R->plane_div = make_fastdiv(R->plane);
+  R->cta_begin = 0;
+  return UNIGIST_OK;
+}
+
+template <typename Kern, typename Params>
+int32_t go_fwd(Kern kern, size_t smem, dim3 grid, const Params& P, const unigist_problem& p, float scale, bool il,
+               cudaStream_t st) {
+  const int Hq = p.num_q_heads, Hkv = p.num_kv_heads, pair = fwd_pair_heads(p);
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return fail(UNIGIST_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
+  {
+    KernelScope ks("attn_fwd_sm100_kernel", st);
+    kern<<<grid, kThreads, smem, st>>>(P, Hq, make_fastdiv(p.ratio), make_fastdiv(pair ? (Hq / Hkv) / 2 : Hq / Hkv),
+                                       scale * 1.4426950408889634f, pair, il ? 1 : 0);
+  }
+  return check_launch("tcgen05 forward kernel");
+}
+
+}  // namespace
+
+int32_t launch_fwd_sm100(const Geom& g, const unigist_problem& p, float scale, const void* q, const void* k,
+                         const void* v, void* o, float* lse, cudaStream_t st, const QueryRows* chunk) {
+  const bool il = (p.flags & UNIGIST_FLAG_INTERLEAVED) != 0 && !chunk;
+  FwdRuns<1> P;
+  P.n = 1;
+  if (int32_t rc = fill_fwd_run(&P.run[0], g, p, p.batch, il, q, k, v, o, lse, chunk)) return rc;
+  const dim3 grid(P.run[0].n_units, fwd_pair_heads(p) ? p.num_q_heads / 2 : p.num_q_heads, p.batch);
+  return p.head_dim == 64 ? go_fwd(attn_fwd_sm100_kernel<64, 1>, FwdSmem<64>::kBytes, grid, P, p, scale, il, st)
+                          : go_fwd(attn_fwd_sm100_kernel<128, 1>, FwdSmem<128>::kBytes, grid, P, p, scale, il, st);
+}
+
+int32_t launch_fwd_sm100_runs(const SeqRun* runs, int n_runs, const unigist_problem& p, float scale, const void* q,
+                              const void* k, const void* v, void* o, float* lse, cudaStream_t st) {
+  const bool il = (p.flags & UNIGIST_FLAG_INTERLEAVED) != 0;
+  const size_t rq = (size_t)p.num_q_heads * p.head_dim * 2, rk = (size_t)p.num_kv_heads * p.head_dim * 2;
+  for (int first = 0; first < n_runs; first += kMaxRunsPerLaunch) {  // one launch per kMaxRunsPerLaunch units
+    FwdRuns<kMaxRunsPerLaunch> P;
+    P.n = n_runs - first < kMaxRunsPerLaunch ? n_runs - first : kMaxRunsPerLaunch;
+    int order[kMaxRunsPerLaunch];  // the longest run's blocks start first
+    for (int i = 0; i < P.n; ++i) order[i] = i;
+    std::stable_sort(order, order + P.n, [&](int a, int b) {
+      return (long long)runs[first + a].g.N * runs[first + a].batch > (long long)runs[first + b].g.N * runs[first + b].batch;
+    });
+    long long ctas = 0;
+    for (int i = 0; i < P.n; ++i) {
+      const SeqRun& r = runs[first + order[i]];
+      if (int32_t rc = fill_fwd_run(&P.run[i], r.g, p, r.batch, il, (const char*)q + r.first_row * rq,
+                                    (const char*)k + r.first_row * rk, (const char*)v + r.first_row * rk,
+                                    (char*)o + r.first_row * rq, lse + r.first_row * p.num_q_heads, nullptr))
+        return rc;
+      P.run[i].cta_begin = (int)ctas;
+      ctas += (long long)P.run[i].plane * r.batch;
+      if (ctas > 0x7fffffffLL) return fail(UNIGIST_ERR_SHAPE, "packed sample too large for one grid");
     }
-    return check_launch("tcgen05 forward kernel");
-  };
-  return D == 64 ? go(attn_fwd_sm100_kernel<64>, FwdSmem<64>::kBytes) : go(attn_fwd_sm100_kernel<128>, FwdSmem<128>::kBytes);
+    for (int i = P.n; i < kMaxRunsPerLaunch; ++i) P.run[i] = P.run[0];  // unused slots: defined contents, never selected
+    const dim3 grid((unsigned)ctas, 1, 1);
+    const int32_t rc = p.head_dim == 64 ? go_fwd(attn_fwd_sm100_kernel<64, kMaxRunsPerLaunch>, FwdSmem<64>::kBytes, grid, P, p, scale, il, st)
+                                        : go_fwd(attn_fwd_sm100_kernel<128, kMaxRunsPerLaunch>, FwdSmem<128>::kBytes, grid, P, p, scale, il, st);
+    if (rc) return rc;
+  }
+  return UNIGIST_OK;
 }
 
 int32_t fwd_sm100_take_timeout(bool* timed_out) {

@@ -151,16 +151,29 @@ struct QueryRows {
 int32_t launch_fwd_sm100(const Geom& g, const unigist_problem& p, float scale, const void* q,
                          const void* k, const void* v, void* o, float* lse, cudaStream_t st,
                          const QueryRows* chunk = nullptr);
+// A run of `batch` consecutive sequences of one geometry inside packed [N_total, heads, D] tensors (a packed
+// sample under cross-document masking), starting at packed row first_row.  The *_runs launchers take the
+// tensors' base pointers and put up to twelve runs into one launch.
+struct SeqRun {
+  Geom g;
+  int batch;
+  long long first_row;
+};
+int32_t launch_fwd_sm100_runs(const SeqRun* runs, int n_runs, const unigist_problem& p, float scale, const void* q,
+                              const void* k, const void* v, void* o, float* lse, cudaStream_t st);
 int32_t fwd_sm100_take_timeout(bool* timed_out);
 int32_t launch_bwd_sm100(const Geom& g, const unigist_problem& p, float scale, const void* q,
                          const void* k, const void* v, const void* o, const float* lse,
                          const void* d_o, void* dq, void* dk, void* dv, void* workspace,
                          cudaStream_t st);
+// The same over a packed sample (head_dim 128; `runs` in token order, `tokens` = rows of the packed tensors).
+int32_t launch_bwd_sm100_runs(const SeqRun* runs, int n_runs, long long tokens, const unigist_problem& p, float scale,
+                              const void* q, const void* k, const void* v, const void* o, const float* lse,
+                              const void* d_o, void* dq, void* dk, void* dv, void* workspace, cudaStream_t st);
+// Bytes of backward scratch for `tokens` packed tokens: Delta, the bf16 copy of an fp32 dO, and for head_dim 128
+// the fp32 dQ accumulator.
+size_t bwd_scratch_bytes(long long tokens, int Hq, int D, bool dout_fp32);
 int32_t bwd_sm100_take_timeout(bool* timed_out);
-int32_t launch_bwd_simt(const Geom& g, const unigist_problem& p, float scale, const void* q,
-                        const void* k, const void* v, const void* o, const float* lse,
-                        const void* d_o, void* dq, void* dk, void* dv, float* delta,
-                        cudaStream_t st);
 int32_t launch_compact_gather(const Geom& g, const unigist_problem& p, const void* k,
                               const void* v, void* kc, void* vc, int num_blocks,
                               const int32_t* table, int max_blocks, int32_t* seq_lens,

@@ -16,7 +16,10 @@ CASES = [
     (8, 8, 16, [40, 304, 8], 2, 1, 128, False),         # sinks in every document; a one-unit document
     (8, 8, 16, [40, 304, 8], 2, 1, 128, True),
     (0, 2, 4, [66, 130], 2, 2, 64, False),              # head_dim 64 (two-kernel backward)
-    (0, 4, 8, [64, 128, 64, 192, 64, 256], 2, 2, 128, True),  # six runs: more than the library has streams
+    (0, 4, 8, [64, 128, 64, 192, 64, 256], 2, 2, 128, True),  # six units of different lengths in one launch
+    # fifteen units: more than one launch holds (twelve), with sinks, a batch of three equal documents and a tiny one
+    (4, 4, 8, [64, 32, 96, 32, 32, 32, 160, 8, 64, 128, 36, 72, 40, 44, 48, 52, 56], 4, 2, 128, False),
+    (0, 8, 16, [64, 32, 96, 32, 32, 32, 160, 8, 64, 128, 16, 72, 40, 24, 48, 56, 80], 2, 2, 128, True),
 ]
 
 
@@ -92,8 +95,8 @@ def test_docs_reject_bad_lists():
 
 
 def test_docs_calls_can_be_captured_in_a_cuda_graph():
-    """The runs of a packed sample fork onto the library's side streams and join again by events only, so
-    the whole forward + backward is capturable; a replay gives what the eager calls gave."""
+    """A packed sample's forward + backward only enqueues kernels on the caller's stream (the documents' tensor
+    maps are kernel parameters), so it is capturable; a replay gives what the eager calls gave."""
     s, r, W, doc_T, Hq, Hkv, D = 0, 4, 8, [256, 128, 64, 64, 192], 4, 2, 128
     p = ug.Problem(1, doc_T[0], r, W, Hq, Hkv, D, num_sinks=s, flags=ug.FLAG_INTERLEAVED)
     n_tot = ug.unigist_docs_total_len(p, doc_T)
@@ -108,7 +111,7 @@ def test_docs_calls_can_be_captured_in_a_cuda_graph():
         ug.unigist_attn_fwd_docs(p, doc_T, q, k, v, o, lse)
         ug.unigist_attn_bwd_docs(p, doc_T, q, k, v, o, lse, do, dq, dk, dv, ws)
 
-    run()  # eager: also creates the side streams outside the capture
+    run()
     torch.cuda.synchronize()
     want = [t.clone() for t in (o, lse, dk, dv)]
     want_dq = dq.clone()
