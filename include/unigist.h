@@ -156,11 +156,13 @@ int32_t unigist_attn_fwd(const unigist_problem* p, const void* q, const void* k,
  *   dQ = scale dS K, dK = scale dS^T Q;  dK, dV summed over the query heads of a KV head.
  * q, k, v, o, lse as in the forward; d_o [B,N,Hq,D] device bf16 (fp32 with
  * UNIGIST_FLAG_DOUT_FP32); dq [B,N,Hq,D], dk, dv [B,N,Hkv,D] device bf16, all shifted.
- * dK/dV are accumulated without atomics: each key tile is owned by one thread block, so they are the
- * same bit for bit from run to run.  For head_dim 128 dQ is the sum, over the key tiles that see a query
- * tile, of fp32 partial tiles reduced into the workspace in whatever order the blocks arrive: its last bit
- * may differ between runs.  workspace: unigist_workspace_bytes(p, UNIGIST_OP_BWD) bytes (Delta, a bf16
- * copy of an fp32 dO, and for head_dim 128 the fp32 dQ accumulator), 16-byte aligned.
+ * dK/dV are accumulated without atomics: a key tile is owned by one thread block, or, where very many queries see
+ * it (sink and gist keys of a long sequence), by one block per chunk of those queries whose fp32 partial sums a
+ * small kernel adds in chunk order; either way they are the same bit for bit from run to run.  For head_dim 128
+ * dQ is the sum, over the key tiles that see a query tile, of fp32 partial tiles reduced into the workspace in
+ * whatever order the blocks arrive: its last bit may differ between runs.  workspace:
+ * unigist_workspace_bytes(p, UNIGIST_OP_BWD) bytes (Delta, a bf16 copy of an fp32 dO, and for head_dim 128 the
+ * fp32 dQ accumulator and the chunks' partial dK / dV), 16-byte aligned.
  */
 int32_t unigist_attn_bwd(const unigist_problem* p, const void* q, const void* k, const void* v,
                          const void* o, const float* lse, const void* d_o, void* dq, void* dk,
@@ -339,6 +341,14 @@ int32_t unigist_decode_static(int32_t num_seqs, int32_t num_q_heads, int32_t num
  * UNIGIST_OK otherwise.  No counterpart in the paper.
  */
 int32_t unigist_device_status(void);
+
+/*
+ * Self-check of that mechanism (no counterpart in the paper): enqueues one small thread block that waits on a
+ * barrier nothing ever completes.  Its wait runs out after about a second, the block leaves the way the
+ * attention kernels leave after a wait that gave up (tensor memory freed, flag raised), and the next
+ * unigist_device_status() returns UNIGIST_ERR_TIMEOUT once; the device stays usable.  Nothing faults or hangs.
+ */
+int32_t unigist_selftest_wait_timeout(void* stream);
 
 /* Number of kernels the library has launched in this process (all threads). */
 int64_t unigist_launch_count(void);

@@ -29,7 +29,7 @@ SYMBOLS = [
     "unigist_device_status", "unigist_decode_static", "unigist_prefill_workspace_bytes", "unigist_prefill_chunk",
     "unigist_cache_state_bytes", "unigist_cache_state_init", "unigist_cache_append", "unigist_decode_step",
     "unigist_rope", "unigist_docs_total_len", "unigist_docs_workspace_bytes", "unigist_attn_fwd_docs",
-    "unigist_attn_bwd_docs",
+    "unigist_attn_bwd_docs", "unigist_selftest_wait_timeout",
 ]
 
 
@@ -107,6 +107,7 @@ def lib() -> ctypes.CDLL:
             "unigist_kernel_timing_count": (i32, []),
             "unigist_kernel_timing_get": (i32, [i32, ctypes.c_char_p, i32, ctypes.POINTER(ctypes.c_float)]),
             "unigist_device_status": (i32, []),
+            "unigist_selftest_wait_timeout": (i32, [vp]),
             "unigist_decode_static": (i32, [i32, i32, i32, i32, f32, vp, vp, vp, i32, vp, i32, vp, vp, vp, vp]),
             "unigist_launch_count": (i64, []),
             "unigist_last_error_string": (ctypes.c_char_p, []),
@@ -197,6 +198,11 @@ def unigist_decode_static(q, k_cache, v_cache, block_table, seq_lens, o, lse=Non
 def unigist_device_status() -> None:
     """Synchronise the device; raise UnigistError if a kernel gave up on a bounded wait."""
     _check(lib().unigist_device_status())
+
+
+def unigist_selftest_wait_timeout(stream=None) -> None:
+    """Enqueue the self-check block whose bounded wait runs out (see unigist_device_status)."""
+    _check(lib().unigist_selftest_wait_timeout(_stream(stream)))
 
 
 def unigist_last_error_string() -> str:

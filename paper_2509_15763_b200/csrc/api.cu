@@ -42,6 +42,26 @@ int sm_count() {
   return n;
 }
 
+size_t l2_bytes() {
+  constexpr int kMaxDevices = 64;
+  constexpr size_t kB200 = 126u << 20;
+  static std::atomic<size_t> cached[kMaxDevices];  // 0 = not asked yet
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
+    cudaGetLastError();
+    return kB200;
+  }
+  size_t n = cached[dev].load(std::memory_order_relaxed);
+  if (n > 0) return n;
+  int v = 0;
+  if (cudaDeviceGetAttribute(&v, cudaDevAttrL2CacheSize, dev) != cudaSuccess || v < 1) {
+    cudaGetLastError();
+    return kB200;
+  }
+  cached[dev].store((size_t)v, std::memory_order_relaxed);
+  return (size_t)v;
+}
+
 namespace {
 struct TimingRecord {
   const char* name;
@@ -169,7 +189,8 @@ size_t unigist_workspace_bytes(const unigist_problem* p, int32_t op) {
       // Delta [B,Hq,N] fp32, a bf16 copy of dO when it arrives as fp32, and for head_dim 128 the fp32 dQ
       // accumulator of the fused tensor-core backward
       return bwd_scratch_bytes((long long)p->batch * g.N, p->num_q_heads, p->head_dim,
-                               (p->flags & UNIGIST_FLAG_DOUT_FP32) != 0);
+                               (p->flags & UNIGIST_FLAG_DOUT_FP32) != 0) +
+             bwd_partial_bytes(g, p->batch, p->num_q_heads, p->num_kv_heads, p->head_dim);
     case UNIGIST_OP_COMPACT: {
       const size_t L = (size_t)g.s + g.n + (size_t)g.k * g.r;
       return align_up(2 * (size_t)p->batch * L * p->num_kv_heads * p->head_dim * 2, 256);
@@ -265,7 +286,9 @@ int32_t unigist_device_status(void) {
   if (int32_t rc = bwd_sm100_take_timeout(&bwd_timed_out)) return rc;
   bool dec_timed_out = false;
   if (int32_t rc = decode_take_timeout(&dec_timed_out)) return rc;
-  if (timed_out || bwd_timed_out || dec_timed_out) return fail(UNIGIST_ERR_TIMEOUT, "a kernel gave up on a bounded wait; its outputs are invalid");
+  bool self_timed_out = false;
+  if (int32_t rc = selftest_take_timeout(&self_timed_out)) return rc;
+  if (timed_out || bwd_timed_out || dec_timed_out || self_timed_out) return fail(UNIGIST_ERR_TIMEOUT, "a kernel gave up on a bounded wait; its outputs are invalid");
   return UNIGIST_OK;
 }
 
@@ -358,9 +381,17 @@ int64_t unigist_docs_total_len(const unigist_problem* p, int32_t num_docs, const
 size_t unigist_docs_workspace_bytes(const unigist_problem* p, int32_t op, int32_t num_docs, const int32_t* doc_raw_len) {
   if (check_docs(p, num_docs, doc_raw_len) != UNIGIST_OK) return 0;
   if (op != UNIGIST_OP_BWD) return 0;
-  if (p->head_dim == 128)  // one scratch layout over all packed tokens
-    return bwd_scratch_bytes(unigist_docs_total_len(p, num_docs, doc_raw_len), p->num_q_heads, p->head_dim,
-                             (p->flags & UNIGIST_FLAG_DOUT_FP32) != 0);
+  if (p->head_dim == 128) {  // one scratch layout over all packed tokens, then the runs' partial dK / dV
+    size_t need = bwd_scratch_bytes(unigist_docs_total_len(p, num_docs, doc_raw_len), p->num_q_heads, p->head_dim,
+                                    (p->flags & UNIGIST_FLAG_DOUT_FP32) != 0);
+    for_each_doc_run(p, num_docs, doc_raw_len, [&](const unigist_problem& run, int64_t, int32_t) {
+      Geom g;
+      if (check_problem(&run, &g, nullptr) == UNIGIST_OK)
+        need += bwd_partial_bytes(g, run.batch, run.num_q_heads, run.num_kv_heads, run.head_dim);
+      return (int32_t)UNIGIST_OK;
+    });
+    return need;
+  }
   size_t need = 0;  // head_dim 64: one launch set per run, each with its own slice
   for_each_doc_run(p, num_docs, doc_raw_len, [&](const unigist_problem& run, int64_t, int32_t) {
     need += align_up(unigist_workspace_bytes(&run, op), 256);
@@ -578,6 +609,8 @@ int32_t unigist_decode_step(const unigist_problem* p, const void* q, const void*
   return launch_decode(S, Hq, Hkv, D, scale, q, kc, vc, num_blocks, table, max_blocks, seq_lens, o, lse, workspace,
                        (cudaStream_t)stream, state, stride, free_off);
 }
+
+int32_t unigist_selftest_wait_timeout(void* stream) { return launch_selftest_wait((cudaStream_t)stream); }
 
 int32_t unigist_kernel_timing(int32_t enable) {
   for (int i = 0; i < g_num_records; ++i) {

@@ -13,6 +13,7 @@
 //                              the visible 64-key tiles: S, dP, dS as above, dQ += dS K in TMEM.
 // Tiles without a visible pair are never loaded; only "partial" tiles evaluate the mask.
 #include <algorithm>
+#include <vector>
 
 #include "sm100_ptx.cuh"
 #include "ug_common.cuh"
@@ -789,7 +790,12 @@ struct alignas(64) BwdRun {
   __nv_bfloat16* dv;
   int n_sink_kt, n_gist_kt, n_raw_kt;
   int cta_begin, plane;  // flat grid: first block of the unit; blocks per batch index
-  FastDiv heavy_div, raw_div, plane_div;
+  // A sink or gist key tile's walk over its query tiles is cut into n_chunks chunks of chunk_tiles tiles, one
+  // block each; `partial` receives the fp32 dK / dV of the chunks of key tiles that have more than one
+  // ([batch][KV head][heavy key tile][chunk][dK | dV][128 keys][128]).
+  int n_chunks, chunk_tiles;
+  float* partial;
+  FastDiv heavy_div /* by n_chunks * heavy tiles */, tile_div /* by heavy tiles */, raw_div, plane_div;
 };
 template <int kRuns>
 struct BwdRuns {
@@ -842,21 +848,25 @@ attn_bwd_fused_sm100_kernel(const __grid_constant__ BwdRuns<kRuns> P, int Hq, in
   volatile int* q_issued = reinterpret_cast<volatile int*>(gen + SM::kOffBars + 144);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  // Block order (the hardware starts blocks in the order of their index): sink and gist key tiles are seen by
-  // every later query, so they are the heaviest and come first, for all KV heads, before any raw key tile;
-  // inside each of the two classes the key tiles of ONE KV head are consecutive.  The blocks that run side by
-  // side then belong to one or two KV heads and walk the same Q / dO / dQ tiles at about the same time, so a
-  // tile comes from DRAM once and from L2 for every other block that needs it (with the KV heads interleaved
-  // instead, a head's sweep over its queries was repeated by every wave of its blocks: about 8 times the
-  // algorithmic DRAM traffic, and a fifth more time).
+  // Block order (the hardware starts blocks in the order of their index).  Sink and gist key tiles are seen by
+  // every later query: they are the heaviest and come first, before any raw key tile.  Their walk over the query
+  // tiles (which starts at the last query tile for every one of them) is cut into chunks of the same query tiles,
+  // one block per (key tile, chunk), ordered KV head, chunk, key tile: the blocks that run side by side are the key
+  // tiles of ONE KV head over ONE chunk of queries, they start together, take the same time and read the same
+  // Q / dO / dQ tiles, which therefore come from DRAM once and from L2 for every other block.  (One block per
+  // key tile over all its queries had blocks of very different lengths start whenever an SM fell free, each
+  // sweeping the head's queries on its own: 7 times the algorithmic DRAM traffic.)  The raw key tiles of one KV
+  // head are consecutive too; their windows of query tiles overlap.
   const int G = Hq / Hkv;
   const int n_heavy_kt = n_sink_kt + n_gist_kt;
-  int hk, rank;
-  if (bx < n_heavy_kt * Hkv) {
+  int hk, rank, chunk = 0;
+  if (bx < n_heavy_kt * R.n_chunks * Hkv) {
     hk = fdiv(R.heavy_div, bx);
-    rank = bx - hk * n_heavy_kt;
+    const int rem = bx - hk * n_heavy_kt * R.n_chunks;
+    chunk = fdiv(R.tile_div, rem);
+    rank = rem - chunk * n_heavy_kt;
   } else {
-    const int y = bx - n_heavy_kt * Hkv;
+    const int y = bx - n_heavy_kt * R.n_chunks * Hkv;
     hk = fdiv(R.raw_div, y);
     rank = n_heavy_kt + (y - hk * n_raw_kt);
   }
@@ -878,7 +888,14 @@ attn_bwd_fused_sm100_kernel(const __grid_constant__ BwdRuns<kRuns> P, int Hq, in
   key_q_interval3(g, kseg, key_a, true, kSegSink, lo_a, hi_a);
   key_q_interval3(g, kseg, key_b, true, kSegSink, lo_b, hi_b);
   const int n_sink_q = hi_b >= lo_a ? hi_b / 128 - lo_a / 128 + 1 : 0, sq_lo = lo_a / 128, sink_t_lo = lo_b, sink_t_hi = hi_a;
-  const int n_iter = (n_raw_q + n_gist_q + n_sink_q) * G;
+  // this block's part of the walk: tiles [t_begin, t_end) of the order below (all of them for a raw key tile)
+  const int n_tiles = n_raw_q + n_gist_q + n_sink_q;
+  const bool heavy = kseg != kSegRaw;
+  const int t_begin = heavy ? chunk * R.chunk_tiles : 0;
+  const int t_end = heavy ? min(t_begin + R.chunk_tiles, n_tiles) : n_tiles;
+  if (chunk > 0 && t_begin >= n_tiles) return;  // this key tile has no such chunk (whole block, before any barrier)
+  const bool to_partial = heavy && n_tiles > R.chunk_tiles;  // several chunks: fp32 partial sums, reduced afterwards
+  const int n_iter = (t_end - t_begin) * G;
 
   if (threadIdx.x == 0) {
     mbar_init(bar_kv, 1);
@@ -913,7 +930,6 @@ attn_bwd_fused_sm100_kernel(const __grid_constant__ BwdRuns<kRuns> P, int Hq, in
   // and share Q / dO / dQ lines in L2.  A raw key tile sees a window of query tiles that moves with the key tile:
   // its neighbour is one tile behind, i.e. G steps with the heads innermost but a single step with the tiles
   // innermost (head by head), which keeps the shared lines in L2 between the two uses.
-  const int n_tiles = n_raw_q + n_gist_q + n_sink_q;
   const bool tiles_inner = kseg == kSegRaw;
   struct StepIter {
     int t, hd;  // tile index in the order above, head of the group
@@ -972,7 +988,7 @@ attn_bwd_fused_sm100_kernel(const __grid_constant__ BwdRuns<kRuns> P, int Hq, in
           st_d[i] = valid ? delta[row_base + row] : 0.f;
         }
       };
-      StepIter cur{0, 0}, ahead{0, 0};
+      StepIter cur{t_begin, 0}, ahead{t_begin, 0};
       if (n_iter > 0) fetch_stats(ahead);
       for (int it = 0; it < n_iter; ++it, advance(cur)) {
         const int st = it & 1;
@@ -1106,7 +1122,7 @@ attn_bwd_fused_sm100_kernel(const __grid_constant__ BwdRuns<kRuns> P, int Hq, in
     const uint32_t lane_base = static_cast<uint32_t>(qd * 32) << 16;
     float* stage_gen = reinterpret_cast<float*>(gen + SM::kOffStage) + (warp - 8) * 1024 + lane;
     const uint32_t stage_sh = base + SM::kOffStage + (warp - 8) * 4096;
-    StepIter cur{0, 0};
+    StepIter cur{t_begin, 0};
     for (int it = 0; it < n_iter && ok; ++it, advance(cur)) {
       int qseg, qt, head;
       tile_of(cur, qseg, qt, head);
@@ -1168,7 +1184,7 @@ attn_bwd_fused_sm100_kernel(const __grid_constant__ BwdRuns<kRuns> P, int Hq, in
     unsigned char* ds_row = gen + SM::kOffDS + hf * SM::kSlab + krow * 128;
     const int swz = krow & 7;
 
-    StepIter cur{0, 0};
+    StepIter cur{t_begin, 0};
     for (int it = 0; it < n_iter && ok; ++it, advance(cur)) {
       const int st = it & 1;
       int qseg, qt, head;
@@ -1236,6 +1252,8 @@ attn_bwd_fused_sm100_kernel(const __grid_constant__ BwdRuns<kRuns> P, int Hq, in
     if (ok) {
       tc_fence_after();
       const long long tok = (long long)b * g.N + seg_row_to_token(g, interleaved != 0, kseg, key_valid ? key : key_a);
+      // where this key's row of the chunk's fp32 partial sums goes when the key tile has several chunks
+      float* part_row = R.partial + (((((long long)b * Hkv + hk) * n_heavy_kt + rank) * R.n_chunks + chunk) * 2 * 128 + krow) * 128 + 64 * hf;
       // this warp stores columns [64 hf, 64 hf + 64) of dK and of dV
 #pragma unroll
       for (int which = 0; which < 2; ++which) {
@@ -1253,7 +1271,15 @@ attn_bwd_fused_sm100_kernel(const __grid_constant__ BwdRuns<kRuns> P, int Hq, in
 #pragma unroll
             for (int i = 0; i < 32; ++i) v[i] = 0u;
           }
-          if (key_valid) {
+          if (to_partial) {
+            if (key_valid) {
+              float4* pd = reinterpret_cast<float4*>(part_row + which * 128 * 128 + 32 * c);
+#pragma unroll
+              for (int i = 0; i < 32; i += 4)
+                pd[i / 4] = make_float4(__uint_as_float(v[i]), __uint_as_float(v[i + 1]), __uint_as_float(v[i + 2]),
+                                        __uint_as_float(v[i + 3]));
+            }
+          } else if (key_valid) {
 #pragma unroll
             for (int i = 0; i < 32; i += 8) {
               uint4 pk;
@@ -1275,6 +1301,52 @@ attn_bwd_fused_sm100_kernel(const __grid_constant__ BwdRuns<kRuns> P, int Hq, in
   if (warp == kFuMmaWarp) {
     __syncwarp();
     tmem_dealloc(tmem, 512);
+  }
+}
+
+// Number of 128-query tiles that see a key tile [key_a, key_b] of segment kseg (all query segments).
+__device__ __forceinline__ int count_q_tiles(const Geom& g, int kseg, int key_a, int key_b) {
+  int n = 0;
+#pragma unroll
+  for (int qseg = 0; qseg < 3; ++qseg) {
+    int lo_a, hi_a, lo_b, hi_b;
+    key_q_interval3(g, kseg, key_a, true, qseg, lo_a, hi_a);
+    key_q_interval3(g, kseg, key_b, true, qseg, lo_b, hi_b);
+    n += hi_b >= lo_a ? hi_b / 128 - lo_a / 128 + 1 : 0;
+  }
+  return n;
+}
+
+// dK, dV of the sink and gist key tiles whose walk was cut into several chunks: the chunks' fp32 partial sums
+// added in chunk order (the same bits on every run), scaled, rounded to bf16 and stored at the keys' rows.
+// One block per (16 rows of a heavy key tile, KV head, batch index), a warp per key row.
+__global__ void __launch_bounds__(128)
+dkdv_reduce_kernel(Geom g, int interleaved, int Hkv, int n_sink_kt, int n_gist_kt, int n_chunks, int chunk_tiles,
+                   const float* __restrict__ partial, __nv_bfloat16* __restrict__ dk, __nv_bfloat16* __restrict__ dv,
+                   float scale) {
+  const int rank = blockIdx.x >> 3, row0 = (blockIdx.x & 7) * 16, hk = blockIdx.y, b = blockIdx.z;
+  const int n_heavy_kt = n_sink_kt + n_gist_kt;
+  const int kseg = rank < n_sink_kt ? kSegSink : kSegGist;
+  const int kt = rank - (kseg == kSegSink ? 0 : n_sink_kt);
+  const int key_a = kt * 128, key_b = min(key_a + 127, seg_len(g, kseg) - 1);
+  const int n_tiles = count_q_tiles(g, kseg, key_a, key_b);
+  if (n_tiles <= chunk_tiles) return;  // a single chunk: the fused kernel stored dK, dV itself
+  const int chunks = (n_tiles + chunk_tiles - 1) / chunk_tiles;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const float* base = partial + ((((long long)b * Hkv + hk) * n_heavy_kt + rank) * n_chunks) * 2 * 128 * 128;
+  for (int krow = row0 + warp; krow < row0 + 16 && key_a + krow <= key_b; krow += 4) {
+    const long long tok = (long long)b * g.N + seg_row_to_token(g, interleaved != 0, kseg, key_a + krow);
+#pragma unroll
+    for (int which = 0; which < 2; ++which) {
+      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+      for (int c = 0; c < chunks; ++c) {
+        const float4 x = __ldcs(reinterpret_cast<const float4*>(base + ((long long)(c * 2 + which) * 128 + krow) * 128) + lane);
+        acc.x += x.x, acc.y += x.y, acc.z += x.z, acc.w += x.w;
+      }
+      const float mul = which == 0 ? scale : 1.f;
+      __nv_bfloat16* dst = (which == 0 ? dk : dv) + (tok * Hkv + hk) * 128 + lane * 4;
+      *reinterpret_cast<uint2*>(dst) = make_uint2(pack_bf16(acc.x * mul, acc.y * mul), pack_bf16(acc.z * mul, acc.w * mul));
+    }
   }
 }
 
@@ -1365,11 +1437,31 @@ int32_t launch_convert(const TokRuns<kRuns>& T, const unigist_problem& p, long l
   return check_launch("dQ convert kernel");
 }
 
+// How the walk of a sink or gist key tile over its query tiles is cut (head_dim 128).  Not at all while the rows
+// one KV head's blocks sweep (Q, dO and the fp32 dQ of its G query heads: 1 KB per token and head) fit in three
+// quarters of the L2: however the blocks start, what one has read is still there for the next.  Otherwise into at
+// most four chunks of at least 16 query tiles, fewer where the chunks' fp32 partial sums would take more than
+// half the room of the dQ accumulator.
+// -> tiles per chunk, number of chunks of the longest walk (1 = no cutting, no partial sums).
+void bwd_chunking(const Geom& g, int batch, int Hq, int Hkv, int* n_chunks, int* chunk_tiles) {
+  const int n_heavy = (g.s + 127) / 128 + (g.n + 127) / 128;
+  const int max_tiles = n_heavy + (g.T + 127) / 128;  // the first sink / gist key tile is seen by every query tile
+  const size_t dq_bytes = (size_t)batch * g.N * Hq * 128 * sizeof(float);
+  const size_t sweep_bytes = (size_t)g.N * (Hq / Hkv) * 1024;
+  int C = sweep_bytes > l2_bytes() / 4 * 3 ? 4 : 1;
+  while (C > 1 && ((max_tiles + C - 1) / C < 16 ||
+                   (size_t)batch * Hkv * n_heavy * C * 2 * 128 * 128 * sizeof(float) > dq_bytes / 2))
+    --C;
+  *chunk_tiles = (max_tiles + C - 1) / C;
+  *n_chunks = (max_tiles + *chunk_tiles - 1) / *chunk_tiles;
+}
+
 // Tensor maps and tile counts of one launch unit of the fused backward: `batch` sequences of geometry g whose
 // first rows are the given pointers.  128-row tile maps per segment (sinks, raw, gists) that read shifted or
 // interleaved tensors, and reduction maps over the fp32 dQ tensor (always shifted).
 int32_t fill_bwd_run(BwdRun* R, const Geom& g, const unigist_problem& p, int batch, const void* q, const void* do_src,
-                     const void* k, const void* v, float* dq32, const float* lse, const float* delta, void* dk, void* dv) {
+                     const void* k, const void* v, float* dq32, const float* lse, const float* delta, void* dk, void* dv,
+                     float* partial) {
   const int D = p.head_dim, Hq = p.num_q_heads, Hkv = p.num_kv_heads;
   const bool il = (p.flags & UNIGIST_FLAG_INTERLEAVED) != 0;
   for (int sg = 0; sg < 3; ++sg) {
@@ -1388,9 +1480,13 @@ int32_t fill_bwd_run(BwdRun* R, const Geom& g, const unigist_problem& p, int bat
   R->n_sink_kt = (g.s + 127) / 128;
   R->n_gist_kt = (g.n + 127) / 128;
   R->n_raw_kt = (g.T + 127) / 128;
-  R->plane = (R->n_sink_kt + R->n_gist_kt + R->n_raw_kt) * Hkv;
+  bwd_chunking(g, batch, Hq, Hkv, &R->n_chunks, &R->chunk_tiles);
+  R->partial = partial;
+  const int n_heavy = R->n_sink_kt + R->n_gist_kt;
+  R->plane = (n_heavy * R->n_chunks + R->n_raw_kt) * Hkv;
   R->cta_begin = 0;
-  R->heavy_div = make_fastdiv(R->n_sink_kt + R->n_gist_kt);
+  R->heavy_div = make_fastdiv(n_heavy * R->n_chunks);
+  R->tile_div = make_fastdiv(n_heavy);
   R->raw_div = make_fastdiv(R->n_raw_kt);
   R->plane_div = make_fastdiv(R->plane);
   return UNIGIST_OK;
@@ -1409,6 +1505,18 @@ int32_t launch_fused(const BwdRuns<kRuns>& P, dim3 grid, const unigist_problem& 
   return check_launch("tcgen05 fused backward kernel");
 }
 
+// Adds up the chunks' partial dK / dV of one launch unit (nothing to do where no key tile has several chunks).
+int32_t launch_dkdv_reduce(const BwdRun& R, int batch, const unigist_problem& p, float scale, cudaStream_t st) {
+  if (R.n_chunks <= 1) return UNIGIST_OK;
+  {
+    KernelScope ks("dkdv_reduce_kernel", st);
+    dkdv_reduce_kernel<<<dim3((R.n_sink_kt + R.n_gist_kt) * 8, p.num_kv_heads, batch), 128, 0, st>>>(
+        R.g, (p.flags & UNIGIST_FLAG_INTERLEAVED) ? 1 : 0, p.num_kv_heads, R.n_sink_kt, R.n_gist_kt, R.n_chunks,
+        R.chunk_tiles, R.partial, R.dk, R.dv, scale);
+  }
+  return check_launch("dK/dV reduce kernel");
+}
+
 }  // namespace
 
 size_t bwd_scratch_bytes(long long tokens, int Hq, int D, bool dout_fp32) {
@@ -1416,6 +1524,15 @@ size_t bwd_scratch_bytes(long long tokens, int Hq, int D, bool dout_fp32) {
   if (dout_fp32) b += align256((size_t)tokens * Hq * D * 2);
   if (D == 128) b += align256((size_t)tokens * Hq * D * sizeof(float));
   return b;
+}
+
+size_t bwd_partial_bytes(const Geom& g, int batch, int Hq, int Hkv, int D) {
+  if (D != 128) return 0;
+  int C, tiles;
+  bwd_chunking(g, batch, Hq, Hkv, &C, &tiles);
+  if (C <= 1) return 0;
+  const size_t n_heavy = (g.s + 127) / 128 + (g.n + 127) / 128;
+  return align256((size_t)batch * Hkv * n_heavy * C * 2 * 128 * 128 * sizeof(float));
 }
 
 int32_t launch_bwd_sm100(const Geom& g, const unigist_problem& p, float scale, const void* q, const void* k,
@@ -1472,8 +1589,10 @@ int32_t launch_bwd_sm100(const Geom& g, const unigist_problem& p, float scale, c
   }
   BwdRuns<1> P;
   P.n = 1;
-  if (int32_t rc = fill_bwd_run(&P.run[0], g, p, B, q, do_src, k, v, sc.dq32, lse, delta, dk, dv)) return rc;
+  float* partial = reinterpret_cast<float*>(static_cast<char*>(workspace) + bwd_scratch_bytes(tokens, Hq, D, f32));
+  if (int32_t rc = fill_bwd_run(&P.run[0], g, p, B, q, do_src, k, v, sc.dq32, lse, delta, dk, dv, partial)) return rc;
   if (int32_t rc = launch_fused(P, dim3(P.run[0].plane, 1, B), p, scale, st)) return rc;
+  if (int32_t rc = launch_dkdv_reduce(P.run[0], B, p, scale, st)) return rc;
   return launch_convert(T, p, tokens, sc, dq, scale, st);
 }
 
@@ -1487,6 +1606,15 @@ int32_t launch_bwd_sm100_runs(const SeqRun* runs, int n_runs, long long tokens, 
   const BwdScratch sc = carve_scratch(workspace, tokens, Hq, D, f32);
   const void* do_src = f32 ? static_cast<const void*>(sc.do_bf16) : d_o;
   const size_t rq = (size_t)Hq * D * 2, rk = (size_t)Hkv * D * 2;
+  // the chunks' partial dK / dV: one slice per run, behind the scratch of the packed tokens
+  std::vector<float*> partial_of(n_runs);
+  {
+    char* at = static_cast<char*>(workspace) + bwd_scratch_bytes(tokens, Hq, D, f32);
+    for (int i = 0; i < n_runs; ++i) {
+      partial_of[i] = reinterpret_cast<float*>(at);
+      at += bwd_partial_bytes(runs[i].g, runs[i].batch, Hq, Hkv, D);
+    }
+  }
   for (int first = 0; first < n_runs; first += kMaxRunsPerLaunch) {
     const int n = n_runs - first < kMaxRunsPerLaunch ? n_runs - first : kMaxRunsPerLaunch;
     // the runs of one launch hold consecutive packed tokens [tok_lo, tok_hi)
@@ -1512,7 +1640,7 @@ int32_t launch_bwd_sm100_runs(const SeqRun* runs, int n_runs, long long tokens, 
                                     (const char*)do_src + r.first_row * rq, (const char*)k + r.first_row * rk,
                                     (const char*)v + r.first_row * rk, sc.dq32 + r.first_row * Hq * D,
                                     lse + r.first_row * Hq, sc.delta + r.first_row * Hq, (char*)dk + r.first_row * rk,
-                                    (char*)dv + r.first_row * rk))
+                                    (char*)dv + r.first_row * rk, partial_of[first + order[i]]))
         return rc;
       P.run[i].cta_begin = (int)ctas;
       ctas += (long long)P.run[i].plane * r.batch;
@@ -1527,6 +1655,8 @@ int32_t launch_bwd_sm100_runs(const SeqRun* runs, int n_runs, long long tokens, 
     if (int32_t rc = launch_prep(T, p, tok_hi - tok_lo, (const char*)d_o + tok_lo * rdo, (const char*)o + tok_lo * rq, part, st))
       return rc;
     if (int32_t rc = launch_fused(P, dim3((unsigned)ctas, 1, 1), p, scale, st)) return rc;
+    for (int i = 0; i < n; ++i)
+      if (int32_t rc = launch_dkdv_reduce(P.run[i], runs[first + order[i]].batch, p, scale, st)) return rc;
     if (int32_t rc = launch_convert(T, p, tok_hi - tok_lo, part, (char*)dq + tok_lo * rq, scale, st)) return rc;
   }
   return UNIGIST_OK;

@@ -125,6 +125,8 @@ void count_launch(int n = 1);
 // Streaming multiprocessors of the current device (asked once per device); 148, the B200's count, when no
 // device can be asked (a size query on a machine without a GPU).
 int sm_count();
+// Bytes of L2 cache of the current device (asked once per device); 126 MB, the B200's, when no device can be asked.
+size_t l2_bytes();
 // Records a CUDA event before and after the kernels launched in its scope when per-kernel
 // timing is switched on; also counts the launch.
 struct KernelScope {
@@ -173,6 +175,9 @@ int32_t launch_bwd_sm100_runs(const SeqRun* runs, int n_runs, long long tokens, 
 // Bytes of backward scratch for `tokens` packed tokens: Delta, the bf16 copy of an fp32 dO, and for head_dim 128
 // the fp32 dQ accumulator.
 size_t bwd_scratch_bytes(long long tokens, int Hq, int D, bool dout_fp32);
+// Bytes behind that scratch for the fp32 partial dK / dV of the sink and gist key tiles whose walk over the
+// queries is cut into chunks (0 where nothing is cut), for `batch` sequences of geometry g.
+size_t bwd_partial_bytes(const Geom& g, int batch, int Hq, int Hkv, int D);
 int32_t bwd_sm100_take_timeout(bool* timed_out);
 int32_t launch_compact_gather(const Geom& g, const unigist_problem& p, const void* k,
                               const void* v, void* kc, void* vc, int num_blocks,
@@ -196,5 +201,7 @@ int32_t launch_cache_append(const Geom& g, const unigist_problem& p, int is_gist
                             int32_t* seq_lens, int32_t* state, cudaStream_t st);
 int decode_num_splits(int S, int Hkv, int max_blocks);
 int32_t decode_take_timeout(bool* timed_out);
+int32_t launch_selftest_wait(cudaStream_t st);
+int32_t selftest_take_timeout(bool* timed_out);
 
 }  // namespace ug
