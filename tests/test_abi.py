@@ -95,3 +95,28 @@ def test_null_and_misaligned_pointers_are_rejected_before_any_launch():
     rc = lib.unigist_decode(1, 6, 4, 128, 0.0, a, a, a, 1, a, 1, a, a, None, a, 1 << 20, None)
     assert rc == 2
     assert ug.unigist_launch_count() == before
+
+
+def test_backward_workspace_sizes_hold_every_part():
+    """Host arithmetic only: the backward's scratch is Delta + (a bf16 copy of an fp32 dO) + (head_dim 128: the fp32
+    dQ accumulator) + (the partial dK / dV of walks that are cut, only where one KV head's sweep exceeds the L2)."""
+    def need(B, T, r, W, Hq, Hkv, D, flags=0, s=0):
+        return ug.unigist_workspace_bytes(ug.Problem(B, T, r, W, Hq, Hkv, D, num_sinks=s, flags=flags), ug.OP_BWD)
+
+    al = lambda x: -(-x // 256) * 256
+    N = 16384 + 2048
+    base = al(32 * N * 4) + al(N * 32 * 128 * 4)
+    assert need(1, 16384, 8, 1024, 32, 8, 128) == base                      # 75 MB per KV head: no cut walks
+    assert need(1, 16384, 8, 1024, 32, 8, 128, ug.FLAG_DOUT_FP32) == base + al(N * 32 * 128 * 2)
+    assert need(1, 16384, 8, 1024, 32, 8, 64) == al(32 * N * 4)              # head_dim 64: Delta only
+    # the training workload: 168 MB per KV head > 3/4 of the L2 -> 4 chunks over 64 gist key tiles per KV head
+    Nt = 32768 + 8192
+    got = need(4, 32768, 4, 2048, 32, 8, 128)
+    assert got == al(4 * 32 * Nt * 4) + al(4 * Nt * 32 * 128 * 4) + 4 * 8 * 64 * 4 * 2 * 128 * 128 * 4
+    # a packed sample: one scratch over all tokens; short documents cut nothing
+    p = ug.Problem(1, 64, 4, 8, 4, 2, 128)
+    docs = [256, 64, 64, 132]
+    n_tot = ug.unigist_docs_total_len(p, docs)
+    assert n_tot == sum(t + t // 4 for t in docs)
+    assert ug.unigist_docs_workspace_bytes(p, ug.OP_BWD, docs) == al(4 * n_tot * 4) + al(n_tot * 4 * 128 * 4)
+    assert ug.unigist_docs_workspace_bytes(p, ug.OP_FWD, docs) == 0
