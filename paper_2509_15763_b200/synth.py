@@ -30,6 +30,7 @@ class Workload:
     head_dim: int
     num_sinks: int = 0
     k_scale: float = 1.0
+    dout_scale: float = 1.0  # dO is drawn as N(0, 1) * dout_scale
     seed: int = BASE_SEED
     forward_only: bool = False  # the workload is a prefill: no backward pass
 
@@ -104,7 +105,7 @@ def attention_inputs(w: Workload, with_grad: bool = True, dout_fp32: bool = Fals
     v = draw(w.num_kv_heads).to(torch.bfloat16)
     out = {"q": q, "k": k, "v": v}
     if with_grad:
-        d = draw(w.num_q_heads)
+        d = draw(w.num_q_heads) * w.dout_scale
         out["dout"] = d if dout_fp32 else d.to(torch.bfloat16)
     return out
 

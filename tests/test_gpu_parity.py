@@ -73,6 +73,10 @@ SMALL = [
     # gist units longer than a tile: plain causal attention as a single unit, and two-tile units with a one-unit window
     synth.Workload("single_unit_causal", 1, 640, 640, 640, 2, 2, 128, seed=116),
     synth.Workload("long_units", 2, 1024, 256, 256, 4, 2, 128, num_sinks=5, seed=117),
+    # 32 query heads on one KV head: the rows one KV head's blocks sweep (133 MB) exceed the L2, so the backward cuts
+    # the walks of the sink and gist key tiles (2 + 4 tiles, 34 query tiles) into two chunks and adds partial dK / dV
+    # (dO scaled down: 32 heads add into one KV head, and the gradient tolerance is absolute)
+    synth.Workload("cut_walks_sinks", 2, 3584, 8, 256, 32, 1, 128, num_sinks=130, dout_scale=0.25, seed=118),
 ]
 
 
