@@ -696,7 +696,9 @@ def run_ours(args, w):
                        "neighbouring steps run on two side streams under the kernels (two device buffer sets)"},
         "explicit_shift_step": None if explicit_ms is None else {
             "ms_per_step": explicit_ms, "value": path.flops / (explicit_ms * 1e-3) / 1e12, "unit": UNIT,
-            "note": "the same step with 4 shift and 4 unshift launches around shifted-order attention calls"},
+            "shift_unshift_ms": explicit_ms - total_ms / args.steps,
+            "note": "the same step with 4 shift and 4 unshift launches around shifted-order attention calls; "
+                    "shift_unshift_ms is what those 8 launches add"},
         "gpu_launches": launches,
         "clocks": clocks,
         # clock-normalised step: milliseconds x median SM MHz = thousands of SM cycles per step

@@ -789,18 +789,23 @@ struct alignas(64) BwdRun {
   __nv_bfloat16* dk;
   __nv_bfloat16* dv;
   int n_sink_kt, n_gist_kt, n_raw_kt;
-  int cta_begin, plane;  // flat grid: first block of the unit; blocks per batch index
+  int plane;  // blocks per batch index
+  // flat grid (several units in one launch): the sink / gist blocks of ALL units come first, then the raw blocks;
+  // the unit's first block in each of the two ranges, and its blocks per batch index there
+  int heavy_begin, raw_begin, heavy_plane, raw_plane;
+  FastDiv heavy_plane_div, raw_plane_div;
   // A sink or gist key tile's walk over its query tiles is cut into n_chunks chunks of chunk_tiles tiles, one
   // block each; `partial` receives the fp32 dK / dV of the chunks of key tiles that have more than one
   // ([batch][KV head][heavy key tile][chunk][dK | dV][128 keys][128]).
   int n_chunks, chunk_tiles;
   float* partial;
-  FastDiv heavy_div /* by n_chunks * heavy tiles */, tile_div /* by heavy tiles */, raw_div, plane_div;
+  FastDiv heavy_div /* by n_chunks * heavy tiles */, tile_div /* by heavy tiles */, raw_div;
 };
 template <int kRuns>
 struct BwdRuns {
   BwdRun run[kRuns];
   int n;
+  int total_heavy;  // flat grid: blocks of the sink / gist range
 };
 constexpr int kMaxRunsPerLaunch = 12;  // 12 units are 24 KB of kernel parameters (the limit is 32 KB)
 
@@ -813,10 +818,17 @@ attn_bwd_fused_sm100_kernel(const __grid_constant__ BwdRuns<kRuns> P, int Hq, in
     bx = blockIdx.x, b = blockIdx.z;
   } else {
     const int c = blockIdx.x;
-    while (ri + 1 < P.n && c >= P.run[ri + 1].cta_begin) ++ri;
-    const int local = c - P.run[ri].cta_begin;
-    b = fdiv(P.run[ri].plane_div, local);
-    bx = local - b * P.run[ri].plane;
+    if (c < P.total_heavy) {
+      while (ri + 1 < P.n && c >= P.run[ri + 1].heavy_begin) ++ri;
+      const int local = c - P.run[ri].heavy_begin;
+      b = fdiv(P.run[ri].heavy_plane_div, local);
+      bx = local - b * P.run[ri].heavy_plane;  // < heavy_plane: a sink / gist block of the unit
+    } else {
+      while (ri + 1 < P.n && c >= P.run[ri + 1].raw_begin) ++ri;
+      const int local = c - P.run[ri].raw_begin;
+      b = fdiv(P.run[ri].raw_plane_div, local);
+      bx = P.run[ri].heavy_plane + (local - b * P.run[ri].raw_plane);
+    }
   }
   const BwdRun& R = P.run[ri];
   const Geom g = R.g;
@@ -1483,12 +1495,15 @@ int32_t fill_bwd_run(BwdRun* R, const Geom& g, const unigist_problem& p, int bat
   bwd_chunking(g, batch, Hq, Hkv, &R->n_chunks, &R->chunk_tiles);
   R->partial = partial;
   const int n_heavy = R->n_sink_kt + R->n_gist_kt;
-  R->plane = (n_heavy * R->n_chunks + R->n_raw_kt) * Hkv;
-  R->cta_begin = 0;
+  R->heavy_plane = n_heavy * R->n_chunks * Hkv;
+  R->raw_plane = R->n_raw_kt * Hkv;
+  R->plane = R->heavy_plane + R->raw_plane;
+  R->heavy_begin = R->raw_begin = 0;
+  R->heavy_plane_div = make_fastdiv(R->heavy_plane);
+  R->raw_plane_div = make_fastdiv(R->raw_plane);
   R->heavy_div = make_fastdiv(n_heavy * R->n_chunks);
   R->tile_div = make_fastdiv(n_heavy);
   R->raw_div = make_fastdiv(R->n_raw_kt);
-  R->plane_div = make_fastdiv(R->plane);
   return UNIGIST_OK;
 }
 
@@ -1589,6 +1604,7 @@ int32_t launch_bwd_sm100(const Geom& g, const unigist_problem& p, float scale, c
   }
   BwdRuns<1> P;
   P.n = 1;
+  P.total_heavy = 0;  // not used with the (blocks, 1, batch) grid
   float* partial = reinterpret_cast<float*>(static_cast<char*>(workspace) + bwd_scratch_bytes(tokens, Hq, D, f32));
   if (int32_t rc = fill_bwd_run(&P.run[0], g, p, B, q, do_src, k, v, sc.dq32, lse, delta, dk, dv, partial)) return rc;
   if (int32_t rc = launch_fused(P, dim3(P.run[0].plane, 1, B), p, scale, st)) return rc;
@@ -1642,9 +1658,19 @@ int32_t launch_bwd_sm100_runs(const SeqRun* runs, int n_runs, long long tokens, 
                                     lse + r.first_row * Hq, sc.delta + r.first_row * Hq, (char*)dk + r.first_row * rk,
                                     (char*)dv + r.first_row * rk, partial_of[first + order[i]]))
         return rc;
-      P.run[i].cta_begin = (int)ctas;
       ctas += (long long)P.run[i].plane * r.batch;
       if (ctas > 0x7fffffffLL) return fail(UNIGIST_ERR_SHAPE, "packed sample too large for one grid");
+    }
+    // block ranges: every unit's sink / gist blocks (the long ones) before any unit's raw blocks
+    int at = 0;
+    for (int i = 0; i < n; ++i) {
+      P.run[i].heavy_begin = at;
+      at += P.run[i].heavy_plane * runs[first + order[i]].batch;
+    }
+    P.total_heavy = at;
+    for (int i = 0; i < n; ++i) {
+      P.run[i].raw_begin = at;
+      at += P.run[i].raw_plane * runs[first + order[i]].batch;
     }
     for (int i = n; i < kMaxRunsPerLaunch; ++i) T.run[i] = T.run[0], P.run[i] = P.run[0];  // never selected
     // the per-token kernels of this launch see the tensors from packed token tok_lo on
