@@ -808,6 +808,7 @@ struct BwdRuns {
   int total_heavy;  // flat grid: blocks of the sink / gist range
 };
 constexpr int kMaxRunsPerLaunch = 12;  // 12 units are 24 KB of kernel parameters (the limit is 32 KB)
+static_assert(sizeof(BwdRuns<kMaxRunsPerLaunch>) + 256 <= 32764, "the launch units must fit the kernel parameter space");
 
 template <int kRuns>
 __global__ void __launch_bounds__(kFuThreads, 1)

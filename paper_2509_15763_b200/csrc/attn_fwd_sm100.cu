@@ -255,6 +255,7 @@ struct FwdRuns {
   int n;
 };
 constexpr int kMaxRunsPerLaunch = 12;  // 12 units are 20 KB of kernel parameters (the limit is 32 KB)
+static_assert(sizeof(FwdRuns<kMaxRunsPerLaunch>) + 256 <= 32764, "the launch units must fit the kernel parameter space");
 
 template <int D, int kRuns>
 __global__ void __launch_bounds__(kThreads, 1)
