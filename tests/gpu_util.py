@@ -88,3 +88,25 @@ def check_close(name, got: np.ndarray, want: np.ndarray, tol_max: float, tol_mea
     assert err.max() <= tol_max, f"{name}: max-abs {err.max():.4g} > {tol_max}"
     if tol_mean is not None:
         assert err.mean() <= tol_mean, f"{name}: mean-abs {err.mean():.4g} > {tol_mean}"
+
+
+def edge_positions(s, T, r, k):
+    """SHIFTED positions of the rows / keys the 128-row tile kernels branch on: the first and last row of the first
+    tile of each segment, of the tile in which the window starts to clip (raw row (k + 1) r, gist k + 1), of a middle
+    tile and of the last tile, the rows on either side of the clipping point, a row inside a tile, and the sinks' ends."""
+    n = T // r
+    pos = set()
+
+    def tiles(base, length, first_clipped):
+        last_tile = (length - 1) // 128
+        for j in {0, min(first_clipped // 128, last_tile), last_tile // 2, last_tile}:
+            pos.update(base + x for x in (128 * j, min(128 * j + 127, length - 1)))
+        for x in (first_clipped - 1, first_clipped, length // 3 + 5):
+            if 0 <= x < length:
+                pos.add(base + x)
+
+    tiles(s, T, (k + 1) * r)      # raw rows: unit k + 1 is the first whose window no longer reaches unit 0
+    tiles(s + T, n, k + 1)        # gist rows
+    if s:
+        pos.update((0, s - 1))
+    return np.array(sorted(pos), dtype=np.int64)

@@ -7,7 +7,7 @@ import paper_2509_15763_b200 as ug
 from paper_2509_15763_b200 import synth
 from oracle import oracle
 
-from gpu_util import (TOL_GRAD, TOL_LSE, TOL_O_MAX, TOL_O_MEAN, check_close, f64, problem_of,
+from gpu_util import (TOL_GRAD, TOL_LSE, TOL_O_MAX, TOL_O_MEAN, check_close, edge_positions, f64, problem_of,
                       run_attention, run_attention_interleaved)
 
 pytestmark = pytest.mark.gpu
@@ -145,28 +145,6 @@ def test_forward_is_deterministic():
 
 
 # ------------------------------------------------------------------ full-size workloads, sampled outputs
-def _edge_positions(s, T, r, k):
-    """SHIFTED positions of the rows / keys the 128-row tile kernels branch on: the first and last row of the first
-    tile of each segment, of the tile in which the window starts to clip (raw row (k + 1) r, gist k + 1), of a middle
-    tile and of the last tile, the rows on either side of the clipping point, a row inside a tile, and the sinks' ends."""
-    n = T // r
-    pos = set()
-
-    def tiles(base, length, first_clipped):
-        last_tile = (length - 1) // 128
-        for j in {0, min(first_clipped // 128, last_tile), last_tile // 2, last_tile}:
-            pos.update(base + x for x in (128 * j, min(128 * j + 127, length - 1)))
-        for x in (first_clipped - 1, first_clipped, length // 3 + 5):
-            if 0 <= x < length:
-                pos.add(base + x)
-
-    tiles(s, T, (k + 1) * r)      # raw rows: unit k + 1 is the first whose window no longer reaches unit 0
-    tiles(s + T, n, k + 1)        # gist rows
-    if s:
-        pos.update((0, s - 1))
-    return np.array(sorted(pos), dtype=np.int64)
-
-
 @pytest.mark.parametrize("name,backward,route", [("llama8b_layer", True, "explicit"), ("train_batch", True, "explicit"),
                                                  ("long_prefill", False, "explicit"),
                                                  # the route bench.py times: interleaved tensors, no shift launches
@@ -184,7 +162,7 @@ def test_full_size_sampled(name, backward, route):
     scale = w.head_dim ** -0.5
     rng = np.random.default_rng(w.seed)
     sp, _, _ = oracle.layout(s, T, r)
-    edge = sp[_edge_positions(s, T, r, min(k, T // r))].astype(np.int64)  # interleaved indices of the edge rows
+    edge = sp[edge_positions(s, T, r, min(k, T // r))].astype(np.int64)  # interleaved indices of the edge rows
     hk0 = int(rng.integers(0, w.num_kv_heads))
     kv_heads = sorted({hk0, (hk0 + max(1, w.num_kv_heads // 2)) % w.num_kv_heads})
     # no row anywhere was left unwritten
