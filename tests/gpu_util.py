@@ -17,12 +17,12 @@ def problem_of(w: synth.Workload, flags: int = 0) -> ug.Problem:
                       w.head_dim, num_sinks=w.num_sinks, flags=flags)
 
 
-def run_attention_interleaved(w: synth.Workload, backward: bool = True, inputs=None):
+def run_attention_interleaved(w: synth.Workload, backward: bool = True, inputs=None, dout_fp32: bool = False):
     """The same results as run_attention, computed with UNIGIST_FLAG_INTERLEAVED: the library reads the
     interleaved tensors as they are and writes o, dq, dk, dv interleaved; no shift / unshift call."""
     dev = torch.device("cuda:0")
-    inp = inputs or synth.attention_inputs(w, with_grad=backward)
-    p = problem_of(w, ug.FLAG_INTERLEAVED)
+    inp = inputs or synth.attention_inputs(w, with_grad=backward, dout_fp32=dout_fp32)
+    p = problem_of(w, ug.FLAG_INTERLEAVED | (ug.FLAG_DOUT_FP32 if (backward and dout_fp32) else 0))
     N = ug.unigist_total_len(p)
     d = {k: v.to(dev) for k, v in inp.items()}
     o = torch.full_like(d["q"], float("nan"))

@@ -82,6 +82,32 @@ def test_docs_match_oracle(case):
     check_close("dv", f64(from_lib(dv)), dv_ref, TOL_GRAD)
 
 
+@pytest.mark.parametrize("D,il", [(128, True), (128, False), (64, False)])
+def test_docs_backward_takes_an_fp32_dout(D, il):
+    """UNIGIST_FLAG_DOUT_FP32 on a packed sample: the gradients of the same dO rounded to bf16, bit for bit."""
+    s, r, W, doc_T, Hq, Hkv = 4, 4, 8, [64, 132, 64, 64, 8], 4, 2
+    flags = ug.FLAG_INTERLEAVED if il else 0
+    p16 = ug.Problem(1, doc_T[0], r, W, Hq, Hkv, D, num_sinks=s, flags=flags)
+    p32 = ug.Problem(1, doc_T[0], r, W, Hq, Hkv, D, num_sinks=s, flags=flags | ug.FLAG_DOUT_FP32)
+    n_tot = ug.unigist_docs_total_len(p16, doc_T)
+    dev = torch.device("cuda:0")
+    q, k, v, _ = (t.to(dev) for t in _packed_inputs(n_tot, Hq, Hkv, D, 31))
+    do32 = torch.randn(n_tot, Hq, D, generator=torch.Generator().manual_seed(32)).to(dev)
+    o = torch.empty_like(q)
+    lse = torch.empty(Hq * n_tot, device=dev)
+    ug.unigist_attn_fwd_docs(p16, doc_T, q, k, v, o, lse)
+    got = {}
+    for p, do in ((p16, do32.to(torch.bfloat16)), (p32, do32)):
+        ws = torch.empty(max(ug.unigist_docs_workspace_bytes(p, ug.OP_BWD, doc_T), 16), dtype=torch.uint8, device=dev)
+        dq, dk, dv = (torch.full_like(t, float("nan")) for t in (q, k, v))
+        ug.unigist_attn_bwd_docs(p, doc_T, q, k, v, o, lse, do, dq, dk, dv, ws)
+        ug.unigist_device_status()
+        got[p is p32] = (dq, dk, dv)
+    assert torch.isfinite(got[True][0].float()).all()
+    assert torch.equal(got[True][1], got[False][1]) and torch.equal(got[True][2], got[False][2])
+    assert (got[True][0].float() - got[False][0].float()).abs().max().item() <= 2.0 ** -7
+
+
 def test_docs_reject_bad_lists():
     p = ug.Problem(1, 16, 4, 8, 2, 2, 128)
     x = torch.zeros(64, 2, 128, dtype=torch.bfloat16, device="cuda")

@@ -122,6 +122,29 @@ def test_interleaved_tensors_match_oracle(w):
     assert (out["dq"].float() - ref["dq"].float()).abs().max().item() <= 2.0 ** -7
 
 
+@pytest.mark.parametrize("name", ["gqa_128", "sinks_300", "ragged_group3_128", "ragged_64"])
+def test_fp32_dout_is_rounded_to_bf16_on_load(name):
+    """UNIGIST_FLAG_DOUT_FP32: the gradients are those of the same dO rounded to bf16 (round to nearest even), bit
+    for bit, on both backward paths and in both tensor orders; and they match the oracle on the rounded dO."""
+    w = next(x for x in SMALL if x.name == name)
+    inp32 = synth.attention_inputs(w, dout_fp32=True)
+    assert inp32["dout"].dtype == torch.float32
+    inp16 = dict(inp32, dout=inp32["dout"].to(torch.bfloat16))
+    routes = [run_attention] + ([run_attention_interleaved] if w in INTERLEAVED else [])
+    for run in routes:
+        a = run(w, inputs=inp32, dout_fp32=True)
+        b = run(w, inputs=inp16)
+        for n in ("dk", "dv"):
+            assert torch.equal(a[n], b[n]), (run.__name__, n)
+        assert (a["dq"].float() - b["dq"].float()).abs().max().item() <= 2.0 ** -7
+    k = oracle.window_units(w.window, w.ratio)
+    dq, dk, dv = oracle.attn_bwd(w.num_sinks, w.raw_len, w.ratio, k, w.head_dim ** -0.5,
+                                 *(f64(inp16[n]) for n in ("q", "k", "v", "dout")))
+    check_close("dQ", f64(a["dq"]), dq, TOL_GRAD)
+    check_close("dK", f64(a["dk"]), dk, TOL_GRAD)
+    check_close("dV", f64(a["dv"]), dv, TOL_GRAD)
+
+
 def test_interleaved_flag_is_refused_where_the_tiles_do_not_line_up():
     for w in (SMALL[0], synth.Workload("r7", 1, 448, 7, 64, 2, 1, 128, seed=1)):
         p = problem_of(w, ug.FLAG_INTERLEAVED)
