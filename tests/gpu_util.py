@@ -12,17 +12,18 @@ from paper_2509_15763_b200 import synth
 TOL_O_MAX, TOL_O_MEAN, TOL_LSE, TOL_GRAD = 2e-2, 2e-3, 1e-3, 5e-2
 
 
-def problem_of(w: synth.Workload, flags: int = 0) -> ug.Problem:
+def problem_of(w: synth.Workload, flags: int = 0, softmax_scale: float = 0.0) -> ug.Problem:
     return ug.Problem(w.batch, w.raw_len, w.ratio, w.window, w.num_q_heads, w.num_kv_heads,
-                      w.head_dim, num_sinks=w.num_sinks, flags=flags)
+                      w.head_dim, num_sinks=w.num_sinks, softmax_scale=softmax_scale, flags=flags)
 
 
-def run_attention_interleaved(w: synth.Workload, backward: bool = True, inputs=None, dout_fp32: bool = False):
+def run_attention_interleaved(w: synth.Workload, backward: bool = True, inputs=None, dout_fp32: bool = False,
+                              softmax_scale: float = 0.0):
     """The same results as run_attention, computed with UNIGIST_FLAG_INTERLEAVED: the library reads the
     interleaved tensors as they are and writes o, dq, dk, dv interleaved; no shift / unshift call."""
     dev = torch.device("cuda:0")
     inp = inputs or synth.attention_inputs(w, with_grad=backward, dout_fp32=dout_fp32)
-    p = problem_of(w, ug.FLAG_INTERLEAVED | (ug.FLAG_DOUT_FP32 if (backward and dout_fp32) else 0))
+    p = problem_of(w, ug.FLAG_INTERLEAVED | (ug.FLAG_DOUT_FP32 if (backward and dout_fp32) else 0), softmax_scale)
     N = ug.unigist_total_len(p)
     d = {k: v.to(dev) for k, v in inp.items()}
     o = torch.full_like(d["q"], float("nan"))
@@ -41,11 +42,12 @@ def run_attention_interleaved(w: synth.Workload, backward: bool = True, inputs=N
     return out
 
 
-def run_attention(w: synth.Workload, backward: bool = True, dout_fp32: bool = False, inputs=None):
+def run_attention(w: synth.Workload, backward: bool = True, dout_fp32: bool = False, inputs=None,
+                  softmax_scale: float = 0.0):
     """-> dict of CUDA tensors in INTERLEAVED order: o, lse [B,Hq,N], dq, dk, dv, plus inputs."""
     dev = torch.device("cuda:0")
     inp = inputs or synth.attention_inputs(w, with_grad=backward, dout_fp32=dout_fp32)
-    p = problem_of(w, ug.FLAG_DOUT_FP32 if (backward and dout_fp32) else 0)
+    p = problem_of(w, ug.FLAG_DOUT_FP32 if (backward and dout_fp32) else 0, softmax_scale)
     N = ug.unigist_total_len(p)
     d = {k: v.to(dev) for k, v in inp.items()}
     sh = {}

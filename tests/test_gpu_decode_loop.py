@@ -24,6 +24,7 @@ CASES = [
     (2, 0, 120, 8, 1000, 8, 2, 2),    # the window never fills: nothing is ever evicted
     (1, 130, 70, 7, 15, 4, 4, 1),     # sinks over two pages, window of ceil(15 / 7) = 3 units
 ]
+CASES = [c + (0.0,) for c in CASES] + [(2, 2, 64, 4, 8, 4, 2, 2, 0.05)]  # the last: a caller-given softmax scale
 
 
 def read_cache(cache, table_row, length):
@@ -31,15 +32,15 @@ def read_cache(cache, table_row, length):
     return blocks.permute(0, 2, 1, 3).reshape(-1, cache.shape[1], cache.shape[3])[:length]
 
 
-@pytest.mark.parametrize("B,s,T,r,W,Hq,Hkv,units0", CASES)
-def test_decode_loop_matches_the_one_pass_forward(B, s, T, r, W, Hq, Hkv, units0):
+@pytest.mark.parametrize("B,s,T,r,W,Hq,Hkv,units0,given_scale", CASES)
+def test_decode_loop_matches_the_one_pass_forward(B, s, T, r, W, Hq, Hkv, units0, given_scale):
     D = 128
     w = synth.Workload("loop", B, T, r, W, Hq, Hkv, D, num_sinks=s, seed=777 + T + r)
     inp = synth.attention_inputs(w, with_grad=False)
     k_units = oracle.window_units(W, r)
-    scale = D ** -0.5
+    scale = given_scale or D ** -0.5
     o_ref, lse_ref = oracle.attn_fwd(s, T, r, k_units, scale, *(f64(inp[n]) for n in ("q", "k", "v")))
-    p = ug.Problem(B, T, r, W, Hq, Hkv, D, num_sinks=s)
+    p = ug.Problem(B, T, r, W, Hq, Hkv, D, num_sinks=s, softmax_scale=given_scale)
     n = T // r
     per_seq = -(-(s + n + (k_units + 1) * r + 1) // PG)
     nblocks = B * per_seq + 1

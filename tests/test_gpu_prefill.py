@@ -24,6 +24,11 @@ CASES = [
     (1, 3, 640, 4, 0, 2, 2, 128, [100, 60]),             # no window: gists and sinks only
     (1, 0, 512, 8, 64, 2, 1, 128, [64]),                 # one chunk = the whole prompt
 ]
+CASES = [c + (0.0,) for c in CASES] + [
+    # a caller-given softmax scale instead of 1 / sqrt(head_dim)
+    (2, 4, 768, 8, 64, 4, 2, 128, [24, 40, 32], 0.05),
+    (1, 0, 330, 5, 48, 2, 1, 64, [30, 36], 0.3),
+]
 
 
 def read_cache(cache, table_row, length):
@@ -31,15 +36,15 @@ def read_cache(cache, table_row, length):
     return blocks.permute(0, 2, 1, 3).reshape(-1, cache.shape[1], cache.shape[3])[:length]
 
 
-@pytest.mark.parametrize("B,s,T,r,W,Hq,Hkv,D,chunks", CASES)
-def test_chunked_prefill_matches_the_one_pass_forward(B, s, T, r, W, Hq, Hkv, D, chunks):
+@pytest.mark.parametrize("B,s,T,r,W,Hq,Hkv,D,chunks,given_scale", CASES)
+def test_chunked_prefill_matches_the_one_pass_forward(B, s, T, r, W, Hq, Hkv, D, chunks, given_scale):
     assert sum(chunks) == T // r
     w = synth.Workload("prefill", B, T, r, W, Hq, Hkv, D, num_sinks=s, seed=4242 + T + r)
     inp = synth.attention_inputs(w, with_grad=False)
     k_units = oracle.window_units(W, r)
-    scale = D ** -0.5
+    scale = given_scale or D ** -0.5
     o_ref, lse_ref = oracle.attn_fwd(s, T, r, k_units, scale, *(f64(inp[n]) for n in ("q", "k", "v")))
-    p = ug.Problem(B, T, r, W, Hq, Hkv, D, num_sinks=s)
+    p = ug.Problem(B, T, r, W, Hq, Hkv, D, num_sinks=s, softmax_scale=given_scale)
     L_max = s + T // r + min(k_units, T // r) * r
     per_seq = -(-L_max // PG)
     nblocks = B * per_seq + 2
@@ -77,7 +82,7 @@ def test_chunked_prefill_matches_the_one_pass_forward(B, s, T, r, W, Hq, Hkv, D,
     qd = torch.randn(B, Hq, D, generator=g).to(torch.bfloat16)
     od = torch.empty(B, Hq, D, dtype=torch.bfloat16, device=DEV)
     wsd = torch.empty(ug.unigist_decode_workspace_bytes(B, Hq, Hkv, D, per_seq), dtype=torch.uint8, device=DEV)
-    ug.unigist_decode(qd.to(DEV), kc, vc, table_d, lens, od, None, wsd)
+    ug.unigist_decode(qd.to(DEV), kc, vc, table_d, lens, od, None, wsd, softmax_scale=given_scale)
     kept = torch.from_numpy(oracle.kept_set(s, T, r, min(k_units, T // r))).long()
     od_ref, _ = oracle.decode(scale, f64(qd), [f64(inp["k"][b, kept]) for b in range(B)],
                               [f64(inp["v"][b, kept]) for b in range(B)])
