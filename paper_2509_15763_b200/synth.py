@@ -30,6 +30,7 @@ class Workload:
     head_dim: int
     num_sinks: int = 0
     k_scale: float = 1.0
+    v_scale: float = 1.0
     dout_scale: float = 1.0  # dO is drawn as N(0, 1) * dout_scale
     seed: int = BASE_SEED
     forward_only: bool = False  # the workload is a prefill: no backward pass
@@ -102,7 +103,7 @@ def attention_inputs(w: Workload, with_grad: bool = True, dout_fp32: bool = Fals
 
     q = draw(w.num_q_heads).to(torch.bfloat16)
     k = (draw(w.num_kv_heads) * w.k_scale).to(torch.bfloat16)
-    v = draw(w.num_kv_heads).to(torch.bfloat16)
+    v = (draw(w.num_kv_heads) * w.v_scale).to(torch.bfloat16)
     out = {"q": q, "k": k, "v": v}
     if with_grad:
         d = draw(w.num_q_heads) * w.dout_scale
