@@ -30,6 +30,21 @@ COMPACT_CASES = [
 ]
 
 
+def _random_compact_cases(count, seed):
+    rng = np.random.default_rng(seed)
+    out = []
+    while len(out) < count:
+        r = int(rng.choice([1, 2, 3, 4, 7, 8, 16, 64, 128]))
+        T = int(rng.integers(1, 2400 // r + 1)) * r
+        s = int(rng.choice([0, 0, 1, 63, 64, 65, 128, 200]))
+        W = int(rng.choice([0, r, 2 * r + 1, 64, 128, 500, 10 ** 6]))
+        out.append((int(rng.choice([1, 2, 3])), s, T, r, W, int(rng.choice([1, 2, 8])), int(rng.choice([64, 128]))))
+    return out
+
+
+COMPACT_CASES += _random_compact_cases(12, 5)
+
+
 @pytest.mark.parametrize("B,s,T,r,W,Hkv,D", COMPACT_CASES)
 @pytest.mark.parametrize("mode", ["gather", "gather_interleaved", "inplace"])
 def test_compaction_matches_oracle(B, s, T, r, W, Hkv, D, mode):

@@ -24,6 +24,21 @@ CASES = [
     (2, 0, 120, 8, 1000, 8, 2, 2),    # the window never fills: nothing is ever evicted
     (1, 130, 70, 7, 15, 4, 4, 1),     # sinks over two pages, window of ceil(15 / 7) = 3 units
 ]
+
+
+def _random_loop_cases(count, seed):
+    rng = np.random.default_rng(seed)
+    out = []
+    while len(out) < count:
+        r = int(rng.choice([1, 2, 3, 4, 8, 16]))
+        n = int(rng.integers(2, 160 // (r + 1) + 2))
+        Hkv = int(rng.choice([1, 2]))
+        out.append((int(rng.choice([1, 2])), int(rng.choice([0, 0, 2, 65])), n * r, r, int(rng.choice([0, r, 2 * r + 1, 40, 10 ** 6])),
+                    Hkv * int(rng.choice([1, 2, 4])), Hkv, int(rng.integers(0, n))))
+    return out
+
+
+CASES += _random_loop_cases(6, 9)
 CASES = [c + (0.0,) for c in CASES] + [(2, 2, 64, 4, 8, 4, 2, 2, 0.05)]  # the last: a caller-given softmax scale
 
 

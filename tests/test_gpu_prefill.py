@@ -24,6 +24,23 @@ CASES = [
     (1, 3, 640, 4, 0, 2, 2, 128, [100, 60]),             # no window: gists and sinks only
     (1, 0, 512, 8, 64, 2, 1, 128, [64]),                 # one chunk = the whole prompt
 ]
+def _random_prefill_cases(count, seed):
+    rng = np.random.default_rng(seed)
+    out = []
+    while len(out) < count:
+        r = int(rng.choice([1, 2, 4, 5, 8, 16, 32]))
+        n = int(rng.integers(2, 1200 // (r + 1) + 1))
+        s = int(rng.choice([0, 0, 3, 64, 130]))
+        W = int(rng.choice([0, r, 3 * r, 100, 10 ** 6]))
+        cuts = sorted(set(rng.integers(1, n, size=int(rng.integers(0, 5))).tolist()))
+        chunks = [b - a for a, b in zip([0] + cuts, cuts + [n])]
+        Hkv = int(rng.choice([1, 2]))
+        out.append((int(rng.choice([1, 2])), s, n * r, r, W, Hkv * int(rng.choice([1, 2, 4])), Hkv,
+                    int(rng.choice([64, 128])), chunks))
+    return out
+
+
+CASES += _random_prefill_cases(10, 3)
 CASES = [c + (0.0,) for c in CASES] + [
     # a caller-given softmax scale instead of 1 / sqrt(head_dim)
     (2, 4, 768, 8, 64, 4, 2, 128, [24, 40, 32], 0.05),
