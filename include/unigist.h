@@ -146,6 +146,7 @@ int32_t unigist_rope(const unigist_problem* p, const void* src, void* dst, int32
  *   S_tj = scale * q_t . k_j over visible j,  LSE_t = log sum_j exp(S_tj),  O_t = softmax(S_t) V.
  * q [B,N,Hq,D], k, v [B,N,Hkv,D], o [B,N,Hq,D]: device bf16, SHIFTED order.
  * lse [B,Hq,N]: device fp32, natural log, shifted order.  Masked-out tiles are never read.
+ * The forward needs no scratch: workspace may be NULL with ws_bytes 0 (unigist_workspace_bytes(p, UNIGIST_OP_FWD) is 0).
  */
 int32_t unigist_attn_fwd(const unigist_problem* p, const void* q, const void* k, const void* v,
                          void* o, float* lse, void* workspace, size_t ws_bytes, void* stream);
