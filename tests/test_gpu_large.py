@@ -157,3 +157,38 @@ def test_decode_over_a_cache_beyond_four_gib():
         oo, ll = oracle.decode(D ** -0.5, f64(q[i:i + 1]), [f64(rows_of(k_pool, i))], [f64(rows_of(v_pool, i))])
         check_close(f"decode O seq {i}", f64(o[i:i + 1]), oo, TOL_O_MAX, TOL_O_MEAN)
         check_close(f"decode LSE seq {i}", f64(lse[i:i + 1]), ll, TOL_LSE)
+
+
+def test_compaction_of_tensors_beyond_four_gib():
+    """Sixteen prompts of the long-prefill geometry (K and V 4.6 GB each) gathered into their compressed caches:
+    the kept rows of the last batch index, bit for bit, are the oracle's kept set of its sample."""
+    B = 16
+    w = synth.WORKLOADS["long_prefill"]
+    s, T, r, Hkv, D = w.num_sinks, w.raw_len, w.ratio, w.num_kv_heads, w.head_dim
+    p = ug.Problem(B, T, r, w.window, Hkv, Hkv, D, num_sinks=s, flags=ug.FLAG_INTERLEAVED)
+    N, L = ug.unigist_total_len(p), ug.unigist_compact_len(p)
+    assert B * N * Hkv * D * 2 > 2 ** 32
+    g = torch.Generator().manual_seed(w.seed + 2000)
+    k2 = torch.randn(2, N, Hkv, D, generator=g).to(torch.bfloat16)  # interleaved order (Eq. 2)
+    v2 = torch.randn(2, N, Hkv, D, generator=g).to(torch.bfloat16)
+    kept = torch.from_numpy(oracle.kept_set(s, T, r, oracle.window_units(w.window, r))).long()  # interleaved indices
+    assert len(kept) == L
+    per_seq = -(-L // PG)
+    nb = B * per_seq + 7
+    table = torch.randperm(nb, generator=g)[:B * per_seq].to(torch.int32).reshape(B, per_seq)
+    kc = torch.zeros(nb, Hkv, PG, D, dtype=torch.bfloat16, device=DEV)
+    vc = torch.zeros_like(kc)
+    lens = torch.zeros(B, dtype=torch.int32, device=DEV)
+    ug.unigist_kv_compact(p, _spread(k2, B), _spread(v2, B), kc, vc, table.to(DEV), lens)
+    torch.cuda.synchronize()
+    assert lens.cpu().tolist() == [L] * B
+
+    def rows(cache, b):
+        return cache[table[b].long().to(DEV)].permute(0, 2, 1, 3).reshape(-1, Hkv, D)[:L]
+
+    for cache, src in ((kc, k2), (vc, v2)):
+        assert torch.equal(rows(cache, B - 1).cpu(), src[1, kept])
+        first = rows(cache, 0)
+        assert torch.equal(first.cpu(), src[0, kept])
+        for b in range(1, B - 1):
+            assert torch.equal(rows(cache, b), first), b
