@@ -72,7 +72,7 @@ typedef enum {
 
 /* Problem statement of Section 4.1: (s, T, r, window) plus the attention shape. */
 typedef struct {
-  int32_t batch;        /* B >= 1 */
+  int32_t batch;        /* B >= 1; B and Hq at most 65535 */
   int32_t raw_len;      /* T, multiple of ratio */
   int32_t num_sinks;    /* s >= 0 */
   int32_t ratio;        /* r >= 1 */
@@ -283,7 +283,7 @@ size_t unigist_decode_workspace_bytes(int32_t num_seqs, int32_t num_q_heads, int
  * cache is visible by construction; the caller appends the new token's K/V first).
  * q, o [num_seqs, Hq, D] device bf16; k_cache, v_cache [num_blocks, Hkv, 64, D] device bf16;
  * block_table [num_seqs, max_blocks_per_seq], seq_lens [num_seqs] device int32 (>= 0);
- * lse [num_seqs, Hq] device fp32, nullable.  head_dim must be 128, Hq / Hkv at most 8.
+ * lse [num_seqs, Hq] device fp32, nullable.  head_dim must be 128, Hq / Hkv at most 8, num_seqs at most 65535.
  * A sequence with nothing to attend to (length 0: a padding slot of the batch) gets O = 0 and LSE = -inf.
  */
 int32_t unigist_decode(int32_t num_seqs, int32_t num_q_heads, int32_t num_kv_heads,

@@ -97,6 +97,8 @@ int32_t check_launch(const char* what) {
   return UNIGIST_OK;
 }
 
+constexpr int kMaxGridYZ = 65535;
+
 int32_t check_problem(const unigist_problem* p, Geom* g, float* scale) {
   if (!p) return fail(UNIGIST_ERR_INVALID_ARG, "problem is NULL");
   if (p->batch < 1 || p->raw_len < 1 || p->num_sinks < 0 || p->ratio < 1 || p->window < 0 ||
@@ -110,6 +112,9 @@ int32_t check_problem(const unigist_problem* p, Geom* g, float* scale) {
                 p->num_q_heads, p->num_kv_heads);
   if (p->head_dim != 64 && p->head_dim != 128)
     return fail(UNIGIST_ERR_SHAPE, "head_dim %d is not 64 or 128", p->head_dim);
+  // batch entries and heads are grid dimensions y / z of the kernels
+  if (p->batch > kMaxGridYZ || p->num_q_heads > kMaxGridYZ)
+    return fail(UNIGIST_ERR_SHAPE, "batch %d or num_q_heads %d exceeds %d", p->batch, p->num_q_heads, kMaxGridYZ);
   const int64_t n = p->raw_len / p->ratio;
   const int64_t N = (int64_t)p->num_sinks + p->raw_len + n;
   if (N > (int64_t)1 << 30) return fail(UNIGIST_ERR_SHAPE, "sequence too long");
@@ -572,6 +577,8 @@ int32_t unigist_decode(int32_t S, int32_t Hq, int32_t Hkv, int32_t D, float soft
                        float* lse, void* workspace, size_t ws_bytes, void* stream) {
   if (S < 1 || Hq < 1 || Hkv < 1 || max_blocks < 1 || num_blocks < 1)
     return fail(UNIGIST_ERR_INVALID_ARG, "decode has a non-positive size");
+  if (S > kMaxGridYZ || Hkv > kMaxGridYZ)
+    return fail(UNIGIST_ERR_SHAPE, "num_seqs %d or num_kv_heads %d exceeds %d", S, Hkv, kMaxGridYZ);
   if (Hq % Hkv) return fail(UNIGIST_ERR_SHAPE, "num_q_heads %d is not a multiple of num_kv_heads %d", Hq, Hkv);
   if (D != 128) return fail(UNIGIST_ERR_SHAPE, "decode supports head_dim 128, got %d", D);
   if (Hq / Hkv > 8) return fail(UNIGIST_ERR_UNSUPPORTED, "decode supports at most 8 query heads per KV head");

@@ -70,7 +70,10 @@ def test_interleaved_flag_is_validated_on_the_host():
 def test_malformed_problems_are_rejected():
     bad = [ug.Problem(1, 10, 3, 4, 1, 1, 64), ug.Problem(1, 16, 4, 4, 3, 2, 64),
            ug.Problem(1, 16, 4, 4, 1, 1, 96), ug.Problem(0, 16, 4, 4, 1, 1, 64),
-           ug.Problem(1, 16, 4, -1, 1, 1, 64)]
+           ug.Problem(1, 16, 4, -1, 1, 1, 64),
+           # batch entries and heads are grid dimensions of the kernels (at most 65535)
+           ug.Problem(65536, 16, 4, 4, 1, 1, 64), ug.Problem(1, 16, 4, 4, 65536, 1, 64)]
+    assert ug.unigist_total_len(ug.Problem(65535, 16, 4, 4, 1, 1, 64)) == 20
     for p in bad:
         assert ug.unigist_total_len(p) < 0
         assert ug.unigist_last_error_string()
