@@ -258,24 +258,46 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
   }
 }
 
-// One block per (seq, q head): merge the splits.
+constexpr int kMaxSplits = 32;  // one lane of a warp per split in the combine kernel
+
+// One block per (seq, q head): merge the splits.  Lane t of the first warp takes split t's maximum and
+// sum, so that all of them are in flight at once, and the warp reduces them; the weighted sum over the splits then
+// runs with eight splits' loads in flight instead of one dependent load after the other.
 __global__ void __launch_bounds__(DD)
 decode_combine_kernel(int splits, const float* __restrict__ part, __nv_bfloat16* __restrict__ o,
                       float* __restrict__ lse) {
+  __shared__ float s_w[kMaxSplits];
+  __shared__ float s_ml[2];
   const long long sh = blockIdx.x;
   const float* base = part + sh * splits * (DD + 2);
-  float M = -INFINITY;
-  for (int i = 0; i < splits; ++i) M = fmaxf(M, base[i * (DD + 2) + DD]);
-  float L = 0.f, acc = 0.f;
-  for (int i = 0; i < splits; ++i) {
-    const float m = base[i * (DD + 2) + DD];
+  const int t = threadIdx.x;
+  if (t < 32) {
+    float m = -INFINITY, l = 0.f;
+    if (t < splits) {
+      m = base[t * (DD + 2) + DD];
+      l = base[t * (DD + 2) + DD + 1];
+    }
+    float M = m;
+#pragma unroll
+    for (int off = 16; off >= 1; off >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, off));
     const float w = m == -INFINITY ? 0.f : exp2f(m - M);
-    L += w * base[i * (DD + 2) + DD + 1];
-    acc += w * base[i * (DD + 2) + threadIdx.x];
+    float L = w * l;
+#pragma unroll
+    for (int off = 16; off >= 1; off >>= 1) L += __shfl_xor_sync(0xffffffffu, L, off);
+    s_w[t] = w;
+    if (t == 0) {
+      s_ml[0] = M;
+      s_ml[1] = L;
+    }
   }
+  __syncthreads();
+  float acc = 0.f;
+#pragma unroll 8
+  for (int i = 0; i < splits; ++i) acc += s_w[i] * base[i * (DD + 2) + t];
+  const float M = s_ml[0], L = s_ml[1];
   // a sequence with nothing to attend to (length 0, or every slot freed): O = 0, LSE = -inf, not 0 / 0
-  o[sh * DD + threadIdx.x] = __float2bfloat16_rn(L > 0.f ? acc / L : 0.f);
-  if (lse && threadIdx.x == 0) lse[sh] = L > 0.f ? (M + log2f(L)) * 0.6931471805599453f : -INFINITY;
+  o[sh * DD + t] = __float2bfloat16_rn(L > 0.f ? acc / L : 0.f);
+  if (lse && t == 0) lse[sh] = L > 0.f ? (M + log2f(L)) * 0.6931471805599453f : -INFINITY;
 }
 
 }  // namespace
@@ -286,7 +308,7 @@ int decode_num_splits(int S, int Hkv, int max_blocks) {
   const long long base = (long long)S * Hkv;
   int best = 1;
   double best_eff = -1.0;
-  for (int sp = 1; sp <= 32; ++sp) {
+  for (int sp = 1; sp <= kMaxSplits; ++sp) {
     const int bps = (max_blocks + sp - 1) / sp;
     if (sp > 1 && bps < 4) break;
     if ((max_blocks + bps - 1) / bps != sp) continue;  // this count leaves an empty split
