@@ -62,6 +62,15 @@ typedef enum {
  */
 #define UNIGIST_FLAG_INTERLEAVED 2u
 
+/*
+ * unigist_attn_bwd / unigist_attn_bwd_docs with head_dim 128: dq, too, is the same bit for bit from run to run.
+ * dQ of a query tile is then summed in tensor memory by ONE thread block that walks the tile's keys (a second
+ * kernel that recomputes S and dP: seven matrix products per tile pair instead of five, 1.5 to 2 times the time)
+ * instead of being reduced into memory in the order in which key tiles' blocks arrive.  No effect for head_dim 64,
+ * whose backward always works this way.  Not together with UNIGIST_FLAG_INTERLEAVED (UNIGIST_ERR_UNSUPPORTED).
+ */
+#define UNIGIST_FLAG_DETERMINISTIC_DQ 4u
+
 enum { UNIGIST_PAGE_TOKENS = 64 }; /* tokens per KV-cache block */
 
 typedef enum {
@@ -161,7 +170,8 @@ int32_t unigist_attn_fwd(const unigist_problem* p, const void* q, const void* k,
  * it (sink and gist keys of a long sequence), by one block per chunk of those queries whose fp32 partial sums a
  * small kernel adds in chunk order; either way they are the same bit for bit from run to run.  For head_dim 128
  * dQ is the sum, over the key tiles that see a query tile, of fp32 partial tiles reduced into the workspace in
- * whatever order the blocks arrive: its last bit may differ between runs.  workspace:
+ * whatever order the blocks arrive: its last bit may differ between runs (UNIGIST_FLAG_DETERMINISTIC_DQ trades
+ * speed for a fixed order).  workspace:
  * unigist_workspace_bytes(p, UNIGIST_OP_BWD) bytes (Delta, a bf16 copy of an fp32 dO, and for head_dim 128 the
  * fp32 dQ accumulator and the chunks' partial dK / dV), 16-byte aligned.
  */

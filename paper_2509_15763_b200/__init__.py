@@ -1,5 +1,5 @@
 """UniGist gist-masked attention for B200 (sm_100a): Python binding of the C-ABI library."""
-from .binding import (DECODE_STATIC_SCRATCH_BYTES, FLAG_DOUT_FP32, FLAG_INTERLEAVED, ROPE_FROM_SHIFTED, ROPE_INVERSE, ROPE_TO_SHIFTED, unigist_rope, unigist_attn_bwd_docs, unigist_attn_fwd_docs, unigist_docs_total_len,
+from .binding import (DECODE_STATIC_SCRATCH_BYTES, FLAG_DETERMINISTIC_DQ, FLAG_DOUT_FP32, FLAG_INTERLEAVED, ROPE_FROM_SHIFTED, ROPE_INVERSE, ROPE_TO_SHIFTED, unigist_rope, unigist_attn_bwd_docs, unigist_attn_fwd_docs, unigist_docs_total_len,
                       unigist_docs_workspace_bytes, OP_BWD, OP_COMPACT, OP_FWD, PAGE_TOKENS, Problem, UnigistError,  # noqa: F401
                       unigist_attn_bwd, unigist_attn_fwd, unigist_cache_append, unigist_cache_state_bytes,
                       unigist_cache_state_init, unigist_compact_len, unigist_decode,

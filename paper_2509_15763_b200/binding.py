@@ -17,6 +17,7 @@ LIB_PATH = _PKG / "libunigist.so"
 
 OP_FWD, OP_BWD, OP_COMPACT = 0, 1, 2
 FLAG_DOUT_FP32 = 1
+FLAG_DETERMINISTIC_DQ = 4
 FLAG_INTERLEAVED = 2
 PAGE_TOKENS = 64
 

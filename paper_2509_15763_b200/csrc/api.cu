@@ -139,6 +139,9 @@ static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 // UNIGIST_FLAG_INTERLEAVED needs the tile addressing of the tensor-core kernels for head_dim 128.
 int32_t check_interleaved(const unigist_problem* p, const Geom& g) {
   if (!(p->flags & UNIGIST_FLAG_INTERLEAVED)) return UNIGIST_OK;
+  if (p->flags & UNIGIST_FLAG_DETERMINISTIC_DQ)
+    return fail(UNIGIST_ERR_UNSUPPORTED,
+                "UNIGIST_FLAG_DETERMINISTIC_DQ takes shifted tensors: its kernels do not address interleaved ones");
   if (p->head_dim != 128 || 128 % g.r != 0)
     return fail(UNIGIST_ERR_UNSUPPORTED,
                 "interleaved tensors need head_dim 128 and a ratio that divides 128 (got D = %d, r = %d): "
@@ -440,10 +443,10 @@ int32_t unigist_attn_bwd_docs(const unigist_problem* p, int32_t num_docs, const 
   if (int32_t rc = doc_runs(p, num_docs, doc_raw_len, &runs, &tokens)) return rc;
   if (int32_t rc = check_interleaved(p, runs[0].g)) return rc;
   const float scale = p->softmax_scale > 0.f ? p->softmax_scale : 1.0f / sqrtf((float)p->head_dim);
-  if (p->head_dim == 128)
+  if (p->head_dim == 128 && !(p->flags & UNIGIST_FLAG_DETERMINISTIC_DQ))
     return launch_bwd_sm100_runs(runs.data(), (int)runs.size(), tokens, *p, scale, q, k, v, o, lse, d_o, dq, dk, dv,
                                  workspace, (cudaStream_t)stream);
-  // head_dim 64 (two kernels per run): the runs one after the other on the caller's stream
+  // the two-kernel backward (head_dim 64, or a fixed summation order asked for): the runs one after the other on the caller's stream
   const size_t rq = (size_t)p->num_q_heads * p->head_dim * 2, rk = (size_t)p->num_kv_heads * p->head_dim * 2;
   const size_t rdo = (p->flags & UNIGIST_FLAG_DOUT_FP32) ? 2 * rq : rq;
   size_t ws_off = 0;

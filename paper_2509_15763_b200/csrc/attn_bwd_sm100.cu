@@ -1533,6 +1533,48 @@ int32_t launch_dkdv_reduce(const BwdRun& R, int batch, const unigist_problem& p,
   return check_launch("dK/dV reduce kernel");
 }
 
+// The two-kernel backward (head_dim 64; head_dim 128 when dQ has to be the same bit for bit from run to run): a
+// block of the first kernel owns a key tile (dK, dV), a block of the second a query tile (dQ, over 64-key tiles).
+template <int D>
+int32_t launch_two_kernels(const Geom& g, const unigist_problem& p, float scale, const void* q, const void* do_src,
+                           const void* k, const void* v, const float* lse, const float* delta, void* dq, void* dk,
+                           void* dv, cudaStream_t st) {
+  const int Hq = p.num_q_heads, Hkv = p.num_kv_heads, B = p.batch;
+  const int n_sink_t = (g.s + 127) / 128, n_raw_t = (g.T + 127) / 128, n_gist_t = (g.n + 127) / 128;
+  // one map per segment (sinks, raw, gists; a tensor map cannot be empty) with 128-row boxes, and 64-row boxes
+  // over K and V for the dQ kernel
+  CUtensorMap mq[3], md[3], mk[3], mv[3], mk64[3], mv64[3];
+  for (int sg = 0; sg < 3; ++sg) {
+    const long long first = seg_base(g, sg), len = seg_len(g, sg) > 0 ? seg_len(g, sg) : 1;
+    if (int32_t rc = encode_segment_map(&mq[sg], q, D, Hq, g.N, B, first, len, 128)) return rc;
+    if (int32_t rc = encode_segment_map(&md[sg], do_src, D, Hq, g.N, B, first, len, 128)) return rc;
+    if (int32_t rc = encode_segment_map(&mk[sg], k, D, Hkv, g.N, B, first, len, 128)) return rc;
+    if (int32_t rc = encode_segment_map(&mv[sg], v, D, Hkv, g.N, B, first, len, 128)) return rc;
+    if (int32_t rc = encode_segment_map(&mk64[sg], k, D, Hkv, g.N, B, first, len, DQ_BN)) return rc;
+    if (int32_t rc = encode_segment_map(&mv64[sg], v, D, Hkv, g.N, B, first, len, DQ_BN)) return rc;
+  }
+  const int n_tiles = n_sink_t + n_raw_t + n_gist_t;
+  cudaError_t e = cudaFuncSetAttribute(attn_bwd_dkdv_sm100_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       KvSmem<D>::kBytes);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(attn_bwd_dq_sm100_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, DqSmem<D>::kBytes);
+  if (e != cudaSuccess) return fail(UNIGIST_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
+  {
+    KernelScope ks("attn_bwd_dkdv_sm100_kernel", st);
+    attn_bwd_dkdv_sm100_kernel<D><<<dim3(n_tiles, Hkv, B), kKvThreads, KvSmem<D>::kBytes, st>>>(
+        mq[0], mq[1], mq[2], md[0], md[1], md[2], mk[0], mk[1], mk[2], mv[0], mv[1], mv[2], g, Hq, Hkv, scale, lse, delta,
+        (__nv_bfloat16*)dk, (__nv_bfloat16*)dv, n_sink_t, n_gist_t);
+  }
+  if (int32_t rc = check_launch("tcgen05 dK/dV kernel")) return rc;
+  {
+    KernelScope ks("attn_bwd_dq_sm100_kernel", st);
+    attn_bwd_dq_sm100_kernel<D><<<dim3(n_tiles, Hq, B), kDqThreads, DqSmem<D>::kBytes, st>>>(
+        mq[0], mq[1], mq[2], md[0], md[1], md[2], mk64[0], mk64[1], mk64[2], mv64[0], mv64[1], mv64[2], g, Hq, Hkv, scale,
+        lse, delta, (__nv_bfloat16*)dq, n_sink_t, n_raw_t);
+  }
+  return check_launch("tcgen05 dQ kernel");
+}
+
 }  // namespace
 
 size_t bwd_scratch_bytes(long long tokens, int Hq, int D, bool dout_fp32) {
@@ -1560,49 +1602,21 @@ int32_t launch_bwd_sm100(const Geom& g, const unigist_problem& p, float scale, c
   const BwdScratch sc = carve_scratch(workspace, tokens, Hq, D, f32);
   float* delta = sc.delta;
   const void* do_src = f32 ? static_cast<const void*>(sc.do_bf16) : d_o;
-  const bool fused = D == 128;  // head_dim 64 takes the two-kernel path
+  // head_dim 64 takes the two-kernel path, and so does head_dim 128 when dQ must not depend on the order in which
+  // blocks arrive
+  const bool fused = D == 128 && !(p.flags & UNIGIST_FLAG_DETERMINISTIC_DQ);
   TokRuns<1> T;
   T.n = 1;
   T.run[0].g = g;
   T.run[0].tok_begin = 0;
   T.run[0].delta = delta;
-  if (int32_t rc = launch_prep(T, p, tokens, d_o, o, sc, st)) return rc;
+  BwdScratch sc_prep = sc;
+  if (!fused) sc_prep.dq32 = nullptr;  // no fp32 dQ accumulator to clear
+  if (int32_t rc = launch_prep(T, p, tokens, d_o, o, sc_prep, st)) return rc;
 
-  const int n_sink_t = (g.s + 127) / 128, n_raw_t = (g.T + 127) / 128, n_gist_t = (g.n + 127) / 128;
-  if (!fused) {
-    // head_dim 64: one map per segment (sinks, raw, gists; a tensor map cannot be empty) with 128-row boxes,
-    // and 64-row boxes over K and V for the dQ kernel
-    CUtensorMap mq[3], md[3], mk[3], mv[3], mk64[3], mv64[3];
-    for (int sg = 0; sg < 3; ++sg) {
-      const long long first = seg_base(g, sg), len = seg_len(g, sg) > 0 ? seg_len(g, sg) : 1;
-      if (int32_t rc = encode_segment_map(&mq[sg], q, D, Hq, g.N, B, first, len, 128)) return rc;
-      if (int32_t rc = encode_segment_map(&md[sg], do_src, D, Hq, g.N, B, first, len, 128)) return rc;
-      if (int32_t rc = encode_segment_map(&mk[sg], k, D, Hkv, g.N, B, first, len, 128)) return rc;
-      if (int32_t rc = encode_segment_map(&mv[sg], v, D, Hkv, g.N, B, first, len, 128)) return rc;
-      if (int32_t rc = encode_segment_map(&mk64[sg], k, D, Hkv, g.N, B, first, len, DQ_BN)) return rc;
-      if (int32_t rc = encode_segment_map(&mv64[sg], v, D, Hkv, g.N, B, first, len, DQ_BN)) return rc;
-    }
-    const int n_tiles = n_sink_t + n_raw_t + n_gist_t;
-    cudaError_t e = cudaFuncSetAttribute(attn_bwd_dkdv_sm100_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         KvSmem<64>::kBytes);
-    if (e == cudaSuccess)
-      e = cudaFuncSetAttribute(attn_bwd_dq_sm100_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, DqSmem<64>::kBytes);
-    if (e != cudaSuccess) return fail(UNIGIST_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
-    {
-      KernelScope ks("attn_bwd_dkdv_sm100_kernel", st);
-      attn_bwd_dkdv_sm100_kernel<64><<<dim3(n_tiles, Hkv, B), kKvThreads, KvSmem<64>::kBytes, st>>>(
-          mq[0], mq[1], mq[2], md[0], md[1], md[2], mk[0], mk[1], mk[2], mv[0], mv[1], mv[2], g, Hq, Hkv, scale, lse, delta,
-          (__nv_bfloat16*)dk, (__nv_bfloat16*)dv, n_sink_t, n_gist_t);
-    }
-    if (int32_t rc = check_launch("tcgen05 dK/dV kernel")) return rc;
-    {
-      KernelScope ks("attn_bwd_dq_sm100_kernel", st);
-      attn_bwd_dq_sm100_kernel<64><<<dim3(n_tiles, Hq, B), kDqThreads, DqSmem<64>::kBytes, st>>>(
-          mq[0], mq[1], mq[2], md[0], md[1], md[2], mk64[0], mk64[1], mk64[2], mv64[0], mv64[1], mv64[2], g, Hq, Hkv, scale,
-          lse, delta, (__nv_bfloat16*)dq, n_sink_t, n_raw_t);
-    }
-    return check_launch("tcgen05 dQ kernel");
-  }
+  if (!fused)
+    return D == 64 ? launch_two_kernels<64>(g, p, scale, q, do_src, k, v, lse, delta, dq, dk, dv, st)
+                   : launch_two_kernels<128>(g, p, scale, q, do_src, k, v, lse, delta, dq, dk, dv, st);
   BwdRuns<1> P;
   P.n = 1;
   P.total_heavy = 0;  // not used with the (blocks, 1, batch) grid

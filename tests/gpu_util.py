@@ -43,11 +43,11 @@ def run_attention_interleaved(w: synth.Workload, backward: bool = True, inputs=N
 
 
 def run_attention(w: synth.Workload, backward: bool = True, dout_fp32: bool = False, inputs=None,
-                  softmax_scale: float = 0.0):
+                  softmax_scale: float = 0.0, flags: int = 0):
     """-> dict of CUDA tensors in INTERLEAVED order: o, lse [B,Hq,N], dq, dk, dv, plus inputs."""
     dev = torch.device("cuda:0")
     inp = inputs or synth.attention_inputs(w, with_grad=backward, dout_fp32=dout_fp32)
-    p = problem_of(w, ug.FLAG_DOUT_FP32 if (backward and dout_fp32) else 0, softmax_scale)
+    p = problem_of(w, flags | (ug.FLAG_DOUT_FP32 if (backward and dout_fp32) else 0), softmax_scale)
     N = ug.unigist_total_len(p)
     d = {k: v.to(dev) for k, v in inp.items()}
     sh = {}

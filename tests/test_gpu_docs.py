@@ -108,6 +108,46 @@ def test_docs_backward_takes_an_fp32_dout(D, il):
     assert (got[True][0].float() - got[False][0].float()).abs().max().item() <= 2.0 ** -7
 
 
+def test_docs_backward_with_a_fixed_dq_order():
+    """UNIGIST_FLAG_DETERMINISTIC_DQ on a packed sample (head_dim 128): against the oracle, and the same bits twice."""
+    s, r, W, doc_T, Hq, Hkv, D = 4, 4, 8, [64, 132, 64, 64, 8, 256], 4, 2, 128
+    k_units = (W + r - 1) // r
+    p = ug.Problem(1, doc_T[0], r, W, Hq, Hkv, D, num_sinks=s, flags=ug.FLAG_DETERMINISTIC_DQ)
+    n_tot = ug.unigist_docs_total_len(p, doc_T)
+    q, k, v, do = _packed_inputs(n_tot, Hq, Hkv, D, 41)  # interleaved order, packed
+    scale = 1.0 / np.sqrt(D)
+    dq_ref, dk_ref, dv_ref = oracle.docs_attn_bwd(s, doc_T, r, k_units, scale, f64(q), f64(k), f64(v), f64(do))
+    perm, base = [], 0
+    for T in doc_T:
+        sp, _, _ = oracle.layout(s, T, r)
+        perm.append(base + sp.astype(np.int64))
+        base += len(sp)
+    perm = torch.from_numpy(np.concatenate(perm))
+    dev = torch.device("cuda:0")
+    qd, kd, vd, dod = (t[perm].contiguous().to(dev) for t in (q, k, v, do))
+    o = torch.empty_like(qd)
+    lse = torch.empty(Hq * n_tot, device=dev)
+    ug.unigist_attn_fwd_docs(p, doc_T, qd, kd, vd, o, lse)
+    ws = torch.empty(max(ug.unigist_docs_workspace_bytes(p, ug.OP_BWD, doc_T), 16), dtype=torch.uint8, device=dev)
+    got = []
+    for _ in range(2):
+        dq, dk, dv = (torch.full_like(t, float("nan")) for t in (qd, kd, vd))
+        ug.unigist_attn_bwd_docs(p, doc_T, qd, kd, vd, o, lse, dod, dq, dk, dv, ws)
+        ug.unigist_device_status()
+        got.append((dq, dk, dv))
+    for a, b in zip(*got):
+        assert torch.equal(a, b)
+
+    def from_lib(t):
+        out = torch.empty_like(t.cpu())
+        out[perm] = t.cpu()
+        return out
+
+    check_close("dq", f64(from_lib(got[0][0])), dq_ref, TOL_GRAD)
+    check_close("dk", f64(from_lib(got[0][1])), dk_ref, TOL_GRAD)
+    check_close("dv", f64(from_lib(got[0][2])), dv_ref, TOL_GRAD)
+
+
 def test_docs_reject_bad_lists():
     p = ug.Problem(1, 16, 4, 8, 2, 2, 128)
     x = torch.zeros(64, 2, 128, dtype=torch.bfloat16, device="cuda")

@@ -156,6 +156,32 @@ def test_fp32_dout_is_rounded_to_bf16_on_load(name):
     check_close("dV", f64(a["dv"]), dv, TOL_GRAD)
 
 
+@pytest.mark.parametrize("name", ["gqa_128", "sinks_300", "ragged_group3_128", "long_units", "cut_walks_sinks", "peaky_128"])
+def test_deterministic_dq_flag(name):
+    """UNIGIST_FLAG_DETERMINISTIC_DQ (head_dim 128): the gradients match the oracle, and two runs give the same bits
+    in dq as well; dk, dv and the forward are what the default backward gives."""
+    w = next(x for x in SMALL + PEAKY if x.name == name)
+    assert w.head_dim == 128
+    a = run_attention(w, flags=ug.FLAG_DETERMINISTIC_DQ)
+    b = run_attention(w, inputs=a["inputs"], flags=ug.FLAG_DETERMINISTIC_DQ)
+    for n in ("o", "lse", "dq", "dk", "dv"):
+        assert torch.equal(a[n], b[n]), n
+    inp = a["inputs"]
+    k = oracle.window_units(w.window, w.ratio)
+    dq, dk, dv = oracle.attn_bwd(w.num_sinks, w.raw_len, w.ratio, k, w.head_dim ** -0.5,
+                                 *(f64(inp[n]) for n in ("q", "k", "v", "dout")))
+    check_close("dQ", f64(a["dq"]), dq, TOL_GRAD)
+    check_close("dK", f64(a["dk"]), dk, TOL_GRAD)
+    check_close("dV", f64(a["dv"]), dv, TOL_GRAD)
+    p = problem_of(w, ug.FLAG_DETERMINISTIC_DQ | ug.FLAG_INTERLEAVED)
+    x = torch.zeros(w.batch, w.total_len, w.num_q_heads, 128, dtype=torch.bfloat16, device=DEV)
+    kv = torch.zeros(w.batch, w.total_len, w.num_kv_heads, 128, dtype=torch.bfloat16, device=DEV)
+    lse = torch.zeros(w.batch, w.num_q_heads, w.total_len, device=DEV)
+    ws = torch.empty(max(16, ug.unigist_workspace_bytes(p, ug.OP_BWD)), dtype=torch.uint8, device=DEV)
+    with pytest.raises(ug.UnigistError):  # the flag's kernels take shifted tensors
+        ug.unigist_attn_bwd(p, x, kv, kv, x, lse, x, torch.empty_like(x), torch.empty_like(kv), torch.empty_like(kv), ws)
+
+
 def test_interleaved_flag_is_refused_where_the_tiles_do_not_line_up():
     for w in (SMALL[0], synth.Workload("r7", 1, 448, 7, 64, 2, 1, 128, seed=1)):
         p = problem_of(w, ug.FLAG_INTERLEAVED)
@@ -185,10 +211,15 @@ def test_forward_is_deterministic():
                                                  ("llama8b_layer", True, "interleaved"),
                                                  ("train_batch", True, "interleaved"),
                                                  ("long_prefill", False, "interleaved"),
-                                                 ("table4_16k_r8", True, "interleaved")])
+                                                 ("table4_16k_r8", True, "interleaved"),
+                                                 # the two-kernel backward at head_dim 128 (a fixed dQ summation order)
+                                                 ("llama8b_layer", True, "deterministic")])
 def test_full_size_sampled(name, backward, route):
     w = synth.WORKLOADS[name]
-    out = run_attention(w, backward=backward) if route == "explicit" else run_attention_interleaved(w, backward=backward)
+    if route == "interleaved":
+        out = run_attention_interleaved(w, backward=backward)
+    else:
+        out = run_attention(w, backward=backward, flags=ug.FLAG_DETERMINISTIC_DQ if route == "deterministic" else 0)
     inp = out["inputs"]
     s, T, r = w.num_sinks, w.raw_len, w.ratio
     k = oracle.window_units(w.window, r)
@@ -201,10 +232,10 @@ def test_full_size_sampled(name, backward, route):
     kv_heads = sorted({hk0, (hk0 + max(1, w.num_kv_heads // 2)) % w.num_kv_heads})
     # no row anywhere was left unwritten
     assert torch.isfinite(out["lse_shifted"]).all()
-    assert torch.isfinite(out["o_shifted" if route == "explicit" else "o"].float()).all()
+    assert torch.isfinite(out["o_shifted" if route != "interleaved" else "o"].float()).all()
     if backward:
         for n in ("dq", "dk", "dv"):
-            assert torch.isfinite(out[n + "_shifted" if route == "explicit" else n].float()).all(), n
+            assert torch.isfinite(out[n + "_shifted" if route != "interleaved" else n].float()).all(), n
     # forward: every batch index, two KV heads; the edge rows one by one and three blocks of 16 consecutive rows
     for b in range(w.batch):
         for hk in kv_heads:
