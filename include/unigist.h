@@ -67,7 +67,8 @@ typedef enum {
  * dQ of a query tile is then summed in tensor memory by ONE thread block that walks the tile's keys (a second
  * kernel that recomputes S and dP: seven matrix products per tile pair instead of five, 1.5 to 2 times the time)
  * instead of being reduced into memory in the order in which key tiles' blocks arrive.  No effect for head_dim 64,
- * whose backward always works this way.  Not together with UNIGIST_FLAG_INTERLEAVED (UNIGIST_ERR_UNSUPPORTED).
+ * whose backward always works this way.  The workspace then holds no fp32 accumulator (the size queries follow the
+ * flag).  Not together with UNIGIST_FLAG_INTERLEAVED (UNIGIST_ERR_UNSUPPORTED).
  */
 #define UNIGIST_FLAG_DETERMINISTIC_DQ 4u
 

@@ -194,11 +194,11 @@ size_t unigist_workspace_bytes(const unigist_problem* p, int32_t op) {
     case UNIGIST_OP_FWD:
       return 0;
     case UNIGIST_OP_BWD:
-      // Delta [B,Hq,N] fp32, a bf16 copy of dO when it arrives as fp32, and for head_dim 128 the fp32 dQ
-      // accumulator of the fused tensor-core backward
+      // Delta [B,Hq,N] fp32, a bf16 copy of dO when it arrives as fp32, and for the fused tensor-core backward
+      // the fp32 dQ accumulator and the chunks' partial dK / dV
       return bwd_scratch_bytes((long long)p->batch * g.N, p->num_q_heads, p->head_dim,
-                               (p->flags & UNIGIST_FLAG_DOUT_FP32) != 0) +
-             bwd_partial_bytes(g, p->batch, p->num_q_heads, p->num_kv_heads, p->head_dim);
+                               (p->flags & UNIGIST_FLAG_DOUT_FP32) != 0, bwd_is_fused(p->head_dim, p->flags)) +
+             bwd_partial_bytes(g, p->batch, p->num_q_heads, p->num_kv_heads, bwd_is_fused(p->head_dim, p->flags));
     case UNIGIST_OP_COMPACT: {
       const size_t L = (size_t)g.s + g.n + (size_t)g.k * g.r;
       return align_up(2 * (size_t)p->batch * L * p->num_kv_heads * p->head_dim * 2, 256);
@@ -389,13 +389,13 @@ int64_t unigist_docs_total_len(const unigist_problem* p, int32_t num_docs, const
 size_t unigist_docs_workspace_bytes(const unigist_problem* p, int32_t op, int32_t num_docs, const int32_t* doc_raw_len) {
   if (check_docs(p, num_docs, doc_raw_len) != UNIGIST_OK) return 0;
   if (op != UNIGIST_OP_BWD) return 0;
-  if (p->head_dim == 128) {  // one scratch layout over all packed tokens, then the runs' partial dK / dV
+  if (bwd_is_fused(p->head_dim, p->flags)) {  // one scratch layout over all packed tokens, then the runs' partial dK / dV
     size_t need = bwd_scratch_bytes(unigist_docs_total_len(p, num_docs, doc_raw_len), p->num_q_heads, p->head_dim,
-                                    (p->flags & UNIGIST_FLAG_DOUT_FP32) != 0);
+                                    (p->flags & UNIGIST_FLAG_DOUT_FP32) != 0, true);
     for_each_doc_run(p, num_docs, doc_raw_len, [&](const unigist_problem& run, int64_t, int32_t) {
       Geom g;
       if (check_problem(&run, &g, nullptr) == UNIGIST_OK)
-        need += bwd_partial_bytes(g, run.batch, run.num_q_heads, run.num_kv_heads, run.head_dim);
+        need += bwd_partial_bytes(g, run.batch, run.num_q_heads, run.num_kv_heads, true);
       return (int32_t)UNIGIST_OK;
     });
     return need;
@@ -443,7 +443,7 @@ int32_t unigist_attn_bwd_docs(const unigist_problem* p, int32_t num_docs, const 
   if (int32_t rc = doc_runs(p, num_docs, doc_raw_len, &runs, &tokens)) return rc;
   if (int32_t rc = check_interleaved(p, runs[0].g)) return rc;
   const float scale = p->softmax_scale > 0.f ? p->softmax_scale : 1.0f / sqrtf((float)p->head_dim);
-  if (p->head_dim == 128 && !(p->flags & UNIGIST_FLAG_DETERMINISTIC_DQ))
+  if (bwd_is_fused(p->head_dim, p->flags))
     return launch_bwd_sm100_runs(runs.data(), (int)runs.size(), tokens, *p, scale, q, k, v, o, lse, d_o, dq, dk, dv,
                                  workspace, (cudaStream_t)stream);
   // the two-kernel backward (head_dim 64, or a fixed summation order asked for): the runs one after the other on the caller's stream

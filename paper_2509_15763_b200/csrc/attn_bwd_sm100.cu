@@ -1403,20 +1403,20 @@ namespace {
 size_t align256(size_t x) { return (x + 255) / 256 * 256; }
 
 // The backward's scratch for `tokens` packed tokens: Delta (fp32, per run a [batch, Hq, N] block that starts at
-// float Hq * first token), the bf16 copy of an fp32 dO, and for head_dim 128 the fp32 dQ accumulator.
+// float Hq * first token), the bf16 copy of an fp32 dO, and for the fused backward the fp32 dQ accumulator.
 struct BwdScratch {
   float* delta;
   __nv_bfloat16* do_bf16;
   float* dq32;
 };
-BwdScratch carve_scratch(void* workspace, long long tokens, int Hq, int D, bool f32) {
+BwdScratch carve_scratch(void* workspace, long long tokens, int Hq, int D, bool f32, bool fused) {
   char* ws = static_cast<char*>(workspace);
   BwdScratch sc;
   sc.delta = reinterpret_cast<float*>(ws);
   ws += align256((size_t)tokens * Hq * sizeof(float));
   sc.do_bf16 = f32 ? reinterpret_cast<__nv_bfloat16*>(ws) : nullptr;
   if (f32) ws += align256((size_t)tokens * Hq * D * 2);
-  sc.dq32 = D == 128 ? reinterpret_cast<float*>(ws) : nullptr;
+  sc.dq32 = fused ? reinterpret_cast<float*>(ws) : nullptr;
   return sc;
 }
 
@@ -1577,15 +1577,15 @@ int32_t launch_two_kernels(const Geom& g, const unigist_problem& p, float scale,
 
 }  // namespace
 
-size_t bwd_scratch_bytes(long long tokens, int Hq, int D, bool dout_fp32) {
+size_t bwd_scratch_bytes(long long tokens, int Hq, int D, bool dout_fp32, bool fused) {
   size_t b = align256((size_t)tokens * Hq * sizeof(float));
   if (dout_fp32) b += align256((size_t)tokens * Hq * D * 2);
-  if (D == 128) b += align256((size_t)tokens * Hq * D * sizeof(float));
+  if (fused) b += align256((size_t)tokens * Hq * D * sizeof(float));
   return b;
 }
 
-size_t bwd_partial_bytes(const Geom& g, int batch, int Hq, int Hkv, int D) {
-  if (D != 128) return 0;
+size_t bwd_partial_bytes(const Geom& g, int batch, int Hq, int Hkv, bool fused) {
+  if (!fused) return 0;
   int C, tiles;
   bwd_chunking(g, batch, Hq, Hkv, &C, &tiles);
   if (C <= 1) return 0;
@@ -1599,20 +1599,18 @@ int32_t launch_bwd_sm100(const Geom& g, const unigist_problem& p, float scale, c
   const int D = p.head_dim, Hq = p.num_q_heads, Hkv = p.num_kv_heads, B = p.batch;
   const bool f32 = (p.flags & UNIGIST_FLAG_DOUT_FP32) != 0;
   const long long tokens = (long long)B * g.N;
-  const BwdScratch sc = carve_scratch(workspace, tokens, Hq, D, f32);
-  float* delta = sc.delta;
-  const void* do_src = f32 ? static_cast<const void*>(sc.do_bf16) : d_o;
   // head_dim 64 takes the two-kernel path, and so does head_dim 128 when dQ must not depend on the order in which
   // blocks arrive
-  const bool fused = D == 128 && !(p.flags & UNIGIST_FLAG_DETERMINISTIC_DQ);
+  const bool fused = bwd_is_fused(D, p.flags);
+  const BwdScratch sc = carve_scratch(workspace, tokens, Hq, D, f32, fused);
+  float* delta = sc.delta;
+  const void* do_src = f32 ? static_cast<const void*>(sc.do_bf16) : d_o;
   TokRuns<1> T;
   T.n = 1;
   T.run[0].g = g;
   T.run[0].tok_begin = 0;
   T.run[0].delta = delta;
-  BwdScratch sc_prep = sc;
-  if (!fused) sc_prep.dq32 = nullptr;  // no fp32 dQ accumulator to clear
-  if (int32_t rc = launch_prep(T, p, tokens, d_o, o, sc_prep, st)) return rc;
+  if (int32_t rc = launch_prep(T, p, tokens, d_o, o, sc, st)) return rc;
 
   if (!fused)
     return D == 64 ? launch_two_kernels<64>(g, p, scale, q, do_src, k, v, lse, delta, dq, dk, dv, st)
@@ -1620,7 +1618,7 @@ int32_t launch_bwd_sm100(const Geom& g, const unigist_problem& p, float scale, c
   BwdRuns<1> P;
   P.n = 1;
   P.total_heavy = 0;  // not used with the (blocks, 1, batch) grid
-  float* partial = reinterpret_cast<float*>(static_cast<char*>(workspace) + bwd_scratch_bytes(tokens, Hq, D, f32));
+  float* partial = reinterpret_cast<float*>(static_cast<char*>(workspace) + bwd_scratch_bytes(tokens, Hq, D, f32, true));
   if (int32_t rc = fill_bwd_run(&P.run[0], g, p, B, q, do_src, k, v, sc.dq32, lse, delta, dk, dv, partial)) return rc;
   if (int32_t rc = launch_fused(P, dim3(P.run[0].plane, 1, B), p, scale, st)) return rc;
   if (int32_t rc = launch_dkdv_reduce(P.run[0], B, p, scale, st)) return rc;
@@ -1634,16 +1632,16 @@ int32_t launch_bwd_sm100_runs(const SeqRun* runs, int n_runs, long long tokens, 
                               const void* d_o, void* dq, void* dk, void* dv, void* workspace, cudaStream_t st) {
   const int D = p.head_dim, Hq = p.num_q_heads, Hkv = p.num_kv_heads;
   const bool f32 = (p.flags & UNIGIST_FLAG_DOUT_FP32) != 0;
-  const BwdScratch sc = carve_scratch(workspace, tokens, Hq, D, f32);
+  const BwdScratch sc = carve_scratch(workspace, tokens, Hq, D, f32, true);
   const void* do_src = f32 ? static_cast<const void*>(sc.do_bf16) : d_o;
   const size_t rq = (size_t)Hq * D * 2, rk = (size_t)Hkv * D * 2;
   // the chunks' partial dK / dV: one slice per run, behind the scratch of the packed tokens
   std::vector<float*> partial_of(n_runs);
   {
-    char* at = static_cast<char*>(workspace) + bwd_scratch_bytes(tokens, Hq, D, f32);
+    char* at = static_cast<char*>(workspace) + bwd_scratch_bytes(tokens, Hq, D, f32, true);
     for (int i = 0; i < n_runs; ++i) {
       partial_of[i] = reinterpret_cast<float*>(at);
-      at += bwd_partial_bytes(runs[i].g, runs[i].batch, Hq, Hkv, D);
+      at += bwd_partial_bytes(runs[i].g, runs[i].batch, Hq, Hkv, true);
     }
   }
   for (int first = 0; first < n_runs; first += kMaxRunsPerLaunch) {

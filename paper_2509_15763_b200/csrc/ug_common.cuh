@@ -172,12 +172,15 @@ int32_t launch_bwd_sm100(const Geom& g, const unigist_problem& p, float scale, c
 int32_t launch_bwd_sm100_runs(const SeqRun* runs, int n_runs, long long tokens, const unigist_problem& p, float scale,
                               const void* q, const void* k, const void* v, const void* o, const float* lse,
                               const void* d_o, void* dq, void* dk, void* dv, void* workspace, cudaStream_t st);
-// Bytes of backward scratch for `tokens` packed tokens: Delta, the bf16 copy of an fp32 dO, and for head_dim 128
-// the fp32 dQ accumulator.
-size_t bwd_scratch_bytes(long long tokens, int Hq, int D, bool dout_fp32);
+// The fused backward serves head_dim 128 unless a fixed dQ summation order is asked for; otherwise two kernels.
+inline bool bwd_is_fused(int D, uint32_t flags) { return D == 128 && !(flags & UNIGIST_FLAG_DETERMINISTIC_DQ); }
+// Bytes of backward scratch for `tokens` packed tokens: Delta, the bf16 copy of an fp32 dO, and for the fused
+// backward the fp32 dQ accumulator.
+size_t bwd_scratch_bytes(long long tokens, int Hq, int D, bool dout_fp32, bool fused);
 // Bytes behind that scratch for the fp32 partial dK / dV of the sink and gist key tiles whose walk over the
-// queries is cut into chunks (0 where nothing is cut), for `batch` sequences of geometry g.
-size_t bwd_partial_bytes(const Geom& g, int batch, int Hq, int Hkv, int D);
+// queries is cut into chunks (0 where nothing is cut, or the backward is not the fused one), for `batch` sequences
+// of geometry g.
+size_t bwd_partial_bytes(const Geom& g, int batch, int Hq, int Hkv, bool fused);
 int32_t bwd_sm100_take_timeout(bool* timed_out);
 int32_t launch_compact_gather(const Geom& g, const unigist_problem& p, const void* k,
                               const void* v, void* kc, void* vc, int num_blocks,

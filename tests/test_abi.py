@@ -112,6 +112,9 @@ def test_backward_workspace_sizes_hold_every_part():
     assert need(1, 16384, 8, 1024, 32, 8, 128) == base                      # 75 MB per KV head: no cut walks
     assert need(1, 16384, 8, 1024, 32, 8, 128, ug.FLAG_DOUT_FP32) == base + al(N * 32 * 128 * 2)
     assert need(1, 16384, 8, 1024, 32, 8, 64) == al(32 * N * 4)              # head_dim 64: Delta only
+    # a fixed dQ order takes the two-kernel backward: no accumulator, no partial dK / dV
+    assert need(1, 16384, 8, 1024, 32, 8, 128, ug.FLAG_DETERMINISTIC_DQ) == al(32 * N * 4)
+    assert need(4, 32768, 4, 2048, 32, 8, 128, ug.FLAG_DETERMINISTIC_DQ) == al(4 * 32 * (32768 + 8192) * 4)
     # the training workload: 168 MB per KV head > 3/4 of the L2 -> 4 chunks over 64 gist key tiles per KV head
     Nt = 32768 + 8192
     got = need(4, 32768, 4, 2048, 32, 8, 128)
